@@ -1,0 +1,23 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+
+
+@pytest.fixture(scope="session")
+def tiny():
+    """(shape, weights, prompt, oracle model) of the tiny configuration."""
+    import synth_inputs as si
+    import oracle
+
+    sh = si.SHAPES["tiny"]
+    w = si.make_weights(sh)
+    return sh, w, si.make_prompts(sh)[0], oracle.Model(sh, w)
