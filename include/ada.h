@@ -1,0 +1,158 @@
+/* ada.h -- C ABI of the adaptive speculative-decoding iteration (AdaEAGLE) for one B200.
+ *
+ * One iteration = predict a draft length n with the Lightweight Draft Length
+ * Predictor (Eq. 3), draft n tokens with the EAGLE head as a chain (Eq. 2),
+ * verify the n+1 candidate positions with the target in one pass over its KV
+ * cache (Eq. 1), accept the longest correct prefix plus one bonus token, and
+ * roll the caches back to the accepted length (Algorithm 1).
+ *
+ * Conventions
+ *  - Every pointer named d_* is DEVICE memory, everything else is host memory.
+ *  - The caller owns weights, workspace and all I/O buffers; they are borrowed
+ *    for the lifetime of the context.  The library allocates no device memory.
+ *  - Weights are bf16, row-major [out][in].  Token ids and lengths are int32.
+ *  - All calls enqueue on the stream given to ada_init and return without
+ *    synchronising, except ada_get_counters and ada_destroy.
+ *  - Return value: 0 or a negative ADA_ERR_* code.  Argument errors are found on
+ *    the host before anything is launched.  Device-side range errors (cache full)
+ *    set a status word that ada_get_counters reports; the offending rows are skipped.
+ *  - Sequences of a batch are independent; per-sequence arrays are indexed [seq].
+ *  - Calling ada_ldlp_predict, ada_draft, ada_verify, ada_accept in that order
+ *    gives exactly what one ada_step gives.
+ */
+#ifndef ADA_H
+#define ADA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ADA_OK 0
+#define ADA_ERR_BAD_CONFIG (-1)
+#define ADA_ERR_NULL (-2)
+#define ADA_ERR_RANGE (-3)
+#define ADA_ERR_KV_FULL (-4)
+#define ADA_ERR_CUDA (-5)
+#define ADA_ERR_WORKSPACE (-6)
+#define ADA_ERR_STATE (-7)
+
+#define ADA_MAX_LAYERS 128
+#define ADA_MAX_BATCH 8
+#define ADA_MAX_NMAX 15
+
+typedef struct ada_ctx ada_ctx; /* opaque, host memory, owned by the library */
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  float rope_theta, rms_eps;
+  int32_t ldlp_hidden;  /* hidden width of the predictor MLP */
+  int32_t n_max;        /* largest draft length (k_max of Eq. 3), 1..15 */
+  int32_t ldlp_mode;    /* 0: class logits, n = argmax + 1 (the classification variant of Section 4.3.2) */
+  int32_t max_batch;    /* sequences decoded together, 1..8 */
+  int32_t kv_capacity;  /* positions per sequence, multiple of page_size */
+  int32_t page_size;    /* KV page length in positions: 64 */
+} ada_config;
+
+/* Device pointers to bf16 tensors.  Per-layer members are HOST arrays of n_layers device pointers. */
+typedef struct {
+  const void *embed;      /* [vocab][d]  shared by target, draft head and predictor        */
+  const void *lm_head;    /* [vocab][d]  shared by target and draft head (Section 2.2)     */
+  const void *final_norm; /* [d]                                                            */
+  const void *const *wq, *const *wk, *const *wv, *const *wo;   /* [d][d]                    */
+  const void *const *w_gate, *const *w_up;                     /* [d_ffn][d]                */
+  const void *const *w_down;                                   /* [d][d_ffn]                */
+  const void *const *norm_attn, *const *norm_mlp;              /* [d]                       */
+  const void *eagle_fc;   /* [d][2d], input [embedding ; feature]                           */
+  const void *e_wq, *e_wk, *e_wv, *e_wo, *e_gate, *e_up, *e_down, *e_norm_attn, *e_norm_mlp;
+  const void *ldlp_w1, *ldlp_b1; /* [hid][2d], [hid]   input [embedding ; feature] (Section 3.3) */
+  const void *ldlp_w2, *ldlp_b2; /* [n_max][hid], [n_max]                                   */
+} ada_weights;
+
+/* Bytes of device workspace (KV pools, feature rows, scratch) ada_init needs for this config;
+ * 0 if the config is invalid. */
+size_t ada_workspace_bytes(const ada_config *cfg);
+
+/* Validates cfg, carves d_workspace (256-byte aligned, >= ada_workspace_bytes) and builds the
+ * rotary table.  cuda_stream is a cudaStream_t (NULL = default stream). */
+int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights *w, void *d_workspace,
+             size_t workspace_bytes, void *cuda_stream);
+
+/* Algorithm 1, first pass (draft length 0): the target reads the m prompt tokens of sequence
+ * `seq`, fills its cache and emits the first new token, which becomes the pending token; the
+ * draft head is brought up to date on prompt positions 0..m-2.  d_first_token (optional)
+ * receives that token.  1 <= m, m + n_max + 2 <= kv_capacity. */
+int ada_prefill(ada_ctx *ctx, int seq, const int32_t *d_prompt, int32_t m, int32_t *d_first_token);
+
+/* Eq. 3: n[seq] = predictor([e ; f]) of the last token of the validated prefix (the token before
+ * the pending one) for every sequence; n in [1, n_max], clipped so that n+1 rows fit the cache.
+ * An override installed by ada_force_n replaces the prediction.  d_n: [max_batch]. */
+int ada_ldlp_predict(ada_ctx *ctx, int32_t *d_n);
+
+/* Eq. 2: the draft head emits d_n[seq] tokens per sequence as a chain (first bringing its cache
+ * up to date with the target features of the positions accepted last time).
+ * d_draft: [max_batch][n_max], entries beyond n are left untouched. */
+int ada_draft(ada_ctx *ctx, const int32_t *d_n, int32_t *d_draft);
+
+/* Eq. 1, forward part: the target runs over the pending token and the n draft tokens of every
+ * sequence (n may be 0: plain autoregressive step) and returns its greedy choice after each row.
+ * d_target_tok: [max_batch][n_max+1].  d_logits (optional): [max_batch][n_max+1][vocab] fp32. */
+int ada_verify(ada_ctx *ctx, const int32_t *d_draft, const int32_t *d_n, int32_t *d_target_tok,
+               float *d_logits);
+
+/* Eq. 1, decision part (footnote of Section 3.1) and the roll-back: accept_len = longest draft
+ * prefix matching the target's choices; emitted = accepted drafts + bonus token; target cache
+ * length and pending token advance; draft cache keeps only rows made from target features.
+ * Uses the drafts and target tokens of the last ada_verify.  All outputs optional:
+ * d_accept_len [max_batch], d_emitted [max_batch][n_max+1], d_n_emitted [max_batch]. */
+int ada_accept(ada_ctx *ctx, int32_t *d_accept_len, int32_t *d_emitted, int32_t *d_n_emitted);
+
+/* One whole iteration of Algorithm 1 (predict -> draft -> verify -> accept) replayed as a
+ * captured CUDA graph; draft lengths never visit the host.  Outputs as in ada_accept plus
+ * d_n_used [max_batch] (the draft lengths used); all optional. */
+int ada_step(ada_ctx *ctx, int32_t *d_emitted, int32_t *d_n_emitted, int32_t *d_n_used,
+             int32_t *d_accept_len);
+
+/* Test and measurement hooks ------------------------------------------------------------- */
+
+/* Fixed draft lengths instead of the predictor: n[seq] (host array of max_batch entries, each
+ * 0..n_max; 0 = plain autoregressive decoding, after which the draft head is out of date and
+ * ada_draft refuses to run).  NULL restores the predictor. */
+int ada_force_n(ada_ctx *ctx, const int32_t *n);
+
+/* Teacher forcing: after every draft step the drafted token of sequence seq is replaced by
+ * d_tokens[seq][step] (device, [max_batch][n_max]).  NULL switches it off. */
+int ada_force_draft(ada_ctx *ctx, const int32_t *d_tokens);
+
+/* Replace the outcome of the iteration that just ran for sequence `seq`: rewind to its start and
+ * commit the `count` given tokens instead (count-1 accepted drafts and a bonus token, 1 <= count
+ * <= n_max+1), recomputing cache rows and features from them.  Used to keep a run on a reference
+ * trajectory. */
+int ada_force_commit(ada_ctx *ctx, int seq, const int32_t *d_tokens, int32_t count);
+
+/* Synchronises the stream and returns, summed over sequences:
+ * out[0] N_target (verify passes), out[1] N_draft, out[2] N_waste, out[3] tokens emitted
+ * (Table 2's counters), out[4] device status word (0 = no device-side error),
+ * out[5] kernels launched by this context so far, out[6..7] 0. */
+int ada_get_counters(ada_ctx *ctx, int64_t out[8]);
+
+/* Device pointer and byte size of an internal buffer, for inspection by tests:
+ * which = 0 features f [max_batch][kv_capacity][d] fp32 (row = position),
+ *         1 predictor outputs z [max_batch][16] fp32, 2 committed tokens [max_batch][kv_capacity] int32,
+ *         3 lengths [max_batch][8] int32 (len, draft-cache len, n, accept_len, ...),
+ *         4 draft-head features of the last draft call [max_batch][n_max][d] fp32,
+ *         5 top-2 logits of every verify row [max_batch][n_max+1][2] fp32,
+ *         6 top-2 logits of every draft step [max_batch][n_max][2] fp32. */
+int ada_debug_buffer(ada_ctx *ctx, int which, void **d_ptr, size_t *bytes);
+
+/* Text of the last host-side error of this context ("" if none). */
+const char *ada_last_error(const ada_ctx *ctx);
+
+int ada_destroy(ada_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADA_H */
