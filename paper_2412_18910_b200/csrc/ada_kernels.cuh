@@ -1,0 +1,908 @@
+// Device kernels of the adaptive speculative-decoding iteration (sm_100a).
+//
+// Numerics shared by all kernels: weights and KV caches are bf16; the residual
+// stream, norms, softmax, every accumulator and every GEMM output are fp32.
+// A GEMM input row x is carried as two bf16 rows hi = bf16(x), lo = bf16(x - hi);
+// the tensor-core product W*hi + W*lo then equals W*x to ~2^-17 relative, which
+// keeps logits within 2e-2 of an fp32 evaluation over 40 layers.  Every output
+// element depends only on its own input row and on a fixed split of K, never on
+// how many rows share the launch, so speculative and autoregressive runs of the
+// library agree bit for bit.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ada {
+
+constexpr int kMaxBatch = 8;
+constexpr int kMaxRows = 128;   // rows of one pass (all sequences together)
+constexpr int kAttnSplits = 8;  // KV splits per (sequence, head)
+constexpr int kRowGroup = 16;   // query rows an attention warp keeps in registers
+template <int HD>
+constexpr int attn_smem_bytes() { return (kRowGroup * HD + 4 * kRowGroup * 32 + 8 * kRowGroup + 4 * kRowGroup * HD) * 4; }
+
+// status bits (device status word)
+constexpr int kStatKvFull = 1;
+constexpr int kStatStale = 2;
+
+struct SeqState {
+  int len;     // committed tokens, the last one pending (its row is not in the target cache)
+  int dlen;    // draft-cache rows computed from target features
+  int n;       // draft length of this iteration
+  int k_acc;   // accepted drafts of the last accept
+  int j_prev;  // index of the pending token when the last verify started
+  int n_emit;  // tokens emitted by the last accept
+  int stale;   // draft head is behind by more rows than one pass holds
+  int pad;
+};
+
+struct Counters {
+  unsigned long long n_target, n_draft, n_waste, n_tokens;
+  int status;
+  int pad;
+};
+
+// Row list of the pass being computed.  Rows of one sequence are contiguous.
+struct Pass {
+  int T;                   // rows in this pass
+  int lmT;                 // rows that go through the LM head (draft: one per active sequence)
+  int row_seq[kMaxRows];
+  int row_pos[kMaxRows];   // absolute position (RoPE angle, cache row)
+  int row_tok[kMaxRows];   // token whose embedding enters the row
+  int row_out[kMaxRows];   // output slot of the row
+  int lm_row[kMaxRows];    // draft: pass row of LM row i
+  int lm_out[kMaxRows];    // draft: output slot of LM row i
+  int seq_row0[kMaxBatch];
+  int seq_rows[kMaxBatch];
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// block-wide sum for blockDim.x <= 1024, result to all threads
+__device__ __forceinline__ float block_sum(float v, float *sh) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += sh[i];  // fixed order
+  return t;
+}
+
+// ---------------------------------------------------------------------------------------------
+// top-2 bookkeeping for the greedy choice: (v1, i1) best value / lowest index among equals, v2 second
+struct Top2 {
+  float v1;
+  int i1;
+  float v2;
+};
+__device__ __forceinline__ Top2 top2_merge(Top2 a, Top2 b) {
+  Top2 r;
+  const bool a_wins = (a.v1 > b.v1) || (a.v1 == b.v1 && a.i1 <= b.i1);
+  if (a_wins) {
+    r.v1 = a.v1; r.i1 = a.i1; r.v2 = fmaxf(a.v2, b.v1);
+  } else {
+    r.v1 = b.v1; r.i1 = b.i1; r.v2 = fmaxf(b.v2, a.v1);
+  }
+  return r;
+}
+__device__ __forceinline__ Top2 top2_shfl_xor(Top2 a, int m) {
+  Top2 b;
+  b.v1 = __shfl_xor_sync(0xffffffffu, a.v1, m);
+  b.i1 = __shfl_xor_sync(0xffffffffu, a.i1, m);
+  b.v2 = __shfl_xor_sync(0xffffffffu, a.v2, m);
+  return top2_merge(a, b);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Skinny GEMM  Y[t][n] = sum_k X[t][k] * W[n][k],  t < T <= 8*NT rows, W bf16 [N][K] streamed once.
+// The weight tile is the 16-row operand of mma.sync m16n8k16 (swap-AB) and is loaded straight from
+// global memory with 128-bit loads: lane (g, q) reads 8 consecutive k of rows g and g+8, and the
+// same k permutation is applied to the activation operand, so no shared-memory staging of W is
+// needed.  Activations (hi and lo halves) sit in shared memory for the CTA's K chunk.
+// A CTA = 4 warps = 64 weight rows; grid.y splits K; partial sums go to a scratch buffer and the
+// CTA that arrives last adds them in split order and runs the epilogue (deterministic).
+enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_ARGMAX = 3 };
+
+struct GemmArgs {
+  const __nv_bfloat16 *W[3];  // STORE: up to 3 row segments; SWIGLU: W[0] = gate, W[1] = up
+  int nseg, Nseg, K;
+  int KS;                     // k range of one split (multiple of KC)
+  int KC;                     // k chunk held in shared memory (multiple of 64)
+  int S;                      // splits
+  const __nv_bfloat16 *Xhi, *Xlo;
+  int ldx;
+  float *Y;                   // STORE / RESID target
+  int ldy;
+  __nv_bfloat16 *Ohi, *Olo;   // SWIGLU target
+  int ldo;
+  float *part;                // [S][8*NT][Ntot] partial sums
+  int *cnt;                   // [tiles] arrival counters (zero between launches)
+  float *logits;              // ARGMAX: optional logits [slot][ldl]
+  int ldl;
+  float4 *amax;               // ARGMAX: [tiles][8*NT] (v1, i1, v2)
+  const Pass *pass;
+  int use_lm_rows;            // ARGMAX in the draft: T = pass->lmT, slots = pass->lm_out
+};
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+template <int NT, int EPI>
+__global__ void __launch_bounds__(128) k_gemm(const GemmArgs a) {
+  constexpr int NA = (EPI == EPI_SWIGLU) ? 2 : 1;  // weight matrices per warp
+  constexpr int U = (NT > 2) ? 2 : 4;              // 32-k blocks in flight per thread
+  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
+  if (T <= 0) return;
+  const int nt_act = (T + 7) >> 3;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q = lane & 3;
+
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int xstride = a.KC * 2 + 64;  // bytes per activation row in shared memory
+  unsigned char *xs_hi = smem;
+  unsigned char *xs_lo = smem + (size_t)NT * 8 * xstride;
+  __shared__ int s_last;
+  __shared__ Top2 s_top[4][NT * 8];
+
+  const int tiles_per_seg = (a.Nseg + 63) >> 6;
+  const int seg = (EPI == EPI_SWIGLU) ? 0 : blockIdx.x / tiles_per_seg;
+  const int tile = (EPI == EPI_SWIGLU) ? blockIdx.x : blockIdx.x % tiles_per_seg;
+  const int n0 = tile * 64 + warp * 16;
+  const int ra = n0 + g, rb = n0 + g + 8;
+  const bool va = ra < a.Nseg, vb = rb < a.Nseg;
+
+  const int kbeg = blockIdx.y * a.KS;
+  const int kend = min(a.K, kbeg + a.KS);
+
+  float acc[NA][NT][4];
+#pragma unroll
+  for (int m = 0; m < NA; ++m)
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[m][i][j] = 0.f;
+
+  const __nv_bfloat16 *wa[NA], *wb[NA];
+#pragma unroll
+  for (int m = 0; m < NA; ++m) {
+    const __nv_bfloat16 *base = (EPI == EPI_SWIGLU) ? a.W[m] : a.W[seg];
+    wa[m] = base + (size_t)(va ? ra : 0) * a.K + 8 * q;
+    wb[m] = base + (size_t)(vb ? rb : 0) * a.K + 8 * q;
+  }
+
+  for (int kc = kbeg; kc < kend; kc += a.KC) {
+    const int kc_end = min(kend, kc + a.KC);
+    __syncthreads();
+    {  // stage activations [nt_act*8][KC] (hi, lo); 16-byte granules, zero beyond K
+      const int gran = a.KC >> 3;
+      const int total = nt_act * 8 * gran * 2;
+      for (int i = tid; i < total; i += 128) {
+        const int which = i / (nt_act * 8 * gran);
+        const int rem = i - which * (nt_act * 8 * gran);
+        const int row = rem / gran, gk = rem - row * gran;
+        const int k = kc + gk * 8;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (k < kc_end) v = *reinterpret_cast<const uint4 *>((which ? a.Xlo : a.Xhi) + (size_t)row * a.ldx + k);
+        *reinterpret_cast<uint4 *>((which ? xs_lo : xs_hi) + (size_t)row * xstride + gk * 16) = v;
+      }
+    }
+    __syncthreads();
+
+    const int nblk = (kc_end - kc + 31) >> 5;
+    uint4 A0[NA][U], A1[NA][U];
+    auto load_blocks = [&](uint4 (&P0)[NA][U], uint4 (&P1)[NA][U], int blk0) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int k = kc + (blk0 + u) * 32 + 8 * q;
+        const bool ok = (blk0 + u) < nblk && k < kc_end;
+#pragma unroll
+        for (int m = 0; m < NA; ++m) {
+          P0[m][u] = (ok && va) ? ldg_stream(wa[m] + kc + (blk0 + u) * 32) : make_uint4(0, 0, 0, 0);
+          P1[m][u] = (ok && vb) ? ldg_stream(wb[m] + kc + (blk0 + u) * 32) : make_uint4(0, 0, 0, 0);
+        }
+      }
+    };
+    load_blocks(A0, A1, 0);
+    for (int blk = 0; blk < nblk; blk += U) {
+      uint4 N0[NA][U], N1[NA][U];
+      load_blocks(N0, N1, blk + U);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        if (blk + u < nblk) {
+          const int koff = ((blk + u) * 32 + 8 * q) * 2;
+#pragma unroll
+          for (int i = 0; i < NT; ++i) {
+            if (i < nt_act) {
+              const uint4 bh = *reinterpret_cast<const uint4 *>(xs_hi + (size_t)(i * 8 + g) * xstride + koff);
+              const uint4 bl = *reinterpret_cast<const uint4 *>(xs_lo + (size_t)(i * 8 + g) * xstride + koff);
+#pragma unroll
+              for (int m = 0; m < NA; ++m) {
+                mma_bf16(acc[m][i], A0[m][u].x, A1[m][u].x, A0[m][u].y, A1[m][u].y, bh.x, bh.y);
+                mma_bf16(acc[m][i], A0[m][u].z, A1[m][u].z, A0[m][u].w, A1[m][u].w, bh.z, bh.w);
+                mma_bf16(acc[m][i], A0[m][u].x, A1[m][u].x, A0[m][u].y, A1[m][u].y, bl.x, bl.y);
+                mma_bf16(acc[m][i], A0[m][u].z, A1[m][u].z, A0[m][u].w, A1[m][u].w, bl.z, bl.w);
+              }
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int m = 0; m < NA; ++m) {
+          A0[m][u] = N0[m][u];
+          A1[m][u] = N1[m][u];
+        }
+    }
+  }
+
+  // element (m, i, j) of acc: weight row n = n0 + g + 8*(j>>1), pass row t = 8*i + 2*q + (j&1)
+  const int Ntot = (EPI == EPI_SWIGLU) ? 2 * a.Nseg : a.nseg * a.Nseg;
+  if (a.S > 1) {
+    const int TP = NT * 8;
+#pragma unroll
+    for (int m = 0; m < NA; ++m)
+#pragma unroll
+      for (int i = 0; i < NT; ++i)
+        if (i < nt_act)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
+            if (n < a.Nseg) {
+              const int col = ((EPI == EPI_SWIGLU) ? m : seg) * a.Nseg + n;
+              __stcg(a.part + ((size_t)blockIdx.y * TP + t) * Ntot + col, acc[m][i][j]);
+            }
+          }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(a.cnt + blockIdx.x, 1) == a.S - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+#pragma unroll
+    for (int m = 0; m < NA; ++m)
+#pragma unroll
+      for (int i = 0; i < NT; ++i)
+        if (i < nt_act)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
+            float s = 0.f;
+            if (n < a.Nseg) {
+              const int col = ((EPI == EPI_SWIGLU) ? m : seg) * a.Nseg + n;
+              for (int sp = 0; sp < a.S; ++sp) s += __ldcg(a.part + ((size_t)sp * TP + t) * Ntot + col);
+            }
+            acc[m][i][j] = s;
+          }
+    if (tid == 0) a.cnt[blockIdx.x] = 0;
+  }
+
+  if (EPI == EPI_STORE || EPI == EPI_RESID) {
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+      if (i < nt_act)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
+          if (n < a.Nseg && t < T) {
+            float *p = a.Y + (size_t)t * a.ldy + seg * a.Nseg + n;
+            if (EPI == EPI_RESID) *p += acc[0][i][j]; else *p = acc[0][i][j];
+          }
+        }
+  } else if (EPI == EPI_SWIGLU) {
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+      if (i < nt_act)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
+          if (n < a.Nseg && t < T) {
+            const float gt = acc[0][i][j], up = acc[NA - 1][i][j];
+            const float o = (gt / (1.f + __expf(-gt))) * up;
+            __nv_bfloat16 hi, lo;
+            split_bf16(o, hi, lo);
+            a.Ohi[(size_t)t * a.ldo + n] = hi;
+            a.Olo[(size_t)t * a.ldo + n] = lo;
+          }
+        }
+  } else {  // EPI_ARGMAX
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      if (i < nt_act) {
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const int t = 8 * i + 2 * q + jj;
+          const int slot = (t < T) ? (a.use_lm_rows ? a.pass->lm_out[t] : a.pass->row_out[t]) : 0;
+          Top2 best;
+          best.v1 = -INFINITY; best.i1 = 0x7fffffff; best.v2 = -INFINITY;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int n = n0 + g + 8 * h;
+            if (n < a.Nseg) {
+              const float v = acc[0][i][jj + 2 * h];
+              if (a.logits && t < T) a.logits[(size_t)slot * a.ldl + n] = v;
+              Top2 c; c.v1 = v; c.i1 = n; c.v2 = -INFINITY;
+              best = top2_merge(best, c);
+            }
+          }
+          best = top2_shfl_xor(best, 4);
+          best = top2_shfl_xor(best, 8);
+          best = top2_shfl_xor(best, 16);
+          if (g == 0) s_top[warp][t] = best;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < nt_act * 8) {
+      Top2 b = s_top[0][tid];
+      for (int w = 1; w < 4; ++w) b = top2_merge(b, s_top[w][tid]);
+      a.amax[(size_t)blockIdx.x * (NT * 8) + tid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+    }
+  }
+}
+
+// Final greedy choice per row: merge the per-tile candidates in tile order.
+// tok_out[slot] = argmax; top_out[slot] = (top1, top2).  forced (optional) overrides the token.
+__global__ void k_argmax_final(const float4 *amax, int tiles, int TP, const Pass *pass, int use_lm_rows,
+                               int *tok_out, float2 *top_out, const int *forced) {
+  const int T = use_lm_rows ? pass->lmT : pass->T;
+  const int t = blockIdx.x;
+  if (t >= T) return;
+  Top2 b;
+  b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+  for (int i = threadIdx.x; i < tiles; i += 32) {
+    const float4 c = amax[(size_t)i * TP + t];
+    Top2 x; x.v1 = c.x; x.i1 = __float_as_int(c.y); x.v2 = c.z;
+    b = top2_merge(b, x);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+  if (threadIdx.x == 0) {
+    const int slot = use_lm_rows ? pass->lm_out[t] : pass->row_out[t];
+    tok_out[slot] = forced ? forced[slot] : b.i1;
+    if (top_out) top_out[slot] = make_float2(b.v1, b.v2);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// h[t][:] = embedding of row_tok[t]
+__global__ void k_embed(const Pass *pass, const __nv_bfloat16 *embed, float *h, int d) {
+  const int t = blockIdx.x;
+  if (t >= pass->T) return;
+  const __nv_bfloat16 *e = embed + (size_t)pass->row_tok[t] * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)t * d + i] = __bfloat162float(e[i]);
+}
+
+// x = h / sqrt(mean(h^2) + eps) * gain  ->  hi/lo halves; optionally also fp32 rows to
+// feat[(seq*cap + pos)][d] (the target feature f after the final norm).
+__global__ void k_rmsnorm(const Pass *pass, const float *h, const __nv_bfloat16 *gain, float eps, int d,
+                          __nv_bfloat16 *xhi, __nv_bfloat16 *xlo, int ldx, float *feat, int cap) {
+  __shared__ float sh[32];
+  const int t = blockIdx.x;
+  if (t >= pass->T) return;
+  const float *hr = h + (size_t)t * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += hr[i] * hr[i];
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  float *fr = feat ? feat + ((size_t)pass->row_seq[t] * cap + pass->row_pos[t]) * d : nullptr;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float x = (hr[i] * inv) * __bfloat162float(gain[i]);
+    __nv_bfloat16 hi, lo;
+    split_bf16(x, hi, lo);
+    xhi[(size_t)t * ldx + i] = hi;
+    xlo[(size_t)t * ldx + i] = lo;
+    if (fr) fr[i] = x;
+  }
+}
+
+// hi/lo halves of selected rows of h without normalisation (draft head output -> LM head);
+// also keeps the fp32 row as the head's own feature for its next step.
+__global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bfloat16 *xhi,
+                                __nv_bfloat16 *xlo, int ldx, float *dfeat, int nmax, int step) {
+  const int i = blockIdx.x;
+  if (i >= pass->lmT) return;
+  const int t = pass->lm_row[i];
+  const int b = pass->row_seq[t];
+  const float *hr = h + (size_t)t * d;
+  float *fo = dfeat + ((size_t)b * nmax + step) * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float x = hr[c];
+    __nv_bfloat16 hi, lo;
+    split_bf16(x, hi, lo);
+    xhi[(size_t)i * ldx + c] = hi;
+    xlo[(size_t)i * ldx + c] = lo;
+    fo[c] = x;
+  }
+}
+
+// Rotary embedding (rotate-half pairing) of q and k, scaling of q by 1/sqrt(hd), and the write of
+// k, v (bf16) into the paged cache.  qkv: [T][3d] fp32.  rope: [cap][hd/2] (cos, sin).
+// Cache element (page, layer, head, slot, i): ((page*L + layer)*H + head)*page_size*hd + slot*hd + i.
+__global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope, float *qout,
+                          __nv_bfloat16 *kpool, __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
+                          int page_size, int L, int layer, int H, int hd, float qscale) {
+  const int t = blockIdx.x;
+  if (t >= pass->T) return;
+  const int d = H * hd, half = hd >> 1;
+  const int pos = pass->row_pos[t], b = pass->row_seq[t];
+  const int page = page_table[b * pages_per_seq + pos / page_size], slot = pos % page_size;
+  const float *q = qkv + (size_t)t * 3 * d, *k = q + d, *v = k + d;
+  for (int idx = threadIdx.x; idx < H * half; idx += blockDim.x) {
+    const int hh = idx / half, i = idx - hh * half;
+    const float2 cs = rope[(size_t)pos * half + i];
+    const int o = hh * hd + i;
+    const float qa = q[o], qb = q[o + half], ka = k[o], kb = k[o + half];
+    qout[(size_t)t * d + o] = (qa * cs.x - qb * cs.y) * qscale;
+    qout[(size_t)t * d + o + half] = (qb * cs.x + qa * cs.y) * qscale;
+    const size_t base = (((size_t)page * L + layer) * H + hh) * page_size * hd + (size_t)slot * hd;
+    kpool[base + i] = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
+    kpool[base + i + half] = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
+    vpool[base + i] = __float2bfloat16_rn(v[o]);
+    vpool[base + i + half] = __float2bfloat16_rn(v[o + half]);
+  }
+}
+
+// Attention of the rows of one sequence for one head over one split of the cache.
+// Row r (absolute position pos0 + r) sees cache positions 0..pos0+r: the whole history and the
+// earlier rows of its own block.  Lane = key in the score phase, lane = 4 channels in the
+// value phase.  Partial (m, l, o[hd]) per (head, split, row) goes to `part`.
+// HD must be 64 or 128.
+template <int HD>
+__global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
+                                                      const __nv_bfloat16 *vpool, const int *page_table,
+                                                      int pages_per_seq, int page_size, int L, int layer, int H,
+                                                      float *part) {
+  constexpr int VPL = HD / 32;  // value channels per lane
+  const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
+  const int R = pass->seq_rows[b];
+  if (pass->T <= 0 || R <= 0) return;
+  const int row0 = pass->seq_row0[b];
+  const int pos0 = pass->row_pos[row0];
+  const int nkeys = pos0 + R;
+  int chunk = (nkeys + kAttnSplits - 1) / kAttnSplits;
+  chunk = ((chunk + 31) / 32) * 32;
+  const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int d = H * HD;
+
+  extern __shared__ __align__(16) float attn_smem[];
+  float (*q_s)[HD] = reinterpret_cast<float (*)[HD]>(attn_smem);
+  float (*p_s)[kRowGroup][32] = reinterpret_cast<float (*)[kRowGroup][32]>(attn_smem + kRowGroup * HD);
+  float (*m_s)[kRowGroup] = reinterpret_cast<float (*)[kRowGroup]>(attn_smem + kRowGroup * HD + 4 * kRowGroup * 32);
+  float (*l_s)[kRowGroup] = m_s + 4;
+  float (*o_s)[kRowGroup][HD] =
+      reinterpret_cast<float (*)[kRowGroup][HD]>(attn_smem + kRowGroup * HD + 4 * kRowGroup * 32 + 8 * kRowGroup);
+
+  for (int rg = 0; rg < R; rg += kRowGroup) {
+    const int nr = min(kRowGroup, R - rg);
+    __syncthreads();
+    for (int i = threadIdx.x; i < nr * HD; i += 128) {
+      const int r = i / HD, c = i - r * HD;
+      q_s[r][c] = q[(size_t)(row0 + rg + r) * d + hh * HD + c];
+    }
+    __syncthreads();
+    float m[kRowGroup], l[kRowGroup], o[kRowGroup][VPL];
+#pragma unroll
+    for (int r = 0; r < kRowGroup; ++r) {
+      m[r] = -INFINITY; l[r] = 0.f;
+#pragma unroll
+      for (int c = 0; c < VPL; ++c) o[r][c] = 0.f;
+    }
+    for (int kb = kbeg + warp * 32; kb < kend; kb += 128) {
+      const int key = kb + lane;
+      const bool kv = key < kend;
+      float s[kRowGroup];
+#pragma unroll
+      for (int r = 0; r < kRowGroup; ++r) s[r] = 0.f;
+      if (kv) {
+        const int page = page_table[b * pages_per_seq + key / page_size], slot = key % page_size;
+        const uint4 *kr = reinterpret_cast<const uint4 *>(
+            kpool + (((size_t)page * L + layer) * H + hh) * page_size * HD + (size_t)slot * HD);
+#pragma unroll 4
+        for (int c = 0; c < HD / 8; ++c) {
+          const uint4 kk = kr[c];
+          float kf[8];
+          kf[0] = bf16_bits_to_float(kk.x & 0xffffu); kf[1] = bf16_bits_to_float(kk.x >> 16);
+          kf[2] = bf16_bits_to_float(kk.y & 0xffffu); kf[3] = bf16_bits_to_float(kk.y >> 16);
+          kf[4] = bf16_bits_to_float(kk.z & 0xffffu); kf[5] = bf16_bits_to_float(kk.z >> 16);
+          kf[6] = bf16_bits_to_float(kk.w & 0xffffu); kf[7] = bf16_bits_to_float(kk.w >> 16);
+#pragma unroll
+          for (int r = 0; r < kRowGroup; ++r) {
+            if (r < nr) {
+              const float4 qa = *reinterpret_cast<const float4 *>(&q_s[r][c * 8]);
+              const float4 qb = *reinterpret_cast<const float4 *>(&q_s[r][c * 8 + 4]);
+              s[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                      qb.z * kf[6] + qb.w * kf[7];
+            }
+          }
+        }
+      }
+      // online softmax per row over this block of 32 keys
+#pragma unroll
+      for (int r = 0; r < kRowGroup; ++r) {
+        if (r < nr) {
+          const bool seen = kv && key <= pos0 + rg + r;
+          const float sv = seen ? s[r] : -INFINITY;
+          const float mx = warp_max(sv);
+          const float mn = fmaxf(m[r], mx);
+          float p = 0.f, corr = 1.f;
+          if (mn > -INFINITY) {
+            p = seen ? __expf(sv - mn) : 0.f;
+            corr = __expf(m[r] - mn);  // m = -inf gives 0
+          }
+          l[r] = l[r] * corr + warp_sum(p);
+#pragma unroll
+          for (int c = 0; c < VPL; ++c) o[r][c] *= corr;
+          m[r] = mn;
+          p_s[warp][r][lane] = p;
+        }
+      }
+      __syncwarp();
+      const int nk = min(32, kend - kb);
+      for (int kk = 0; kk < nk; ++kk) {
+        const int key2 = kb + kk;
+        const int page = page_table[b * pages_per_seq + key2 / page_size], slot = key2 % page_size;
+        const __nv_bfloat16 *vr = vpool + (((size_t)page * L + layer) * H + hh) * page_size * HD + (size_t)slot * HD;
+        float vf[VPL];
+        if (VPL == 4) {
+          const uint2 vv = *reinterpret_cast<const uint2 *>(vr + lane * 4);
+          vf[0] = bf16_bits_to_float(vv.x & 0xffffu); vf[1] = bf16_bits_to_float(vv.x >> 16);
+          vf[VPL - 2] = bf16_bits_to_float(vv.y & 0xffffu); vf[VPL - 1] = bf16_bits_to_float(vv.y >> 16);
+        } else {
+          const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr + lane * 2);
+          vf[0] = bf16_bits_to_float(vv & 0xffffu); vf[VPL - 1] = bf16_bits_to_float(vv >> 16);
+        }
+#pragma unroll
+        for (int r = 0; r < kRowGroup; ++r) {
+          if (r < nr) {
+            const float p = p_s[warp][r][kk];
+#pragma unroll
+            for (int c = 0; c < VPL; ++c) o[r][c] += p * vf[c];
+          }
+        }
+      }
+      __syncwarp();
+    }
+    // combine the 4 warps in warp order
+#pragma unroll
+    for (int r = 0; r < kRowGroup; ++r) {
+      if (r < nr) {
+        if (lane == 0) { m_s[warp][r] = m[r]; l_s[warp][r] = l[r]; }
+#pragma unroll
+        for (int c = 0; c < VPL; ++c) o_s[warp][r][lane * VPL + c] = o[r][c];
+      }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < nr * HD; i += 128) {
+      const int r = i / HD, c = i - r * HD;
+      float M = m_s[0][r];
+      for (int w = 1; w < 4; ++w) M = fmaxf(M, m_s[w][r]);
+      float lo = 0.f, oo = 0.f;
+      if (M > -INFINITY) {
+        for (int w = 0; w < 4; ++w) {
+          const float e = __expf(m_s[w][r] - M);
+          lo += l_s[w][r] * e;
+          oo += o_s[w][r][c] * e;
+        }
+      }
+      float *pp = part + (((size_t)hh * kAttnSplits + split) * kMaxRows + (row0 + rg + r)) * (HD + 2);
+      pp[c] = oo;
+      if (c == 0) { pp[HD] = M; pp[HD + 1] = lo; }
+    }
+  }
+}
+
+// Merge the cache splits in split order and emit the attention output row as hi/lo halves.
+template <int HD>
+__global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat16 *xhi, __nv_bfloat16 *xlo,
+                               int ldx) {
+  const int hh = blockIdx.x, t = blockIdx.y;
+  if (t >= pass->T) return;
+  const int c = threadIdx.x;
+  const float *base = part + (((size_t)hh * kAttnSplits) * kMaxRows + t) * (HD + 2);
+  const size_t sstride = (size_t)kMaxRows * (HD + 2);
+  const int b = pass->row_seq[t];
+  const int nkeys = pass->row_pos[pass->seq_row0[b]] + pass->seq_rows[b];
+  int chunk = (nkeys + kAttnSplits - 1) / kAttnSplits;
+  chunk = ((chunk + 31) / 32) * 32;
+  const int nsp = (nkeys + chunk - 1) / chunk;  // splits that held keys
+  float M = -INFINITY;
+  for (int s = 0; s < nsp; ++s) M = fmaxf(M, base[s * sstride + HD]);
+  float l = 0.f, o = 0.f;
+  for (int s = 0; s < nsp; ++s) {
+    const float e = __expf(base[s * sstride + HD] - M);
+    l += base[s * sstride + HD + 1] * e;
+    o += base[s * sstride + c] * e;
+  }
+  const float x = o / l;
+  __nv_bfloat16 hi, lo;
+  split_bf16(x, hi, lo);
+  xhi[(size_t)t * ldx + hh * HD + c] = hi;
+  xlo[(size_t)t * ldx + hh * HD + c] = lo;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Draft-head input rows: X[t] = [embedding(row_tok[t]) ; feature] as hi/lo halves (K = 2d).
+// Catch-up rows (step 0) read the target feature of their position; later steps read the head's
+// own previous output dfeat[seq][step-1].
+__global__ void k_eagle_input(const Pass *pass, const __nv_bfloat16 *embed, const float *feat, int cap,
+                              const float *dfeat, int nmax, int step, int d, __nv_bfloat16 *xhi,
+                              __nv_bfloat16 *xlo, int ldx) {
+  const int t = blockIdx.x;
+  if (t >= pass->T) return;
+  const int b = pass->row_seq[t];
+  const __nv_bfloat16 *e = embed + (size_t)pass->row_tok[t] * d;
+  const float *f = step == 0 ? feat + ((size_t)b * cap + pass->row_pos[t]) * d
+                             : dfeat + ((size_t)b * nmax + (step - 1)) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    xhi[(size_t)t * ldx + i] = e[i];
+    xlo[(size_t)t * ldx + i] = __float2bfloat16_rn(0.f);
+    __nv_bfloat16 hi, lo;
+    split_bf16(f[i], hi, lo);
+    xhi[(size_t)t * ldx + d + i] = hi;
+    xlo[(size_t)t * ldx + d + i] = lo;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Length predictor (Eq. 3), class-logit form.  Stage 1: hidden unit per warp:
+// h[b][u] = ReLU(W1[u] . [e(tok[len-2]) ; f[len-2]] + b1[u]).
+__global__ void k_ldlp_hidden(const SeqState *st, const int *tok, const float *feat, int cap,
+                              const __nv_bfloat16 *embed, const __nv_bfloat16 *w1, const __nv_bfloat16 *b1, int d,
+                              int hid, float *hbuf) {
+  const int b = blockIdx.y;
+  const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int p = st[b].len - 2;
+  if (u >= hid || p < 0) return;
+  const __nv_bfloat16 *e = embed + (size_t)tok[(size_t)b * cap + p] * d;
+  const float *f = feat + ((size_t)b * cap + p) * d;
+  const __nv_bfloat16 *w = w1 + (size_t)u * 2 * d;
+  float s = 0.f;
+  for (int i = lane; i < d; i += 32) s += __bfloat162float(w[i]) * __bfloat162float(e[i]);
+  for (int i = lane; i < d; i += 32) s += __bfloat162float(w[d + i]) * f[i];
+  s = warp_sum(s);
+  if (lane == 0) hbuf[(size_t)b * hid + u] = fmaxf(s + __bfloat162float(b1[u]), 0.f);
+}
+
+// Stage 2: z = W2 h + b2, n = argmax + 1 (lowest index among equals), then the override and the
+// clip to the cache capacity.  One warp per sequence.
+__global__ void k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 *w2, const __nv_bfloat16 *b2,
+                           int hid, int nmax, int cap, const int *force_n, int has_force, float *zbuf,
+                           int *n_out, Counters *cnt) {
+  const int b = blockIdx.x, lane = threadIdx.x;
+  const int len = st[b].len;
+  if (len < 2) { if (lane == 0) { st[b].n = 0; if (n_out) n_out[b] = 0; } return; }
+  float best = -INFINITY;
+  int bi = 0;
+  for (int c = 0; c < nmax; ++c) {
+    float s = 0.f;
+    for (int i = lane; i < hid; i += 32) s += __bfloat162float(w2[(size_t)c * hid + i]) * hbuf[(size_t)b * hid + i];
+    s = warp_sum(s) + __bfloat162float(b2[c]);
+    if (lane == 0) zbuf[b * 16 + c] = s;
+    if (s > best) { best = s; bi = c; }
+  }
+  if (lane == 0) {
+    int n = bi + 1;
+    if (has_force) n = force_n[b];
+    const int room = cap - len;  // rows j..j+n need j + n + 1 <= cap, j = len - 1
+    if (n > room) { n = room < 0 ? 0 : room; atomicOr(&cnt->status, kStatKvFull); }
+    st[b].n = n;
+    if (n_out) n_out[b] = n;
+  }
+}
+
+// n[b] <- user array (separate-call API), with the same clip
+__global__ void k_set_n(SeqState *st, const int *n_in, int B, int nmax, int cap, Counters *cnt) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  int n = n_in[b];
+  n = max(0, min(n, nmax));
+  const int room = cap - st[b].len;
+  if (n > room) { n = room < 0 ? 0 : room; atomicOr(&cnt->status, kStatKvFull); }
+  st[b].n = n;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row lists.  One thread block of one warp; B <= 8, rows <= kMaxRows.
+//
+// Verify (Eq. 1): rows of sequence b = pending token then its n drafts, positions j..j+n.
+__global__ void k_rows_verify(Pass *pass, SeqState *st, const int *tok, int cap, const int *draft, int nmax, int B,
+                              int only_seq) {
+  if (threadIdx.x != 0) return;
+  int T = 0;
+  for (int b = 0; b < B; ++b) {
+    pass->seq_row0[b] = T;
+    pass->seq_rows[b] = 0;
+    if (only_seq >= 0 && b != only_seq) continue;
+    const int len = st[b].len;
+    if (len < 1) continue;
+    const int j = len - 1, n = st[b].n;
+    if (j + n + 1 > cap) continue;
+    st[b].j_prev = j;
+    for (int i = 0; i <= n; ++i) {
+      pass->row_seq[T] = b;
+      pass->row_pos[T] = j + i;
+      pass->row_tok[T] = i == 0 ? tok[(size_t)b * cap + j] : draft[b * nmax + i - 1];
+      pass->row_out[T] = b * (nmax + 1) + i;
+      ++T;
+    }
+    pass->seq_rows[b] = n + 1;
+  }
+  pass->T = T;
+  pass->lmT = T;
+}
+
+// Prefill chunk: rows pos0..pos0+R-1 of sequence b, tokens from the committed-token array.
+__global__ void k_rows_chunk(Pass *pass, const int *tok, int cap, int b, int pos0, int R, int tok_shift, int B) {
+  if (threadIdx.x != 0) return;
+  for (int i = 0; i < B; ++i) { pass->seq_row0[i] = 0; pass->seq_rows[i] = 0; }
+  for (int i = 0; i < R; ++i) {
+    pass->row_seq[i] = b;
+    pass->row_pos[i] = pos0 + i;
+    pass->row_tok[i] = tok[(size_t)b * cap + pos0 + i + tok_shift];
+    pass->row_out[i] = i;
+    pass->lm_row[i] = i;
+    pass->lm_out[i] = i;
+  }
+  pass->seq_rows[b] = R;
+  pass->T = R;
+  pass->lmT = R;
+}
+
+// Draft (Eq. 2).  step 0: catch-up rows p = dlen..j-1 of every sequence with n >= 1; row p pairs the
+// target feature of p with the embedding of token p+1; the last row feeds the LM head.
+// step s >= 1: one row per sequence with n > s at position j+s-1, token = draft[s-1].
+__global__ void k_rows_draft(Pass *pass, SeqState *st, const int *tok, int cap, const int *draft, int nmax, int B,
+                             int step, int max_rows, Counters *cnt) {
+  if (threadIdx.x != 0) return;
+  int T = 0, lmT = 0;
+  for (int b = 0; b < B; ++b) {
+    pass->seq_row0[b] = T;
+    pass->seq_rows[b] = 0;
+    const int n = st[b].n, j = st[b].len - 1;
+    if (n <= step || j < 1) continue;
+    if (step == 0) {
+      const int R = j - st[b].dlen;
+      if (R < 1 || T + R > max_rows || st[b].stale) { st[b].n = 0; atomicOr(&cnt->status, kStatStale); continue; }
+      for (int i = 0; i < R; ++i) {
+        const int p = st[b].dlen + i;
+        pass->row_seq[T] = b;
+        pass->row_pos[T] = p;
+        pass->row_tok[T] = tok[(size_t)b * cap + p + 1];
+        pass->row_out[T] = 0;
+        ++T;
+      }
+      pass->seq_rows[b] = R;
+      st[b].dlen = j;
+    } else {
+      pass->row_seq[T] = b;
+      pass->row_pos[T] = j + step - 1;
+      pass->row_tok[T] = draft[b * nmax + step - 1];
+      pass->row_out[T] = 0;
+      ++T;
+      pass->seq_rows[b] = 1;
+    }
+    pass->lm_row[lmT] = T - 1;
+    pass->lm_out[lmT] = b * nmax + step;
+    ++lmT;
+  }
+  pass->T = T;
+  pass->lmT = lmT;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Accept (Eq. 1 and the footnote of Section 3.1) and roll-back.  One thread per sequence.
+// forced_count > 0 (force_commit of sequence only_seq): accept count-1 drafts and take the bonus
+// from forced_tok instead of the target's choice.
+__global__ void k_accept(SeqState *st, int *tok, int cap, const int *draft, const int *target, int nmax, int B,
+                         Counters *cnt, int only_seq, const int *forced_tok, int forced_count, int *acc_out,
+                         int *emit_out, int *nemit_out, int *nused_out) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  if (only_seq >= 0 && b != only_seq) return;
+  const int len = st[b].len;
+  if (len < 1) return;
+  const int n = st[b].n;
+  const int j = st[b].j_prev;
+  if (j != len - 1 || j + n + 1 > cap) {  // no verify ran for this sequence
+    if (acc_out) acc_out[b] = 0;
+    if (nemit_out) nemit_out[b] = 0;
+    if (nused_out) nused_out[b] = n;
+    st[b].n_emit = 0;
+    return;
+  }
+  int k = 0;
+  if (forced_count > 0) {
+    k = forced_count - 1;
+  } else {
+    while (k < n && draft[b * nmax + k] == target[b * (nmax + 1) + k]) ++k;
+  }
+  for (int i = 0; i <= k; ++i) {
+    int t;
+    if (forced_count > 0) t = forced_tok[i];
+    else t = i < k ? draft[b * nmax + i] : target[b * (nmax + 1) + k];
+    tok[(size_t)b * cap + j + 1 + i] = t;
+    if (emit_out) emit_out[b * (nmax + 1) + i] = t;
+  }
+  st[b].len = j + k + 2;
+  st[b].k_acc = k;
+  st[b].n_emit = k + 1;
+  if (n == 0) st[b].stale = (j + 1 - st[b].dlen) > nmax + 1;  // the head falls behind while not drafting
+  if (acc_out) acc_out[b] = k;
+  if (nemit_out) nemit_out[b] = k + 1;
+  if (nused_out) nused_out[b] = n;
+  if (forced_count == 0) {
+    atomicAdd(&cnt->n_target, 1ull);
+    atomicAdd(&cnt->n_draft, (unsigned long long)n);
+    atomicAdd(&cnt->n_waste, (unsigned long long)(n - k));
+    atomicAdd(&cnt->n_tokens, (unsigned long long)(k + 1));
+  }
+}
+
+// Small state edits used by prefill and force_commit.
+__global__ void k_copy_prompt(int *tok, int cap, int b, const int *prompt, int m) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < m; i += gridDim.x * blockDim.x)
+    tok[(size_t)b * cap + i] = prompt[i];
+}
+__global__ void k_finish_prefill(SeqState *st, int *tok, int cap, int b, int m, const int *first_tok_slot,
+                                 int *user_out) {
+  if (threadIdx.x != 0) return;
+  const int t = first_tok_slot[0];
+  tok[(size_t)b * cap + m] = t;
+  st[b].len = m + 1;
+  st[b].dlen = m - 1;
+  st[b].n = 0; st[b].k_acc = 0; st[b].j_prev = -1; st[b].n_emit = 0; st[b].stale = 0;
+  if (user_out) *user_out = t;
+}
+__global__ void k_rewind(SeqState *st, int b, int count, const int *forced_tok, int *draft, int nmax,
+                         Counters *cnt) {
+  if (threadIdx.x != 0) return;
+  const int j = st[b].j_prev;
+  if (j < 0) return;
+  atomicAdd(&cnt->n_tokens, (unsigned long long)(count - st[b].n_emit));  // wraps correctly for negatives
+  st[b].len = j + 1;
+  st[b].n = count - 1;
+  for (int i = 0; i + 1 < count; ++i) draft[b * nmax + i] = forced_tok[i];
+}
+__global__ void k_copy_i32(int *dst, const int *src, int n) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = src[i];
+}
+__global__ void k_gather_n(const SeqState *st, int *out, int B) {
+  if (threadIdx.x < B) out[threadIdx.x] = st[threadIdx.x].n;
+}
+
+}  // namespace ada
