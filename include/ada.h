@@ -144,7 +144,9 @@ int ada_get_counters(ada_ctx *ctx, int64_t out[8]);
  *         3 lengths [max_batch][8] int32 (len, draft-cache len, n, accept_len, ...),
  *         4 draft-head features of the last draft call [max_batch][n_max][d] fp32,
  *         5 top-2 logits of every verify row [max_batch][n_max+1][2] fp32,
- *         6 top-2 logits of every draft step [max_batch][n_max][2] fp32. */
+ *         6 top-2 logits of every draft step [max_batch][n_max][2] fp32,
+ *         7 draft tokens of the last draft [max_batch][n_max] int32,
+ *         8 target choices of the last verify [max_batch][n_max+1] int32. */
 int ada_debug_buffer(ada_ctx *ctx, int which, void **d_ptr, size_t *bytes);
 
 /* Text of the last host-side error of this context ("" if none). */

@@ -1,0 +1,604 @@
+// Host side of the C ABI declared in include/ada.h: argument checks, workspace carving, and the
+// order in which the kernels of ada_kernels.cuh are enqueued for each step of Algorithm 1.
+// Every step of the path runs in those kernels; nothing is computed on the host except the
+// rotary table at initialisation.
+#include "ada.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "ada_kernels.cuh"
+
+using namespace ada;
+typedef __nv_bfloat16 bf16;
+
+namespace {
+
+struct LayerW {
+  const bf16 *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nm;
+};
+
+struct GemmPlan {
+  int KC, KS, S;
+};
+
+}  // namespace
+
+struct ada_ctx {
+  ada_config c;
+  cudaStream_t stream;
+  int B, TM, NT;          // batch, rows per pass, n8 tiles
+  int pages_per_seq, n_pages;
+  std::vector<LayerW> layers;
+  LayerW eagle;
+  const bf16 *embed, *lm_head, *final_norm, *eagle_fc, *ldlp_w1, *ldlp_b1, *ldlp_w2, *ldlp_b2;
+  // workspace pieces (device)
+  bf16 *tk, *tv, *dk, *dv;          // KV pools: target [page][L][H][ps][hd], draft [page][1][H][ps][hd]
+  int *page_table;                  // [B][pages_per_seq]
+  float2 *rope;                     // [cap][hd/2]
+  float *feat;                      // [B][cap][d]
+  float *dfeat;                     // [B][nmax][d]
+  int *tok;                         // [B][cap]
+  SeqState *st;                     // [B]
+  Counters *cnt;
+  Pass *pass;
+  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_z;
+  bf16 *xhi, *xlo, *x2hi, *x2lo;    // [TP][ldx], [TP][ldx2]
+  int ldx, ldx2;
+  int *gemm_cnt;
+  float4 *amax;
+  int *draft, *target, *force_n_dev, *chunk_tok;
+  float2 *vtop, *dtop;
+  float *chunk_logits_unused;
+  const int *force_draft;           // user device pointer or null
+  int has_force_n;
+  int host_force_n[ADA_MAX_BATCH];
+  size_t part_floats;
+  // bookkeeping
+  long long launches;
+  cudaGraphExec_t graph;
+  int graph_launches;
+  int graph_key;                    // configuration the graph was captured for
+  int *out_acc, *out_emit, *out_nemit, *out_nused;   // internal outputs of ada_step
+  std::string err;
+};
+
+namespace {
+
+int fail(ada_ctx *ctx, int code, const char *msg) {
+  if (ctx) ctx->err = msg;
+  return code;
+}
+
+#define LAUNCH(ctx, kernel, grid, block, smem, ...)                         \
+  do {                                                                      \
+    kernel<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);              \
+    (ctx)->launches++;                                                      \
+  } while (0)
+
+struct Carver {
+  char *base;
+  size_t off;
+  template <typename T>
+  T *take(size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+bool config_ok(const ada_config *c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->n_layers > ADA_MAX_LAYERS) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_heads < 1 || c->d_model != c->n_heads * c->head_dim) return false;
+  if (c->d_model % 64 || c->d_ffn % 16 || c->d_ffn < 16 || c->vocab % 16 || c->vocab < 16) return false;
+  if (c->ldlp_hidden < 1 || c->n_max < 1 || c->n_max > ADA_MAX_NMAX) return false;
+  if (c->ldlp_mode != 0) return false;
+  if (c->max_batch < 1 || c->max_batch > ADA_MAX_BATCH) return false;
+  if (c->max_batch * (c->n_max + 1) > 88) return false;
+  if (c->page_size != 64 || c->kv_capacity < 64 || c->kv_capacity % c->page_size) return false;
+  if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+  return true;
+}
+
+int rows_per_pass(const ada_config *c) {
+  int t = c->max_batch * (c->n_max + 1);
+  return t < 16 ? 16 : ((t + 7) / 8) * 8;
+}
+
+GemmPlan plan_gemm(int NT, int K, int tiles) {
+  GemmPlan p;
+  const int Kr = ((K + 63) / 64) * 64;
+  if (NT <= 2) {
+    p.KC = Kr < 1024 ? Kr : 1024;
+    p.KS = p.KC;
+  } else {
+    p.KC = Kr < 256 ? Kr : 256;
+    int chunks = (K + p.KC - 1) / p.KC;
+    int want = (592 + tiles - 1) / tiles;  // about four CTAs per SM in total
+    if (want < 1) want = 1;
+    if (want > chunks) want = chunks;
+    int per = (chunks + want - 1) / want;
+    p.KS = per * p.KC;
+  }
+  p.S = (K + p.KS - 1) / p.KS;
+  return p;
+}
+
+size_t part_need(int NT, int Ntot, int K, int tiles) {
+  GemmPlan p = plan_gemm(NT, K, tiles);
+  return p.S > 1 ? (size_t)p.S * NT * 8 * Ntot : 0;
+}
+
+// Lays the workspace out; with base == nullptr only measures it.
+size_t carve(ada_ctx *x, const ada_config *c, char *base) {
+  Carver w{base, 0};
+  const size_t d = c->d_model, F = c->d_ffn, V = c->vocab, L = c->n_layers, H = c->n_heads, hd = c->head_dim;
+  const size_t B = c->max_batch, cap = c->kv_capacity, ps = c->page_size;
+  const int TM = rows_per_pass(c), NT = TM / 8 > 2 ? 11 : 2;
+  const size_t TP = (size_t)NT * 8;
+  const size_t pps = cap / ps, pages = pps * B;
+  x->B = (int)B; x->TM = TM; x->NT = NT; x->pages_per_seq = (int)pps; x->n_pages = (int)pages;
+  x->tk = w.take<bf16>(pages * L * H * ps * hd);
+  x->tv = w.take<bf16>(pages * L * H * ps * hd);
+  x->dk = w.take<bf16>(pages * H * ps * hd);
+  x->dv = w.take<bf16>(pages * H * ps * hd);
+  x->page_table = w.take<int>(B * pps);
+  x->rope = w.take<float2>(cap * (hd / 2));
+  x->feat = w.take<float>(B * cap * d);
+  x->dfeat = w.take<float>(B * c->n_max * d);
+  x->tok = w.take<int>(B * cap);
+  x->st = w.take<SeqState>(B);
+  x->cnt = w.take<Counters>(1);
+  x->pass = w.take<Pass>(1);
+  x->h = w.take<float>(TP * d);
+  x->qkv = w.take<float>(TP * 3 * d);
+  x->qrot = w.take<float>(TP * d);
+  x->attn_part = w.take<float>(H * kAttnSplits * (size_t)kMaxRows * (hd + 2));
+  const size_t ldx = 2 * d, ldx2 = ((F + 63) / 64) * 64 > d ? ((F + 63) / 64) * 64 : d;
+  x->ldx = (int)ldx; x->ldx2 = (int)ldx2;
+  x->xhi = w.take<bf16>(TP * ldx);
+  x->xlo = w.take<bf16>(TP * ldx);
+  x->x2hi = w.take<bf16>(TP * ldx2);
+  x->x2lo = w.take<bf16>(TP * ldx2);
+  size_t pf = 0;
+  auto upd = [&](size_t v) { if (v > pf) pf = v; };
+  upd(part_need(NT, (int)(3 * d), (int)d, (int)(3 * ((d + 63) / 64))));
+  upd(part_need(NT, (int)d, (int)d, (int)((d + 63) / 64)));
+  upd(part_need(NT, (int)(2 * F), (int)d, (int)((F + 63) / 64)));
+  upd(part_need(NT, (int)d, (int)F, (int)((d + 63) / 64)));
+  upd(part_need(NT, (int)V, (int)d, (int)((V + 63) / 64)));
+  upd(part_need(NT, (int)d, (int)(2 * d), (int)((d + 63) / 64)));
+  x->part_floats = pf;
+  x->gemm_part = w.take<float>(pf ? pf : 1);
+  x->gemm_cnt = w.take<int>(4096);
+  x->amax = w.take<float4>(((V + 63) / 64) * TP);
+  x->ldlp_h = w.take<float>(B * c->ldlp_hidden);
+  x->ldlp_z = w.take<float>(B * 16);
+  x->draft = w.take<int>(B * c->n_max);
+  x->target = w.take<int>(B * (c->n_max + 1));
+  x->force_n_dev = w.take<int>(B);
+  x->chunk_tok = w.take<int>(kMaxRows);
+  x->vtop = w.take<float2>(B * (c->n_max + 1) + kMaxRows);
+  x->dtop = w.take<float2>(B * c->n_max + kMaxRows);
+  x->out_acc = w.take<int>(B);
+  x->out_emit = w.take<int>(B * (c->n_max + 1));
+  x->out_nemit = w.take<int>(B);
+  x->out_nused = w.take<int>(B);
+  return (w.off + 255) & ~(size_t)255;
+}
+
+template <int NT>
+int launch_gemm_nt(ada_ctx *x, int epi, GemmArgs &a, dim3 grid, size_t smem) {
+  switch (epi) {
+    case EPI_STORE: LAUNCH(x, (k_gemm<NT, EPI_STORE>), grid, 128, smem, a); break;
+    case EPI_RESID: LAUNCH(x, (k_gemm<NT, EPI_RESID>), grid, 128, smem, a); break;
+    case EPI_SWIGLU: LAUNCH(x, (k_gemm<NT, EPI_SWIGLU>), grid, 128, smem, a); break;
+    default: LAUNCH(x, (k_gemm<NT, EPI_ARGMAX>), grid, 128, smem, a); break;
+  }
+  return 0;
+}
+
+template <int NT>
+cudaError_t gemm_attr_nt(int bytes) {
+  cudaError_t e;
+  e = cudaFuncSetAttribute(k_gemm<NT, EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_gemm<NT, EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_gemm<NT, EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_gemm<NT, EPI_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+// Y = X W^T with one of the epilogues.  W0..W2: row segments (STORE) or gate/up (SWIGLU).
+void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, int nseg, int Nseg, int K,
+          const bf16 *Xhi, const bf16 *Xlo, int ldx, float *Y, int ldy, bf16 *Ohi, bf16 *Olo, int ldo,
+          float *logits, int use_lm_rows) {
+  GemmArgs a;
+  memset(&a, 0, sizeof(a));
+  a.W[0] = W0; a.W[1] = W1; a.W[2] = W2;
+  a.nseg = nseg; a.Nseg = Nseg; a.K = K;
+  const int tiles_per_seg = (Nseg + 63) / 64;
+  const int tiles = epi == EPI_SWIGLU ? tiles_per_seg : tiles_per_seg * nseg;
+  GemmPlan p = plan_gemm(x->NT, K, tiles);
+  a.KC = p.KC; a.KS = p.KS; a.S = p.S;
+  a.Xhi = Xhi; a.Xlo = Xlo; a.ldx = ldx;
+  a.Y = Y; a.ldy = ldy; a.Ohi = Ohi; a.Olo = Olo; a.ldo = ldo;
+  a.part = x->gemm_part; a.cnt = x->gemm_cnt;
+  a.logits = logits; a.ldl = x->c.vocab; a.amax = x->amax;
+  a.pass = x->pass; a.use_lm_rows = use_lm_rows;
+  const size_t smem = (size_t)2 * x->NT * 8 * (p.KC * 2 + 64);
+  dim3 grid(tiles, p.S);
+  if (x->NT == 2) launch_gemm_nt<2>(x, epi, a, grid, smem);
+  else launch_gemm_nt<11>(x, epi, a, grid, smem);
+}
+
+void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
+  const ada_config &c = x->c;
+  dim3 g1(c.n_heads, kAttnSplits, x->B);
+  dim3 g2(c.n_heads, x->TM);
+  if (c.head_dim == 128) {
+    LAUNCH(x, k_attn_partial<128>, g1, 128, attn_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
+    LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
+  } else {
+    LAUNCH(x, k_attn_partial<64>, g1, 128, attn_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
+    LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
+  }
+}
+
+// One pre-norm decoder block over the rows of x->pass; residual stream in x->h.
+void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L, int layer) {
+  const ada_config &c = x->c;
+  const int d = c.d_model, F = c.d_ffn;
+  LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.na, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
+  gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->ldx, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
+  LAUNCH(x, k_rope_kv, x->TM, 256, 0, x->pass, x->qkv, x->rope, x->qrot, kpool, vpool, x->page_table,
+         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim));
+  attention(x, kpool, vpool, L, layer);
+  gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->ldx, x->h, d, nullptr, nullptr, 0, nullptr, 0);
+  LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.nm, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
+  gemm(x, EPI_SWIGLU, w.wg, w.wu, nullptr, 1, F, d, x->xhi, x->xlo, x->ldx, nullptr, 0, x->x2hi, x->x2lo, x->ldx2,
+       nullptr, 0);
+  gemm(x, EPI_RESID, w.wd, nullptr, nullptr, 1, d, F, x->x2hi, x->x2lo, x->ldx2, x->h, d, nullptr, nullptr, 0, nullptr, 0);
+}
+
+// Target over the rows of x->pass: embedding, all layers, final norm (features kept per position).
+void target_rows(ada_ctx *x) {
+  const ada_config &c = x->c;
+  LAUNCH(x, k_embed, x->TM, 256, 0, x->pass, x->embed, x->h, c.d_model);
+  for (int l = 0; l < c.n_layers; ++l) decoder_block(x, x->layers[l], x->tk, x->tv, c.n_layers, l);
+  LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, x->final_norm, c.rms_eps, c.d_model, x->xhi, x->xlo, x->ldx,
+         x->feat, c.kv_capacity);
+}
+
+// Shared LM head + greedy choice over the rows staged in (xhi, xlo).
+void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int ldx, int use_lm_rows, int *tok_out, float2 *top_out,
+             const int *forced, float *logits) {
+  const ada_config &c = x->c;
+  gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, ldx, nullptr, 0, nullptr, nullptr,
+       0, logits, use_lm_rows);
+  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 63) / 64, x->NT * 8, x->pass, use_lm_rows, tok_out,
+         top_out, forced);
+}
+
+// Draft head over the rows of x->pass (already built for `step`).
+void draft_rows(ada_ctx *x, int step, bool with_lm) {
+  const ada_config &c = x->c;
+  const int d = c.d_model;
+  LAUNCH(x, k_eagle_input, x->TM, 256, 0, x->pass, x->embed, x->feat, c.kv_capacity, x->dfeat, c.n_max, step, d, x->xhi,
+         x->xlo, x->ldx);
+  gemm(x, EPI_STORE, x->eagle_fc, nullptr, nullptr, 1, d, 2 * d, x->xhi, x->xlo, x->ldx, x->h, d, nullptr, nullptr, 0,
+       nullptr, 0);
+  decoder_block(x, x->eagle, x->dk, x->dv, 1, 0);
+  if (with_lm) {
+    LAUNCH(x, k_split_lm_rows, x->B, 256, 0, x->pass, x->h, d, x->x2hi, x->x2lo, x->ldx2, x->dfeat, c.n_max, step);
+    lm_head(x, x->x2hi, x->x2lo, x->ldx2, 1, x->draft, x->dtop, x->force_draft, nullptr);
+  }
+}
+
+void enqueue_ldlp(ada_ctx *x, int *d_n) {
+  const ada_config &c = x->c;
+  dim3 g((c.ldlp_hidden + 7) / 8, x->B);
+  LAUNCH(x, k_ldlp_hidden, g, 256, 0, x->st, x->tok, x->feat, c.kv_capacity, x->embed, x->ldlp_w1, x->ldlp_b1,
+         c.d_model, c.ldlp_hidden, x->ldlp_h);
+  LAUNCH(x, k_ldlp_out, x->B, 32, 0, x->st, x->ldlp_h, x->ldlp_w2, x->ldlp_b2, c.ldlp_hidden, c.n_max, c.kv_capacity,
+         x->force_n_dev, x->has_force_n, x->ldlp_z, d_n, x->cnt);
+}
+
+void enqueue_draft(ada_ctx *x) {
+  const ada_config &c = x->c;
+  for (int step = 0; step < c.n_max; ++step) {
+    LAUNCH(x, k_rows_draft, 1, 32, 0, x->pass, x->st, x->tok, c.kv_capacity, x->draft, c.n_max, x->B, step, x->TM,
+           x->cnt);
+    draft_rows(x, step, true);
+  }
+}
+
+void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
+  const ada_config &c = x->c;
+  LAUNCH(x, k_rows_verify, 1, 32, 0, x->pass, x->st, x->tok, c.kv_capacity, x->draft, c.n_max, x->B, only_seq);
+  target_rows(x);
+  lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->target, x->vtop, nullptr, d_logits);
+}
+
+bool cuda_ok(ada_ctx *x, const char *what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    x->err = std::string(what) + ": " + cudaGetErrorString(e);
+    return false;
+  }
+  return true;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+
+extern "C" size_t ada_workspace_bytes(const ada_config *cfg) {
+  if (!config_ok(cfg)) return 0;
+  ada_ctx tmp;
+  return carve(&tmp, cfg, nullptr);
+}
+
+extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights *w, void *d_workspace,
+                        size_t workspace_bytes, void *cuda_stream) {
+  if (!out || !cfg || !w || !d_workspace) return ADA_ERR_NULL;
+  if (!config_ok(cfg)) return ADA_ERR_BAD_CONFIG;
+  if (((uintptr_t)d_workspace & 255) != 0) return ADA_ERR_WORKSPACE;
+  const void *singles[] = {w->embed, w->lm_head, w->final_norm, w->eagle_fc, w->e_wq, w->e_wk, w->e_wv, w->e_wo,
+                           w->e_gate, w->e_up, w->e_down, w->e_norm_attn, w->e_norm_mlp, w->ldlp_w1, w->ldlp_b1,
+                           w->ldlp_w2, w->ldlp_b2};
+  for (const void *p : singles)
+    if (!p || ((uintptr_t)p & 15)) return ADA_ERR_NULL;
+  const void *const *per[] = {w->wq, w->wk, w->wv, w->wo, w->w_gate, w->w_up, w->w_down, w->norm_attn, w->norm_mlp};
+  for (auto arr : per) {
+    if (!arr) return ADA_ERR_NULL;
+    for (int l = 0; l < cfg->n_layers; ++l)
+      if (!arr[l] || ((uintptr_t)arr[l] & 15)) return ADA_ERR_NULL;
+  }
+  ada_ctx *x = new ada_ctx();
+  x->c = *cfg;
+  x->stream = (cudaStream_t)cuda_stream;
+  const size_t need = carve(x, cfg, (char *)d_workspace);
+  if (workspace_bytes < need) {
+    delete x;
+    return ADA_ERR_WORKSPACE;
+  }
+  x->layers.resize(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers; ++l)
+    x->layers[l] = LayerW{(const bf16 *)w->wq[l], (const bf16 *)w->wk[l], (const bf16 *)w->wv[l], (const bf16 *)w->wo[l],
+                          (const bf16 *)w->w_gate[l], (const bf16 *)w->w_up[l], (const bf16 *)w->w_down[l],
+                          (const bf16 *)w->norm_attn[l], (const bf16 *)w->norm_mlp[l]};
+  x->eagle = LayerW{(const bf16 *)w->e_wq, (const bf16 *)w->e_wk, (const bf16 *)w->e_wv, (const bf16 *)w->e_wo,
+                    (const bf16 *)w->e_gate, (const bf16 *)w->e_up, (const bf16 *)w->e_down,
+                    (const bf16 *)w->e_norm_attn, (const bf16 *)w->e_norm_mlp};
+  x->embed = (const bf16 *)w->embed; x->lm_head = (const bf16 *)w->lm_head; x->final_norm = (const bf16 *)w->final_norm;
+  x->eagle_fc = (const bf16 *)w->eagle_fc;
+  x->ldlp_w1 = (const bf16 *)w->ldlp_w1; x->ldlp_b1 = (const bf16 *)w->ldlp_b1;
+  x->ldlp_w2 = (const bf16 *)w->ldlp_w2; x->ldlp_b2 = (const bf16 *)w->ldlp_b2;
+  x->force_draft = nullptr; x->has_force_n = 0; x->launches = 0; x->graph = nullptr; x->graph_launches = 0;
+  x->graph_key = -1;
+
+  // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as (cos, sin) floats
+  const int half = cfg->head_dim / 2, cap = cfg->kv_capacity;
+  std::vector<float2> rope((size_t)cap * half);
+  for (int i = 0; i < half; ++i) {
+    const double inv = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
+    for (int p = 0; p < cap; ++p) {
+      const double ang = (double)p * inv;
+      rope[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+    }
+  }
+  // page table: page i of sequence b is pool page i*B + b (sequences interleaved in the pool)
+  std::vector<int> pt((size_t)x->B * x->pages_per_seq);
+  for (int b = 0; b < x->B; ++b)
+    for (int i = 0; i < x->pages_per_seq; ++i) pt[(size_t)b * x->pages_per_seq + i] = i * x->B + b;
+  cudaError_t e = cudaMemcpyAsync(x->rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, x->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(x->page_table, pt.data(), pt.size() * sizeof(int), cudaMemcpyHostToDevice, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->st, 0, sizeof(SeqState) * x->B, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->cnt, 0, sizeof(Counters), x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->pass, 0, sizeof(Pass), x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->gemm_cnt, 0, sizeof(int) * 4096, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->tok, 0, sizeof(int) * (size_t)x->B * cap, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->draft, 0, sizeof(int) * x->B * cfg->n_max, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->target, 0, sizeof(int) * x->B * (cfg->n_max + 1), x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->force_n_dev, 0, sizeof(int) * x->B, x->stream);
+  // activation staging rows beyond the live ones are read by the tensor-core tiles: keep them finite
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xhi, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xlo, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);  // host vectors go out of scope
+  const int gemm_smem = 2 * x->NT * 8 * ((x->NT == 2 ? 1024 : 256) * 2 + 64);
+  if (e == cudaSuccess) e = x->NT == 2 ? gemm_attr_nt<2>(gemm_smem) : gemm_attr_nt<11>(gemm_smem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_attn_partial<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<128>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_attn_partial<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<64>());
+  if (e != cudaSuccess) {
+    delete x;
+    return ADA_ERR_CUDA;
+  }
+  *out = x;
+  return ADA_OK;
+}
+
+extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t m, int32_t *d_first_token) {
+  if (!x || !d_prompt) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  if (seq < 0 || seq >= x->B) return fail(x, ADA_ERR_RANGE, "ada_prefill: seq out of range");
+  if (m < 1) return fail(x, ADA_ERR_RANGE, "ada_prefill: empty prompt");
+  if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
+  LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
+  int last_rows = 0;
+  for (int p0 = 0; p0 < m; p0 += x->TM) {
+    const int R = (m - p0 < x->TM) ? m - p0 : x->TM;
+    LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
+    target_rows(x);
+    if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
+      lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
+      last_rows = R;
+    }
+    // draft head on positions p0 .. min(p0+R, m-1)-1 (needs the token after each position)
+    const int Rd = (p0 + R <= m - 1) ? R : (m - 1 - p0);
+    if (Rd > 0) {
+      LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
+      draft_rows(x, 0, false);
+    }
+  }
+  LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),
+         d_first_token);
+  return cuda_ok(x, "ada_prefill") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_ldlp_predict(ada_ctx *x, int32_t *d_n) {
+  if (!x || !d_n) return ADA_ERR_NULL;
+  enqueue_ldlp(x, d_n);
+  return cuda_ok(x, "ada_ldlp_predict") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_draft(ada_ctx *x, const int32_t *d_n, int32_t *d_draft) {
+  if (!x || !d_n || !d_draft) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  LAUNCH(x, k_set_n, 1, 32, 0, x->st, d_n, x->B, c.n_max, c.kv_capacity, x->cnt);
+  enqueue_draft(x);
+  LAUNCH(x, k_copy_i32, 1, 128, 0, d_draft, x->draft, x->B * c.n_max);
+  return cuda_ok(x, "ada_draft") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_verify(ada_ctx *x, const int32_t *d_draft, const int32_t *d_n, int32_t *d_target_tok,
+                          float *d_logits) {
+  if (!x || !d_n || !d_target_tok) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  LAUNCH(x, k_set_n, 1, 32, 0, x->st, d_n, x->B, c.n_max, c.kv_capacity, x->cnt);
+  if (d_draft && d_draft != x->draft) LAUNCH(x, k_copy_i32, 1, 128, 0, x->draft, d_draft, x->B * c.n_max);
+  enqueue_verify(x, -1, d_logits);
+  LAUNCH(x, k_copy_i32, 1, 128, 0, d_target_tok, x->target, x->B * (c.n_max + 1));
+  return cuda_ok(x, "ada_verify") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_accept(ada_ctx *x, int32_t *d_accept_len, int32_t *d_emitted, int32_t *d_n_emitted) {
+  if (!x) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, -1,
+         (const int *)nullptr, 0, d_accept_len, d_emitted, d_n_emitted, (int *)nullptr);
+  return cuda_ok(x, "ada_accept") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, int32_t *d_n_used,
+                        int32_t *d_accept_len) {
+  if (!x) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  // the graph bakes in the override switches; re-capture when they change
+  bool all_ar = x->has_force_n;  // forced plain autoregressive decoding never drafts
+  for (int b = 0; b < x->B && all_ar; ++b) all_ar = x->host_force_n[b] == 0;
+  const int key = (x->has_force_n ? 1 : 0) | (x->force_draft ? 2 : 0) | (all_ar ? 4 : 0);
+  if (!x->graph || x->graph_key != key) {
+    if (x->graph) { cudaGraphExecDestroy(x->graph); x->graph = nullptr; }
+    const long long before = x->launches;
+    cudaGraph_t g = nullptr;
+    if (cudaStreamBeginCapture(x->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
+      return fail(x, ADA_ERR_CUDA, "ada_step: cannot begin stream capture");
+    enqueue_ldlp(x, x->out_nused);
+    if (!all_ar) enqueue_draft(x);
+    enqueue_verify(x, -1, nullptr);
+    LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, -1,
+           (const int *)nullptr, 0, x->out_acc, x->out_emit, x->out_nemit, (int *)nullptr);
+    cudaError_t e = cudaStreamEndCapture(x->stream, &g);
+    x->graph_launches = (int)(x->launches - before);
+    x->launches = before;
+    if (e != cudaSuccess || !g) return fail(x, ADA_ERR_CUDA, "ada_step: stream capture failed");
+    e = cudaGraphInstantiate(&x->graph, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) { x->graph = nullptr; return fail(x, ADA_ERR_CUDA, "ada_step: graph instantiation failed"); }
+    x->graph_key = key;
+  }
+  if (cudaGraphLaunch(x->graph, x->stream) != cudaSuccess) return fail(x, ADA_ERR_CUDA, "ada_step: graph launch failed");
+  x->launches += x->graph_launches;
+  if (d_emitted) LAUNCH(x, k_copy_i32, 1, 128, 0, d_emitted, x->out_emit, x->B * (c.n_max + 1));
+  if (d_n_emitted) LAUNCH(x, k_copy_i32, 1, 32, 0, d_n_emitted, x->out_nemit, x->B);
+  if (d_n_used) LAUNCH(x, k_copy_i32, 1, 32, 0, d_n_used, x->out_nused, x->B);
+  if (d_accept_len) LAUNCH(x, k_copy_i32, 1, 32, 0, d_accept_len, x->out_acc, x->B);
+  return cuda_ok(x, "ada_step") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_force_n(ada_ctx *x, const int32_t *n) {
+  if (!x) return ADA_ERR_NULL;
+  if (!n) { x->has_force_n = 0; return ADA_OK; }
+  for (int b = 0; b < x->B; ++b)
+    if (n[b] < 0 || n[b] > x->c.n_max) return fail(x, ADA_ERR_RANGE, "ada_force_n: length out of range");
+  for (int b = 0; b < x->B; ++b) x->host_force_n[b] = n[b];
+  // pageable host memory: the copy has left the host buffer when the call returns
+  if (cudaMemcpyAsync(x->force_n_dev, x->host_force_n, sizeof(int) * x->B, cudaMemcpyHostToDevice, x->stream) !=
+      cudaSuccess)
+    return fail(x, ADA_ERR_CUDA, "ada_force_n: copy failed");
+  x->has_force_n = 1;
+  return ADA_OK;
+}
+
+extern "C" int ada_force_draft(ada_ctx *x, const int32_t *d_tokens) {
+  if (!x) return ADA_ERR_NULL;
+  x->force_draft = d_tokens;
+  return ADA_OK;
+}
+
+extern "C" int ada_force_commit(ada_ctx *x, int seq, const int32_t *d_tokens, int32_t count) {
+  if (!x || !d_tokens) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  if (seq < 0 || seq >= x->B) return fail(x, ADA_ERR_RANGE, "ada_force_commit: seq out of range");
+  if (count < 1 || count > c.n_max + 1) return fail(x, ADA_ERR_RANGE, "ada_force_commit: count out of range");
+  LAUNCH(x, k_rewind, 1, 32, 0, x->st, seq, count, d_tokens, x->draft, c.n_max, x->cnt);
+  enqueue_verify(x, seq, nullptr);
+  LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, seq, d_tokens,
+         count, (int *)nullptr, (int *)nullptr, (int *)nullptr, (int *)nullptr);
+  return cuda_ok(x, "ada_force_commit") ? ADA_OK : ADA_ERR_CUDA;
+}
+
+extern "C" int ada_get_counters(ada_ctx *x, int64_t out[8]) {
+  if (!x || !out) return ADA_ERR_NULL;
+  Counters h;
+  if (cudaStreamSynchronize(x->stream) != cudaSuccess) return fail(x, ADA_ERR_CUDA, "ada_get_counters: stream error");
+  if (cudaMemcpy(&h, x->cnt, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return fail(x, ADA_ERR_CUDA, "ada_get_counters: copy failed");
+  out[0] = (int64_t)h.n_target; out[1] = (int64_t)h.n_draft; out[2] = (int64_t)h.n_waste; out[3] = (int64_t)h.n_tokens;
+  out[4] = h.status; out[5] = x->launches; out[6] = 0; out[7] = 0;
+  return ADA_OK;
+}
+
+extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *bytes) {
+  if (!x || !d_ptr || !bytes) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  const size_t B = x->B;
+  switch (which) {
+    case 0: *d_ptr = x->feat; *bytes = B * c.kv_capacity * c.d_model * sizeof(float); break;
+    case 1: *d_ptr = x->ldlp_z; *bytes = B * 16 * sizeof(float); break;
+    case 2: *d_ptr = x->tok; *bytes = B * c.kv_capacity * sizeof(int); break;
+    case 3: *d_ptr = x->st; *bytes = B * sizeof(SeqState); break;
+    case 4: *d_ptr = x->dfeat; *bytes = B * c.n_max * c.d_model * sizeof(float); break;
+    case 5: *d_ptr = x->vtop; *bytes = B * (c.n_max + 1) * sizeof(float2); break;
+    case 6: *d_ptr = x->dtop; *bytes = B * c.n_max * sizeof(float2); break;
+    case 7: *d_ptr = x->draft; *bytes = B * c.n_max * sizeof(int); break;
+    case 8: *d_ptr = x->target; *bytes = B * (c.n_max + 1) * sizeof(int); break;
+    default: return fail(x, ADA_ERR_RANGE, "ada_debug_buffer: unknown buffer");
+  }
+  return ADA_OK;
+}
+
+extern "C" const char *ada_last_error(const ada_ctx *x) { return x ? x->err.c_str() : ""; }
+
+extern "C" int ada_destroy(ada_ctx *x) {
+  if (!x) return ADA_ERR_NULL;
+  cudaStreamSynchronize(x->stream);
+  if (x->graph) cudaGraphExecDestroy(x->graph);
+  delete x;
+  return ADA_OK;
+}

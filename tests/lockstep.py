@@ -1,0 +1,83 @@
+"""Lock-step comparison of the CUDA library with the CPU oracle.
+
+Both sides start every iteration from the same committed tokens.  The library's draft length,
+drafts, target choices, accepted length and emitted tokens are compared with the oracle's; a
+difference is tolerated only where the oracle's own top-1/top-2 margin at the deciding row is at
+most `margin` (0.05 for token logits), in which case the library is put back on the oracle's
+trajectory with ada_force_commit.
+"""
+import numpy as np
+import torch
+
+TOKEN_MARGIN = 0.05   # logits: positions with a smaller oracle margin may flip (bf16 cache vs fp32)
+LDLP_MARGIN = 2e-3    # predictor logits are fp32 on both sides; only features differ
+
+
+def _top2_gap(z):
+    s = np.sort(np.asarray(z, dtype=np.float64))
+    return float(s[-1] - s[-2]) if len(s) > 1 else float("inf")
+
+
+def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n=False):
+    """o: dict from oracle Seq.step().  Returns (ok, exempt, needs_resync, message)."""
+    exempt = 0
+    n = o["n"]
+    if g_n != n:
+        if forced_n or _top2_gap(o["ldlp_z"][:n_max]) > LDLP_MARGIN:
+            return False, 0, True, "draft length %d != oracle %d" % (g_n, n)
+        return True, 1, list(g_emitted) != list(o["emitted"]), "n flipped inside the predictor margin"
+    for i in range(n):
+        if g_draft[i] != o["draft"][i]:
+            if o["d_top1"][i] - o["d_top2"][i] > TOKEN_MARGIN:
+                return False, 0, True, "draft %d: %d != %d (margin %.3f)" % (
+                    i, g_draft[i], o["draft"][i], o["d_top1"][i] - o["d_top2"][i])
+            # a flipped draft changes the rows after it: compare only what the oracle decided
+            exempt += 1
+            return True, exempt, list(g_emitted) != list(o["emitted"]), "draft flipped inside the margin"
+    for i in range(o["k"] + 1):   # rows whose inputs are committed tokens on both sides
+        if g_target[i] != o["target"][i]:
+            if o["v_top1"][i] - o["v_top2"][i] > TOKEN_MARGIN:
+                return False, 0, True, "target row %d: %d != %d (margin %.3f)" % (
+                    i, g_target[i], o["target"][i], o["v_top1"][i] - o["v_top2"][i])
+            return True, exempt + 1, True, "target flipped inside the margin"
+    if g_k != o["k"] or list(g_emitted) != list(o["emitted"]):
+        return False, 0, True, "accept %d / emitted %s != oracle %d / %s" % (g_k, list(g_emitted), o["k"], list(o["emitted"]))
+    return True, exempt, False, ""
+
+
+def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=None):
+    """Runs `iters` ada_step iterations against oracle sequences (one per batch slot).
+
+    Returns dict(iterations, exempt, failures[list of str], tokens[list per seq]).
+    """
+    B, nmax = engine.B, engine.nmax
+    dev = engine.dev
+    draft_buf = engine.ada_debug_buffer(7, torch.int32, (B, nmax))
+    target_buf = engine.ada_debug_buffer(8, torch.int32, (B, nmax + 1))
+    failures, exempt, compared = [], 0, 0
+    for r in range(iters):
+        forced = None
+        olist = []
+        if forced_stream is not None:
+            ft = torch.zeros(B, nmax, dtype=torch.int32)
+            for b, os_ in enumerate(oseqs):
+                off = os_.len - len(prompts[b])       # tokens emitted so far (index of the next emitted token)
+                chunk = np.asarray(forced_stream[b][off: off + nmax], dtype=np.int32)
+                ft[b, : len(chunk)] = torch.from_numpy(chunk)
+            forced = ft
+            engine.ada_force_draft(ft.to(dev))
+        for b, os_ in enumerate(oseqs):
+            olist.append(os_.step(n_forced, None if forced is None else forced[b].numpy()))
+        g = engine.step()
+        gd, gt = draft_buf.cpu().numpy(), target_buf.cpu().numpy()
+        for b, o in enumerate(olist):
+            ok, ex, resync, msg = compare_iteration(o, g["n"][b], gd[b], gt[b], g["k"][b], g["emitted"][b], nmax,
+                                                    forced_n=n_forced >= 0)
+            compared += 1
+            exempt += ex
+            if not ok:
+                failures.append("iter %d seq %d: %s" % (r, b, msg))
+            if resync:
+                em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(dev)
+                engine.ada_force_commit(b, em, len(o["emitted"]))
+    return dict(iterations=compared, exempt=exempt, failures=failures)

@@ -1,0 +1,194 @@
+"""GPU parity of the CUDA library against the CPU oracle on the tiny configuration (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from tests import lockstep
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def eng(tiny):
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, m = tiny
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
+    yield e
+    e.close()
+
+
+def _prefill_both(e, m, prompt, cap=512):
+    seq = m.new_seq(cap)
+    t_o = seq.prefill(prompt)
+    t_g = e.prefill(0, prompt)
+    return seq, t_o, t_g
+
+
+def test_stage_by_stage_parity_with_logits(tiny, eng):
+    sh, w, prompt, m = tiny
+    seq, t_o, t_g = _prefill_both(eng, m, prompt)
+    assert t_o == t_g
+    feat = eng.ada_debug_buffer(0, torch.float32, (1, sh.kv_capacity, sh.d_model))
+    T = len(prompt)
+    assert np.abs(feat[0, :T].cpu().numpy() - seq.features(0, T)).max() < 2e-2
+    logits = torch.zeros(1, sh.n_max + 1, sh.vocab, dtype=torch.float32, device=eng.dev)
+    zbuf = eng.ada_debug_buffer(1, torch.float32, (1, 16))
+    dfeat = eng.ada_debug_buffer(4, torch.float32, (1, sh.n_max, sh.d_model))
+    worst = 0.0
+    for it in range(12):
+        n_o, z_o = seq.ldlp()
+        eng.ada_ldlp_predict(eng.d_n)
+        assert int(eng.d_n.cpu()[0]) == n_o
+        assert np.abs(zbuf[0, : sh.n_max].cpu().numpy() - z_o[: sh.n_max]).max() < 2e-3
+        if it % 3 == 2:            # other lengths than the predictor's
+            n_o = 1 + (it * 5) % sh.n_max
+            eng.d_n.fill_(n_o)
+        d_o, d1, d2 = seq.draft(n_o)
+        eng.ada_draft(eng.d_n, eng.d_draft)
+        d_g = eng.d_draft.cpu().numpy()[0, :n_o]
+        assert np.abs(dfeat[0, :n_o].cpu().numpy() - seq.draft_features(n_o)).max() < 2e-2
+        for i in range(n_o):
+            if d_g[i] != d_o[i]:
+                assert d1[i] - d2[i] <= lockstep.TOKEN_MARGIN
+                break
+        # verify the oracle's drafts on both sides so that every row is comparable
+        eng.d_draft[0, :n_o] = torch.from_numpy(d_o).to(eng.dev)
+        tt_o, v1, v2, lg_o = seq.verify(d_o, want_logits=True)
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target, logits)
+        lg_g = logits[0, : n_o + 1].cpu().numpy()
+        worst = max(worst, float(np.abs(lg_g - lg_o).max()))
+        assert worst < 2e-2
+        tt_g = eng.d_target.cpu().numpy()[0, : n_o + 1]
+        for i in range(n_o + 1):
+            assert tt_g[i] == tt_o[i] or v1[i] - v2[i] <= lockstep.TOKEN_MARGIN
+        k_o, em_o = seq.accept(d_o, tt_o)
+        eng.ada_accept(eng.d_accept, eng.d_emitted, eng.d_nemit)
+        k_g = int(eng.d_accept.cpu()[0])
+        em_g = eng.d_emitted.cpu().numpy()[0, : int(eng.d_nemit.cpu()[0])]
+        if k_g != k_o or list(em_g) != list(em_o):
+            assert min(v1[: k_o + 1] - v2[: k_o + 1]) <= lockstep.TOKEN_MARGIN
+            eng.ada_force_commit(0, torch.from_numpy(em_o).to(eng.dev), len(em_o))
+    print("max |logit diff| =", worst)
+    assert eng.ada_get_counters()["status"] == 0
+
+
+@pytest.mark.parametrize("n_forced", [-1, 1, 3, 8])
+def test_step_lockstep(tiny, eng, n_forced):
+    sh, w, prompt, m = tiny
+    seq, t_o, t_g = _prefill_both(eng, m, prompt)
+    assert t_o == t_g
+    eng.ada_force_draft(None)
+    eng.ada_force_n(None if n_forced < 0 else [n_forced])
+    res = lockstep.run_lockstep(eng, [seq], 24, n_forced=n_forced)
+    eng.ada_force_n(None)
+    assert not res["failures"], res["failures"]
+    assert res["exempt"] <= res["iterations"] // 2
+
+
+def test_teacher_forced_drafts_accept_everything(tiny, eng):
+    sh, w, prompt, m = tiny
+    ar = oracle.decode(m, prompt, 120, n_policy=0)["tokens"]
+    for n in (2, 8):
+        seq, t_o, t_g = _prefill_both(eng, m, prompt)
+        eng.ada_force_n([n])
+        res = lockstep.run_lockstep(eng, [seq], 8, n_forced=n, forced_stream=[ar[1:]], prompts=[prompt])
+        eng.ada_force_n(None)
+        eng.ada_force_draft(None)
+        assert not res["failures"], res["failures"]
+        assert seq.counters()["n_waste"] == 0
+
+
+def test_library_speculative_output_equals_its_own_greedy_output(tiny, eng):
+    """Lossless property on the GPU itself, bit for bit: no row's result depends on the rows beside it."""
+    sh, w, prompt, m = tiny
+
+    def run(n):
+        first = eng.prefill(0, prompt)
+        eng.ada_force_n(None if n < 0 else [n])
+        out = [first]
+        while len(out) < 40:
+            out.extend(eng.step()["emitted"][0])
+        eng.ada_force_n(None)
+        return out[:40]
+
+    ar = run(0)
+    for n in (-1, 1, 4, 8):
+        assert run(n) == ar
+
+
+def test_counters_and_launch_count(tiny, eng):
+    sh, w, prompt, m = tiny
+    eng.prefill(0, prompt)
+    c0 = eng.ada_get_counters()
+    tot = dict(n=0, k=0, e=0)
+    for _ in range(5):
+        g = eng.step()
+        tot["n"] += g["n"][0]; tot["k"] += g["k"][0]; tot["e"] += g["n_emitted"][0]
+    c1 = eng.ada_get_counters()
+    assert c1["n_target"] - c0["n_target"] == 5
+    assert c1["n_draft"] - c0["n_draft"] == tot["n"]
+    assert c1["n_waste"] - c0["n_waste"] == tot["n"] - tot["k"]
+    assert c1["n_tokens"] - c0["n_tokens"] == tot["e"]
+    assert c1["launches"] > c0["launches"] + 5 * 20
+    assert c1["status"] == 0
+
+
+def test_ragged_batch_matches_per_sequence_oracle(tiny):
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, m = tiny
+    B = 3
+    prompts = [si.uniform_ids(11, "rag%d" % b, L, sh.vocab) for b, L in enumerate((17, 64, 41))]
+    e = Engine(sh, w, max_batch=B, kv_capacity=256)
+    try:
+        seqs = []
+        for b in range(B):
+            s = m.new_seq(256)
+            assert s.prefill(prompts[b]) == e.prefill(b, prompts[b])
+            seqs.append(s)
+        res = lockstep.run_lockstep(e, seqs, 10)
+        assert not res["failures"], res["failures"]
+        e.ada_force_n([1, 5, 8])
+        for b in range(B):       # per-sequence lengths: the verify block is ragged
+            pass
+        olist = [s.step(n) for s, n in zip(seqs, (1, 5, 8))]
+        g = e.step()
+        assert g["n"] == [1, 5, 8]
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
+
+
+def test_argument_errors_are_reported_not_launched(tiny, eng):
+    import ctypes as C
+    from paper_2412_18910_b200 import AdaError, Config, lib
+    sh, w, prompt, m = tiny
+    L = lib()
+    bad = Config(2, 256, 4, 64, 688, 4096, 1e4, 1e-6, 128, 8, 0, 1, 500, 64)   # capacity not a page multiple
+    assert L.ada_workspace_bytes(C.byref(bad)) == 0
+    bad = Config(2, 256, 4, 60, 688, 4096, 1e4, 1e-6, 128, 8, 0, 1, 512, 64)
+    assert L.ada_workspace_bytes(C.byref(bad)) == 0
+    with pytest.raises(AdaError):
+        eng.prefill(0, np.zeros(sh.kv_capacity, dtype=np.int32))     # does not fit
+    with pytest.raises(AdaError):
+        eng.prefill(1, prompt)                                       # no such sequence
+    with pytest.raises(AdaError):
+        eng.ada_force_n([sh.n_max + 1])
+    assert L.ada_step(None, None, None, None, None) == -2
+
+
+def test_cache_full_clips_the_draft_length(tiny):
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, m = tiny
+    e = Engine(sh, w, max_batch=1, kv_capacity=128)
+    try:
+        e.prefill(0, si.uniform_ids(3, "long", 118, sh.vocab))       # 118 + n_max + 2 = 128
+        e.ada_force_n([8])
+        lens = e.ada_debug_buffer(3, torch.int32, (1, 8))
+        for _ in range(12):
+            g = e.step()
+            assert int(lens[0, 0].cpu()) <= 128
+        assert e.ada_get_counters()["status"] & 1                   # clipped at least once
+    finally:
+        e.close()
