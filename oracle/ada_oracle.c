@@ -407,7 +407,7 @@ int orc_draft(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int3
               float *top1, float *top2v) {
   const int d = m->c.d_model, V = m->c.vocab;
   const int j = s->len - 1; /* index of the pending token */
-  if (n < 1 || n > m->c.n_max || j + n + 1 > s->cap) return -1;
+  if (n < 1 || n > m->c.n_max || j + n + 2 > s->cap) return -1;
   float *logits = (float *)malloc(sizeof(float) * (size_t)V);
   const int R = j - s->dlen; /* catch-up rows: positions dlen .. j-1 */
   if (R < 1) { free(logits); return -2; }
@@ -440,7 +440,7 @@ int orc_verify(const orc_model *m, orc_seq *s, const int32_t *draft, int n, int3
                float *logits_out, float *top1, float *top2v) {
   const int d = m->c.d_model, V = m->c.vocab;
   const int j = s->len - 1;
-  if (n < 0 || j + n + 1 > s->cap) return -1;
+  if (n < 0 || j + n + 2 > s->cap) return -1; /* up to n + 1 new tokens must fit the token array */
   const int R = n + 1;
   int32_t *rows = (int32_t *)malloc(sizeof(int32_t) * (size_t)R);
   rows[0] = s->tok[j];
@@ -495,8 +495,8 @@ int orc_step(const orc_model *m, orc_seq *s, int n_forced, const int32_t *forced
   if (n < 0) n = orc_ldlp(m, s, ldlp_z);
   if (n < 0) return -1;
   const int j = s->len - 1;
-  if (j + 1 > s->cap) return -2;
-  if (j + n + 1 > s->cap) n = s->cap - j - 1;
+  if (j + 2 > s->cap) return -2;
+  if (j + n + 2 > s->cap) n = s->cap - j - 2;
   if (n >= 1 && orc_draft(m, s, n, forced_draft, draft, d_top1, d_top2)) return -3;
   if (orc_verify(m, s, draft, n, target, NULL, v_top1, v_top2)) return -4;
   int k = orc_accept(m, s, draft, target, n, emitted, n_emitted);

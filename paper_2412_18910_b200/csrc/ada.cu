@@ -30,6 +30,7 @@ struct GemmPlan {
 struct ada_ctx {
   ada_config c;
   cudaStream_t stream;
+  cudaStream_t capture_stream;  // private, only ever used to record the step graph (nothing executes on it)
   int B, TM, NT;          // batch, rows per pass, n8 tiles
   int pages_per_seq, n_pages;
   std::vector<LayerW> layers;
@@ -386,6 +387,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   x->ldlp_w2 = (const bf16 *)w->ldlp_w2; x->ldlp_b2 = (const bf16 *)w->ldlp_b2;
   x->force_draft = nullptr; x->has_force_n = 0; x->launches = 0; x->graph = nullptr; x->graph_launches = 0;
   x->graph_key = -1;
+  x->capture_stream = nullptr;
 
   // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as (cos, sin) floats
   const int half = cfg->head_dim / 2, cap = cfg->kv_capacity;
@@ -506,14 +508,24 @@ extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, in
     if (x->graph) { cudaGraphExecDestroy(x->graph); x->graph = nullptr; }
     const long long before = x->launches;
     cudaGraph_t g = nullptr;
-    if (cudaStreamBeginCapture(x->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
+    // record on the private stream (the caller's may be the legacy default stream, which cannot be
+    // captured); the graph is then replayed on the caller's stream
+    if (!x->capture_stream &&
+        cudaStreamCreateWithFlags(&x->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
+      return fail(x, ADA_ERR_CUDA, "ada_step: cannot create the capture stream");
+    cudaStream_t user_stream = x->stream;
+    x->stream = x->capture_stream;
+    if (cudaStreamBeginCapture(x->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      x->stream = user_stream;
       return fail(x, ADA_ERR_CUDA, "ada_step: cannot begin stream capture");
+    }
     enqueue_ldlp(x, x->out_nused);
     if (!all_ar) enqueue_draft(x);
     enqueue_verify(x, -1, nullptr);
     LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, -1,
            (const int *)nullptr, 0, x->out_acc, x->out_emit, x->out_nemit, (int *)nullptr);
     cudaError_t e = cudaStreamEndCapture(x->stream, &g);
+    x->stream = user_stream;
     x->graph_launches = (int)(x->launches - before);
     x->launches = before;
     if (e != cudaSuccess || !g) return fail(x, ADA_ERR_CUDA, "ada_step: stream capture failed");
@@ -599,6 +611,7 @@ extern "C" int ada_destroy(ada_ctx *x) {
   if (!x) return ADA_ERR_NULL;
   cudaStreamSynchronize(x->stream);
   if (x->graph) cudaGraphExecDestroy(x->graph);
+  if (x->capture_stream) cudaStreamDestroy(x->capture_stream);
   delete x;
   return ADA_OK;
 }

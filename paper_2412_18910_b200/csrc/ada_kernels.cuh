@@ -718,7 +718,7 @@ __global__ void k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 
   if (lane == 0) {
     int n = bi + 1;
     if (has_force) n = force_n[b];
-    const int room = cap - len;  // rows j..j+n need j + n + 1 <= cap, j = len - 1
+    const int room = cap - len - 1;  // the n + 1 tokens this iteration may commit must fit: len + n + 1 <= cap
     if (n > room) { n = room < 0 ? 0 : room; atomicOr(&cnt->status, kStatKvFull); }
     st[b].n = n;
     if (n_out) n_out[b] = n;
@@ -731,7 +731,7 @@ __global__ void k_set_n(SeqState *st, const int *n_in, int B, int nmax, int cap,
   if (b >= B) return;
   int n = n_in[b];
   n = max(0, min(n, nmax));
-  const int room = cap - st[b].len;
+  const int room = cap - st[b].len - 1;
   if (n > room) { n = room < 0 ? 0 : room; atomicOr(&cnt->status, kStatKvFull); }
   st[b].n = n;
 }
@@ -751,7 +751,7 @@ __global__ void k_rows_verify(Pass *pass, SeqState *st, const int *tok, int cap,
     const int len = st[b].len;
     if (len < 1) continue;
     const int j = len - 1, n = st[b].n;
-    if (j + n + 1 > cap) continue;
+    if (len + n + 1 > cap) continue;  // a full sequence takes no further step
     st[b].j_prev = j;
     for (int i = 0; i <= n; ++i) {
       pass->row_seq[T] = b;
@@ -838,7 +838,7 @@ __global__ void k_accept(SeqState *st, int *tok, int cap, const int *draft, cons
   if (len < 1) return;
   const int n = st[b].n;
   const int j = st[b].j_prev;
-  if (j != len - 1 || j + n + 1 > cap) {  // no verify ran for this sequence
+  if (j != len - 1 || len + n + 1 > cap) {  // no verify ran for this sequence
     if (acc_out) acc_out[b] = 0;
     if (nemit_out) nemit_out[b] = 0;
     if (nused_out) nused_out[b] = n;

@@ -61,7 +61,7 @@ def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=
         if forced_stream is not None:
             ft = torch.zeros(B, nmax, dtype=torch.int32)
             for b, os_ in enumerate(oseqs):
-                off = os_.len - len(prompts[b])       # tokens emitted so far (index of the next emitted token)
+                off = os_.len - len(prompts[b])       # tokens emitted so far = index of the next one in the stream
                 chunk = np.asarray(forced_stream[b][off: off + nmax], dtype=np.int32)
                 ft[b, : len(chunk)] = torch.from_numpy(chunk)
             forced = ft

@@ -93,7 +93,7 @@ def test_teacher_forced_drafts_accept_everything(tiny, eng):
     for n in (2, 8):
         seq, t_o, t_g = _prefill_both(eng, m, prompt)
         eng.ada_force_n([n])
-        res = lockstep.run_lockstep(eng, [seq], 8, n_forced=n, forced_stream=[ar[1:]], prompts=[prompt])
+        res = lockstep.run_lockstep(eng, [seq], 8, n_forced=n, forced_stream=[ar], prompts=[prompt])
         eng.ada_force_n(None)
         eng.ada_force_draft(None)
         assert not res["failures"], res["failures"]
