@@ -1,0 +1,336 @@
+"""Benchmark of the adaptive speculative-decoding iteration on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 7b]
+
+A step is one whole iteration of Algorithm 1 (predict length -> draft -> verify -> accept).  The
+metric is decode tokens per second at batch 1, timed on the device over exactly K steps after W
+warm-up steps (prefill excluded), on seeded synthetic weights and prompts of the named shape.
+With N > 1 (launched by torchrun, one rank per GPU) every rank decodes its own replica: the path
+has no exchange step, so there is no collective on it; ranks meet only at the timing barriers.
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores over a bounded sample.
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode tokens/sec at batch 1 (device-timed)"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    """Measured HBM copy bandwidth (GB/s) of this machine's B200s, else the stated fallback."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- algorithmic bytes
+
+def verify_weight_bytes(sh) -> int:
+    """bf16 bytes of every weight a verify pass reads once: L layers + LM head."""
+    d, f, v = sh.d_model, sh.d_ffn, sh.vocab
+    return 2 * (sh.n_layers * (4 * d * d + 3 * d * f) + v * d)
+
+
+def draft_step_bytes(sh) -> int:
+    """bf16 bytes of one draft-head step: fc + one layer + LM head."""
+    d, f, v = sh.d_model, sh.d_ffn, sh.vocab
+    return 2 * (2 * d * d + 4 * d * d + 3 * d * f + v * d)
+
+
+def kv_bytes_per_token(sh) -> int:
+    return 2 * 2 * sh.n_layers * sh.d_model
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()   # our own child, by handle
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- multi-rank plumbing
+
+def dist_setup(n_gpus: int):
+    """(rank, world, local_rank, dist or None).  One process per GPU under torchrun."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1:
+        return 0, 1, 0, None
+    import torch.distributed as dist
+    backend = os.environ.get("ADA_BENCH_BACKEND", "nccl")
+    if not dist.is_initialized():
+        dist.init_process_group(backend=backend)
+    return rank, world, local, dist
+
+
+def aggregate(dist, local_ms: float, local_units: float, device=None):
+    """Whole-job figures: max over ranks of the elapsed time, sum over ranks of the units."""
+    if dist is None:
+        return local_ms, local_units
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ----------------------------------------------------------------------------- the CPU oracle arm
+
+def oracle_sample(sh, weights, prompt, iters: int, warm: int, prefill_tokens: int = 32):
+    """Times `iters` oracle iterations (after `warm`) on a short prefix of the prompt.  Returns
+    (tokens per second, ms per step, threads, description)."""
+    import oracle
+    m = oracle.Model(sh, weights)
+    seq = m.new_seq(prefill_tokens + (iters + warm + 2) * (sh.n_max + 1) + 4)
+    seq.prefill(prompt[:prefill_tokens])
+    for _ in range(warm):
+        seq.step(-1)
+    toks, t0 = 0, time.perf_counter()
+    for _ in range(iters):
+        toks += len(seq.step(-1)["emitted"])
+    dt = time.perf_counter() - t0
+    desc = "%d iterations (predictor-chosen lengths) after a %d-token prefill of the same prompt" % (iters, prefill_tokens)
+    return toks / dt, 1e3 * dt / iters, oracle.num_threads(), desc
+
+
+# ----------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b", choices=["tiny", "7b", "13b"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    import numpy as np
+    import synth_inputs as si
+
+    sh = si.SHAPES[args.workload]
+    K, W = max(1, args.steps), max(0, args.warmup)
+    config = {"workload": "%s shape: %d layers, d=%d, %d heads x %d, ffn %d, vocab %d, n_max %d; batch 1, prompt %d "
+                          "uniform-random ids, predictor-chosen draft lengths, greedy"
+                          % (sh.name, sh.n_layers, sh.d_model, sh.n_heads, sh.head_dim, sh.d_ffn, sh.vocab, sh.n_max,
+                             sh.prompt_len),
+              "kv_capacity": sh.kv_capacity, "seed": si.DEFAULT_SEED,
+              "l2": "inputs larger than L2 (weights %.1f GB per verify pass)" % (verify_weight_bytes(sh) / 1e9)}
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        if rank != 0:
+            return 0
+        weights = si.make_weights(sh)
+        prompt = si.make_prompts(sh)[0]
+        # bounded sample: the oracle needs about a second per 7B iteration
+        iters = min(K, 12 if sh.name != "tiny" else 256)
+        warm = min(W, 2)
+        tps, ms, threads, desc = oracle_sample(sh, weights, prompt, iters, warm)
+        line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": iters,
+                "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+                "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    from paper_2412_18910_b200 import Engine
+
+    rank, world, local, dist = dist_setup(args.gpus)
+    dev = torch.device("cuda:%d" % local)
+    torch.cuda.set_device(dev)
+    weights = si.make_weights(sh)
+    prompt = si.uniform_ids(si.DEFAULT_SEED + rank, "prompt0", sh.prompt_len, sh.vocab)
+    eng = Engine(sh, weights, max_batch=1, kv_capacity=sh.kv_capacity, device=str(dev))
+    per_episode = max(1, (sh.kv_capacity - sh.prompt_len - sh.n_max - 4) // (sh.n_max + 1))
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+
+    # ---- device-timed leg: K steps, inputs resident, no host round trip between steps
+    d_prompt = torch.from_numpy(prompt).to(dev)
+    eng.ada_prefill(0, d_prompt, None)
+    for _ in range(max(W, 3)):
+        eng.ada_step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    c0 = eng.ada_get_counters()
+    total_ms, done = 0.0, 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    used_in_episode = max(W, 3)
+    while done < K:
+        todo = min(K - done, per_episode - used_in_episode)
+        if todo <= 0:                      # cache nearly full: start again from the prompt (not timed)
+            eng.ada_prefill(0, d_prompt, None)
+            used_in_episode = 0
+            continue
+        barrier()
+        ev0.record(eng.stream)
+        for _ in range(todo):
+            eng.ada_step()
+        ev1.record(eng.stream)
+        barrier()
+        total_ms += ev0.elapsed_time(ev1)
+        done += todo
+        used_in_episode += todo
+    c1 = eng.ada_get_counters()
+    clocks = sampler.stop()
+    tokens = c1["n_tokens"] - c0["n_tokens"]
+    launches = c1["launches"] - c0["launches"]
+    n_draft = c1["n_draft"] - c0["n_draft"]
+    n_target = c1["n_target"] - c0["n_target"]
+    job_ms, job_tokens = aggregate(dist, total_ms, float(tokens), dev)
+    value = job_tokens / (job_ms * 1e-3)
+
+    # ---- end-to-end leg: prompt from pinned host memory, prefill, K steps each followed by a
+    # device->host read of what it emitted (a serving loop must see tokens to stop on a terminator)
+    h_prompt = torch.from_numpy(prompt).pin_memory()
+    h_out = torch.zeros(sh.n_max + 3, dtype=torch.int32).pin_memory()
+    d_out = torch.zeros(sh.n_max + 3, dtype=torch.int32, device=dev)
+    Ke = min(K, per_episode)
+    barrier()
+    t0 = time.perf_counter()
+    d_p2 = torch.empty_like(d_prompt)
+    d_p2.copy_(h_prompt, non_blocking=True)
+    eng.ada_prefill(0, d_p2, d_out[sh.n_max + 2:])
+    e_tokens = 0
+    for _ in range(Ke):
+        eng.ada_step(d_out[: sh.n_max + 1], d_out[sh.n_max + 1: sh.n_max + 2])
+        h_out.copy_(d_out, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        e_tokens += int(h_out[sh.n_max + 1])
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    e_ms, e_tok = aggregate(dist, e2e_ms, float(e_tokens), dev)
+    e2e = {"value": e_tok / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": prompt.nbytes / Ke,
+           "d2h_bytes_per_step": h_out.numel() * 4, "steps": Ke,
+           "note": "request latency: pinned-host prompt copy + prefill + steps with a host read-back each"}
+
+    # ---- roofline leg: the dominant kernel (skinny GEMM) and the whole verify pass, timed with
+    # events on the library's stream at the context length the timed region ended at
+    peak, peak_kind = load_peaks()
+    eng.ada_prefill(0, d_prompt, None)
+    eng.ada_ldlp_predict(eng.d_n)
+    n_now = int(eng.d_n.cpu()[0])
+    eng.ada_draft(eng.d_n, eng.d_draft)
+    reps = 8
+    for _ in range(2):
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)     # same rows again: nothing is committed
+    torch.cuda.synchronize(dev)
+    eng.ada_profile(True)
+    va, vb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    va.record(eng.stream)
+    for _ in range(reps):
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+    vb.record(eng.stream)
+    prof = eng.ada_get_profile()
+    eng.ada_profile(False)
+    verify_ms_prof = va.elapsed_time(vb) / reps
+    va.record(eng.stream)
+    for _ in range(reps):
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+    vb.record(eng.stream)
+    torch.cuda.synchronize(dev)
+    verify_ms = va.elapsed_time(vb) / reps
+    ctx_len = sh.prompt_len + 1
+    vbytes = verify_weight_bytes(sh) + ctx_len * kv_bytes_per_token(sh)
+    gemm_gbs = prof["gemm_bytes"] / (prof["gemm_ms"] * 1e-3) / 1e9 if prof["gemm_ms"] > 0 else None
+    roofline = {"bound": "hbm", "kernel": "k_gemm (all weight GEMMs of a verify pass)",
+                "achieved": gemm_gbs, "peak": peak, "unit": "GB/s",
+                "frac": (gemm_gbs / peak) if gemm_gbs else None, "peak_kind": "of " + peak_kind, "traffic": None,
+                "launches_timed": prof["gemm_launches"], "avg_launch_us": 1e3 * prof["gemm_ms"] / max(1, prof["gemm_launches"]),
+                "bytes_per_launch": prof["gemm_bytes"] / max(1, prof["gemm_launches"]),
+                "verify_pass": {"rows": n_now + 1, "ctx": ctx_len, "ms": verify_ms, "bytes": vbytes,
+                                "gbs": vbytes / (verify_ms * 1e-3) / 1e9,
+                                "frac_of_measured": vbytes / (verify_ms * 1e-3) / 1e9 / peak,
+                                "frac_of_8000": vbytes / (verify_ms * 1e-3) / 1e9 / 8000.0,
+                                "attn_ms": prof["attn_ms"] / reps, "gemm_ms": prof["gemm_ms"] / reps}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
+            "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 weights and KV cache, f32 accumulate", "data": "synthetic", "config": config,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "tau": tokens / max(1, n_target), "mean_draft_len": n_draft / max(1, n_target)}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tps, ms, threads, desc = oracle_sample(sh, weights, prompt, 10 if sh.name != "tiny" else 64, 1)
+        line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    eng.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -149,6 +149,15 @@ int ada_get_counters(ada_ctx *ctx, int64_t out[8]);
  *         8 target choices of the last verify [max_batch][n_max+1] int32. */
 int ada_debug_buffer(ada_ctx *ctx, int which, void **d_ptr, size_t *bytes);
 
+/* Measurement hook for roofline reports.  ada_profile(ctx, 1) clears the records and from then on
+ * brackets every GEMM launch and every attention launch pair of the separately called steps
+ * (not of the ada_step graph) with CUDA events on the context's stream; ada_profile(ctx, 0) stops.
+ * ada_get_profile synchronises and returns out[0] GEMM launches, out[1] their summed duration (ms),
+ * out[2] the weight bytes they streamed (each weight once per launch), out[3] attention launch
+ * pairs, out[4] their summed duration (ms), out[5..7] 0.  At most 4096 launches are recorded. */
+int ada_profile(ada_ctx *ctx, int enable);
+int ada_get_profile(ada_ctx *ctx, double out[8]);
+
 /* Text of the last host-side error of this context ("" if none). */
 const char *ada_last_error(const ada_ctx *ctx);
 

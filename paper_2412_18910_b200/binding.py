@@ -16,7 +16,8 @@ ADA_ERRORS = {0: "ADA_OK", -1: "ADA_ERR_BAD_CONFIG", -2: "ADA_ERR_NULL", -3: "AD
 
 exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
-                    "ada_get_counters", "ada_debug_buffer", "ada_last_error", "ada_destroy")
+                    "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
+                    "ada_destroy")
 
 
 class AdaError(RuntimeError):
@@ -66,6 +67,8 @@ def lib():
     L.ada_force_commit.argtypes = [vp, C.c_int, vp, i32]
     L.ada_get_counters.argtypes = [vp, C.POINTER(C.c_int64)]
     L.ada_debug_buffer.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t)]
+    L.ada_profile.argtypes = [vp, C.c_int]
+    L.ada_get_profile.argtypes = [vp, C.POINTER(C.c_double)]
     L.ada_last_error.restype = C.c_char_p
     L.ada_last_error.argtypes = [vp]
     L.ada_destroy.argtypes = [vp]
@@ -197,6 +200,15 @@ class Engine:
         out = (C.c_int64 * 8)()
         self._check(self.L.ada_get_counters(self.h, out), "ada_get_counters")
         return dict(n_target=out[0], n_draft=out[1], n_waste=out[2], n_tokens=out[3], status=out[4], launches=out[5])
+
+    def ada_profile(self, enable: bool):
+        self._check(self.L.ada_profile(self.h, 1 if enable else 0), "ada_profile")
+
+    def ada_get_profile(self) -> dict:
+        out = (C.c_double * 8)()
+        self._check(self.L.ada_get_profile(self.h, out), "ada_get_profile")
+        return dict(gemm_launches=int(out[0]), gemm_ms=out[1], gemm_bytes=out[2], attn_launches=int(out[3]),
+                    attn_ms=out[4])
 
     def ada_debug_buffer(self, which: int, dtype, shape):
         """A torch view (no copy) of an internal buffer."""

@@ -64,6 +64,12 @@ struct ada_ctx {
   int graph_launches;
   int graph_key;                    // configuration the graph was captured for
   int *out_acc, *out_emit, *out_nemit, *out_nused;   // internal outputs of ada_step
+  // per-kernel timing for roofline reports (off by default): event pairs around GEMM / attention launches
+  int prof;
+  std::vector<cudaEvent_t> ev_pool;
+  struct ProfRec { int cls; int ev; double bytes; };
+  std::vector<ProfRec> prof_recs;
+  int ev_used;
   std::string err;
 };
 
@@ -79,6 +85,18 @@ int fail(ada_ctx *ctx, int code, const char *msg) {
     kernel<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);              \
     (ctx)->launches++;                                                      \
   } while (0)
+
+// Event pair around the launches made by `body` when profiling is on.
+template <typename F>
+void timed(ada_ctx *x, int cls, double bytes, F body) {
+  if (!x->prof || x->ev_used + 2 > (int)x->ev_pool.size()) { body(); return; }
+  const int e0 = x->ev_used;
+  x->ev_used += 2;
+  cudaEventRecord(x->ev_pool[e0], x->stream);
+  body();
+  cudaEventRecord(x->ev_pool[e0 + 1], x->stream);
+  x->prof_recs.push_back({cls, e0, bytes});
+}
 
 struct Carver {
   char *base;
@@ -236,14 +254,18 @@ void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   a.pass = x->pass; a.use_lm_rows = use_lm_rows;
   const size_t smem = (size_t)2 * x->NT * 8 * (p.KC * 2 + 64);
   dim3 grid(tiles, p.S);
-  if (x->NT == 2) launch_gemm_nt<2>(x, epi, a, grid, smem);
-  else launch_gemm_nt<11>(x, epi, a, grid, smem);
+  const double wbytes = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
+  timed(x, 0, wbytes, [&] {
+    if (x->NT == 2) launch_gemm_nt<2>(x, epi, a, grid, smem);
+    else launch_gemm_nt<11>(x, epi, a, grid, smem);
+  });
 }
 
 void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   const ada_config &c = x->c;
   dim3 g1(c.n_heads, kAttnSplits, x->B);
   dim3 g2(c.n_heads, x->TM);
+  timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
     LAUNCH(x, k_attn_partial<128>, g1, 128, attn_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
@@ -253,6 +275,7 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
     LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   }
+  });
 }
 
 // One pre-norm decoder block over the rows of x->pass; residual stream in x->h.
@@ -388,6 +411,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   x->force_draft = nullptr; x->has_force_n = 0; x->launches = 0; x->graph = nullptr; x->graph_launches = 0;
   x->graph_key = -1;
   x->capture_stream = nullptr;
+  x->prof = 0; x->ev_used = 0;
 
   // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as (cos, sin) floats
   const int half = cfg->head_dim / 2, cap = cfg->kv_capacity;
@@ -514,9 +538,12 @@ extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, in
         cudaStreamCreateWithFlags(&x->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
       return fail(x, ADA_ERR_CUDA, "ada_step: cannot create the capture stream");
     cudaStream_t user_stream = x->stream;
+    const int user_prof = x->prof;
+    x->prof = 0;
     x->stream = x->capture_stream;
     if (cudaStreamBeginCapture(x->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
       x->stream = user_stream;
+      x->prof = user_prof;
       return fail(x, ADA_ERR_CUDA, "ada_step: cannot begin stream capture");
     }
     enqueue_ldlp(x, x->out_nused);
@@ -526,6 +553,7 @@ extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, in
            (const int *)nullptr, 0, x->out_acc, x->out_emit, x->out_nemit, (int *)nullptr);
     cudaError_t e = cudaStreamEndCapture(x->stream, &g);
     x->stream = user_stream;
+    x->prof = user_prof;
     x->graph_launches = (int)(x->launches - before);
     x->launches = before;
     if (e != cudaSuccess || !g) return fail(x, ADA_ERR_CUDA, "ada_step: stream capture failed");
@@ -605,6 +633,32 @@ extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *byt
   return ADA_OK;
 }
 
+extern "C" int ada_profile(ada_ctx *x, int enable) {
+  if (!x) return ADA_ERR_NULL;
+  if (enable && x->ev_pool.empty()) {
+    x->ev_pool.resize(8192);
+    for (auto &e : x->ev_pool)
+      if (cudaEventCreate(&e) != cudaSuccess) return fail(x, ADA_ERR_CUDA, "ada_profile: cannot create events");
+  }
+  x->prof = enable ? 1 : 0;
+  x->ev_used = 0;
+  x->prof_recs.clear();
+  return ADA_OK;
+}
+
+extern "C" int ada_get_profile(ada_ctx *x, double out[8]) {
+  if (!x || !out) return ADA_ERR_NULL;
+  if (cudaStreamSynchronize(x->stream) != cudaSuccess) return fail(x, ADA_ERR_CUDA, "ada_get_profile: stream error");
+  for (int i = 0; i < 8; ++i) out[i] = 0.0;
+  for (const auto &r : x->prof_recs) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, x->ev_pool[r.ev], x->ev_pool[r.ev + 1]) != cudaSuccess) continue;
+    const int o = r.cls == 0 ? 0 : 3;
+    out[o] += 1.0; out[o + 1] += ms; out[o + 2] += r.bytes;
+  }
+  return ADA_OK;
+}
+
 extern "C" const char *ada_last_error(const ada_ctx *x) { return x ? x->err.c_str() : ""; }
 
 extern "C" int ada_destroy(ada_ctx *x) {
@@ -612,6 +666,7 @@ extern "C" int ada_destroy(ada_ctx *x) {
   cudaStreamSynchronize(x->stream);
   if (x->graph) cudaGraphExecDestroy(x->graph);
   if (x->capture_stream) cudaStreamDestroy(x->capture_stream);
+  for (auto &e : x->ev_pool) cudaEventDestroy(e);
   delete x;
   return ADA_OK;
 }

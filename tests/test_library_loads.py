@@ -1,0 +1,27 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU and exports what include/ada.h declares."""
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_every_declared_symbol_is_exported():
+    import paper_2412_18910_b200 as pkg
+    L = pkg.lib()
+    header = open(os.path.join(ROOT, "include", "ada.h")).read()
+    declared = set(re.findall(r"\b(ada_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations found"
+    for name in declared:
+        assert hasattr(L, name), name
+    assert declared == set(pkg.exported_symbols)
+
+
+def test_workspace_size_is_reported_without_a_gpu():
+    import ctypes as C
+    import paper_2412_18910_b200 as pkg
+    L = pkg.lib()
+    ok = pkg.Config(32, 4096, 32, 128, 11008, 32000, 1e4, 1e-6, 512, 10, 0, 1, 4096, 64)
+    n = L.ada_workspace_bytes(C.byref(ok))
+    assert 2 * 2 * 32 * 4096 * 4096 < n < 8 * 2**30          # at least the KV pool, well under 8 GiB
+    bad = pkg.Config(32, 4096, 32, 128, 11008, 32000, 1e4, 1e-6, 512, 16, 0, 1, 4096, 64)   # n_max too large
+    assert L.ada_workspace_bytes(C.byref(bad)) == 0
