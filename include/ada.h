@@ -38,6 +38,7 @@ extern "C" {
 #define ADA_ERR_CUDA (-5)
 #define ADA_ERR_WORKSPACE (-6)
 #define ADA_ERR_STATE (-7)
+#define ADA_ERR_TOO_LARGE (-8) /* a size exceeds a fixed maximum of the library (see ada_ldlp_eval_static) */
 
 #define ADA_MAX_LAYERS 128
 #define ADA_MAX_BATCH 8
@@ -157,6 +158,30 @@ int ada_debug_buffer(ada_ctx *ctx, int which, void **d_ptr, size_t *bytes);
  * pairs, out[4] their summed duration (ms), out[5..7] 0.  At most 4096 launches are recorded. */
 int ada_profile(ada_ctx *ctx, int enable);
 int ada_get_profile(ada_ctx *ctx, double out[8]);
+
+/* Length predictor for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a packaging variant of ada_ldlp_predict, not a step of the method).
+ * Every other call runs inside a workspace that the caller allocated; this one needs none.  It is
+ * meant for code that cannot call cudaMalloc at all: a plugin inside a host application that owns
+ * all device memory, code running while another allocator holds the whole GPU, or a latency-bound
+ * path where an allocation would stall the device.  Its only scratch, the predictor's hidden
+ * activations, lives in a fixed array inside the library image: ADA_STATIC_MAX_HIDDEN floats
+ * (16 KiB) on every GPU that loads the library, until the process exits.
+ *   z = W2 ReLU(W1 [e ; f] + b1) + b2,  n = argmax(z) + 1 (lowest index among equals)
+ * d_w1 [hidden][2*d_model], d_b1 [hidden], d_w2 [n_max][hidden], d_b2 [n_max], d_embed_row [d_model]
+ * are bf16; d_feature [d_model] fp32; outputs d_n (one int32) and d_z ([n_max] fp32, optional).
+ * All pointers are device memory owned by the caller; the call enqueues on cuda_stream and returns.
+ * No override and no cache-capacity clip are applied (there is no context).
+ * Errors: ADA_ERR_TOO_LARGE if hidden > ADA_STATIC_MAX_HIDDEN (nothing is launched),
+ * ADA_ERR_RANGE for other bad sizes, ADA_ERR_NULL, ADA_ERR_CUDA.
+ * The first call on each device looks up the array's device address (that device must be current);
+ * make that first call before any stream capture begins.  All calls on a device share the array,
+ * which keeps the previous call's contents (nothing in it needs clearing: each call overwrites
+ * what it reads); calls that overlap on the GPU race on it, so order them on one stream. */
+#define ADA_STATIC_MAX_HIDDEN 4096
+int ada_ldlp_eval_static(const void *d_w1, const void *d_b1, const void *d_w2, const void *d_b2,
+                         const void *d_embed_row, const float *d_feature, int32_t d_model, int32_t hidden,
+                         int32_t n_max, int32_t *d_n, float *d_z, void *cuda_stream);
 
 /* Text of the last host-side error of this context ("" if none). */
 const char *ada_last_error(const ada_ctx *ctx);

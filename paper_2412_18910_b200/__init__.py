@@ -4,4 +4,4 @@ The product is the CUDA library `libada.so` (sources under csrc/, interface in i
 This package only marshals arguments; PyTorch supplies device memory and streams.
 Importing it does not need a GPU; creating an Engine does.
 """
-from .binding import (ADA_ERRORS, AdaError, Config, Engine, lib, exported_symbols)  # noqa: F401
+from .binding import (ADA_ERRORS, AdaError, Config, Engine, ada_ldlp_eval_static, lib, exported_symbols)  # noqa: F401

@@ -12,12 +12,13 @@ import os
 from . import build as _build
 
 ADA_ERRORS = {0: "ADA_OK", -1: "ADA_ERR_BAD_CONFIG", -2: "ADA_ERR_NULL", -3: "ADA_ERR_RANGE", -4: "ADA_ERR_KV_FULL",
-              -5: "ADA_ERR_CUDA", -6: "ADA_ERR_WORKSPACE", -7: "ADA_ERR_STATE"}
+              -5: "ADA_ERR_CUDA", -6: "ADA_ERR_WORKSPACE", -7: "ADA_ERR_STATE",
+              -8: "ADA_ERR_TOO_LARGE (a size exceeds a fixed maximum of the library)"}
 
 exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
                     "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
-                    "ada_destroy")
+                    "ada_destroy", "ada_ldlp_eval_static")
 
 
 class AdaError(RuntimeError):
@@ -69,6 +70,7 @@ def lib():
     L.ada_debug_buffer.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t)]
     L.ada_profile.argtypes = [vp, C.c_int]
     L.ada_get_profile.argtypes = [vp, C.POINTER(C.c_double)]
+    L.ada_ldlp_eval_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
     L.ada_last_error.restype = C.c_char_p
     L.ada_last_error.argtypes = [vp]
     L.ada_destroy.argtypes = [vp]
@@ -81,6 +83,17 @@ def lib():
 
 def _dp(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def ada_ldlp_eval_static(w1, b1, w2, b2, embed_row, feature, n_out, z_out=None, stream=None) -> int:
+    """Length predictor without a context or workspace, for callers that cannot allocate device memory
+    (its scratch is a fixed 16 KiB array inside the library).  All arguments are torch device tensors:
+    bf16 w1 [hid][2d], b1 [hid], w2 [n_max][hid], b2 [n_max], embed_row [d]; fp32 feature [d];
+    int32 n_out [1]; optional fp32 z_out [n_max].  Returns the library's status code (0 = enqueued)."""
+    hid, d2 = w1.shape
+    return lib().ada_ldlp_eval_static(_dp(w1), _dp(b1), _dp(w2), _dp(b2), _dp(embed_row), _dp(feature), d2 // 2, hid,
+                                      w2.shape[0], _dp(n_out), _dp(z_out),
+                                      C.c_void_p(stream.cuda_stream if stream is not None else 0))
 
 
 class Engine:

@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB = os.path.join(_HERE, "libada.so")
-SOURCES = [os.path.join(_HERE, "csrc", "ada.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", "ada.cu"), os.path.join(_HERE, "csrc", "ada_static.cu")]
 DEPS = SOURCES + [os.path.join(_HERE, "csrc", "ada_kernels.cuh"), os.path.join(_ROOT, "include", "ada.h")]
 
 
