@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "ada_kernels.cuh"
+#include "ada_pass.cuh"
 
 using namespace ada;
 typedef __nv_bfloat16 bf16;
@@ -58,6 +59,13 @@ struct ada_ctx {
   int has_force_n;
   int host_force_n[ADA_MAX_BATCH];
   size_t part_floats;
+  // persistent pass kernel (batch 1): device copies of the layer pointer tables and its scratch
+  int use_pass, n_sm, attn_splits;
+  LayerPtrs *d_layers, *d_eagle;
+  float *attn_out, *act, *ss_part, *attn_part2;
+  int *attn_cnt;
+  float4 *amax2;
+  unsigned *gbar;
   // bookkeeping
   long long launches;
   cudaGraphExec_t graph;
@@ -209,6 +217,15 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->out_emit = w.take<int>(B * (c->n_max + 1));
   x->out_nemit = w.take<int>(B);
   x->out_nused = w.take<int>(B);
+  x->d_layers = w.take<LayerPtrs>(L);
+  x->d_eagle = w.take<LayerPtrs>(1);
+  x->attn_out = w.take<float>(16 * d);
+  x->act = w.take<float>(16 * F);
+  x->ss_part = w.take<float>(256 * 16);
+  x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
+  x->attn_cnt = w.take<int>(H);
+  x->amax2 = w.take<float4>(256 * 16);
+  x->gbar = w.take<unsigned>(64);
   return (w.off + 255) & ~(size_t)255;
 }
 
@@ -328,6 +345,48 @@ void draft_rows(ada_ctx *x, int step, bool with_lm) {
   }
 }
 
+// Bytes of weights one pass streams (each once): for the per-launch roofline record.
+double pass_weight_bytes(const ada_ctx *x, int mode, int with_lm) {
+  const ada_config &c = x->c;
+  const double d = c.d_model, F = c.d_ffn, V = c.vocab;
+  const double layer = 4 * d * d + 3 * d * F;
+  double p = mode == 0 ? c.n_layers * layer : 2 * d * d + layer;
+  if (with_lm) p += V * d;
+  return 2.0 * p;
+}
+
+// One persistent launch for a whole pass over the rows of x->pass (at most 16 rows, one sequence).
+// mode 0: target (embedding, layers, final norm -> features, LM head -> target choices)
+// mode 1: draft head (fc on [e ; f], its layer, optionally the LM head on the last rows)
+void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *tok_out, float2 *top_out,
+              const int *forced) {
+  const ada_config &c = x->c;
+  PassParams p;
+  memset(&p, 0, sizeof(p));
+  p.pass = x->pass;
+  p.layers = mode == 0 ? x->d_layers : x->d_eagle;
+  p.n_layers = mode == 0 ? c.n_layers : 1;
+  p.cache_layers = p.n_layers;
+  p.d = c.d_model; p.H = c.n_heads; p.hd = c.head_dim; p.F = c.d_ffn; p.V = c.vocab; p.eps = c.rms_eps;
+  p.embed = x->embed; p.lm_head = x->lm_head; p.final_norm = x->final_norm; p.eagle_fc = x->eagle_fc;
+  p.mode = mode; p.draft_step = step; p.with_lm = with_lm;
+  p.h = x->h; p.qkv = x->qkv; p.attn = x->attn_out; p.act = x->act; p.ss_part = x->ss_part;
+  p.feat = x->feat; p.cap = c.kv_capacity; p.dfeat = x->dfeat; p.nmax = c.n_max;
+  p.rope = x->rope;
+  p.kpool = mode == 0 ? x->tk : x->dk; p.vpool = mode == 0 ? x->tv : x->dv;
+  p.page_table = x->page_table; p.pages_per_seq = x->pages_per_seq; p.page_size = c.page_size;
+  p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
+  p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
+  p.gbar = x->gbar; p.cnt = x->cnt;
+  timed(x, 0, pass_weight_bytes(x, mode, with_lm), [&] {
+    cudaMemsetAsync(x->gbar, 0, sizeof(unsigned), x->stream);
+    void *args[] = {&p};
+    cudaLaunchCooperativeKernel((const void *)k_pass, dim3(x->n_sm), dim3(kPassThreads), args, kPassSmemBytes,
+                                x->stream);
+    x->launches++;
+  });
+}
+
 void enqueue_ldlp(ada_ctx *x, int *d_n) {
   const ada_config &c = x->c;
   dim3 g((c.ldlp_hidden + 7) / 8, x->B);
@@ -342,15 +401,20 @@ void enqueue_draft(ada_ctx *x) {
   for (int step = 0; step < c.n_max; ++step) {
     LAUNCH(x, k_rows_draft, 1, 32, 0, x->pass, x->st, x->tok, c.kv_capacity, x->draft, c.n_max, x->B, step, x->TM,
            x->cnt);
-    draft_rows(x, step, true);
+    if (x->use_pass) run_pass(x, 1, step, 1, nullptr, x->draft, x->dtop, x->force_draft);
+    else draft_rows(x, step, true);
   }
 }
 
 void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
   const ada_config &c = x->c;
   LAUNCH(x, k_rows_verify, 1, 32, 0, x->pass, x->st, x->tok, c.kv_capacity, x->draft, c.n_max, x->B, only_seq);
-  target_rows(x);
-  lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->target, x->vtop, nullptr, d_logits);
+  if (x->use_pass) {
+    run_pass(x, 0, 0, 1, d_logits, x->target, x->vtop, nullptr);
+  } else {
+    target_rows(x);
+    lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->target, x->vtop, nullptr, d_logits);
+  }
 }
 
 bool cuda_ok(ada_ctx *x, const char *what) {
@@ -444,6 +508,33 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);  // host vectors go out of scope
+  // persistent pass kernel: used when a pass never has more than 16 rows (batch 1)
+  x->use_pass = 0;
+  if (e == cudaSuccess && x->NT == 2) {
+    int dev = 0, sms = 0, per_sm = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, kPassSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pass, kPassThreads, kPassSmemBytes);
+    if (e == cudaSuccess && per_sm >= 1 && sms >= 1 && sms <= 256) {
+      x->use_pass = 1;
+      x->n_sm = sms;
+      int sp = sms / cfg->n_heads;
+      x->attn_splits = sp < 1 ? 1 : (sp > 8 ? 8 : sp);
+      std::vector<LayerPtrs> lp(cfg->n_layers);
+      for (int l = 0; l < cfg->n_layers; ++l) {
+        const LayerW &a = x->layers[l];
+        lp[l] = LayerPtrs{a.wq, a.wk, a.wv, a.wo, a.wg, a.wu, a.wd, a.na, a.nm};
+      }
+      const LayerW &a = x->eagle;
+      LayerPtrs ep{a.wq, a.wk, a.wv, a.wo, a.wg, a.wu, a.wd, a.na, a.nm};
+      e = cudaMemcpy(x->d_layers, lp.data(), sizeof(LayerPtrs) * lp.size(), cudaMemcpyHostToDevice);
+      if (e == cudaSuccess) e = cudaMemcpy(x->d_eagle, &ep, sizeof(LayerPtrs), cudaMemcpyHostToDevice);
+      if (e == cudaSuccess) e = cudaMemset(x->attn_cnt, 0, sizeof(int) * cfg->n_heads);
+      if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
+    }
+  }
   const int gemm_smem = 2 * x->NT * 8 * ((x->NT == 2 ? 1024 : 256) * 2 + 64);
   if (e == cudaSuccess) e = x->NT == 2 ? gemm_attr_nt<2>(gemm_smem) : gemm_attr_nt<11>(gemm_smem);
   if (e == cudaSuccess)
@@ -469,16 +560,22 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   for (int p0 = 0; p0 < m; p0 += x->TM) {
     const int R = (m - p0 < x->TM) ? m - p0 : x->TM;
     LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
-    target_rows(x);
-    if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
-      lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
-      last_rows = R;
+    if (x->use_pass) {  // the LM phase also writes the features; its choices matter only in the last chunk
+      run_pass(x, 0, 0, 1, nullptr, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr);
+      if (p0 + R == m) last_rows = R;
+    } else {
+      target_rows(x);
+      if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
+        lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
+        last_rows = R;
+      }
     }
     // draft head on positions p0 .. min(p0+R, m-1)-1 (needs the token after each position)
     const int Rd = (p0 + R <= m - 1) ? R : (m - 1 - p0);
     if (Rd > 0) {
       LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
-      draft_rows(x, 0, false);
+      if (x->use_pass) run_pass(x, 1, 0, 0, nullptr, nullptr, nullptr, nullptr);
+      else draft_rows(x, 0, false);
     }
   }
   LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),

@@ -1,0 +1,837 @@
+// Persistent whole-pass kernel for passes of at most 16 rows (batch 1): one CTA per SM runs
+// every phase of a model pass (embedding or draft-head input, all decoder layers, final norm,
+// LM head with greedy choice) with grid barriers between dependent phases.
+//
+// Why: a 7B verify pass streams 13.2 GB of weights in about 2 ms at HBM speed; one layer is ~60 us.
+// Nine separate launches per layer lose a large share of that to launch gaps, ramp-up and tails.
+// Here each CTA owns a fixed slab of rows of every weight matrix (N / gridDim rows), and a
+// producer warp streams those slabs through a shared-memory ring with bulk async copies
+// (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the
+// producer runs ahead across phase boundaries: while the other warps sit in a grid barrier or in
+// the attention phase, the ring is already filling with the next GEMM's weights.
+//
+// Roles inside a CTA (13 warps):
+//   warp 0        producer: walks the static schedule of (phase, k chunk, row pair-tile) stages
+//   warps 1..4    activation loaders: read the fp32 input rows of the current GEMM from L2, apply
+//                 RMSNorm scale and gain where the phase asks for it, split into bf16 hi/lo planes
+//                 in shared memory (the tensor-core B operand)
+//   warps 5..12   consumers: mma.sync m16n8k16 with the weight tile as the 16-row operand
+//                 (swap-AB), fp32 accumulators in registers, epilogues, attention
+//
+// Every wait (mbarrier, grid barrier) is bounded; when a bound is hit the kernel sets a status bit
+// and carries on as if the wait had succeeded, so it always terminates.
+#pragma once
+#include "ada_kernels.cuh"
+
+namespace ada {
+
+constexpr int kPassThreads = 13 * 32;
+constexpr int kNumXWarps = 4;
+constexpr int kNumCWarps = 8;
+constexpr int kKc = 256;                         // k elements per ring stage
+constexpr int kRowStride = kKc * 2 + 64;         // bytes per staged row: 64 mod 128 keeps 128-bit reads conflict free
+constexpr int kStageRows = 32;                   // two 16-row tiles per stage
+constexpr int kStageBytes = kStageRows * kRowStride;
+constexpr int kStages = 8;
+constexpr int kXBufs = 4;                        // one activation chunk in flight per loader warp
+constexpr int kXPlaneBytes = 16 * kRowStride;
+constexpr int kXBufBytes = 2 * kXPlaneBytes;
+constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
+constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
+// attention scratch lives where the activation buffers and the reduction buffer are (both idle
+// during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
+constexpr int kAttnLoopBytes = (3 * 16 * 128 + 8 * 16 * 32) * 4;   // q, k, v rows and softmax weights
+constexpr int kAttnPartBytes = 8 * 16 * 130 * 4;                   // per-warp partial results
+constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
+constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
+constexpr int kPassSmemBytes = kStages * kStageBytes + kMiscBytes + kScratchBytes;
+static_assert(kPassSmemBytes <= 227 * 1024, "shared memory budget");
+constexpr int kStatTimeout = 4;
+constexpr unsigned kSpinLimit = 1u << 22;
+
+struct LayerPtrs {
+  const __nv_bfloat16 *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nm;
+};
+
+struct PassParams {
+  const Pass *pass;
+  const LayerPtrs *layers;     // device array
+  int n_layers;                // layers of this pass (target: L, draft head: 1)
+  int cache_layers;            // layers in the KV pool (stride)
+  int d, H, hd, F, V;
+  float eps;
+  const __nv_bfloat16 *embed, *lm_head, *final_norm, *eagle_fc;
+  int mode;                    // 0 target pass, 1 draft-head pass
+  int draft_step;              // draft: 0 catch-up rows, s >= 1 single-row steps
+  int with_lm;                 // run the LM head
+  // activations
+  float *h, *qkv, *attn, *act; // [16][d], [16][3d], [16][d], [16][F]
+  float *ss_part;              // [grid][16] partial sums of squares of h
+  float *feat; int cap;        // target features by position [seq][cap][d]
+  float *dfeat; int nmax;      // draft features [seq][nmax][d]
+  // attention
+  const float2 *rope;
+  __nv_bfloat16 *kpool, *vpool;
+  const int *page_table; int pages_per_seq, page_size;
+  float *attn_part;            // [H][splits][16][hd+2]
+  int *attn_cnt;               // [H] arrival counters (zero between passes)
+  int attn_splits;
+  // LM head
+  float4 *amax;                // [grid][16]
+  float *logits;               // optional [slot][V]
+  int *tok_out; float2 *top_out; const int *forced;
+  // sync
+  unsigned *gbar;              // grid barrier counter, zero at launch
+  Counters *cnt;
+};
+
+// ---------------------------------------------------------------------------------- primitives
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t *bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait; on give-up records a status bit and returns
+// (*abort_flag is a per-CTA shared word: once any wait of the CTA has given up, later waits do not spin)
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
+  for (unsigned i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try(bar, parity)) return;
+    if (*abort_flag) return;
+    if (i > 64) __nanosleep(40);
+  }
+  *abort_flag = 1;
+  atomicOr(&cnt->status, kStatTimeout);
+}
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void named_bar(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// ---------------------------------------------------------------------------------- GEMM phases
+
+enum { SRC_PLAIN = 0, SRC_NORM = 1, SRC_EAGLE = 2, SRC_LMROWS = 3 };
+
+struct GemmDesc {
+  const __nv_bfloat16 *W[3];
+  int nseg, Nseg, K, epi, src_mode;
+  const float *src; int ldsrc;
+  const __nv_bfloat16 *gain;
+  float *out; int ldout;
+  int write_feat;   // NORM phase also stores the normalised rows as target features (CTA 0)
+  int write_ss;     // RESID / STORE phase also stores partial sums of squares of the new h
+  int lm;           // ARGMAX over lm rows of the draft
+};
+
+// Phase list.  Target: [embed] then per layer QKV, ATTN, O, GATEUP, DOWN, then LM.
+// Draft: FC, then the same five, then LM.  Index -> kind:
+enum { PH_EMBED = 0, PH_FC, PH_QKV, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM, PH_END };
+
+__device__ __forceinline__ int phase_count(const PassParams &p) { return 1 + 5 * p.n_layers + (p.with_lm ? 1 : 0); }
+__device__ __forceinline__ int phase_kind(const PassParams &p, int idx, int &layer) {
+  layer = 0;
+  if (idx == 0) return p.mode == 0 ? PH_EMBED : PH_FC;
+  const int i = idx - 1;
+  if (i < 5 * p.n_layers) {
+    layer = i / 5;
+    return PH_QKV + (i % 5);
+  }
+  return PH_LM;
+}
+
+__device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int layer, GemmDesc &g) {
+  const LayerPtrs &L = p.layers[layer];
+  g.nseg = 1; g.gain = nullptr; g.write_feat = 0; g.write_ss = 0; g.lm = 0;
+  g.W[1] = g.W[2] = nullptr;
+  switch (kind) {
+    case PH_FC:
+      g.W[0] = p.eagle_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE; g.src_mode = SRC_EAGLE;
+      g.src = nullptr; g.ldsrc = 0; g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      return true;
+    case PH_QKV:
+      g.W[0] = L.wq; g.W[1] = L.wk; g.W[2] = L.wv; g.nseg = 3; g.Nseg = p.d; g.K = p.d; g.epi = EPI_STORE;
+      g.src_mode = SRC_NORM; g.src = p.h; g.ldsrc = p.d; g.gain = L.na; g.out = p.qkv; g.ldout = 3 * p.d;
+      return true;
+    case PH_O:
+      g.W[0] = L.wo; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID; g.src_mode = SRC_PLAIN; g.src = p.attn; g.ldsrc = p.d;
+      g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      return true;
+    case PH_GATEUP:
+      g.W[0] = L.wg; g.W[1] = L.wu; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU; g.src_mode = SRC_NORM; g.src = p.h;
+      g.ldsrc = p.d; g.gain = L.nm; g.out = p.act; g.ldout = p.F;
+      return true;
+    case PH_DOWN:
+      g.W[0] = L.wd; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID; g.src_mode = SRC_PLAIN; g.src = p.act; g.ldsrc = p.F;
+      g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      return true;
+    case PH_LM:
+      g.W[0] = p.lm_head; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX; g.src = p.h; g.ldsrc = p.d; g.out = nullptr;
+      g.ldout = 0;
+      if (p.mode == 0) { g.src_mode = SRC_NORM; g.gain = p.final_norm; g.write_feat = 1; }
+      else { g.src_mode = SRC_LMROWS; g.lm = 1; }
+      return true;
+    default:
+      return false;
+  }
+}
+
+// Row slab of this CTA and its 16-row tiles.  Virtual rows: segments concatenated (nseg * Nseg rows);
+// SWIGLU: the slab is over Nseg rows and tiles are listed gate first, then up.
+struct Slab {
+  int r0, rows;     // slab [r0, r0 + rows) in virtual rows
+  int mt;           // tiles per matrix pass (ceil(rows / 16))
+  int ntiles;       // tiles in the list (SWIGLU: 2 * mt)
+  int nstage_rows;  // stages per k chunk = ceil(ntiles / 2)
+};
+__device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) {
+  Slab s;
+  const int N = g.nseg * g.Nseg;
+  const int rpc = (N + ncta - 1) / ncta;
+  s.r0 = cta * rpc;
+  s.rows = max(0, min(N, s.r0 + rpc) - s.r0);
+  s.mt = (s.rows + 15) >> 4;
+  s.ntiles = g.epi == EPI_SWIGLU ? 2 * s.mt : s.mt;
+  s.nstage_rows = (s.ntiles + 1) >> 1;
+  return s;
+}
+// weight row pointer of virtual row v (tile list index -> matrix for SWIGLU)
+__device__ __forceinline__ const __nv_bfloat16 *row_ptr(const GemmDesc &g, const Slab &s, int tile, int r) {
+  if (g.epi == EPI_SWIGLU) {
+    const int m = tile >= s.mt ? 1 : 0;
+    const int v = s.r0 + (tile - m * s.mt) * 16 + r;
+    return g.W[m] + (size_t)v * g.K;
+  }
+  const int v = s.r0 + tile * 16 + r;
+  const int seg = v / g.Nseg;
+  return g.W[seg] + (size_t)(v - seg * g.Nseg) * g.K;
+}
+__device__ __forceinline__ int tile_rows(const GemmDesc &g, const Slab &s, int tile) {
+  const int t = (g.epi == EPI_SWIGLU && tile >= s.mt) ? tile - s.mt : tile;
+  return max(0, min(16, s.rows - t * 16));
+}
+
+struct RingPos {
+  int stage;
+  unsigned parity;
+  __device__ __forceinline__ void advance() {
+    if (++stage == kStages) { stage = 0; parity ^= 1u; }
+  }
+};
+
+// ---------------------------------------------------------------------------------- grid barrier
+
+// All loader and consumer threads (384) take part; the producer warp does not.
+__device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoch, int tid, volatile int *abort_flag) {
+  named_bar(2, (kNumXWarps + kNumCWarps) * 32);
+  ++epoch;
+  if (tid == 32) {
+    __threadfence();
+    atomicAdd(p.gbar, 1u);
+    const unsigned target = epoch * gridDim.x;
+    bool ok = false;
+    for (unsigned i = 0; i < kSpinLimit && !*abort_flag; ++i) {
+      if (ld_acquire(p.gbar) >= target) { ok = true; break; }
+      if ((i & 63) == 63 && (ld_acquire(reinterpret_cast<const unsigned *>(&p.cnt->status)) & kStatTimeout)) break;
+      if (i > 32) __nanosleep(64);
+    }
+    if (!ok) { *abort_flag = 1; atomicOr(&p.cnt->status, kStatTimeout); }
+    __threadfence();
+  }
+  named_bar(2, (kNumXWarps + kNumCWarps) * 32);
+}
+
+// ---------------------------------------------------------------------------------- the kernel
+
+__global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
+  const int T = p.pass->T;
+  if (T <= 0) return;
+  const int lmT = p.pass->lmT;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, ncta = gridDim.x;
+
+  extern __shared__ __align__(128) unsigned char pass_smem[];
+  unsigned char *const smem = pass_smem;
+  unsigned char *ring = smem;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
+  uint64_t *full = bars, *empty = bars + kStages, *xfull = bars + 2 * kStages, *xempty = bars + 2 * kStages + kXBufs;
+  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs);   // [16]
+  float *ssw = inv_rms + 16;                                                       // [8][16]
+  Top2 *topw = reinterpret_cast<Top2 *>(ssw + 8 * 16);                             // [8][16]
+  int *flag_s = reinterpret_cast<int *>(topw + 8 * 16);
+  volatile int *abort_s = flag_s + 1;
+  unsigned char *xbuf = smem + kStages * kStageBytes + kMiscBytes;
+  float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
+  static_assert((2 * kStages + 2 * kXBufs) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
+
+  if (tid == 0) {
+    *abort_s = 0;
+    for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], kNumCWarps); }
+    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], kNumCWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int nphase = phase_count(p);
+
+  // ================================================================= producer warp
+  if (warp == 0) {
+    RingPos rp{0, 0};
+    unsigned filled = 0;  // stages issued so far; the first kStages need no wait
+    for (int ph = 0; ph < nphase; ++ph) {
+      int layer;
+      const int kind = phase_kind(p, ph, layer);
+      GemmDesc g;
+      if (!make_gemm(p, kind, layer, g)) continue;
+      if (kind == PH_LM && p.mode == 1 && lmT <= 0) continue;
+      const Slab s = make_slab(g, cta, ncta);
+      if (s.rows == 0) continue;
+      const int nchunk = (g.K + kKc - 1) / kKc;
+      for (int c = 0; c < nchunk; ++c) {
+        const int kvalid = min(kKc, g.K - c * kKc);
+        for (int sr = 0; sr < s.nstage_rows; ++sr) {
+          if (filled >= (unsigned)kStages) {
+            if (lane == 0) mbar_wait(&empty[rp.stage], rp.parity ^ 1u, p.cnt, abort_s);
+            __syncwarp();
+          }
+          const int t0 = 2 * sr;
+          const int rows0 = tile_rows(g, s, t0), rows1 = (t0 + 1 < s.ntiles) ? tile_rows(g, s, t0 + 1) : 0;
+          if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)((rows0 + rows1) * kvalid * 2));
+          __syncwarp();
+          unsigned char *dst = ring + (size_t)rp.stage * kStageBytes;
+          const int which = lane >> 4, r = lane & 15;
+          const int nr = which ? rows1 : rows0;
+          if (r < nr) {
+            const __nv_bfloat16 *src = row_ptr(g, s, t0 + which, r) + (size_t)c * kKc;
+            bulk_g2s(dst + (size_t)(which * 16 + r) * kRowStride, src, (unsigned)(kvalid * 2), &full[rp.stage]);
+          }
+          ++filled;
+          rp.advance();
+        }
+      }
+    }
+    return;
+  }
+
+  // ================================================================= loaders and consumers
+  const bool is_loader = warp <= kNumXWarps;
+  const int cw = warp - 1 - kNumXWarps;   // consumer warp index 0..7 (consumers only)
+  const int g8 = lane >> 2, q4 = lane & 3;
+  unsigned epoch = 0;
+  RingPos rp{0, 0};
+  int xcount = 0;   // activation chunks produced / consumed so far (buffer = xcount % kXBufs)
+
+  for (int ph = 0; ph < nphase; ++ph) {
+    int layer;
+    const int kind = phase_kind(p, ph, layer);
+
+    // ------------------------------------------------------------- embedding
+    if (kind == PH_EMBED) {
+      // h[t][:] = embedding rows; column slices per CTA; partial sums of squares for the first norm
+      const int ltid = tid - 32, nth = (kNumXWarps + kNumCWarps) * 32;
+      const int cpc = (p.d + ncta - 1) / ncta;
+      const int c0 = cta * cpc, c1 = min(p.d, c0 + cpc);
+      for (int t = 0; t < 16; ++t) {
+        float ss = 0.f;
+        if (t < T) {
+          const __nv_bfloat16 *e = p.embed + (size_t)p.pass->row_tok[t] * p.d;
+          for (int c = c0 + ltid; c < c1; c += nth) {
+            const float v = __bfloat162float(e[c]);
+            p.h[(size_t)t * p.d + c] = v;
+            ss += v * v;
+          }
+        }
+        // CTA-wide sum of ss in a fixed order: warp sums, then warps in order
+        ss = warp_sum(ss);
+        if (lane == 0) red[(warp - 1) * 16 + t] = ss;
+      }
+      named_bar(2, nth);
+      if (tid - 32 < 16) {
+        float s = 0.f;
+        for (int w = 0; w < kNumXWarps + kNumCWarps; ++w) s += red[w * 16 + (tid - 32)];
+        p.ss_part[(size_t)cta * 16 + (tid - 32)] = s;
+      }
+      grid_barrier(p, epoch, tid, abort_s);
+      continue;
+    }
+
+    // ------------------------------------------------------------- attention
+    if (kind == PH_ATTN) {
+      if (!is_loader) {
+        // items (sequence 0, head, split) round-robin over CTAs; batch 1 only on this path
+        const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
+        const int nkeys = pos0 + R, nsp = p.attn_splits;
+        int chunk = (nkeys + nsp - 1) / nsp;
+        chunk = ((chunk + 31) / 32) * 32;
+        const int b = p.pass->row_seq[0];
+        float *q_s = reinterpret_cast<float *>(xbuf);          // [16][128]
+        float *k_s = q_s + 16 * 128;                           // new rows, rotated, bf16-rounded [16][128]
+        float *v_s = k_s + 16 * 128;
+        float *p_s = v_s + 16 * 128;                           // [8][16][32]
+        float *part_s = q_s;                                   // [8][16][130], reuses the loop's scratch
+        const int ctid = tid - 32 * (1 + kNumXWarps);
+        const int VPL = HD / 32;
+        const LayerPtrs &Lw = p.layers[layer];
+        (void)Lw;
+        for (int item = cta; item < p.H * nsp; item += ncta) {
+          const int hh = item / nsp, split = item - hh * nsp;
+          const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
+          named_bar(3, kNumCWarps * 32);
+          // q (scaled), k, v of the block rows with rotary embedding
+          const float qscale = rsqrtf((float)HD);
+          for (int i = ctid; i < R * half; i += kNumCWarps * 32) {
+            const int r = i / half, c = i - r * half;
+            const float2 cs = p.rope[(size_t)(pos0 + r) * half + c];
+            const float *qr = p.qkv + (size_t)r * 3 * d + hh * HD;
+            const float qa = qr[c], qb = qr[c + half], ka = qr[d + c], kb = qr[d + c + half];
+            q_s[r * 128 + c] = (qa * cs.x - qb * cs.y) * qscale;
+            q_s[r * 128 + c + half] = (qb * cs.x + qa * cs.y) * qscale;
+            const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
+            const __nv_bfloat16 k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(qr[2 * d + c]), v1 = __float2bfloat16_rn(qr[2 * d + c + half]);
+            k_s[r * 128 + c] = __bfloat162float(k0); k_s[r * 128 + c + half] = __bfloat162float(k1);
+            v_s[r * 128 + c] = __bfloat162float(v0); v_s[r * 128 + c + half] = __bfloat162float(v1);
+            if (split == 0) {  // one item per head stores the new rows in the cache
+              const int pos = pos0 + r;
+              const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
+              const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD;
+              p.kpool[base + c] = k0; p.kpool[base + c + half] = k1;
+              p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
+            }
+          }
+          named_bar(3, kNumCWarps * 32);
+          float m[16], l[16], o[16][4];
+#pragma unroll
+          for (int r = 0; r < 16; ++r) { m[r] = -INFINITY; l[r] = 0.f; o[r][0] = o[r][1] = o[r][2] = o[r][3] = 0.f; }
+          for (int kb = kbeg + cw * 32; kb < kend; kb += kNumCWarps * 32) {
+            const int key = kb + lane;
+            const bool kv = key < kend;
+            float s[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) s[r] = 0.f;
+            if (kv) {
+              if (key >= pos0) {
+                const float *kr = k_s + (key - pos0) * 128;
+                for (int c = 0; c < HD; c += 4) {
+                  const float4 kk = *reinterpret_cast<const float4 *>(kr + c);
+#pragma unroll
+                  for (int r = 0; r < 16; ++r)
+                    if (r < R) {
+                      const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c);
+                      s[r] += qa.x * kk.x + qa.y * kk.y + qa.z * kk.z + qa.w * kk.w;
+                    }
+                }
+              } else {
+                const int page = p.page_table[b * p.pages_per_seq + key / p.page_size], slot = key % p.page_size;
+                const uint4 *kr = reinterpret_cast<const uint4 *>(
+                    p.kpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD);
+                for (int c = 0; c < HD / 8; ++c) {
+                  const uint4 kk = kr[c];
+                  float kf[8];
+                  kf[0] = bf16_bits_to_float(kk.x & 0xffffu); kf[1] = bf16_bits_to_float(kk.x >> 16);
+                  kf[2] = bf16_bits_to_float(kk.y & 0xffffu); kf[3] = bf16_bits_to_float(kk.y >> 16);
+                  kf[4] = bf16_bits_to_float(kk.z & 0xffffu); kf[5] = bf16_bits_to_float(kk.z >> 16);
+                  kf[6] = bf16_bits_to_float(kk.w & 0xffffu); kf[7] = bf16_bits_to_float(kk.w >> 16);
+#pragma unroll
+                  for (int r = 0; r < 16; ++r)
+                    if (r < R) {
+                      const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8);
+                      const float4 qb = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8 + 4);
+                      s[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                              qb.z * kf[6] + qb.w * kf[7];
+                    }
+                }
+              }
+            }
+#pragma unroll
+            for (int r = 0; r < 16; ++r)
+              if (r < R) {
+                const bool seen = kv && key <= pos0 + r;
+                const float sv = seen ? s[r] : -INFINITY;
+                const float mx = warp_max(sv);
+                const float mn = fmaxf(m[r], mx);
+                float pe = 0.f, corr = 1.f;
+                if (mn > -INFINITY) { pe = seen ? __expf(sv - mn) : 0.f; corr = __expf(m[r] - mn); }
+                l[r] = l[r] * corr + warp_sum(pe);
+                o[r][0] *= corr; o[r][1] *= corr; o[r][2] *= corr; o[r][3] *= corr;
+                m[r] = mn;
+                p_s[(cw * 16 + r) * 32 + lane] = pe;
+              }
+            __syncwarp();
+            const int nk = min(32, kend - kb);
+            for (int kk = 0; kk < nk; ++kk) {
+              const int key2 = kb + kk;
+              float vf[4] = {0.f, 0.f, 0.f, 0.f};
+              if (key2 >= pos0) {
+                const float *vr = v_s + (key2 - pos0) * 128 + lane * VPL;
+                for (int c = 0; c < VPL; ++c) vf[c] = vr[c];
+              } else {
+                const int page = p.page_table[b * p.pages_per_seq + key2 / p.page_size], slot = key2 % p.page_size;
+                const __nv_bfloat16 *vr =
+                    p.vpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD;
+                if (VPL == 4) {
+                  const uint2 vv = *reinterpret_cast<const uint2 *>(vr + lane * 4);
+                  vf[0] = bf16_bits_to_float(vv.x & 0xffffu); vf[1] = bf16_bits_to_float(vv.x >> 16);
+                  vf[2] = bf16_bits_to_float(vv.y & 0xffffu); vf[3] = bf16_bits_to_float(vv.y >> 16);
+                } else {
+                  const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr + lane * 2);
+                  vf[0] = bf16_bits_to_float(vv & 0xffffu); vf[1] = bf16_bits_to_float(vv >> 16);
+                }
+              }
+#pragma unroll
+              for (int r = 0; r < 16; ++r)
+                if (r < R) {
+                  const float pe = p_s[(cw * 16 + r) * 32 + kk];
+                  o[r][0] += pe * vf[0]; o[r][1] += pe * vf[1]; o[r][2] += pe * vf[2]; o[r][3] += pe * vf[3];
+                }
+            }
+            __syncwarp();
+          }
+          // per-warp partials -> shared (over the loop's scratch once every warp has left the loop),
+          // merged in warp order, stored per (head, split)
+          named_bar(3, kNumCWarps * 32);
+#pragma unroll
+          for (int r = 0; r < 16; ++r)
+            if (r < R) {
+              float *pp = part_s + (cw * 16 + r) * 130;
+              for (int c = 0; c < VPL; ++c) pp[lane * VPL + c] = o[r][c];
+              if (lane == 0) { pp[128] = m[r]; pp[129] = l[r]; }
+            }
+          named_bar(3, kNumCWarps * 32);
+          for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
+            const int r = i / HD, c = i - r * HD;
+            float M = -INFINITY;
+            for (int w = 0; w < kNumCWarps; ++w) M = fmaxf(M, part_s[(w * 16 + r) * 130 + 128]);
+            float lo = 0.f, oo = 0.f;
+            if (M > -INFINITY)
+              for (int w = 0; w < kNumCWarps; ++w) {
+                const float e = __expf(part_s[(w * 16 + r) * 130 + 128] - M);
+                lo += part_s[(w * 16 + r) * 130 + 129] * e;
+                oo += part_s[(w * 16 + r) * 130 + c] * e;
+              }
+            float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
+            __stcg(gp + c, oo);
+            if (c == 0) { __stcg(gp + HD, M); __stcg(gp + HD + 1, lo); }
+          }
+          // the item that arrives last for this head merges the splits in split order
+          __threadfence();
+          named_bar(3, kNumCWarps * 32);
+          if (ctid == 0) *flag_s = (atomicAdd(p.attn_cnt + hh, 1) == nsp - 1);
+          named_bar(3, kNumCWarps * 32);
+          if (*flag_s) {
+            __threadfence();
+            for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
+              const int r = i / HD, c = i - r * HD;
+              const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2);
+              const size_t sst = (size_t)16 * (HD + 2);
+              float M = -INFINITY;
+              for (int s2 = 0; s2 < nsp; ++s2) M = fmaxf(M, __ldcg(gp + s2 * sst + HD));
+              float lo = 0.f, oo = 0.f;
+              for (int s2 = 0; s2 < nsp; ++s2) {
+                const float ms = __ldcg(gp + s2 * sst + HD);
+                if (ms > -INFINITY) {
+                  const float e = __expf(ms - M);
+                  lo += __ldcg(gp + s2 * sst + HD + 1) * e;
+                  oo += __ldcg(gp + s2 * sst + c) * e;
+                }
+              }
+              p.attn[(size_t)r * d + hh * HD + c] = oo / lo;
+            }
+            if (ctid == 0) p.attn_cnt[hh] = 0;
+          }
+        }
+      }
+      grid_barrier(p, epoch, tid, abort_s);
+      continue;
+    }
+
+    // ------------------------------------------------------------- GEMM phases
+    GemmDesc g;
+    make_gemm(p, kind, layer, g);
+    const int Tg = g.lm ? lmT : T;
+    if (Tg <= 0) { grid_barrier(p, epoch, tid, abort_s); continue; }
+    const int nt_act = (Tg + 7) >> 3;
+    const Slab s = make_slab(g, cta, ncta);
+    const int nchunk = (g.K + kKc - 1) / kKc;
+
+    if (is_loader) {
+      // ---- activation loaders: chunk by chunk, X = hi/lo planes of the GEMM input rows
+      const int xt = tid - 32;  // 0..127
+      if (g.src_mode == SRC_NORM) {
+        if (xt < 16) {
+          float ssum = 0.f;
+          for (int i = 0; i < ncta; ++i) ssum += __ldcg(p.ss_part + (size_t)i * 16 + xt);
+          inv_rms[xt] = rsqrtf(ssum / (float)p.d + p.eps);
+        }
+        named_bar(4, kNumXWarps * 32);
+      }
+      if (s.rows > 0) {
+        const int lw = warp - 1;   // loader warp index; it converts chunks c with (xcount + c) % 4 == lw
+        for (int c = 0; c < nchunk; ++c) {
+          const int xc = xcount + c;
+          if ((xc % kNumXWarps) != lw) continue;
+          const int buf = xc % kXBufs;
+          if (xc >= kXBufs) {
+            if (lane == 0) mbar_wait(&xempty[buf], ((unsigned)(xc / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
+            __syncwarp();
+          }
+          unsigned char *xh = xbuf + (size_t)buf * kXBufBytes, *xl = xh + kXPlaneBytes;
+          // nt_act*8 rows x 256 k in groups of 4 elements; lane handles groups lane, lane+32, ...
+          const int ngroups = nt_act * 8 * (kKc / 4);
+#pragma unroll 4
+          for (int gi = lane; gi < ngroups; gi += 32) {
+            const int r = gi / (kKc / 4), kk = (gi - r * (kKc / 4)) * 4;
+            const int k = c * kKc + kk;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r < Tg && k < g.K) {
+              if (g.src_mode == SRC_EAGLE) {
+                const int b = p.pass->row_seq[r];
+                if (k < p.d) {
+                  const __nv_bfloat16 *e = p.embed + (size_t)p.pass->row_tok[r] * p.d + k;
+                  v = make_float4(__bfloat162float(e[0]), __bfloat162float(e[1]), __bfloat162float(e[2]),
+                                  __bfloat162float(e[3]));
+                } else {
+                  const float *f = p.draft_step == 0 ? p.feat + ((size_t)b * p.cap + p.pass->row_pos[r]) * p.d
+                                                     : p.dfeat + ((size_t)b * p.nmax + (p.draft_step - 1)) * p.d;
+                  v = __ldcg(reinterpret_cast<const float4 *>(f + (k - p.d)));
+                }
+              } else {
+                const int sr = g.src_mode == SRC_LMROWS ? p.pass->lm_row[r] : r;
+                v = __ldcg(reinterpret_cast<const float4 *>(g.src + (size_t)sr * g.ldsrc + k));
+                if (g.src_mode == SRC_NORM) {
+                  const float iv = inv_rms[r];
+                  const __nv_bfloat16 *gn = g.gain + k;
+                  v.x = (v.x * iv) * __bfloat162float(gn[0]); v.y = (v.y * iv) * __bfloat162float(gn[1]);
+                  v.z = (v.z * iv) * __bfloat162float(gn[2]); v.w = (v.w * iv) * __bfloat162float(gn[3]);
+                  if (g.write_feat && cta == 0)
+                    *reinterpret_cast<float4 *>(p.feat + ((size_t)p.pass->row_seq[r] * p.cap + p.pass->row_pos[r]) * p.d + k) = v;
+                } else if (g.src_mode == SRC_LMROWS && cta == 0) {
+                  const int b = p.pass->row_seq[sr];
+                  *reinterpret_cast<float4 *>(p.dfeat + ((size_t)b * p.nmax + p.draft_step) * p.d + k) = v;
+                }
+              }
+            }
+            __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+            split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
+            uint2 hv, lv;
+            hv.x = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            hv.y = (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16);
+            lv.x = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            lv.y = (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16);
+            *reinterpret_cast<uint2 *>(xh + (size_t)r * kRowStride + kk * 2) = hv;
+            *reinterpret_cast<uint2 *>(xl + (size_t)r * kRowStride + kk * 2) = lv;
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&xfull[buf]);
+        }
+        xcount += nchunk;
+      }
+      grid_barrier(p, epoch, tid, abort_s);
+      continue;
+    }
+
+    // ---- consumers
+    // tile ownership: mt <= 8 tiles (single matrix): tile = cw / ksplit, k blocks split ksplit ways;
+    // otherwise warp cw owns list tiles cw and cw + 8 (SWIGLU: gate tile cw and up tile cw + mt).
+    int tileA = -1, tileB = -1, ksplit = 1, kpart = 0;
+    if (g.epi == EPI_SWIGLU) {
+      if (cw < s.mt) { tileA = cw; tileB = cw + s.mt; }
+    } else if (s.mt <= 8) {
+      ksplit = s.mt <= 1 ? 8 : (s.mt == 2 ? 4 : (s.mt <= 4 ? 2 : 1));
+      if (cw / ksplit < s.mt) { tileA = cw / ksplit; kpart = cw % ksplit; }
+    } else {
+      tileA = cw; if (cw + 8 < s.mt) tileB = cw + 8;
+    }
+    float acc[2][2][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[a][i][j] = 0.f;
+
+    if (s.rows > 0) {
+      const int bpw = 8 / ksplit;  // 32-k blocks of a chunk this warp handles
+      for (int c = 0; c < nchunk; ++c, ++xcount) {
+        const int buf = xcount % kXBufs;
+        mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
+        const unsigned char *xh = xbuf + (size_t)buf * kXBufBytes, *xl = xh + kXPlaneBytes;
+        const int kvalid = min(kKc, g.K - c * kKc);
+        for (int sr = 0; sr < s.nstage_rows; ++sr) {
+          mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
+          const unsigned char *st = ring + (size_t)rp.stage * kStageBytes;
+#pragma unroll
+          for (int slot = 0; slot < 2; ++slot) {
+            const int tile = slot ? tileB : tileA;
+            if (tile >= 0 && (tile >> 1) == sr) {
+              const unsigned char *a_base = st + (size_t)((tile & 1) * 16) * kRowStride;
+#pragma unroll 4
+              for (int bi = 0; bi < bpw; ++bi) {
+                const int blk = kpart * bpw + bi;
+                if (blk * 32 < kvalid) {   // warp-uniform: every lane takes part in the mma
+                  const int koff = blk * 32 + 8 * q4;
+                  const bool okk = koff < kvalid;   // ragged end of K: this lane's 8 k are past it
+                  uint4 A0 = make_uint4(0, 0, 0, 0), A1 = A0;
+                  if (okk) {
+                    A0 = *reinterpret_cast<const uint4 *>(a_base + (size_t)g8 * kRowStride + koff * 2);
+                    A1 = *reinterpret_cast<const uint4 *>(a_base + (size_t)(g8 + 8) * kRowStride + koff * 2);
+                  }
+#pragma unroll
+                  for (int i = 0; i < 2; ++i)
+                    if (i < nt_act) {
+                      const uint4 bh = *reinterpret_cast<const uint4 *>(xh + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
+                      const uint4 bl = *reinterpret_cast<const uint4 *>(xl + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
+                      mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bh.x, bh.y);
+                      mma_bf16(acc[slot][i], A0.z, A1.z, A0.w, A1.w, bh.z, bh.w);
+                      mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bl.x, bl.y);
+                      mma_bf16(acc[slot][i], A0.z, A1.z, A0.w, A1.w, bl.z, bl.w);
+                    }
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&empty[rp.stage]);
+          rp.advance();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&xempty[buf]);
+      }
+    }
+
+    // ---- k-split reduction inside the CTA (fixed order), then the epilogue by the owner warps
+    if (ksplit > 1) {
+      float *mine = red + (size_t)(cw * 32 + lane) * 8;
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mine[i * 4 + j] = acc[0][i][j];
+      named_bar(3, kNumCWarps * 32);
+      if (kpart == 0 && tileA >= 0) {
+        for (int s2 = 1; s2 < ksplit; ++s2) {
+          const float *oth = red + (size_t)((cw + s2) * 32 + lane) * 8;
+#pragma unroll
+          for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[0][i][j] += oth[i * 4 + j];
+        }
+      }
+    }
+    const bool owner = tileA >= 0 && kpart == 0 && s.rows > 0;
+    float ssl[4] = {0.f, 0.f, 0.f, 0.f};   // sums of squares for pass rows 2*q4 + {0,1} + 8*{0,1}
+    Top2 tb[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { tb[i].v1 = -INFINITY; tb[i].i1 = 0x7fffffff; tb[i].v2 = -INFINITY; }
+
+    if (owner) {
+#pragma unroll
+      for (int slot = 0; slot < 2; ++slot) {
+        const int tile = slot ? tileB : tileA;
+        if (tile < 0 || (g.epi == EPI_SWIGLU && slot == 1)) continue;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          if (i >= nt_act) continue;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int rr = g8 + 8 * (j >> 1), t = 8 * i + 2 * q4 + (j & 1);
+            const int vrow = s.r0 + tile * 16 + rr;     // virtual output column
+            if (tile * 16 + rr >= s.rows || t >= Tg) continue;
+            const float y = acc[slot][i][j];
+            if (g.epi == EPI_STORE) {
+              g.out[(size_t)t * g.ldout + vrow] = y;
+              if (g.write_ss) ssl[i * 2 + (j & 1)] += y * y;
+            } else if (g.epi == EPI_RESID) {
+              float *hp = g.out + (size_t)t * g.ldout + vrow;
+              const float hn = __ldcg(hp) + y;
+              *hp = hn;
+              ssl[i * 2 + (j & 1)] += hn * hn;
+            } else if (g.epi == EPI_SWIGLU) {
+              const float up = acc[1][i][j];
+              g.out[(size_t)t * g.ldout + vrow] = (y / (1.f + __expf(-y))) * up;
+            } else {  // ARGMAX
+              if (p.logits) {
+                const int slot_out = g.lm ? p.pass->lm_out[t] : p.pass->row_out[t];
+                p.logits[(size_t)slot_out * p.V + vrow] = y;
+              }
+              Top2 cnd; cnd.v1 = y; cnd.i1 = vrow; cnd.v2 = -INFINITY;
+              tb[i * 2 + (j & 1)] = top2_merge(tb[i * 2 + (j & 1)], cnd);
+            }
+          }
+        }
+      }
+    }
+    if (g.write_ss || g.epi == EPI_RESID) {
+      // reduce over the 8 row groups of the warp, then over warps in order, one value per pass row
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float v = ssl[i];
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (g8 == 0) ssw[cw * 16 + (i >> 1) * 8 + 2 * q4 + (i & 1)] = v;
+      }
+      named_bar(3, kNumCWarps * 32);
+      if (cw == 0 && lane < 16) {
+        float v = 0.f;
+        for (int w = 0; w < kNumCWarps; ++w) v += ssw[w * 16 + lane];
+        p.ss_part[(size_t)cta * 16 + lane] = v;
+      }
+    } else if (g.epi == EPI_ARGMAX) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        Top2 b = tb[i];
+        b = top2_shfl_xor(b, 4); b = top2_shfl_xor(b, 8); b = top2_shfl_xor(b, 16);
+        if (g8 == 0) topw[cw * 16 + (i >> 1) * 8 + 2 * q4 + (i & 1)] = b;
+      }
+      named_bar(3, kNumCWarps * 32);
+      if (cw == 0 && lane < 16) {
+        Top2 b = topw[lane];
+        for (int w = 1; w < kNumCWarps; ++w) b = top2_merge(b, topw[w * 16 + lane]);
+        p.amax[(size_t)cta * 16 + lane] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+      }
+    }
+    grid_barrier(p, epoch, tid, abort_s);
+
+    if (g.epi == EPI_ARGMAX && cta == 0 && cw == 0 && lane < 16 && lane < Tg) {
+      // greedy choice per row: candidates of all CTAs merged in CTA order
+      Top2 b;
+      b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+      for (int i = 0; i < ncta; ++i) {
+        const float4 c4 = __ldcg(p.amax + (size_t)i * 16 + lane);
+        Top2 x; x.v1 = c4.x; x.i1 = __float_as_int(c4.y); x.v2 = c4.z;
+        b = top2_merge(b, x);
+      }
+      const int slot_out = g.lm ? p.pass->lm_out[lane] : p.pass->row_out[lane];
+      p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
+      if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
+    }
+  }
+}
+
+}  // namespace ada
