@@ -147,7 +147,10 @@ int ada_get_counters(ada_ctx *ctx, int64_t out[8]);
  *         5 top-2 logits of every verify row [max_batch][n_max+1][2] fp32,
  *         6 top-2 logits of every draft step [max_batch][n_max][2] fp32,
  *         7 draft tokens of the last draft [max_batch][n_max] int32,
- *         8 target choices of the last verify [max_batch][n_max+1] int32. */
+ *         8 target choices of the last verify [max_batch][n_max+1] int32,
+ *         9 phase clock of the last profiled target pass (batch 1, ada_profile on): 512 uint64
+ *           nanosecond stamps, [0] = start, [i+1] = end of phase i (embedding, then per layer
+ *           QKV, attention, O, gate/up, down, then the LM head). */
 int ada_debug_buffer(ada_ctx *ctx, int which, void **d_ptr, size_t *bytes);
 
 /* Measurement hook for roofline reports.  ada_profile(ctx, 1) clears the records and from then on

@@ -62,10 +62,12 @@ struct ada_ctx {
   // persistent pass kernel (batch 1): device copies of the layer pointer tables and its scratch
   int use_pass, n_sm, attn_splits;
   LayerPtrs *d_layers, *d_eagle;
-  float *attn_out, *act, *ss_part, *attn_part2;
+  float *ss_part, *attn_part2;
+  bf16 *xa_hi, *xa_lo, *at_hi, *at_lo, *ac_hi, *ac_lo, *fc_hi, *fc_lo;
   int *attn_cnt;
   float4 *amax2;
   unsigned *gbar;
+  unsigned long long *phase_ns;
   // bookkeeping
   long long launches;
   cudaGraphExec_t graph;
@@ -219,13 +221,16 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->out_nused = w.take<int>(B);
   x->d_layers = w.take<LayerPtrs>(L);
   x->d_eagle = w.take<LayerPtrs>(1);
-  x->attn_out = w.take<float>(16 * d);
-  x->act = w.take<float>(16 * F);
+  x->xa_hi = w.take<bf16>(16 * d); x->xa_lo = w.take<bf16>(16 * d);
+  x->at_hi = w.take<bf16>(16 * d); x->at_lo = w.take<bf16>(16 * d);
+  x->ac_hi = w.take<bf16>(16 * F); x->ac_lo = w.take<bf16>(16 * F);
+  x->fc_hi = w.take<bf16>(32 * d); x->fc_lo = w.take<bf16>(32 * d);
   x->ss_part = w.take<float>(256 * 16);
   x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
   x->attn_cnt = w.take<int>(H);
   x->amax2 = w.take<float4>(256 * 16);
   x->gbar = w.take<unsigned>(64);
+  x->phase_ns = w.take<unsigned long long>(512);
   return (w.off + 255) & ~(size_t)255;
 }
 
@@ -370,7 +375,9 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.d = c.d_model; p.H = c.n_heads; p.hd = c.head_dim; p.F = c.d_ffn; p.V = c.vocab; p.eps = c.rms_eps;
   p.embed = x->embed; p.lm_head = x->lm_head; p.final_norm = x->final_norm; p.eagle_fc = x->eagle_fc;
   p.mode = mode; p.draft_step = step; p.with_lm = with_lm;
-  p.h = x->h; p.qkv = x->qkv; p.attn = x->attn_out; p.act = x->act; p.ss_part = x->ss_part;
+  p.h = x->h; p.qkv = x->qkv; p.ss_part = x->ss_part;
+  p.xa_hi = x->xa_hi; p.xa_lo = x->xa_lo; p.at_hi = x->at_hi; p.at_lo = x->at_lo;
+  p.ac_hi = x->ac_hi; p.ac_lo = x->ac_lo; p.fc_hi = x->fc_hi; p.fc_lo = x->fc_lo;
   p.feat = x->feat; p.cap = c.kv_capacity; p.dfeat = x->dfeat; p.nmax = c.n_max;
   p.rope = x->rope;
   p.kpool = mode == 0 ? x->tk : x->dk; p.vpool = mode == 0 ? x->tv : x->dv;
@@ -378,6 +385,7 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
   p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
   p.gbar = x->gbar; p.cnt = x->cnt;
+  p.phase_ns = (x->prof && mode == 0) ? x->phase_ns : nullptr;
   timed(x, 0, pass_weight_bytes(x, mode, with_lm), [&] {
     cudaMemsetAsync(x->gbar, 0, sizeof(unsigned), x->stream);
     void *args[] = {&p};
@@ -725,6 +733,7 @@ extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *byt
     case 6: *d_ptr = x->dtop; *bytes = B * c.n_max * sizeof(float2); break;
     case 7: *d_ptr = x->draft; *bytes = B * c.n_max * sizeof(int); break;
     case 8: *d_ptr = x->target; *bytes = B * (c.n_max + 1) * sizeof(int); break;
+    case 9: *d_ptr = x->phase_ns; *bytes = 512 * sizeof(unsigned long long); break;
     default: return fail(x, ADA_ERR_RANGE, "ada_debug_buffer: unknown buffer");
   }
   return ADA_OK;

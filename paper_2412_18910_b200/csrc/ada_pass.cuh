@@ -10,12 +10,16 @@
 // producer runs ahead across phase boundaries: while the other warps sit in a grid barrier or in
 // the attention phase, the ring is already filling with the next GEMM's weights.
 //
-// Roles inside a CTA (13 warps):
-//   warp 0        producer: walks the static schedule of (phase, k chunk, row pair-tile) stages
-//   warps 1..4    activation loaders: read the fp32 input rows of the current GEMM from L2, apply
-//                 RMSNorm scale and gain where the phase asks for it, split into bf16 hi/lo planes
-//                 in shared memory (the tensor-core B operand)
-//   warps 5..12   consumers: mma.sync m16n8k16 with the weight tile as the 16-row operand
+// Every GEMM input lives in global memory already split into two bf16 planes (hi, lo), written by
+// the epilogue that produced it, so activations too are fetched by bulk copies with no conversion
+// on the way.  RMSNorm is folded around the GEMM: the producing epilogue stores split(h * gain) and
+// the per-row sum of squares; the consuming epilogue multiplies its accumulators by 1/rms(row).
+//
+// Roles inside a CTA (10 warps):
+//   warp 0        weight producer: walks the static schedule of (phase, k chunk, row pair-tile) stages
+//   warp 1        activation producer: per GEMM phase (after the grid barrier that makes its input
+//                 visible) copies the input planes chunk by chunk into shared memory
+//   warps 2..9    consumers: mma.sync m16n8k16 with the weight tile as the 16-row operand
 //                 (swap-AB), fp32 accumulators in registers, epilogues, attention
 //
 // Every wait (mbarrier, grid barrier) is bounded; when a bound is hit the kernel sets a status bit
@@ -25,8 +29,8 @@
 
 namespace ada {
 
-constexpr int kPassThreads = 13 * 32;
-constexpr int kNumXWarps = 4;
+constexpr int kPassThreads = 10 * 32;
+constexpr int kNumXWarps = 1;
 constexpr int kNumCWarps = 8;
 constexpr int kKc = 256;                         // k elements per ring stage
 constexpr int kRowStride = kKc * 2 + 64;         // bytes per staged row: 64 mod 128 keeps 128-bit reads conflict free
@@ -64,8 +68,12 @@ struct PassParams {
   int mode;                    // 0 target pass, 1 draft-head pass
   int draft_step;              // draft: 0 catch-up rows, s >= 1 single-row steps
   int with_lm;                 // run the LM head
-  // activations
-  float *h, *qkv, *attn, *act; // [16][d], [16][3d], [16][d], [16][F]
+  // activations: fp32 residual stream and qkv; bf16 (hi, lo) planes of every GEMM input
+  float *h, *qkv;              // [16][d], [16][3d]
+  __nv_bfloat16 *xa_hi, *xa_lo;   // [16][d]   h * gain of the norm that follows
+  __nv_bfloat16 *at_hi, *at_lo;   // [16][d]   attention output
+  __nv_bfloat16 *ac_hi, *ac_lo;   // [16][F]   SwiGLU output
+  __nv_bfloat16 *fc_hi, *fc_lo;   // [16][2d]  draft-head input [e ; f]
   float *ss_part;              // [grid][16] partial sums of squares of h
   float *feat; int cap;        // target features by position [seq][cap][d]
   float *dfeat; int nmax;      // draft features [seq][nmax][d]
@@ -83,6 +91,7 @@ struct PassParams {
   // sync
   unsigned *gbar;              // grid barrier counter, zero at launch
   Counters *cnt;
+  unsigned long long *phase_ns;  // optional [512]: [0] = start, [i+1] = time CTA 0 left barrier i (globaltimer)
 };
 
 // ---------------------------------------------------------------------------------- primitives
@@ -137,28 +146,30 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
 
 // ---------------------------------------------------------------------------------- GEMM phases
 
-enum { SRC_PLAIN = 0, SRC_NORM = 1, SRC_EAGLE = 2, SRC_LMROWS = 3 };
+enum { EPI_STORE_QKV = 0, EPI_RESID_H = 1, EPI_SWIGLU_ACT = 2, EPI_ARGMAX_LM = 3, EPI_STORE_H = 4 };
 
 struct GemmDesc {
   const __nv_bfloat16 *W[3];
-  int nseg, Nseg, K, epi, src_mode;
-  const float *src; int ldsrc;
-  const __nv_bfloat16 *gain;
-  float *out; int ldout;
-  int write_feat;   // NORM phase also stores the normalised rows as target features (CTA 0)
-  int write_ss;     // RESID / STORE phase also stores partial sums of squares of the new h
-  int lm;           // ARGMAX over lm rows of the draft
+  int nseg, Nseg, K, epi;
+  const __nv_bfloat16 *xhi, *xlo;   // input planes
+  int ldx;
+  int scale_inv_rms;                // accumulators are multiplied by 1/rms(row) of h (input was h * gain)
+  int lm_rows;                      // input rows are pass->lm_row[i] (draft LM head)
+  const __nv_bfloat16 *gain_next;   // RESID_H / STORE_H: planes written are split(h * gain_next); null = no gain
 };
 
-// Phase list.  Target: [embed] then per layer QKV, ATTN, O, GATEUP, DOWN, then LM.
-// Draft: FC, then the same five, then LM.  Index -> kind:
-enum { PH_EMBED = 0, PH_FC, PH_QKV, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM, PH_END };
+// Phase list.  Target: EMBED, then per layer QKV, ATTN, O, GATEUP, DOWN, then LM.
+// Draft: EAGLE_IN, FC, then the same five, then LM (optional).
+enum { PH_EMBED = 0, PH_EAGLE_IN, PH_FC, PH_QKV, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM };
 
-__device__ __forceinline__ int phase_count(const PassParams &p) { return 1 + 5 * p.n_layers + (p.with_lm ? 1 : 0); }
+__device__ __forceinline__ int phase_count(const PassParams &p) {
+  return (p.mode == 0 ? 1 : 2) + 5 * p.n_layers + (p.with_lm ? 1 : 0);
+}
 __device__ __forceinline__ int phase_kind(const PassParams &p, int idx, int &layer) {
   layer = 0;
-  if (idx == 0) return p.mode == 0 ? PH_EMBED : PH_FC;
-  const int i = idx - 1;
+  const int pre = p.mode == 0 ? 1 : 2;
+  if (idx < pre) return p.mode == 0 ? PH_EMBED : (idx == 0 ? PH_EAGLE_IN : PH_FC);
+  const int i = idx - pre;
   if (i < 5 * p.n_layers) {
     layer = i / 5;
     return PH_QKV + (i % 5);
@@ -168,34 +179,35 @@ __device__ __forceinline__ int phase_kind(const PassParams &p, int idx, int &lay
 
 __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int layer, GemmDesc &g) {
   const LayerPtrs &L = p.layers[layer];
-  g.nseg = 1; g.gain = nullptr; g.write_feat = 0; g.write_ss = 0; g.lm = 0;
+  g.nseg = 1; g.scale_inv_rms = 0; g.lm_rows = 0; g.gain_next = nullptr;
   g.W[1] = g.W[2] = nullptr;
   switch (kind) {
     case PH_FC:
-      g.W[0] = p.eagle_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE; g.src_mode = SRC_EAGLE;
-      g.src = nullptr; g.ldsrc = 0; g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      g.W[0] = p.eagle_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H;
+      g.xhi = p.fc_hi; g.xlo = p.fc_lo; g.ldx = 2 * p.d; g.gain_next = L.na;
       return true;
     case PH_QKV:
-      g.W[0] = L.wq; g.W[1] = L.wk; g.W[2] = L.wv; g.nseg = 3; g.Nseg = p.d; g.K = p.d; g.epi = EPI_STORE;
-      g.src_mode = SRC_NORM; g.src = p.h; g.ldsrc = p.d; g.gain = L.na; g.out = p.qkv; g.ldout = 3 * p.d;
+      g.W[0] = L.wq; g.W[1] = L.wk; g.W[2] = L.wv; g.nseg = 3; g.Nseg = p.d; g.K = p.d; g.epi = EPI_STORE_QKV;
+      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d; g.scale_inv_rms = 1;
       return true;
     case PH_O:
-      g.W[0] = L.wo; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID; g.src_mode = SRC_PLAIN; g.src = p.attn; g.ldsrc = p.d;
-      g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      g.W[0] = L.wo; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H;
+      g.xhi = p.at_hi; g.xlo = p.at_lo; g.ldx = p.d; g.gain_next = L.nm;
       return true;
     case PH_GATEUP:
-      g.W[0] = L.wg; g.W[1] = L.wu; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU; g.src_mode = SRC_NORM; g.src = p.h;
-      g.ldsrc = p.d; g.gain = L.nm; g.out = p.act; g.ldout = p.F;
+      g.W[0] = L.wg; g.W[1] = L.wu; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU_ACT;
+      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d; g.scale_inv_rms = 1;
       return true;
     case PH_DOWN:
-      g.W[0] = L.wd; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID; g.src_mode = SRC_PLAIN; g.src = p.act; g.ldsrc = p.F;
-      g.out = p.h; g.ldout = p.d; g.write_ss = 1;
+      g.W[0] = L.wd; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H;
+      g.xhi = p.ac_hi; g.xlo = p.ac_lo; g.ldx = p.F;
+      // the norm that follows: next layer's, or the final one; the draft head has none after its layer
+      g.gain_next = (layer + 1 < p.n_layers) ? p.layers[layer + 1].na : (p.mode == 0 ? p.final_norm : nullptr);
       return true;
     case PH_LM:
-      g.W[0] = p.lm_head; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX; g.src = p.h; g.ldsrc = p.d; g.out = nullptr;
-      g.ldout = 0;
-      if (p.mode == 0) { g.src_mode = SRC_NORM; g.gain = p.final_norm; g.write_feat = 1; }
-      else { g.src_mode = SRC_LMROWS; g.lm = 1; }
+      g.W[0] = p.lm_head; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX_LM;
+      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d;
+      if (p.mode == 0) g.scale_inv_rms = 1; else g.lm_rows = 1;
       return true;
     default:
       return false;
@@ -217,13 +229,13 @@ __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) 
   s.r0 = cta * rpc;
   s.rows = max(0, min(N, s.r0 + rpc) - s.r0);
   s.mt = (s.rows + 15) >> 4;
-  s.ntiles = g.epi == EPI_SWIGLU ? 2 * s.mt : s.mt;
+  s.ntiles = g.epi == EPI_SWIGLU_ACT ? 2 * s.mt : s.mt;
   s.nstage_rows = (s.ntiles + 1) >> 1;
   return s;
 }
 // weight row pointer of virtual row v (tile list index -> matrix for SWIGLU)
 __device__ __forceinline__ const __nv_bfloat16 *row_ptr(const GemmDesc &g, const Slab &s, int tile, int r) {
-  if (g.epi == EPI_SWIGLU) {
+  if (g.epi == EPI_SWIGLU_ACT) {
     const int m = tile >= s.mt ? 1 : 0;
     const int v = s.r0 + (tile - m * s.mt) * 16 + r;
     return g.W[m] + (size_t)v * g.K;
@@ -233,7 +245,7 @@ __device__ __forceinline__ const __nv_bfloat16 *row_ptr(const GemmDesc &g, const
   return g.W[seg] + (size_t)(v - seg * g.Nseg) * g.K;
 }
 __device__ __forceinline__ int tile_rows(const GemmDesc &g, const Slab &s, int tile) {
-  const int t = (g.epi == EPI_SWIGLU && tile >= s.mt) ? tile - s.mt : tile;
+  const int t = (g.epi == EPI_SWIGLU_ACT && tile >= s.mt) ? tile - s.mt : tile;
   return max(0, min(16, s.rows - t * 16));
 }
 
@@ -263,6 +275,11 @@ __device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoc
     }
     if (!ok) { *abort_flag = 1; atomicOr(&p.cnt->status, kStatTimeout); }
     __threadfence();
+    if (p.phase_ns && blockIdx.x == 0 && epoch < 511) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      p.phase_ns[epoch] = t;
+    }
   }
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
 }
@@ -289,6 +306,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   unsigned char *xbuf = smem + kStages * kStageBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
   static_assert((2 * kStages + 2 * kXBufs) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
+  (void)red;
 
   if (tid == 0) {
     *abort_s = 0;
@@ -299,6 +317,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   __syncthreads();
 
   const int nphase = phase_count(p);
+  if (p.phase_ns && cta == 0 && tid == 32) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    p.phase_ns[0] = t;
+  }
 
   // ================================================================= producer warp
   if (warp == 0) {
@@ -339,10 +362,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     return;
   }
 
-  // ================================================================= loaders and consumers
-  const bool is_loader = warp <= kNumXWarps;
-  const int cw = warp - 1 - kNumXWarps;   // consumer warp index 0..7 (consumers only)
+  // ================================================================= activation producer + consumers
+  const bool is_xprod = warp == 1;
+  const int cw = warp - 2;                 // consumer warp index 0..7 (consumers only)
   const int g8 = lane >> 2, q4 = lane & 3;
+  const int ntid = tid - 32;               // index among the 288 non-weight-producer threads
+  const int nnth = (kNumXWarps + kNumCWarps) * 32;
+  const int ctid = tid - 64;               // index among the 256 consumer threads
   unsigned epoch = 0;
   RingPos rp{0, 0};
   int xcount = 0;   // activation chunks produced / consumed so far (buffer = xcount % kXBufs)
@@ -351,31 +377,53 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     int layer;
     const int kind = phase_kind(p, ph, layer);
 
-    // ------------------------------------------------------------- embedding
-    if (kind == PH_EMBED) {
-      // h[t][:] = embedding rows; column slices per CTA; partial sums of squares for the first norm
-      const int ltid = tid - 32, nth = (kNumXWarps + kNumCWarps) * 32;
-      const int cpc = (p.d + ncta - 1) / ncta;
-      const int c0 = cta * cpc, c1 = min(p.d, c0 + cpc);
+    // ------------------------------------------------------------- row-wise input phases
+    if (kind == PH_EMBED || kind == PH_EAGLE_IN) {
+      // EMBED: h = embedding rows, planes = split(h * gain of layer 0), partial sums of squares.
+      // EAGLE_IN: planes of [e(token) ; feature] for the draft head's fc.  Column slices per CTA.
+      const int width = kind == PH_EMBED ? p.d : 2 * p.d;
+      const int cpc = (((width + ncta - 1) / ncta) + 3) & ~3;
+      const int c0 = cta * cpc, c1 = min(width, c0 + cpc);
+      const __nv_bfloat16 *gain = p.layers[0].na;
       for (int t = 0; t < 16; ++t) {
         float ss = 0.f;
         if (t < T) {
+          const int b = p.pass->row_seq[t];
           const __nv_bfloat16 *e = p.embed + (size_t)p.pass->row_tok[t] * p.d;
-          for (int c = c0 + ltid; c < c1; c += nth) {
-            const float v = __bfloat162float(e[c]);
-            p.h[(size_t)t * p.d + c] = v;
-            ss += v * v;
+          for (int c = c0 + ntid; c < c1; c += nnth) {
+            if (kind == PH_EMBED) {
+              const float v = __bfloat162float(e[c]);
+              p.h[(size_t)t * p.d + c] = v;
+              ss += v * v;
+              __nv_bfloat16 hi, lo;
+              split_bf16(v * __bfloat162float(gain[c]), hi, lo);
+              p.xa_hi[(size_t)t * p.d + c] = hi; p.xa_lo[(size_t)t * p.d + c] = lo;
+            } else {
+              float v;
+              if (c < p.d) v = __bfloat162float(e[c]);
+              else {
+                const float *f = p.draft_step == 0 ? p.feat + ((size_t)b * p.cap + p.pass->row_pos[t]) * p.d
+                                                   : p.dfeat + ((size_t)b * p.nmax + (p.draft_step - 1)) * p.d;
+                v = __ldcg(f + (c - p.d));
+              }
+              __nv_bfloat16 hi, lo;
+              split_bf16(v, hi, lo);
+              p.fc_hi[(size_t)t * 2 * p.d + c] = hi; p.fc_lo[(size_t)t * 2 * p.d + c] = lo;
+            }
           }
         }
-        // CTA-wide sum of ss in a fixed order: warp sums, then warps in order
-        ss = warp_sum(ss);
-        if (lane == 0) red[(warp - 1) * 16 + t] = ss;
+        if (kind == PH_EMBED) {
+          ss = warp_sum(ss);
+          if (lane == 0) red[(warp - 1) * 16 + t] = ss;
+        }
       }
-      named_bar(2, nth);
-      if (tid - 32 < 16) {
-        float s = 0.f;
-        for (int w = 0; w < kNumXWarps + kNumCWarps; ++w) s += red[w * 16 + (tid - 32)];
-        p.ss_part[(size_t)cta * 16 + (tid - 32)] = s;
+      if (kind == PH_EMBED) {
+        named_bar(2, nnth);
+        if (ntid < 16) {
+          float sum = 0.f;
+          for (int w = 0; w < kNumXWarps + kNumCWarps; ++w) sum += red[w * 16 + ntid];
+          p.ss_part[(size_t)cta * 16 + ntid] = sum;
+        }
       }
       grid_barrier(p, epoch, tid, abort_s);
       continue;
@@ -383,8 +431,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 
     // ------------------------------------------------------------- attention
     if (kind == PH_ATTN) {
-      if (!is_loader) {
-        // items (sequence 0, head, split) round-robin over CTAs; batch 1 only on this path
+      if (!is_xprod) {
+        // items (head, split) round-robin over CTAs; one sequence on this path
         const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
         const int nkeys = pos0 + R, nsp = p.attn_splits;
         int chunk = (nkeys + nsp - 1) / nsp;
@@ -395,10 +443,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         float *v_s = k_s + 16 * 128;
         float *p_s = v_s + 16 * 128;                           // [8][16][32]
         float *part_s = q_s;                                   // [8][16][130], reuses the loop's scratch
-        const int ctid = tid - 32 * (1 + kNumXWarps);
         const int VPL = HD / 32;
-        const LayerPtrs &Lw = p.layers[layer];
-        (void)Lw;
         for (int item = cta; item < p.H * nsp; item += ncta) {
           const int hh = item / nsp, split = item - hh * nsp;
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
@@ -409,12 +454,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const int r = i / half, c = i - r * half;
             const float2 cs = p.rope[(size_t)(pos0 + r) * half + c];
             const float *qr = p.qkv + (size_t)r * 3 * d + hh * HD;
-            const float qa = qr[c], qb = qr[c + half], ka = qr[d + c], kb = qr[d + c + half];
+            const float qa = __ldcg(qr + c), qb = __ldcg(qr + c + half);
+            const float ka = __ldcg(qr + d + c), kb = __ldcg(qr + d + c + half);
             q_s[r * 128 + c] = (qa * cs.x - qb * cs.y) * qscale;
             q_s[r * 128 + c + half] = (qb * cs.x + qa * cs.y) * qscale;
             const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(qr[2 * d + c]), v1 = __float2bfloat16_rn(qr[2 * d + c + half]);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(qr + 2 * d + c));
+            const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(qr + 2 * d + c + half));
             k_s[r * 128 + c] = __bfloat162float(k0); k_s[r * 128 + c + half] = __bfloat162float(k1);
             v_s[r * 128 + c] = __bfloat162float(v0); v_s[r * 128 + c + half] = __bfloat162float(v1);
             if (split == 0) {  // one item per head stores the new rows in the cache
@@ -432,9 +479,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           for (int kb = kbeg + cw * 32; kb < kend; kb += kNumCWarps * 32) {
             const int key = kb + lane;
             const bool kv = key < kend;
-            float s[16];
+            float sc[16];
 #pragma unroll
-            for (int r = 0; r < 16; ++r) s[r] = 0.f;
+            for (int r = 0; r < 16; ++r) sc[r] = 0.f;
             if (kv) {
               if (key >= pos0) {
                 const float *kr = k_s + (key - pos0) * 128;
@@ -444,7 +491,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   for (int r = 0; r < 16; ++r)
                     if (r < R) {
                       const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c);
-                      s[r] += qa.x * kk.x + qa.y * kk.y + qa.z * kk.z + qa.w * kk.w;
+                      sc[r] += qa.x * kk.x + qa.y * kk.y + qa.z * kk.z + qa.w * kk.w;
                     }
                 }
               } else {
@@ -463,8 +510,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                     if (r < R) {
                       const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8);
                       const float4 qb = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8 + 4);
-                      s[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                              qb.z * kf[6] + qb.w * kf[7];
+                      sc[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                               qb.z * kf[6] + qb.w * kf[7];
                     }
                 }
               }
@@ -473,7 +520,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             for (int r = 0; r < 16; ++r)
               if (r < R) {
                 const bool seen = kv && key <= pos0 + r;
-                const float sv = seen ? s[r] : -INFINITY;
+                const float sv = seen ? sc[r] : -INFINITY;
                 const float mx = warp_max(sv);
                 const float mn = fmaxf(m[r], mx);
                 float pe = 0.f, corr = 1.f;
@@ -561,7 +608,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   oo += __ldcg(gp + s2 * sst + c) * e;
                 }
               }
-              p.attn[(size_t)r * d + hh * HD + c] = oo / lo;
+              __nv_bfloat16 hi, lw;
+              split_bf16(oo / lo, hi, lw);
+              p.at_hi[(size_t)r * d + hh * HD + c] = hi;
+              p.at_lo[(size_t)r * d + hh * HD + c] = lw;
             }
             if (ctid == 0) p.attn_cnt[hh] = 0;
           }
@@ -574,93 +624,66 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     // ------------------------------------------------------------- GEMM phases
     GemmDesc g;
     make_gemm(p, kind, layer, g);
-    const int Tg = g.lm ? lmT : T;
+    const int Tg = g.lm_rows ? lmT : T;
     if (Tg <= 0) { grid_barrier(p, epoch, tid, abort_s); continue; }
     const int nt_act = (Tg + 7) >> 3;
     const Slab s = make_slab(g, cta, ncta);
     const int nchunk = (g.K + kKc - 1) / kKc;
 
-    if (is_loader) {
-      // ---- activation loaders: chunk by chunk, X = hi/lo planes of the GEMM input rows
-      const int xt = tid - 32;  // 0..127
-      if (g.src_mode == SRC_NORM) {
-        if (xt < 16) {
-          float ssum = 0.f;
-          for (int i = 0; i < ncta; ++i) ssum += __ldcg(p.ss_part + (size_t)i * 16 + xt);
-          inv_rms[xt] = rsqrtf(ssum / (float)p.d + p.eps);
-        }
-        named_bar(4, kNumXWarps * 32);
-      }
+    if (is_xprod) {
+      // ---- activation producer: the input planes of this GEMM, chunk by chunk, by bulk copies
       if (s.rows > 0) {
-        const int lw = warp - 1;   // loader warp index; it converts chunks c with (xcount + c) % 4 == lw
-        for (int c = 0; c < nchunk; ++c) {
-          const int xc = xcount + c;
-          if ((xc % kNumXWarps) != lw) continue;
-          const int buf = xc % kXBufs;
-          if (xc >= kXBufs) {
-            if (lane == 0) mbar_wait(&xempty[buf], ((unsigned)(xc / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
+        const int plane = lane >> 4, r = lane & 15;
+        const int srow = (r < Tg) ? (g.lm_rows ? p.pass->lm_row[r] : r) : 0;
+        const __nv_bfloat16 *src_row = (plane ? g.xlo : g.xhi) + (size_t)srow * g.ldx;
+        for (int c = 0; c < nchunk; ++c, ++xcount) {
+          const int buf = xcount % kXBufs;
+          if (xcount >= kXBufs) {
+            if (lane == 0) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
             __syncwarp();
           }
-          unsigned char *xh = xbuf + (size_t)buf * kXBufBytes, *xl = xh + kXPlaneBytes;
-          // nt_act*8 rows x 256 k in groups of 4 elements; lane handles groups lane, lane+32, ...
-          const int ngroups = nt_act * 8 * (kKc / 4);
-#pragma unroll 4
-          for (int gi = lane; gi < ngroups; gi += 32) {
-            const int r = gi / (kKc / 4), kk = (gi - r * (kKc / 4)) * 4;
-            const int k = c * kKc + kk;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (r < Tg && k < g.K) {
-              if (g.src_mode == SRC_EAGLE) {
-                const int b = p.pass->row_seq[r];
-                if (k < p.d) {
-                  const __nv_bfloat16 *e = p.embed + (size_t)p.pass->row_tok[r] * p.d + k;
-                  v = make_float4(__bfloat162float(e[0]), __bfloat162float(e[1]), __bfloat162float(e[2]),
-                                  __bfloat162float(e[3]));
-                } else {
-                  const float *f = p.draft_step == 0 ? p.feat + ((size_t)b * p.cap + p.pass->row_pos[r]) * p.d
-                                                     : p.dfeat + ((size_t)b * p.nmax + (p.draft_step - 1)) * p.d;
-                  v = __ldcg(reinterpret_cast<const float4 *>(f + (k - p.d)));
-                }
-              } else {
-                const int sr = g.src_mode == SRC_LMROWS ? p.pass->lm_row[r] : r;
-                v = __ldcg(reinterpret_cast<const float4 *>(g.src + (size_t)sr * g.ldsrc + k));
-                if (g.src_mode == SRC_NORM) {
-                  const float iv = inv_rms[r];
-                  const __nv_bfloat16 *gn = g.gain + k;
-                  v.x = (v.x * iv) * __bfloat162float(gn[0]); v.y = (v.y * iv) * __bfloat162float(gn[1]);
-                  v.z = (v.z * iv) * __bfloat162float(gn[2]); v.w = (v.w * iv) * __bfloat162float(gn[3]);
-                  if (g.write_feat && cta == 0)
-                    *reinterpret_cast<float4 *>(p.feat + ((size_t)p.pass->row_seq[r] * p.cap + p.pass->row_pos[r]) * p.d + k) = v;
-                } else if (g.src_mode == SRC_LMROWS && cta == 0) {
-                  const int b = p.pass->row_seq[sr];
-                  *reinterpret_cast<float4 *>(p.dfeat + ((size_t)b * p.nmax + p.draft_step) * p.d + k) = v;
-                }
-              }
-            }
-            __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-            split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
-            uint2 hv, lv;
-            hv.x = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-            hv.y = (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16);
-            lv.x = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-            lv.y = (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16);
-            *reinterpret_cast<uint2 *>(xh + (size_t)r * kRowStride + kk * 2) = hv;
-            *reinterpret_cast<uint2 *>(xl + (size_t)r * kRowStride + kk * 2) = lv;
-          }
+          const int kvalid = min(kKc, g.K - c * kKc);
+          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(2 * Tg * kvalid * 2));
           __syncwarp();
-          if (lane == 0) mbar_arrive(&xfull[buf]);
+          if (r < Tg)
+            bulk_g2s(xbuf + (size_t)buf * kXBufBytes + (size_t)plane * kXPlaneBytes + (size_t)r * kRowStride,
+                     src_row + (size_t)c * kKc, (unsigned)(kvalid * 2), &xfull[buf]);
         }
-        xcount += nchunk;
       }
       grid_barrier(p, epoch, tid, abort_s);
       continue;
     }
 
     // ---- consumers
+    // 1/rms per row of h for phases whose input was h * gain; features of the rows (target LM phase)
+    if (g.scale_inv_rms) {
+      if (ctid < 16) {
+        float ssum = 0.f;
+        for (int i = 0; i < ncta; ++i) ssum += __ldcg(p.ss_part + (size_t)i * 16 + ctid);
+        inv_rms[ctid] = rsqrtf(ssum / (float)p.d + p.eps);
+      }
+      named_bar(3, kNumCWarps * 32);
+    }
+    if (kind == PH_LM) {
+      // column slice of the feature rows: target f = h / rms * gain (kept per position); draft: the
+      // head's own output rows (kept per step) -- both read by later passes
+      const int cpc = (p.d + ncta - 1) / ncta;
+      const int c0 = cta * cpc, c1 = min(p.d, c0 + cpc);
+      for (int i = ctid; i < Tg * (c1 - c0); i += kNumCWarps * 32) {
+        const int t = i / (c1 - c0), c = c0 + (i - t * (c1 - c0));
+        if (p.mode == 0) {
+          const float v = (__ldcg(p.h + (size_t)t * p.d + c) * inv_rms[t]) * __bfloat162float(p.final_norm[c]);
+          p.feat[((size_t)p.pass->row_seq[t] * p.cap + p.pass->row_pos[t]) * p.d + c] = v;
+        } else {
+          const int sr = p.pass->lm_row[t];
+          p.dfeat[((size_t)p.pass->row_seq[sr] * p.nmax + p.draft_step) * p.d + c] = __ldcg(p.h + (size_t)sr * p.d + c);
+        }
+      }
+    }
     // tile ownership: mt <= 8 tiles (single matrix): tile = cw / ksplit, k blocks split ksplit ways;
     // otherwise warp cw owns list tiles cw and cw + 8 (SWIGLU: gate tile cw and up tile cw + mt).
     int tileA = -1, tileB = -1, ksplit = 1, kpart = 0;
-    if (g.epi == EPI_SWIGLU) {
+    if (g.epi == EPI_SWIGLU_ACT) {
       if (cw < s.mt) { tileA = cw; tileB = cw + s.mt; }
     } else if (s.mt <= 8) {
       ksplit = s.mt <= 1 ? 8 : (s.mt == 2 ? 4 : (s.mt <= 4 ? 2 : 1));
@@ -697,7 +720,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 if (blk * 32 < kvalid) {   // warp-uniform: every lane takes part in the mma
                   const int koff = blk * 32 + 8 * q4;
                   const bool okk = koff < kvalid;   // ragged end of K: this lane's 8 k are past it
-                  uint4 A0 = make_uint4(0, 0, 0, 0), A1 = A0;
+                  const uint4 zero4 = make_uint4(0, 0, 0, 0);
+                  uint4 A0 = zero4, A1 = zero4;
                   if (okk) {
                     A0 = *reinterpret_cast<const uint4 *>(a_base + (size_t)g8 * kRowStride + koff * 2);
                     A1 = *reinterpret_cast<const uint4 *>(a_base + (size_t)(g8 + 8) * kRowStride + koff * 2);
@@ -705,8 +729,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
                   for (int i = 0; i < 2; ++i)
                     if (i < nt_act) {
-                      const uint4 bh = *reinterpret_cast<const uint4 *>(xh + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
-                      const uint4 bl = *reinterpret_cast<const uint4 *>(xl + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
+                      uint4 bh = zero4, bl = zero4;
+                      if (okk) {
+                        bh = *reinterpret_cast<const uint4 *>(xh + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
+                        bl = *reinterpret_cast<const uint4 *>(xl + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
+                      }
                       mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bh.x, bh.y);
                       mma_bf16(acc[slot][i], A0.z, A1.z, A0.w, A1.w, bh.z, bh.w);
                       mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bl.x, bl.y);
@@ -744,7 +771,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       }
     }
     const bool owner = tileA >= 0 && kpart == 0 && s.rows > 0;
-    float ssl[4] = {0.f, 0.f, 0.f, 0.f};   // sums of squares for pass rows 2*q4 + {0,1} + 8*{0,1}
+    const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
+    float ssl[4] = {0.f, 0.f, 0.f, 0.f};   // sums of squares for pass rows 8*i + 2*q4 + (j&1)
     Top2 tb[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) { tb[i].v1 = -INFINITY; tb[i].i1 = 0x7fffffff; tb[i].v2 = -INFINITY; }
@@ -753,30 +781,36 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
       for (int slot = 0; slot < 2; ++slot) {
         const int tile = slot ? tileB : tileA;
-        if (tile < 0 || (g.epi == EPI_SWIGLU && slot == 1)) continue;
+        if (tile < 0 || (g.epi == EPI_SWIGLU_ACT && slot == 1)) continue;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           if (i >= nt_act) continue;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int rr = g8 + 8 * (j >> 1), t = 8 * i + 2 * q4 + (j & 1);
-            const int vrow = s.r0 + tile * 16 + rr;     // virtual output column
+            const int vrow = s.r0 + tile * 16 + rr;     // output column (virtual row of the weight)
             if (tile * 16 + rr >= s.rows || t >= Tg) continue;
-            const float y = acc[slot][i][j];
-            if (g.epi == EPI_STORE) {
-              g.out[(size_t)t * g.ldout + vrow] = y;
-              if (g.write_ss) ssl[i * 2 + (j & 1)] += y * y;
-            } else if (g.epi == EPI_RESID) {
-              float *hp = g.out + (size_t)t * g.ldout + vrow;
-              const float hn = __ldcg(hp) + y;
+            const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
+            const float y = acc[slot][i][j] * sc;
+            if (g.epi == EPI_STORE_QKV) {
+              p.qkv[(size_t)t * 3 * p.d + vrow] = y;
+            } else if (g.epi == EPI_RESID_H || g.epi == EPI_STORE_H) {
+              float *hp = p.h + (size_t)t * p.d + vrow;
+              const float hn = g.epi == EPI_RESID_H ? __ldcg(hp) + y : y;
               *hp = hn;
               ssl[i * 2 + (j & 1)] += hn * hn;
-            } else if (g.epi == EPI_SWIGLU) {
-              const float up = acc[1][i][j];
-              g.out[(size_t)t * g.ldout + vrow] = (y / (1.f + __expf(-y))) * up;
-            } else {  // ARGMAX
+              const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
+              __nv_bfloat16 hi, lo;
+              split_bf16(hn * gn, hi, lo);
+              p.xa_hi[(size_t)t * p.d + vrow] = hi; p.xa_lo[(size_t)t * p.d + vrow] = lo;
+            } else if (g.epi == EPI_SWIGLU_ACT) {
+              const float up = acc[1][i][j] * sc;
+              __nv_bfloat16 hi, lo;
+              split_bf16((y / (1.f + __expf(-y))) * up, hi, lo);
+              p.ac_hi[(size_t)t * p.F + vrow] = hi; p.ac_lo[(size_t)t * p.F + vrow] = lo;
+            } else {  // EPI_ARGMAX_LM
               if (p.logits) {
-                const int slot_out = g.lm ? p.pass->lm_out[t] : p.pass->row_out[t];
+                const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
                 p.logits[(size_t)slot_out * p.V + vrow] = y;
               }
               Top2 cnd; cnd.v1 = y; cnd.i1 = vrow; cnd.v2 = -INFINITY;
@@ -786,7 +820,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         }
       }
     }
-    if (g.write_ss || g.epi == EPI_RESID) {
+    if (has_ss) {
       // reduce over the 8 row groups of the warp, then over warps in order, one value per pass row
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -802,7 +836,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         for (int w = 0; w < kNumCWarps; ++w) v += ssw[w * 16 + lane];
         p.ss_part[(size_t)cta * 16 + lane] = v;
       }
-    } else if (g.epi == EPI_ARGMAX) {
+    } else if (g.epi == EPI_ARGMAX_LM) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         Top2 b = tb[i];
@@ -818,7 +852,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     }
     grid_barrier(p, epoch, tid, abort_s);
 
-    if (g.epi == EPI_ARGMAX && cta == 0 && cw == 0 && lane < 16 && lane < Tg) {
+    if (g.epi == EPI_ARGMAX_LM && cta == 0 && cw == 0 && lane < 16 && lane < Tg) {
       // greedy choice per row: candidates of all CTAs merged in CTA order
       Top2 b;
       b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
@@ -827,7 +861,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         Top2 x; x.v1 = c4.x; x.i1 = __float_as_int(c4.y); x.v2 = c4.z;
         b = top2_merge(b, x);
       }
-      const int slot_out = g.lm ? p.pass->lm_out[lane] : p.pass->row_out[lane];
+      const int slot_out = g.lm_rows ? p.pass->lm_out[lane] : p.pass->row_out[lane];
       p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
       if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
     }
