@@ -4,6 +4,8 @@
 // rotary table at initialisation.
 #include "ada.h"
 
+#include <cuda.h>
+
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -62,6 +64,8 @@ struct ada_ctx {
   // persistent pass kernel (batch 1): device copies of the layer pointer tables and its scratch
   int use_pass, n_sm, attn_splits;
   LayerPtrs *d_layers, *d_eagle;
+  TensorMap128 *d_maps;
+  int n_maps;
   float *ss_part, *attn_part2;
   bf16 *xa_hi, *xa_lo, *at_hi, *at_lo, *ac_hi, *ac_lo, *fc_hi, *fc_lo;
   int *attn_cnt;
@@ -221,6 +225,8 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->out_nused = w.take<int>(B);
   x->d_layers = w.take<LayerPtrs>(L);
   x->d_eagle = w.take<LayerPtrs>(1);
+  x->n_maps = (int)(7 * (L + 1) + 2 + 8);
+  x->d_maps = w.take<TensorMap128>(x->n_maps);
   x->xa_hi = w.take<bf16>(16 * d); x->xa_lo = w.take<bf16>(16 * d);
   x->at_hi = w.take<bf16>(16 * d); x->at_lo = w.take<bf16>(16 * d);
   x->ac_hi = w.take<bf16>(16 * F); x->ac_lo = w.take<bf16>(16 * F);
@@ -230,7 +236,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->attn_cnt = w.take<int>(H);
   x->amax2 = w.take<float4>(256 * 16);
   x->gbar = w.take<unsigned>(64);
-  x->phase_ns = w.take<unsigned long long>(512);
+  x->phase_ns = w.take<unsigned long long>(512 + 4 * 512);
   return (w.off + 255) & ~(size_t)255;
 }
 
@@ -350,6 +356,51 @@ void draft_rows(ada_ctx *x, int step, bool with_lm) {
   }
 }
 
+// 2-D bf16 tensor map over a row-major [rows][cols] matrix: box = 64 columns x box_rows rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_map(EncodeTiledFn fn, TensorMap128 *out, const void *base, size_t rows, size_t cols, unsigned box_rows) {
+  static_assert(sizeof(CUtensorMap) == sizeof(TensorMap128), "tensor map size");
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// All tensor maps of a context, in the order ada_pass.cuh documents.
+bool build_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
+  void *sym = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym) return false;
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(sym);
+  const ada_config &c = x->c;
+  const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+  maps.assign(x->n_maps, TensorMap128());
+  bool ok = true;
+  auto layer = [&](int base, const LayerW &a) {
+    ok = ok && encode_map(fn, &maps[base + MAP_WQ], a.wq, d, d, 32) && encode_map(fn, &maps[base + MAP_WK], a.wk, d, d, 32) &&
+         encode_map(fn, &maps[base + MAP_WV], a.wv, d, d, 32) && encode_map(fn, &maps[base + MAP_WO], a.wo, d, d, 32) &&
+         encode_map(fn, &maps[base + MAP_WG], a.wg, F, d, 32) && encode_map(fn, &maps[base + MAP_WU], a.wu, F, d, 32) &&
+         encode_map(fn, &maps[base + MAP_WD], a.wd, d, F, 32);
+  };
+  for (int l = 0; l < c.n_layers; ++l) layer(7 * l, x->layers[l]);
+  layer(7 * c.n_layers, x->eagle);
+  const int m0 = 7 * (c.n_layers + 1);
+  ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, 32) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, 32);
+  const int pl = m0 + 2;
+  ok = ok && encode_map(fn, &maps[pl + MAPX_XA], x->xa_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_XA + 1], x->xa_lo, 16, d, 16) &&
+       encode_map(fn, &maps[pl + MAPX_AT], x->at_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_AT + 1], x->at_lo, 16, d, 16) &&
+       encode_map(fn, &maps[pl + MAPX_AC], x->ac_hi, 16, F, 16) && encode_map(fn, &maps[pl + MAPX_AC + 1], x->ac_lo, 16, F, 16) &&
+       encode_map(fn, &maps[pl + MAPX_FC], x->fc_hi, 16, 2 * d, 16) && encode_map(fn, &maps[pl + MAPX_FC + 1], x->fc_lo, 16, 2 * d, 16);
+  return ok;
+}
+
 // Bytes of weights one pass streams (each once): for the per-launch roofline record.
 double pass_weight_bytes(const ada_ctx *x, int mode, int with_lm) {
   const ada_config &c = x->c;
@@ -370,6 +421,9 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   memset(&p, 0, sizeof(p));
   p.pass = x->pass;
   p.layers = mode == 0 ? x->d_layers : x->d_eagle;
+  p.maps = x->d_maps;
+  p.map_layer0 = mode == 0 ? 0 : 7 * c.n_layers;
+  p.map_fc = 7 * (c.n_layers + 1); p.map_lm = p.map_fc + 1; p.map_planes = p.map_fc + 2;
   p.n_layers = mode == 0 ? c.n_layers : 1;
   p.cache_layers = p.n_layers;
   p.d = c.d_model; p.H = c.n_heads; p.hd = c.head_dim; p.F = c.d_ffn; p.V = c.vocab; p.eps = c.rms_eps;
@@ -539,6 +593,19 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       LayerPtrs ep{a.wq, a.wk, a.wv, a.wo, a.wg, a.wu, a.wd, a.na, a.nm};
       e = cudaMemcpy(x->d_layers, lp.data(), sizeof(LayerPtrs) * lp.size(), cudaMemcpyHostToDevice);
       if (e == cudaSuccess) e = cudaMemcpy(x->d_eagle, &ep, sizeof(LayerPtrs), cudaMemcpyHostToDevice);
+      std::vector<TensorMap128> maps;
+      if (e == cudaSuccess && !build_maps(x, maps)) e = cudaErrorUnknown;
+      if (e == cudaSuccess) e = cudaMemcpy(x->d_maps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);
+      // planes start finite: rows past the live ones are read by the tensor-core tiles
+      const size_t dd = cfg->d_model, FF = cfg->d_ffn;
+      if (e == cudaSuccess) e = cudaMemset(x->xa_hi, 0, 32 * dd); 
+      if (e == cudaSuccess) e = cudaMemset(x->xa_lo, 0, 32 * dd);
+      if (e == cudaSuccess) e = cudaMemset(x->at_hi, 0, 32 * dd);
+      if (e == cudaSuccess) e = cudaMemset(x->at_lo, 0, 32 * dd);
+      if (e == cudaSuccess) e = cudaMemset(x->ac_hi, 0, 32 * FF);
+      if (e == cudaSuccess) e = cudaMemset(x->ac_lo, 0, 32 * FF);
+      if (e == cudaSuccess) e = cudaMemset(x->fc_hi, 0, 64 * dd);
+      if (e == cudaSuccess) e = cudaMemset(x->fc_lo, 0, 64 * dd);
       if (e == cudaSuccess) e = cudaMemset(x->attn_cnt, 0, sizeof(int) * cfg->n_heads);
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }
@@ -733,7 +800,7 @@ extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *byt
     case 6: *d_ptr = x->dtop; *bytes = B * c.n_max * sizeof(float2); break;
     case 7: *d_ptr = x->draft; *bytes = B * c.n_max * sizeof(int); break;
     case 8: *d_ptr = x->target; *bytes = B * (c.n_max + 1) * sizeof(int); break;
-    case 9: *d_ptr = x->phase_ns; *bytes = 512 * sizeof(unsigned long long); break;
+    case 9: *d_ptr = x->phase_ns; *bytes = (512 + 4 * 512) * sizeof(unsigned long long); break;
     default: return fail(x, ADA_ERR_RANGE, "ada_debug_buffer: unknown buffer");
   }
   return ADA_OK;

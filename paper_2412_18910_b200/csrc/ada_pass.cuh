@@ -5,8 +5,9 @@
 // Why: a 7B verify pass streams 13.2 GB of weights in about 2 ms at HBM speed; one layer is ~60 us.
 // Nine separate launches per layer lose a large share of that to launch gaps, ramp-up and tails.
 // Here each CTA owns a fixed slab of rows of every weight matrix (N / gridDim rows), and a
-// producer warp streams those slabs through a shared-memory ring with bulk async copies
-// (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the
+// producer warp streams those slabs through a shared-memory ring with TMA tiled loads
+// (cp.async.bulk.tensor.2d, 128-byte swizzle, mbarrier transaction counts; one 4 KB box per
+// instruction -- separate 512-byte bulk copies were measured to cap a CTA near 12 GB/s).  Weights do not depend on activations, so the
 // producer runs ahead across phase boundaries: while the other warps sit in a grid barrier or in
 // the attention phase, the ring is already filling with the next GEMM's weights.
 //
@@ -19,8 +20,9 @@
 //   warp 0        weight producer: walks the static schedule of (phase, k chunk, row pair-tile) stages
 //   warp 1        activation producer: per GEMM phase (after the grid barrier that makes its input
 //                 visible) copies the input planes chunk by chunk into shared memory
-//   warps 2..9    consumers: mma.sync m16n8k16 with the weight tile as the 16-row operand
-//                 (swap-AB), fp32 accumulators in registers, epilogues, attention
+//   warps 2..9    consumers: ldmatrix from the swizzled tiles, mma.sync m16n8k16 with the weight
+//                 tile as the 16-row operand (swap-AB), fp32 accumulators in registers,
+//                 epilogues, attention
 //
 // Every wait (mbarrier, grid barrier) is bounded; when a bound is hit the kernel sets a status bit
 // and carries on as if the wait had succeeded, so it always terminates.
@@ -32,13 +34,15 @@ namespace ada {
 constexpr int kPassThreads = 10 * 32;
 constexpr int kNumXWarps = 1;
 constexpr int kNumCWarps = 8;
-constexpr int kKc = 256;                         // k elements per ring stage
-constexpr int kRowStride = kKc * 2 + 64;         // bytes per staged row: 64 mod 128 keeps 128-bit reads conflict free
+constexpr int kKc = 256;                         // k elements per ring stage = 4 boxes of 64
+constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
 constexpr int kStageRows = 32;                   // two 16-row tiles per stage
-constexpr int kStageBytes = kStageRows * kRowStride;
+constexpr int kWBoxBytes = kStageRows * 128;     // 4 KB
+constexpr int kStageBytes = (kKc / kBoxK) * kWBoxBytes;   // 16 KB
 constexpr int kStages = 8;
-constexpr int kXBufs = 4;                        // one activation chunk in flight per loader warp
-constexpr int kXPlaneBytes = 16 * kRowStride;
+constexpr int kXBufs = 4;
+constexpr int kXBoxBytes = 16 * 128;             // activation box: 16 rows x 64 k
+constexpr int kXPlaneBytes = (kKc / kBoxK) * kXBoxBytes;  // 8 KB
 constexpr int kXBufBytes = 2 * kXPlaneBytes;
 constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
@@ -48,7 +52,7 @@ constexpr int kAttnLoopBytes = (3 * 16 * 128 + 8 * 16 * 32) * 4;   // q, k, v ro
 constexpr int kAttnPartBytes = 8 * 16 * 130 * 4;                   // per-warp partial results
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
-constexpr int kPassSmemBytes = kStages * kStageBytes + kMiscBytes + kScratchBytes;
+constexpr int kPassSmemBytes = 1024 + kStages * kStageBytes + kMiscBytes + kScratchBytes;   // 1 KB to align the ring
 static_assert(kPassSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr int kStatTimeout = 4;
 constexpr unsigned kSpinLimit = 1u << 22;
@@ -57,8 +61,21 @@ struct LayerPtrs {
   const __nv_bfloat16 *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nm;
 };
 
+// Tensor maps (CUtensorMap, 128 bytes each) live in a device array, in this order:
+//   7 per target layer (wq wk wv wo w_gate w_up w_down), 7 for the draft head's layer, then
+//   eagle_fc, lm_head, then the activation planes xa_hi xa_lo at_hi at_lo ac_hi ac_lo fc_hi fc_lo.
+// Weight maps: dims {K, N}, box {64, 32}; plane maps: dims {K, 16}, box {64, 16}; 128-byte swizzle.
+struct alignas(64) TensorMap128 {
+  unsigned long long opaque[16];
+};
+enum { MAP_WQ = 0, MAP_WK, MAP_WV, MAP_WO, MAP_WG, MAP_WU, MAP_WD };
+enum { MAPX_XA = 0, MAPX_AT = 2, MAPX_AC = 4, MAPX_FC = 6 };
+
 struct PassParams {
   const Pass *pass;
+  const TensorMap128 *maps;    // device array, see above
+  int map_layer0;              // index of the first map of this pass's first layer
+  int map_fc, map_lm, map_planes;
   const LayerPtrs *layers;     // device array
   int n_layers;                // layers of this pass (target: L, draft head: 1)
   int cache_layers;            // layers in the KV pool (stride)
@@ -135,6 +152,18 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+__device__ __forceinline__ void tma_load_2d(void *dst, const TensorMap128 *map, int x, int y, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
 __device__ __forceinline__ void named_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -149,10 +178,9 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
 enum { EPI_STORE_QKV = 0, EPI_RESID_H = 1, EPI_SWIGLU_ACT = 2, EPI_ARGMAX_LM = 3, EPI_STORE_H = 4 };
 
 struct GemmDesc {
-  const __nv_bfloat16 *W[3];
+  int wmap[3];                      // tensor maps of the weight matrices (segments, or gate / up)
   int nseg, Nseg, K, epi;
-  const __nv_bfloat16 *xhi, *xlo;   // input planes
-  int ldx;
+  int xmap;                         // tensor map of the input's hi plane (lo plane = xmap + 1)
   int scale_inv_rms;                // accumulators are multiplied by 1/rms(row) of h (input was h * gain)
   int lm_rows;                      // input rows are pass->lm_row[i] (draft LM head)
   const __nv_bfloat16 *gain_next;   // RESID_H / STORE_H: planes written are split(h * gain_next); null = no gain
@@ -179,34 +207,35 @@ __device__ __forceinline__ int phase_kind(const PassParams &p, int idx, int &lay
 
 __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int layer, GemmDesc &g) {
   const LayerPtrs &L = p.layers[layer];
+  const int lm = p.map_layer0 + 7 * layer;
   g.nseg = 1; g.scale_inv_rms = 0; g.lm_rows = 0; g.gain_next = nullptr;
-  g.W[1] = g.W[2] = nullptr;
+  g.wmap[1] = g.wmap[2] = -1;
   switch (kind) {
     case PH_FC:
-      g.W[0] = p.eagle_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H;
-      g.xhi = p.fc_hi; g.xlo = p.fc_lo; g.ldx = 2 * p.d; g.gain_next = L.na;
+      g.wmap[0] = p.map_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H;
+      g.xmap = p.map_planes + MAPX_FC; g.gain_next = L.na;
       return true;
     case PH_QKV:
-      g.W[0] = L.wq; g.W[1] = L.wk; g.W[2] = L.wv; g.nseg = 3; g.Nseg = p.d; g.K = p.d; g.epi = EPI_STORE_QKV;
-      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d; g.scale_inv_rms = 1;
+      g.wmap[0] = lm + MAP_WQ; g.wmap[1] = lm + MAP_WK; g.wmap[2] = lm + MAP_WV; g.nseg = 3; g.Nseg = p.d; g.K = p.d;
+      g.epi = EPI_STORE_QKV; g.xmap = p.map_planes + MAPX_XA; g.scale_inv_rms = 1;
       return true;
     case PH_O:
-      g.W[0] = L.wo; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H;
-      g.xhi = p.at_hi; g.xlo = p.at_lo; g.ldx = p.d; g.gain_next = L.nm;
+      g.wmap[0] = lm + MAP_WO; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H;
+      g.xmap = p.map_planes + MAPX_AT; g.gain_next = L.nm;
       return true;
     case PH_GATEUP:
-      g.W[0] = L.wg; g.W[1] = L.wu; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU_ACT;
-      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d; g.scale_inv_rms = 1;
+      g.wmap[0] = lm + MAP_WG; g.wmap[1] = lm + MAP_WU; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU_ACT;
+      g.xmap = p.map_planes + MAPX_XA; g.scale_inv_rms = 1;
       return true;
     case PH_DOWN:
-      g.W[0] = L.wd; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H;
-      g.xhi = p.ac_hi; g.xlo = p.ac_lo; g.ldx = p.F;
+      g.wmap[0] = lm + MAP_WD; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H;
+      g.xmap = p.map_planes + MAPX_AC;
       // the norm that follows: next layer's, or the final one; the draft head has none after its layer
       g.gain_next = (layer + 1 < p.n_layers) ? p.layers[layer + 1].na : (p.mode == 0 ? p.final_norm : nullptr);
       return true;
     case PH_LM:
-      g.W[0] = p.lm_head; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX_LM;
-      g.xhi = p.xa_hi; g.xlo = p.xa_lo; g.ldx = p.d;
+      g.wmap[0] = p.map_lm; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX_LM;
+      g.xmap = p.map_planes + MAPX_XA;
       if (p.mode == 0) g.scale_inv_rms = 1; else g.lm_rows = 1;
       return true;
     default:
@@ -214,39 +243,35 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
   }
 }
 
-// Row slab of this CTA and its 16-row tiles.  Virtual rows: segments concatenated (nseg * Nseg rows);
-// SWIGLU: the slab is over Nseg rows and tiles are listed gate first, then up.
+// Row slab of this CTA.  A GEMM over nseg separate matrices of Nseg rows gives each matrix
+// gridDim / nseg CTAs, so a slab never spans two matrices.  The slab is cut into 16-row tiles;
+// a ring stage holds 32 consecutive rows (two tiles) of ONE matrix.  SWIGLU: the slab is the same
+// row range of the gate and of the up matrix; stages alternate gate, up, gate, up ...
 struct Slab {
-  int r0, rows;     // slab [r0, r0 + rows) in virtual rows
-  int mt;           // tiles per matrix pass (ceil(rows / 16))
-  int ntiles;       // tiles in the list (SWIGLU: 2 * mt)
-  int nstage_rows;  // stages per k chunk = ceil(ntiles / 2)
+  int seg;          // matrix (segment) of this CTA
+  int r0, rows;     // rows [r0, r0 + rows) inside that matrix
+  int mt;           // 16-row tiles of the slab
+  int nstage_rows;  // ring stages per k chunk
 };
 __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) {
   Slab s;
-  const int N = g.nseg * g.Nseg;
-  const int rpc = (N + ncta - 1) / ncta;
-  s.r0 = cta * rpc;
-  s.rows = max(0, min(N, s.r0 + rpc) - s.r0);
+  const int cps = ncta / g.nseg;                  // CTAs per matrix
+  s.seg = cta / cps;
+  const int li = cta - s.seg * cps;
+  const int rpc = (g.Nseg + cps - 1) / cps;
+  s.r0 = li * rpc;
+  s.rows = (s.seg < g.nseg) ? max(0, min(g.Nseg, s.r0 + rpc) - s.r0) : 0;
   s.mt = (s.rows + 15) >> 4;
-  s.ntiles = g.epi == EPI_SWIGLU_ACT ? 2 * s.mt : s.mt;
-  s.nstage_rows = (s.ntiles + 1) >> 1;
+  const int pairs = (s.mt + 1) >> 1;
+  s.nstage_rows = g.epi == EPI_SWIGLU_ACT ? 2 * pairs : pairs;
   return s;
 }
-// weight row pointer of virtual row v (tile list index -> matrix for SWIGLU)
-__device__ __forceinline__ const __nv_bfloat16 *row_ptr(const GemmDesc &g, const Slab &s, int tile, int r) {
-  if (g.epi == EPI_SWIGLU_ACT) {
-    const int m = tile >= s.mt ? 1 : 0;
-    const int v = s.r0 + (tile - m * s.mt) * 16 + r;
-    return g.W[m] + (size_t)v * g.K;
-  }
-  const int v = s.r0 + tile * 16 + r;
-  const int seg = v / g.Nseg;
-  return g.W[seg] + (size_t)(v - seg * g.Nseg) * g.K;
-}
-__device__ __forceinline__ int tile_rows(const GemmDesc &g, const Slab &s, int tile) {
-  const int t = (g.epi == EPI_SWIGLU_ACT && tile >= s.mt) ? tile - s.mt : tile;
-  return max(0, min(16, s.rows - t * 16));
+// stage sr of a chunk -> weight map index and first row; and which two tiles it holds
+__device__ __forceinline__ void stage_source(const GemmDesc &g, const Slab &s, int sr, int &map, int &row0, int &pair,
+                                             int &which) {
+  if (g.epi == EPI_SWIGLU_ACT) { which = sr & 1; pair = sr >> 1; map = g.wmap[which]; }
+  else { which = 0; pair = sr; map = g.wmap[s.seg]; }
+  row0 = s.r0 + pair * 32;
 }
 
 struct RingPos {
@@ -284,6 +309,15 @@ __device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoc
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
 }
 
+// optional fine-grained clock of CTA 0's first consumer lane: 4 stamps per phase after the 512 barrier stamps
+__device__ __forceinline__ void stamp(const PassParams &p, int ph, int k, bool on) {
+  if (on && p.phase_ns && ph < 500) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    p.phase_ns[512 + 4 * ph + k] = t;
+  }
+}
+
 // ---------------------------------------------------------------------------------- the kernel
 
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
@@ -294,7 +328,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   const int cta = blockIdx.x, ncta = gridDim.x;
 
   extern __shared__ __align__(128) unsigned char pass_smem[];
-  unsigned char *const smem = pass_smem;
+  // swizzled TMA boxes need 1024-byte aligned bases
+  unsigned char *const smem = pass_smem + ((1024u - (smem_u32(pass_smem) & 1023u)) & 1023u);
   unsigned char *ring = smem;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
   uint64_t *full = bars, *empty = bars + kStages, *xfull = bars + 2 * kStages, *xempty = bars + 2 * kStages + kXBufs;
@@ -337,23 +372,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       if (s.rows == 0) continue;
       const int nchunk = (g.K + kKc - 1) / kKc;
       for (int c = 0; c < nchunk; ++c) {
-        const int kvalid = min(kKc, g.K - c * kKc);
+        const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;   // boxes that hold any k < K
         for (int sr = 0; sr < s.nstage_rows; ++sr) {
           if (filled >= (unsigned)kStages) {
             if (lane == 0) mbar_wait(&empty[rp.stage], rp.parity ^ 1u, p.cnt, abort_s);
             __syncwarp();
           }
-          const int t0 = 2 * sr;
-          const int rows0 = tile_rows(g, s, t0), rows1 = (t0 + 1 < s.ntiles) ? tile_rows(g, s, t0 + 1) : 0;
-          if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)((rows0 + rows1) * kvalid * 2));
+          int map, row0, pair, which;
+          stage_source(g, s, sr, map, row0, pair, which);
+          if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)(nbox * kWBoxBytes));
           __syncwarp();
-          unsigned char *dst = ring + (size_t)rp.stage * kStageBytes;
-          const int which = lane >> 4, r = lane & 15;
-          const int nr = which ? rows1 : rows0;
-          if (r < nr) {
-            const __nv_bfloat16 *src = row_ptr(g, s, t0 + which, r) + (size_t)c * kKc;
-            bulk_g2s(dst + (size_t)(which * 16 + r) * kRowStride, src, (unsigned)(kvalid * 2), &full[rp.stage]);
-          }
+          if (lane < nbox)   // one 64-k x 32-row box per lane; rows past the matrix and k past K read as zero
+            tma_load_2d(ring + (size_t)rp.stage * kStageBytes + (size_t)lane * kWBoxBytes, p.maps + map,
+                        c * kKc + lane * kBoxK, row0, &full[rp.stage]);
           ++filled;
           rp.advance();
         }
@@ -633,21 +664,20 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     if (is_xprod) {
       // ---- activation producer: the input planes of this GEMM, chunk by chunk, by bulk copies
       if (s.rows > 0) {
-        const int plane = lane >> 4, r = lane & 15;
-        const int srow = (r < Tg) ? (g.lm_rows ? p.pass->lm_row[r] : r) : 0;
-        const __nv_bfloat16 *src_row = (plane ? g.xlo : g.xhi) + (size_t)srow * g.ldx;
+        const int plane = lane >> 2, box = lane & 3;           // lanes 0..7: (plane, box)
+        const int y0 = g.lm_rows ? p.pass->lm_row[0] : 0;       // draft LM head: its single row
         for (int c = 0; c < nchunk; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
           if (xcount >= kXBufs) {
             if (lane == 0) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
             __syncwarp();
           }
-          const int kvalid = min(kKc, g.K - c * kKc);
-          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(2 * Tg * kvalid * 2));
+          const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
+          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(2 * nbox * kXBoxBytes));
           __syncwarp();
-          if (r < Tg)
-            bulk_g2s(xbuf + (size_t)buf * kXBufBytes + (size_t)plane * kXPlaneBytes + (size_t)r * kRowStride,
-                     src_row + (size_t)c * kKc, (unsigned)(kvalid * 2), &xfull[buf]);
+          if (lane < 8 && box < nbox)
+            tma_load_2d(xbuf + (size_t)buf * kXBufBytes + (size_t)plane * kXPlaneBytes + (size_t)box * kXBoxBytes,
+                        p.maps + g.xmap + plane, c * kKc + box * kBoxK, y0, &xfull[buf]);
         }
       }
       grid_barrier(p, epoch, tid, abort_s);
@@ -655,6 +685,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     }
 
     // ---- consumers
+    const bool stamper = cta == 0 && ctid == 0;
+    stamp(p, ph, 0, stamper);
     // 1/rms per row of h for phases whose input was h * gain; features of the rows (target LM phase)
     if (g.scale_inv_rms) {
       if (ctid < 16) {
@@ -684,7 +716,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     // otherwise warp cw owns list tiles cw and cw + 8 (SWIGLU: gate tile cw and up tile cw + mt).
     int tileA = -1, tileB = -1, ksplit = 1, kpart = 0;
     if (g.epi == EPI_SWIGLU_ACT) {
-      if (cw < s.mt) { tileA = cw; tileB = cw + s.mt; }
+      if (cw < s.mt) { tileA = cw; tileB = cw; }
     } else if (s.mt <= 8) {
       ksplit = s.mt <= 1 ? 8 : (s.mt == 2 ? 4 : (s.mt <= 4 ? 2 : 1));
       if (cw / ksplit < s.mt) { tileA = cw / ksplit; kpart = cw % ksplit; }
@@ -700,45 +732,47 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         for (int j = 0; j < 4; ++j) acc[a][i][j] = 0.f;
 
     if (s.rows > 0) {
-      const int bpw = 8 / ksplit;  // 32-k blocks of a chunk this warp handles
+      const int spw = 16 / ksplit;   // k16 steps of a chunk this warp handles
+      // ldmatrix lane addressing inside a 128-byte-swizzled box (row pitch 128 B, 16-byte chunk index
+      // XORed with row & 7): A = weight tile rows, B = activation rows
+      const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_sel = lane >> 4;
+      const int b_row = (lane & 7) + ((lane >> 4) & 1) * 8, b_sel = (lane >> 3) & 1;
+      const uint32_t ring_u = smem_u32(ring), xbuf_u = smem_u32(xbuf);
       for (int c = 0; c < nchunk; ++c, ++xcount) {
         const int buf = xcount % kXBufs;
         mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
-        const unsigned char *xh = xbuf + (size_t)buf * kXBufBytes, *xl = xh + kXPlaneBytes;
-        const int kvalid = min(kKc, g.K - c * kKc);
+        if (c == 0) stamp(p, ph, 1, stamper);
+        const uint32_t xh = xbuf_u + (uint32_t)buf * kXBufBytes, xl = xh + kXPlaneBytes;
+        const int nstep = (min(kKc, g.K - c * kKc) + 15) >> 4;   // k16 steps that hold any k < K
         for (int sr = 0; sr < s.nstage_rows; ++sr) {
           mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
-          const unsigned char *st = ring + (size_t)rp.stage * kStageBytes;
+          const uint32_t st = ring_u + (uint32_t)rp.stage * kStageBytes;
+          int map, row0, pair, which;
+          stage_source(g, s, sr, map, row0, pair, which);
 #pragma unroll
           for (int slot = 0; slot < 2; ++slot) {
             const int tile = slot ? tileB : tileA;
-            if (tile >= 0 && (tile >> 1) == sr) {
-              const unsigned char *a_base = st + (size_t)((tile & 1) * 16) * kRowStride;
+            // slot 0 holds tiles of matrix 0 (or the only one), slot 1 of the up matrix / second tile
+            const bool mine = tile >= 0 && (tile >> 1) == pair &&
+                              (g.epi == EPI_SWIGLU_ACT ? which == slot : true);
+            if (mine) {
+              const uint32_t a_tile = st + (uint32_t)((tile & 1) * 16 + a_row) * 128;
 #pragma unroll 4
-              for (int bi = 0; bi < bpw; ++bi) {
-                const int blk = kpart * bpw + bi;
-                if (blk * 32 < kvalid) {   // warp-uniform: every lane takes part in the mma
-                  const int koff = blk * 32 + 8 * q4;
-                  const bool okk = koff < kvalid;   // ragged end of K: this lane's 8 k are past it
-                  const uint4 zero4 = make_uint4(0, 0, 0, 0);
-                  uint4 A0 = zero4, A1 = zero4;
-                  if (okk) {
-                    A0 = *reinterpret_cast<const uint4 *>(a_base + (size_t)g8 * kRowStride + koff * 2);
-                    A1 = *reinterpret_cast<const uint4 *>(a_base + (size_t)(g8 + 8) * kRowStride + koff * 2);
+              for (int si = 0; si < spw; ++si) {
+                const int ks = kpart * spw + si;
+                if (ks < nstep) {
+                  const int box = ks >> 2, s4 = ks & 3;
+                  uint32_t a0, a1, a2, a3, h0, h1, h2, h3, l0, l1, l2, l3;
+                  ldmatrix_x4(a_tile + box * kWBoxBytes + (((2 * s4 + a_sel) ^ (lane & 7)) << 4), a0, a1, a2, a3);
+                  const uint32_t boff = box * kXBoxBytes + b_row * 128 + (((2 * s4 + b_sel) ^ (lane & 7)) << 4);
+                  ldmatrix_x4(xh + boff, h0, h1, h2, h3);
+                  ldmatrix_x4(xl + boff, l0, l1, l2, l3);
+                  mma_bf16(acc[slot][0], a0, a1, a2, a3, h0, h1);
+                  mma_bf16(acc[slot][0], a0, a1, a2, a3, l0, l1);
+                  if (nt_act > 1) {
+                    mma_bf16(acc[slot][1], a0, a1, a2, a3, h2, h3);
+                    mma_bf16(acc[slot][1], a0, a1, a2, a3, l2, l3);
                   }
-#pragma unroll
-                  for (int i = 0; i < 2; ++i)
-                    if (i < nt_act) {
-                      uint4 bh = zero4, bl = zero4;
-                      if (okk) {
-                        bh = *reinterpret_cast<const uint4 *>(xh + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
-                        bl = *reinterpret_cast<const uint4 *>(xl + (size_t)(i * 8 + g8) * kRowStride + koff * 2);
-                      }
-                      mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bh.x, bh.y);
-                      mma_bf16(acc[slot][i], A0.z, A1.z, A0.w, A1.w, bh.z, bh.w);
-                      mma_bf16(acc[slot][i], A0.x, A1.x, A0.y, A1.y, bl.x, bl.y);
-                      mma_bf16(acc[slot][i], A0.z, A1.z, A0.w, A1.w, bl.z, bl.w);
-                    }
                 }
               }
             }
@@ -752,6 +786,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       }
     }
 
+    stamp(p, ph, 2, stamper);
     // ---- k-split reduction inside the CTA (fixed order), then the epilogue by the owner warps
     if (ksplit > 1) {
       float *mine = red + (size_t)(cw * 32 + lane) * 8;
@@ -788,7 +823,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int rr = g8 + 8 * (j >> 1), t = 8 * i + 2 * q4 + (j & 1);
-            const int vrow = s.r0 + tile * 16 + rr;     // output column (virtual row of the weight)
+            const int vrow = s.seg * g.Nseg + s.r0 + tile * 16 + rr;   // output column
             if (tile * 16 + rr >= s.rows || t >= Tg) continue;
             const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
             const float y = acc[slot][i][j] * sc;
@@ -850,6 +885,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         p.amax[(size_t)cta * 16 + lane] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
       }
     }
+    stamp(p, ph, 3, stamper);
     grid_barrier(p, epoch, tid, abort_s);
 
     if (g.epi == EPI_ARGMAX_LM && cta == 0 && cw == 0 && lane < 16 && lane < Tg) {
