@@ -383,16 +383,21 @@ bool build_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
   const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
   maps.assign(x->n_maps, TensorMap128());
   bool ok = true;
+  // box height of each matrix = rows of one m tile of its slabs (same arithmetic as the kernel's make_slab)
+  const unsigned b_qkv = slab_box_rows(slab_rpc((int)d, 3, x->n_sm), false);
+  const unsigned b_d = slab_box_rows(slab_rpc((int)d, 1, x->n_sm), false);
+  const unsigned b_f = slab_box_rows(slab_rpc((int)F, 1, x->n_sm), true);
+  const unsigned b_v = slab_box_rows(slab_rpc((int)V, 1, x->n_sm), false);
   auto layer = [&](int base, const LayerW &a) {
-    ok = ok && encode_map(fn, &maps[base + MAP_WQ], a.wq, d, d, 32) && encode_map(fn, &maps[base + MAP_WK], a.wk, d, d, 32) &&
-         encode_map(fn, &maps[base + MAP_WV], a.wv, d, d, 32) && encode_map(fn, &maps[base + MAP_WO], a.wo, d, d, 32) &&
-         encode_map(fn, &maps[base + MAP_WG], a.wg, F, d, 32) && encode_map(fn, &maps[base + MAP_WU], a.wu, F, d, 32) &&
-         encode_map(fn, &maps[base + MAP_WD], a.wd, d, F, 32);
+    ok = ok && encode_map(fn, &maps[base + MAP_WQ], a.wq, d, d, b_qkv) && encode_map(fn, &maps[base + MAP_WK], a.wk, d, d, b_qkv) &&
+         encode_map(fn, &maps[base + MAP_WV], a.wv, d, d, b_qkv) && encode_map(fn, &maps[base + MAP_WO], a.wo, d, d, b_d) &&
+         encode_map(fn, &maps[base + MAP_WG], a.wg, F, d, b_f) && encode_map(fn, &maps[base + MAP_WU], a.wu, F, d, b_f) &&
+         encode_map(fn, &maps[base + MAP_WD], a.wd, d, F, b_d);
   };
   for (int l = 0; l < c.n_layers; ++l) layer(7 * l, x->layers[l]);
   layer(7 * c.n_layers, x->eagle);
   const int m0 = 7 * (c.n_layers + 1);
-  ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, 32) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, 32);
+  ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, b_d) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, b_v);
   const int pl = m0 + 2;
   ok = ok && encode_map(fn, &maps[pl + MAPX_XA], x->xa_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_XA + 1], x->xa_lo, 16, d, 16) &&
        encode_map(fn, &maps[pl + MAPX_AT], x->at_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_AT + 1], x->at_lo, 16, d, 16) &&
@@ -579,7 +584,10 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, kPassSmemBytes);
     if (e == cudaSuccess)
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pass, kPassThreads, kPassSmemBytes);
-    if (e == cudaSuccess && per_sm >= 1 && sms >= 1 && sms <= 256) {
+    // slabs must fit the tensor-memory accumulators: one m tile (128 rows) for gate/up, two otherwise
+    const bool fits = sms >= 3 && slab_rpc(cfg->d_ffn, 1, sms) <= 128 && slab_rpc(cfg->vocab, 1, sms) <= 256 &&
+                      slab_rpc(cfg->d_model, 3, sms) <= 256;
+    if (e == cudaSuccess && per_sm >= 1 && sms <= 256 && fits) {
       x->use_pass = 1;
       x->n_sm = sms;
       int sp = sms / cfg->n_heads;

@@ -16,13 +16,22 @@
 // on the way.  RMSNorm is folded around the GEMM: the producing epilogue stores split(h * gain) and
 // the per-row sum of squares; the consuming epilogue multiplies its accumulators by 1/rms(row).
 //
-// Roles inside a CTA (10 warps):
-//   warp 0        weight producer: walks the static schedule of (phase, k chunk, row pair-tile) stages
+// The contraction runs on the 5th-generation tensor cores: one thread issues tcgen05.mma
+// (M = 128 weight rows, N = 32 = 16 activation rows in a hi and a lo bf16 plane, K = 16) straight
+// from the swizzled shared-memory tiles that TMA wrote, accumulating in tensor memory over the
+// whole K range; tcgen05.commit releases ring stages and signals the finished accumulator.  (With
+// mma.sync the same loop was bound by the latency of dependent register accumulators at about
+// 40 % of the streaming rate.)
+//
+// Roles inside a CTA (12 warps):
+//   warp 0        weight producer: walks the static schedule of (phase, k chunk, k boxes, m tile) stages
 //   warp 1        activation producer: per GEMM phase (after the grid barrier that makes its input
 //                 visible) copies the input planes chunk by chunk into shared memory
-//   warps 2..9    consumers: ldmatrix from the swizzled tiles, mma.sync m16n8k16 with the weight
-//                 tile as the 16-row operand (swap-AB), fp32 accumulators in registers,
-//                 epilogues, attention
+//   warp 2        tensor-memory allocation; its lane 0 issues every tcgen05.mma and commit
+//   warp 3        idle (keeps the workers on warp indices whose index mod 4 spans the four
+//                 tensor-memory lane quarters)
+//   warps 4..11   workers: epilogues out of tensor memory (tcgen05.ld: one weight row per thread),
+//                 attention, row-wise phases
 //
 // Every wait (mbarrier, grid barrier) is bounded; when a bound is hit the kernel sets a status bit
 // and carries on as if the wait had succeeded, so it always terminates.
@@ -31,19 +40,18 @@
 
 namespace ada {
 
-constexpr int kPassThreads = 10 * 32;
+constexpr int kPassThreads = 12 * 32;
 constexpr int kNumXWarps = 1;
-constexpr int kNumCWarps = 8;
-constexpr int kKc = 256;                         // k elements per ring stage = 4 boxes of 64
+constexpr int kNumCWarps = 8;                    // workers
+constexpr int kFirstWorker = 4;                  // warp index of worker 0
+constexpr int kKc = 256;                         // k elements per activation chunk = 4 boxes of 64
 constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
-constexpr int kStageRows = 32;                   // two 16-row tiles per stage
-constexpr int kWBoxBytes = kStageRows * 128;     // 4 KB
-constexpr int kStageBytes = (kKc / kBoxK) * kWBoxBytes;   // 16 KB
+constexpr int kStageBytes = 16 * 1024;           // ring stage: kb boxes of [box_rows x 64 k], kb = 1, 2 or 4
 constexpr int kStages = 8;
 constexpr int kXBufs = 4;
-constexpr int kXBoxBytes = 16 * 128;             // activation box: 16 rows x 64 k
-constexpr int kXPlaneBytes = (kKc / kBoxK) * kXBoxBytes;  // 8 KB
-constexpr int kXBufBytes = 2 * kXPlaneBytes;
+constexpr int kXBoxBytes = 32 * 128;             // activation box pair: 16 hi rows then 16 lo rows, 64 k
+constexpr int kXBufBytes = (kKc / kBoxK) * kXBoxBytes;    // 16 KB per chunk
+constexpr int kTmemCols = 64;                    // two accumulators of 32 columns
 constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
@@ -51,7 +59,8 @@ constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA 
 constexpr int kAttnLoopBytes = (3 * 16 * 128 + 8 * 16 * 32) * 4;   // q, k, v rows and softmax weights
 constexpr int kAttnPartBytes = 8 * 16 * 130 * 4;                   // per-warp partial results
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
-constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
+// (the + 16 KB: a tensor-core read of 128 tile rows may run past a short last stage; it must stay inside the allocation)
+constexpr int kScratchBytes = ((kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes) + 16 * 1024;
 constexpr int kPassSmemBytes = 1024 + kStages * kStageBytes + kMiscBytes + kScratchBytes;   // 1 KB to align the ring
 static_assert(kPassSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr int kStatTimeout = 4;
@@ -64,7 +73,8 @@ struct LayerPtrs {
 // Tensor maps (CUtensorMap, 128 bytes each) live in a device array, in this order:
 //   7 per target layer (wq wk wv wo w_gate w_up w_down), 7 for the draft head's layer, then
 //   eagle_fc, lm_head, then the activation planes xa_hi xa_lo at_hi at_lo ac_hi ac_lo fc_hi fc_lo.
-// Weight maps: dims {K, N}, box {64, 32}; plane maps: dims {K, 16}, box {64, 16}; 128-byte swizzle.
+// Weight maps: dims {K, N}, box {64, rows of one m tile of that matrix's slabs}; plane maps: dims {K, 16},
+// box {64, 16}; 128-byte swizzle.
 struct alignas(64) TensorMap128 {
   unsigned long long opaque[16];
 };
@@ -164,6 +174,50 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
 }
+// ---- tcgen05 (5th generation tensor cores, accumulators in tensor memory)
+__device__ __forceinline__ void tmem_alloc(uint32_t *smem_slot, uint32_t ncols) {   // whole warp
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {      // whole warp
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// K-major operand tile in shared memory, 128-byte swizzle: rows 128 B apart, 8-row groups 1024 B apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = 128, N = 32, K = 16
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 consecutive accumulator columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void named_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -244,34 +298,46 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
 }
 
 // Row slab of this CTA.  A GEMM over nseg separate matrices of Nseg rows gives each matrix
-// gridDim / nseg CTAs, so a slab never spans two matrices.  The slab is cut into 16-row tiles;
-// a ring stage holds 32 consecutive rows (two tiles) of ONE matrix.  SWIGLU: the slab is the same
-// row range of the gate and of the up matrix; stages alternate gate, up, gate, up ...
+// gridDim / nseg CTAs, so a slab never spans two matrices.  The slab is cut into at most two m
+// tiles of box_rows <= 128 rows (the tensor map's box height, fixed per matrix at initialisation
+// from the same arithmetic); SWIGLU: the two m tiles are the same row range of the gate and of the
+// up matrix.  A ring stage holds kb boxes (kb * 64 k) of one m tile.
 struct Slab {
   int seg;          // matrix (segment) of this CTA
   int r0, rows;     // rows [r0, r0 + rows) inside that matrix
-  int mt;           // 16-row tiles of the slab
-  int nstage_rows;  // ring stages per k chunk
+  int mtiles;       // accumulators in use (1 or 2)
+  int box_rows;     // rows per m tile = box height of the tensor map
+  int region;       // bytes of one box in shared memory (box_rows rounded up to 8, times 128)
+  int kb;           // boxes per stage
 };
+__host__ __device__ __forceinline__ int slab_rpc(int Nseg, int nseg, int ncta) {
+  const int cps = ncta / nseg;
+  return (Nseg + cps - 1) / cps;
+}
+__host__ __device__ __forceinline__ int slab_box_rows(int rpc, bool swiglu) {
+  const int mt = swiglu ? 1 : (rpc + 127) / 128;
+  return (rpc + mt - 1) / mt;
+}
 __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) {
   Slab s;
+  const bool sw = g.epi == EPI_SWIGLU_ACT;
   const int cps = ncta / g.nseg;                  // CTAs per matrix
   s.seg = cta / cps;
   const int li = cta - s.seg * cps;
-  const int rpc = (g.Nseg + cps - 1) / cps;
+  const int rpc = slab_rpc(g.Nseg, g.nseg, ncta);
   s.r0 = li * rpc;
   s.rows = (s.seg < g.nseg) ? max(0, min(g.Nseg, s.r0 + rpc) - s.r0) : 0;
-  s.mt = (s.rows + 15) >> 4;
-  const int pairs = (s.mt + 1) >> 1;
-  s.nstage_rows = g.epi == EPI_SWIGLU_ACT ? 2 * pairs : pairs;
+  s.box_rows = slab_box_rows(rpc, sw);
+  s.mtiles = sw ? 2 : ((rpc + 127) / 128);
+  if (!sw && s.rows <= s.box_rows) s.mtiles = 1;  // a short last slab may not reach the second tile
+  s.region = ((s.box_rows + 7) & ~7) * 128;
+  s.kb = s.region <= 4096 ? 4 : (s.region <= 8192 ? 2 : 1);
   return s;
 }
-// stage sr of a chunk -> weight map index and first row; and which two tiles it holds
-__device__ __forceinline__ void stage_source(const GemmDesc &g, const Slab &s, int sr, int &map, int &row0, int &pair,
-                                             int &which) {
-  if (g.epi == EPI_SWIGLU_ACT) { which = sr & 1; pair = sr >> 1; map = g.wmap[which]; }
-  else { which = 0; pair = sr; map = g.wmap[s.seg]; }
-  row0 = s.r0 + pair * 32;
+// m tile mi -> weight map index and first row
+__device__ __forceinline__ void tile_source(const GemmDesc &g, const Slab &s, int mi, int &map, int &row0) {
+  if (g.epi == EPI_SWIGLU_ACT) { map = g.wmap[mi]; row0 = s.r0; }
+  else { map = g.wmap[s.seg]; row0 = s.r0 + mi * s.box_rows; }
 }
 
 struct RingPos {
@@ -284,7 +350,7 @@ struct RingPos {
 
 // ---------------------------------------------------------------------------------- grid barrier
 
-// All loader and consumer threads (384) take part; the producer warp does not.
+// Warp 1 and the eight worker warps (288 threads) take part; the producers' and the issuer's warps do not.
 __device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoch, int tid, volatile int *abort_flag) {
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
   ++epoch;
@@ -333,23 +399,30 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   unsigned char *ring = smem;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
   uint64_t *full = bars, *empty = bars + kStages, *xfull = bars + 2 * kStages, *xempty = bars + 2 * kStages + kXBufs;
-  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs);   // [16]
+  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs + 2);   // [16] (after accfull)
   float *ssw = inv_rms + 16;                                                       // [8][16]
   Top2 *topw = reinterpret_cast<Top2 *>(ssw + 8 * 16);                             // [8][16]
   int *flag_s = reinterpret_cast<int *>(topw + 8 * 16);
   volatile int *abort_s = flag_s + 1;
   unsigned char *xbuf = smem + kStages * kStageBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
-  static_assert((2 * kStages + 2 * kXBufs) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
+  static_assert((2 * kStages + 2 * kXBufs + 2) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
   (void)red;
 
+  uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
   if (tid == 0) {
     *abort_s = 0;
-    for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], kNumCWarps); }
-    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], kNumCWarps); }
+    for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
+    mbar_init(accfull, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 2) tmem_alloc(tmem_slot, kTmemCols);
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
   const int nphase = phase_count(p);
   if (p.phase_ns && cta == 0 && tid == 32) {
@@ -358,7 +431,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     p.phase_ns[0] = t;
   }
 
-  // ================================================================= producer warp
+  // ================================================================= weight producer
   if (warp == 0) {
     RingPos rp{0, 0};
     unsigned filled = 0;  // stages issued so far; the first kStages need no wait
@@ -367,42 +440,103 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       const int kind = phase_kind(p, ph, layer);
       GemmDesc g;
       if (!make_gemm(p, kind, layer, g)) continue;
-      if (kind == PH_LM && p.mode == 1 && lmT <= 0) continue;
+      if ((g.lm_rows ? lmT : T) <= 0) continue;
       const Slab s = make_slab(g, cta, ncta);
       if (s.rows == 0) continue;
       const int nchunk = (g.K + kKc - 1) / kKc;
       for (int c = 0; c < nchunk; ++c) {
         const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;   // boxes that hold any k < K
-        for (int sr = 0; sr < s.nstage_rows; ++sr) {
-          if (filled >= (unsigned)kStages) {
-            if (lane == 0) mbar_wait(&empty[rp.stage], rp.parity ^ 1u, p.cnt, abort_s);
+        for (int b0 = 0; b0 < nbox; b0 += s.kb) {
+          const int nb = min(s.kb, nbox - b0);
+          for (int mi = 0; mi < s.mtiles; ++mi) {
+            if (filled >= (unsigned)kStages) {
+              if (lane == 0) mbar_wait(&empty[rp.stage], rp.parity ^ 1u, p.cnt, abort_s);
+              __syncwarp();
+            }
+            int map, row0;
+            tile_source(g, s, mi, map, row0);
+            if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)(nb * s.box_rows * 128));
             __syncwarp();
+            if (lane < nb)   // one box per lane; rows past the matrix and k past K read as zero
+              tma_load_2d(ring + (size_t)rp.stage * kStageBytes + (size_t)lane * s.region, p.maps + map,
+                          c * kKc + (b0 + lane) * kBoxK, row0, &full[rp.stage]);
+            ++filled;
+            rp.advance();
           }
-          int map, row0, pair, which;
-          stage_source(g, s, sr, map, row0, pair, which);
-          if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)(nbox * kWBoxBytes));
-          __syncwarp();
-          if (lane < nbox)   // one 64-k x 32-row box per lane; rows past the matrix and k past K read as zero
-            tma_load_2d(ring + (size_t)rp.stage * kStageBytes + (size_t)lane * kWBoxBytes, p.maps + map,
-                        c * kKc + lane * kBoxK, row0, &full[rp.stage]);
-          ++filled;
-          rp.advance();
         }
       }
     }
     return;
   }
 
-  // ================================================================= activation producer + consumers
+  // ================================================================= tensor-core issuer
+  if (warp == 2) {
+    if (lane == 0) {
+      RingPos rp{0, 0};
+      int xcount = 0;
+      const uint32_t ring_u = smem_u32(ring), xbuf_u = smem_u32(xbuf);
+      for (int ph = 0; ph < nphase; ++ph) {
+        int layer;
+        const int kind = phase_kind(p, ph, layer);
+        GemmDesc g;
+        if (!make_gemm(p, kind, layer, g)) continue;
+        if ((g.lm_rows ? lmT : T) <= 0) continue;
+        const Slab s = make_slab(g, cta, ncta);
+        if (s.rows == 0) continue;
+        const int nchunk = (g.K + kKc - 1) / kKc;
+        unsigned started = 0;   // bit mi set once accumulator mi holds a product of this phase
+        for (int c = 0; c < nchunk; ++c, ++xcount) {
+          const int buf = xcount % kXBufs;
+          mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
+          const int kleft = min(kKc, g.K - c * kKc);
+          const int nbox = (kleft + kBoxK - 1) / kBoxK;
+          for (int b0 = 0; b0 < nbox; b0 += s.kb) {
+            const int nb = min(s.kb, nbox - b0);
+            for (int mi = 0; mi < s.mtiles; ++mi) {
+              mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
+              tc_fence_after();
+              for (int bi = 0; bi < nb; ++bi) {
+                const int box = b0 + bi;
+                const uint32_t a_box = ring_u + (uint32_t)rp.stage * kStageBytes + (uint32_t)bi * s.region;
+                const uint32_t b_box = xbuf_u + (uint32_t)buf * kXBufBytes + (uint32_t)box * kXBoxBytes;
+                const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
+                for (int s4 = 0; s4 < nstep; ++s4) {
+                  umma_bf16(tmem_base + mi * 32, umma_desc(a_box + s4 * 32), umma_desc(b_box + s4 * 32),
+                            (started >> mi) & 1u);
+                  started |= 1u << mi;
+                }
+              }
+              umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
+              rp.advance();
+            }
+          }
+          umma_commit(&xempty[buf]);
+        }
+        umma_commit(accfull);
+      }
+    }
+    __syncwarp();
+    // the workers signal when their last read of tensor memory is done
+    tc_fence_before();
+    named_bar(5, 32 + kNumCWarps * 32);
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+    return;
+  }
+  if (warp == 3) return;
+
+  // ================================================================= activation producer + workers
   const bool is_xprod = warp == 1;
-  const int cw = warp - 2;                 // consumer warp index 0..7 (consumers only)
+  const int cw = warp - kFirstWorker;      // worker warp index 0..7 (workers only)
   const int g8 = lane >> 2, q4 = lane & 3;
-  const int ntid = tid - 32;               // index among the 288 non-weight-producer threads
+  const int ntid = is_xprod ? lane : 32 + (tid - kFirstWorker * 32);   // index among the 288 barrier participants
   const int nnth = (kNumXWarps + kNumCWarps) * 32;
-  const int ctid = tid - 64;               // index among the 256 consumer threads
+  const int ctid = tid - kFirstWorker * 32;   // index among the 256 worker threads
   unsigned epoch = 0;
   RingPos rp{0, 0};
-  int xcount = 0;   // activation chunks produced / consumed so far (buffer = xcount % kXBufs)
+  int xcount = 0;   // activation chunks produced so far (buffer = xcount % kXBufs)
+  unsigned acc_phase = 0;   // GEMM phases of this CTA whose accumulator has been awaited
+  (void)g8; (void)q4; (void)rp;
 
   for (int ph = 0; ph < nphase; ++ph) {
     int layer;
@@ -445,7 +579,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         }
         if (kind == PH_EMBED) {
           ss = warp_sum(ss);
-          if (lane == 0) red[(warp - 1) * 16 + t] = ss;
+          if (lane == 0) red[(ntid >> 5) * 16 + t] = ss;
         }
       }
       if (kind == PH_EMBED) {
@@ -662,7 +796,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     const int nchunk = (g.K + kKc - 1) / kKc;
 
     if (is_xprod) {
-      // ---- activation producer: the input planes of this GEMM, chunk by chunk, by bulk copies
+      // ---- activation producer: the input planes of this GEMM, chunk by chunk, by TMA.
+      // Shared-memory layout of a chunk: per 64-k box, 16 hi rows then 16 lo rows (one 32-row B tile).
       if (s.rows > 0) {
         const int plane = lane >> 2, box = lane & 3;           // lanes 0..7: (plane, box)
         const int y0 = g.lm_rows ? p.pass->lm_row[0] : 0;       // draft LM head: its single row
@@ -673,10 +808,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             __syncwarp();
           }
           const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
-          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(2 * nbox * kXBoxBytes));
+          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(nbox * kXBoxBytes));
           __syncwarp();
           if (lane < 8 && box < nbox)
-            tma_load_2d(xbuf + (size_t)buf * kXBufBytes + (size_t)plane * kXPlaneBytes + (size_t)box * kXBoxBytes,
+            tma_load_2d(xbuf + (size_t)buf * kXBufBytes + (size_t)box * kXBoxBytes + (size_t)plane * (kXBoxBytes / 2),
                         p.maps + g.xmap + plane, c * kKc + box * kBoxK, y0, &xfull[buf]);
         }
       }
@@ -684,15 +819,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       continue;
     }
 
-    // ---- consumers
+    // ---- workers: wait for the accumulator, then the epilogue straight out of tensor memory
     const bool stamper = cta == 0 && ctid == 0;
     stamp(p, ph, 0, stamper);
-    // 1/rms per row of h for phases whose input was h * gain; features of the rows (target LM phase)
+    // 1/rms per row of h for phases whose input was h * gain (partials summed in CTA order)
     if (g.scale_inv_rms) {
-      if (ctid < 16) {
-        float ssum = 0.f;
-        for (int i = 0; i < ncta; ++i) ssum += __ldcg(p.ss_part + (size_t)i * 16 + ctid);
-        inv_rms[ctid] = rsqrtf(ssum / (float)p.d + p.eps);
+      if (cw < 2) {   // 16 rows over two warps; lanes stride over the CTAs, fixed shuffle tree
+        for (int rr = 0; rr < 8; ++rr) {
+          const int t = cw * 8 + rr;
+          float ssum = 0.f;
+          for (int i = lane; i < ncta; i += 32) ssum += __ldcg(p.ss_part + (size_t)i * 16 + t);
+          ssum = warp_sum(ssum);
+          if (lane == 0) inv_rms[t] = rsqrtf(ssum / (float)p.d + p.eps);
+        }
       }
       named_bar(3, kNumCWarps * 32);
     }
@@ -712,134 +851,52 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         }
       }
     }
-    // tile ownership: mt <= 8 tiles (single matrix): tile = cw / ksplit, k blocks split ksplit ways;
-    // otherwise warp cw owns list tiles cw and cw + 8 (SWIGLU: gate tile cw and up tile cw + mt).
-    int tileA = -1, tileB = -1, ksplit = 1, kpart = 0;
-    if (g.epi == EPI_SWIGLU_ACT) {
-      if (cw < s.mt) { tileA = cw; tileB = cw; }
-    } else if (s.mt <= 8) {
-      ksplit = s.mt <= 1 ? 8 : (s.mt == 2 ? 4 : (s.mt <= 4 ? 2 : 1));
-      if (cw / ksplit < s.mt) { tileA = cw / ksplit; kpart = cw % ksplit; }
-    } else {
-      tileA = cw; if (cw + 8 < s.mt) tileB = cw + 8;
-    }
-    float acc[2][2][4];
+    stamp(p, ph, 1, stamper);
+    const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
+    const bool sw = g.epi == EPI_SWIGLU_ACT;
+    // thread <-> weight row: quarter = warp index mod 4 (the tensor-memory lanes this warp may read),
+    // m tile = worker index / 4 (SWIGLU: the first four workers read both accumulators)
+    const int quarter = warp & 3, mi = sw ? 0 : (cw >> 2);
+    const int rloc = quarter * 32 + lane;                       // row inside the m tile
+    const bool active_warp = s.rows > 0 && (sw ? cw < 4 : mi < s.mtiles);
+    const int rslab = mi * s.box_rows + rloc;                   // row inside the slab
+    const bool valid = active_warp && rloc < s.box_rows && rslab < s.rows;
+    const int vrow = s.seg * g.Nseg + s.r0 + rslab;             // output column
+    float ssl[16];
+    Top2 tb[16];
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-      for (int i = 0; i < 2; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[a][i][j] = 0.f;
+    for (int t = 0; t < 16; ++t) { ssl[t] = 0.f; tb[t].v1 = -INFINITY; tb[t].i1 = 0x7fffffff; tb[t].v2 = -INFINITY; }
 
     if (s.rows > 0) {
-      const int spw = 16 / ksplit;   // k16 steps of a chunk this warp handles
-      // ldmatrix lane addressing inside a 128-byte-swizzled box (row pitch 128 B, 16-byte chunk index
-      // XORed with row & 7): A = weight tile rows, B = activation rows
-      const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_sel = lane >> 4;
-      const int b_row = (lane & 7) + ((lane >> 4) & 1) * 8, b_sel = (lane >> 3) & 1;
-      const uint32_t ring_u = smem_u32(ring), xbuf_u = smem_u32(xbuf);
-      for (int c = 0; c < nchunk; ++c, ++xcount) {
-        const int buf = xcount % kXBufs;
-        mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
-        if (c == 0) stamp(p, ph, 1, stamper);
-        const uint32_t xh = xbuf_u + (uint32_t)buf * kXBufBytes, xl = xh + kXPlaneBytes;
-        const int nstep = (min(kKc, g.K - c * kKc) + 15) >> 4;   // k16 steps that hold any k < K
-        for (int sr = 0; sr < s.nstage_rows; ++sr) {
-          mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
-          const uint32_t st = ring_u + (uint32_t)rp.stage * kStageBytes;
-          int map, row0, pair, which;
-          stage_source(g, s, sr, map, row0, pair, which);
-#pragma unroll
-          for (int slot = 0; slot < 2; ++slot) {
-            const int tile = slot ? tileB : tileA;
-            // slot 0 holds tiles of matrix 0 (or the only one), slot 1 of the up matrix / second tile
-            const bool mine = tile >= 0 && (tile >> 1) == pair &&
-                              (g.epi == EPI_SWIGLU_ACT ? which == slot : true);
-            if (mine) {
-              const uint32_t a_tile = st + (uint32_t)((tile & 1) * 16 + a_row) * 128;
-#pragma unroll 4
-              for (int si = 0; si < spw; ++si) {
-                const int ks = kpart * spw + si;
-                if (ks < nstep) {
-                  const int box = ks >> 2, s4 = ks & 3;
-                  uint32_t a0, a1, a2, a3, h0, h1, h2, h3, l0, l1, l2, l3;
-                  ldmatrix_x4(a_tile + box * kWBoxBytes + (((2 * s4 + a_sel) ^ (lane & 7)) << 4), a0, a1, a2, a3);
-                  const uint32_t boff = box * kXBoxBytes + b_row * 128 + (((2 * s4 + b_sel) ^ (lane & 7)) << 4);
-                  ldmatrix_x4(xh + boff, h0, h1, h2, h3);
-                  ldmatrix_x4(xl + boff, l0, l1, l2, l3);
-                  mma_bf16(acc[slot][0], a0, a1, a2, a3, h0, h1);
-                  mma_bf16(acc[slot][0], a0, a1, a2, a3, l0, l1);
-                  if (nt_act > 1) {
-                    mma_bf16(acc[slot][1], a0, a1, a2, a3, h2, h3);
-                    mma_bf16(acc[slot][1], a0, a1, a2, a3, l2, l3);
-                  }
-                }
-              }
-            }
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&empty[rp.stage]);
-          rp.advance();
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&xempty[buf]);
-      }
+      mbar_wait(accfull, acc_phase & 1u, p.cnt, abort_s);
+      ++acc_phase;
+      tc_fence_after();
     }
-
     stamp(p, ph, 2, stamper);
-    // ---- k-split reduction inside the CTA (fixed order), then the epilogue by the owner warps
-    if (ksplit > 1) {
-      float *mine = red + (size_t)(cw * 32 + lane) * 8;
+    if (active_warp) {
+      float v[32], u[32];
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * 32);
+      tmem_ld32(taddr, v);
+      if (sw) tmem_ld32(taddr + 32, u);
+      if (valid) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) mine[i * 4 + j] = acc[0][i][j];
-      named_bar(3, kNumCWarps * 32);
-      if (kpart == 0 && tileA >= 0) {
-        for (int s2 = 1; s2 < ksplit; ++s2) {
-          const float *oth = red + (size_t)((cw + s2) * 32 + lane) * 8;
-#pragma unroll
-          for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[0][i][j] += oth[i * 4 + j];
-        }
-      }
-    }
-    const bool owner = tileA >= 0 && kpart == 0 && s.rows > 0;
-    const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
-    float ssl[4] = {0.f, 0.f, 0.f, 0.f};   // sums of squares for pass rows 8*i + 2*q4 + (j&1)
-    Top2 tb[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { tb[i].v1 = -INFINITY; tb[i].i1 = 0x7fffffff; tb[i].v2 = -INFINITY; }
-
-    if (owner) {
-#pragma unroll
-      for (int slot = 0; slot < 2; ++slot) {
-        const int tile = slot ? tileB : tileA;
-        if (tile < 0 || (g.epi == EPI_SWIGLU_ACT && slot == 1)) continue;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          if (i >= nt_act) continue;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int rr = g8 + 8 * (j >> 1), t = 8 * i + 2 * q4 + (j & 1);
-            const int vrow = s.seg * g.Nseg + s.r0 + tile * 16 + rr;   // output column
-            if (tile * 16 + rr >= s.rows || t >= Tg) continue;
+        for (int t = 0; t < 16; ++t) {
+          if (t < Tg) {
             const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
-            const float y = acc[slot][i][j] * sc;
+            const float y = (v[t] + v[16 + t]) * sc;
             if (g.epi == EPI_STORE_QKV) {
               p.qkv[(size_t)t * 3 * p.d + vrow] = y;
-            } else if (g.epi == EPI_RESID_H || g.epi == EPI_STORE_H) {
+            } else if (has_ss) {
               float *hp = p.h + (size_t)t * p.d + vrow;
               const float hn = g.epi == EPI_RESID_H ? __ldcg(hp) + y : y;
               *hp = hn;
-              ssl[i * 2 + (j & 1)] += hn * hn;
+              ssl[t] = hn * hn;
               const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
               __nv_bfloat16 hi, lo;
               split_bf16(hn * gn, hi, lo);
               p.xa_hi[(size_t)t * p.d + vrow] = hi; p.xa_lo[(size_t)t * p.d + vrow] = lo;
-            } else if (g.epi == EPI_SWIGLU_ACT) {
-              const float up = acc[1][i][j] * sc;
+            } else if (sw) {
+              const float up = (u[t] + u[16 + t]) * sc;
               __nv_bfloat16 hi, lo;
               split_bf16((y / (1.f + __expf(-y))) * up, hi, lo);
               p.ac_hi[(size_t)t * p.F + vrow] = hi; p.ac_lo[(size_t)t * p.F + vrow] = lo;
@@ -848,35 +905,35 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
                 p.logits[(size_t)slot_out * p.V + vrow] = y;
               }
-              Top2 cnd; cnd.v1 = y; cnd.i1 = vrow; cnd.v2 = -INFINITY;
-              tb[i * 2 + (j & 1)] = top2_merge(tb[i * 2 + (j & 1)], cnd);
+              tb[t].v1 = y; tb[t].i1 = vrow;
             }
           }
         }
       }
     }
+    tc_fence_before();
     if (has_ss) {
-      // reduce over the 8 row groups of the warp, then over warps in order, one value per pass row
+      // per pass row: sum over the warp's 32 weight rows, then over the warps in order
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float v = ssl[i];
-        v += __shfl_xor_sync(0xffffffffu, v, 4);
-        v += __shfl_xor_sync(0xffffffffu, v, 8);
-        v += __shfl_xor_sync(0xffffffffu, v, 16);
-        if (g8 == 0) ssw[cw * 16 + (i >> 1) * 8 + 2 * q4 + (i & 1)] = v;
+      for (int t = 0; t < 16; ++t) {
+        const float r = warp_sum(ssl[t]);
+        if (lane == 0) ssw[cw * 16 + t] = r;
       }
       named_bar(3, kNumCWarps * 32);
       if (cw == 0 && lane < 16) {
-        float v = 0.f;
-        for (int w = 0; w < kNumCWarps; ++w) v += ssw[w * 16 + lane];
-        p.ss_part[(size_t)cta * 16 + lane] = v;
+        float r = 0.f;
+        for (int w = 0; w < kNumCWarps; ++w) r += ssw[w * 16 + lane];
+        p.ss_part[(size_t)cta * 16 + lane] = r;
       }
     } else if (g.epi == EPI_ARGMAX_LM) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        Top2 b = tb[i];
-        b = top2_shfl_xor(b, 4); b = top2_shfl_xor(b, 8); b = top2_shfl_xor(b, 16);
-        if (g8 == 0) topw[cw * 16 + (i >> 1) * 8 + 2 * q4 + (i & 1)] = b;
+      for (int t = 0; t < 16; ++t) {
+        Top2 b = tb[t];
+        if (t < Tg) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+        }
+        if (lane == 0) topw[cw * 16 + t] = b;
       }
       named_bar(3, kNumCWarps * 32);
       if (cw == 0 && lane < 16) {
@@ -901,6 +958,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
       if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
     }
+  }
+  // let warp 2 free the tensor memory once every worker has made its last read
+  if (!is_xprod) {
+    tc_fence_before();
+    named_bar(5, 32 + kNumCWarps * 32);
   }
 }
 
