@@ -27,9 +27,8 @@
 //   warp 0        weight producer: walks the static schedule of (phase, k chunk, k boxes, m tile) stages
 //   warp 1        activation producer: per GEMM phase (after the grid barrier that makes its input
 //                 visible) copies the input planes chunk by chunk into shared memory
-//   warp 2        tensor-memory allocation; its lane 0 issues every tcgen05.mma and commit
-//   warp 3        idle (keeps the workers on warp indices whose index mod 4 spans the four
-//                 tensor-memory lane quarters)
+//   warps 2, 3    lane 0 of each issues tcgen05.mma and commit (two issuers: one thread's issue
+//                 rate is too low for short slabs); warp 2 also owns the tensor-memory allocation
 //   warps 4..11   workers: epilogues out of tensor memory (tcgen05.ld: one weight row per thread),
 //                 attention, row-wise phases
 //
@@ -190,12 +189,15 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = 128, N = 32, K = 16
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = 128 or 64, N = 32, K = 16
+// (M = 64 for slabs of at most 64 rows: the tensor core then reads half as much of the A tile)
+__host__ __device__ constexpr uint32_t umma_idesc(uint32_t m) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed
@@ -309,6 +311,7 @@ struct Slab {
   int box_rows;     // rows per m tile = box height of the tensor map
   int region;       // bytes of one box in shared memory (box_rows rounded up to 8, times 128)
   int kb;           // boxes per stage
+  int m64;          // 1: M = 64 products (accumulator row i in lane (i % 16) + 32 * (i / 16))
 };
 __host__ __device__ __forceinline__ int slab_rpc(int Nseg, int nseg, int ncta) {
   const int cps = ncta / nseg;
@@ -332,6 +335,7 @@ __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) 
   if (!sw && s.rows <= s.box_rows) s.mtiles = 1;  // a short last slab may not reach the second tile
   s.region = ((s.box_rows + 7) & ~7) * 128;
   s.kb = s.region <= 4096 ? 4 : (s.region <= 8192 ? 2 : 1);
+  s.m64 = s.box_rows <= 64;
   return s;
 }
 // m tile mi -> weight map index and first row
@@ -414,8 +418,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
-    mbar_init(accfull, 1);
+    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 2); }
+    mbar_init(accfull, 2);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(tmem_slot, kTmemCols);
@@ -469,8 +473,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     return;
   }
 
-  // ================================================================= tensor-core issuer
-  if (warp == 2) {
+  // ================================================================= tensor-core issuers (warps 2 and 3)
+  // One thread's tcgen05.mma issue rate (about 55 cycles each) is below what a 28-row slab needs, so
+  // two threads issue.  With two m tiles issuer i owns m tile i; with one m tile the issuers take
+  // alternate stages and accumulate into tensor-memory regions 0 and 1, which the epilogue adds in
+  // that order.  Every product of an accumulator is thus issued by one thread, in schedule order.
+  if (warp == 2 || warp == 3) {
+    const int me = warp - 2;
     if (lane == 0) {
       RingPos rp{0, 0};
       int xcount = 0;
@@ -484,38 +493,50 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         const Slab s = make_slab(g, cta, ncta);
         if (s.rows == 0) continue;
         const int nchunk = (g.K + kKc - 1) / kKc;
-        unsigned started = 0;   // bit mi set once accumulator mi holds a product of this phase
+        const uint32_t idesc = umma_idesc(s.m64 ? 64u : 128u);
+        const uint32_t region16 = (uint32_t)s.region >> 4;
+        uint32_t started = 0;   // this issuer's accumulator holds a product of this phase
+        int sidx = 0;           // stage index inside the phase
         for (int c = 0; c < nchunk; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
-          mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
           const int kleft = min(kKc, g.K - c * kKc);
           const int nbox = (kleft + kBoxK - 1) / kBoxK;
+          const uint64_t bdesc0 = umma_desc(xbuf_u + (uint32_t)buf * kXBufBytes);
+          // both issuers wait for the chunk even if only one has a stage in it: an issuer can then never
+          // release a buffer twice before the other has released it once
+          mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
           for (int b0 = 0; b0 < nbox; b0 += s.kb) {
             const int nb = min(s.kb, nbox - b0);
-            for (int mi = 0; mi < s.mtiles; ++mi) {
-              mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
-              tc_fence_after();
-              for (int bi = 0; bi < nb; ++bi) {
-                const int box = b0 + bi;
-                const uint32_t a_box = ring_u + (uint32_t)rp.stage * kStageBytes + (uint32_t)bi * s.region;
-                const uint32_t b_box = xbuf_u + (uint32_t)buf * kXBufBytes + (uint32_t)box * kXBoxBytes;
-                const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
-                for (int s4 = 0; s4 < nstep; ++s4) {
-                  umma_bf16(tmem_base + mi * 32, umma_desc(a_box + s4 * 32), umma_desc(b_box + s4 * 32),
-                            (started >> mi) & 1u);
-                  started |= 1u << mi;
+            for (int mi = 0; mi < s.mtiles; ++mi, ++sidx) {
+              const bool mine = (s.mtiles == 2 ? mi : (sidx & 1)) == me;
+              if (mine) {
+                const uint64_t adesc0 = umma_desc(ring_u + (uint32_t)rp.stage * kStageBytes);
+                const uint32_t dcol = tmem_base + (uint32_t)(s.mtiles == 2 ? mi : me) * 32;
+                mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
+                tc_fence_after();
+                for (int bi = 0; bi < nb; ++bi) {
+                  const int box = b0 + bi;
+                  const uint64_t ad = adesc0 + (uint64_t)(bi * region16);
+                  const uint64_t bd = bdesc0 + (uint64_t)(box * (kXBoxBytes >> 4));
+                  const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
+                  for (int s4 = 0; s4 < nstep; ++s4) {
+                    umma_bf16(dcol, ad + 2 * s4, bd + 2 * s4, idesc, started);   // + 32 bytes per k16 step
+                    started = 1;
+                  }
                 }
+                umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
               }
-              umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
               rp.advance();
             }
           }
+          // both issuers release the chunk (an issuer with no stage in it releases it at once)
           umma_commit(&xempty[buf]);
         }
         umma_commit(accfull);
       }
     }
     __syncwarp();
+    if (warp == 3) return;
     // the workers signal when their last read of tensor memory is done
     tc_fence_before();
     named_bar(5, 32 + kNumCWarps * 32);
@@ -523,7 +544,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     tmem_dealloc(tmem_base, kTmemCols);
     return;
   }
-  if (warp == 3) return;
 
   // ================================================================= activation producer + workers
   const bool is_xprod = warp == 1;
@@ -824,13 +844,16 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     stamp(p, ph, 0, stamper);
     // 1/rms per row of h for phases whose input was h * gain (partials summed in CTA order)
     if (g.scale_inv_rms) {
-      if (cw < 2) {   // 16 rows over two warps; lanes stride over the CTAs, fixed shuffle tree
-        for (int rr = 0; rr < 8; ++rr) {
-          const int t = cw * 8 + rr;
-          float ssum = 0.f;
-          for (int i = lane; i < ncta; i += 32) ssum += __ldcg(p.ss_part + (size_t)i * 16 + t);
-          ssum = warp_sum(ssum);
-          if (lane == 0) inv_rms[t] = rsqrtf(ssum / (float)p.d + p.eps);
+      {   // two rows per worker warp; lanes stride over the CTAs, fixed shuffle tree
+        float s0 = 0.f, s1 = 0.f;
+        for (int i = lane; i < ncta; i += 32) {
+          s0 += __ldcg(p.ss_part + (size_t)i * 16 + 2 * cw);
+          s1 += __ldcg(p.ss_part + (size_t)i * 16 + 2 * cw + 1);
+        }
+        s0 = warp_sum(s0); s1 = warp_sum(s1);
+        if (lane == 0) {
+          inv_rms[2 * cw] = rsqrtf(s0 / (float)p.d + p.eps);
+          inv_rms[2 * cw + 1] = rsqrtf(s1 / (float)p.d + p.eps);
         }
       }
       named_bar(3, kNumCWarps * 32);
@@ -854,10 +877,15 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     stamp(p, ph, 1, stamper);
     const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
     const bool sw = g.epi == EPI_SWIGLU_ACT;
+    int nstages_phase = 0;   // ring stages of this phase in this CTA (as the issuers count them)
+    for (int c = 0; c < nchunk; ++c) {
+      const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
+      nstages_phase += ((nbox + s.kb - 1) / s.kb) * s.mtiles;
+    }
     // thread <-> weight row: quarter = warp index mod 4 (the tensor-memory lanes this warp may read),
     // m tile = worker index / 4 (SWIGLU: the first four workers read both accumulators)
     const int quarter = warp & 3, mi = sw ? 0 : (cw >> 2);
-    const int rloc = quarter * 32 + lane;                       // row inside the m tile
+    const int rloc = s.m64 ? (lane < 16 ? quarter * 16 + lane : 1 << 20) : quarter * 32 + lane;   // row inside the m tile
     const bool active_warp = s.rows > 0 && (sw ? cw < 4 : mi < s.mtiles);
     const int rslab = mi * s.box_rows + rloc;                   // row inside the slab
     const bool valid = active_warp && rloc < s.box_rows && rslab < s.rows;
@@ -878,7 +906,16 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * 32);
       tmem_ld32(taddr, v);
       if (sw) tmem_ld32(taddr + 32, u);
+      else if (s.mtiles == 1 && nstages_phase >= 2) {   // one m tile: issuer 1's share sits in region 1
+        tmem_ld32(taddr + 32, u);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] += u[i];
+      }
       if (valid) {
+        float hold[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t)
+          hold[t] = (g.epi == EPI_RESID_H && t < Tg) ? __ldcg(p.h + (size_t)t * p.d + vrow) : 0.f;
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           if (t < Tg) {
@@ -888,7 +925,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               p.qkv[(size_t)t * 3 * p.d + vrow] = y;
             } else if (has_ss) {
               float *hp = p.h + (size_t)t * p.d + vrow;
-              const float hn = g.epi == EPI_RESID_H ? __ldcg(hp) + y : y;
+              const float hn = hold[t] + y;
               *hp = hn;
               ssl[t] = hn * hn;
               const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
