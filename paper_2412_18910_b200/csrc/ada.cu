@@ -67,7 +67,7 @@ struct ada_ctx {
   TensorMap128 *d_maps;
   int n_maps;
   float *ss_part, *attn_part2;
-  bf16 *xa_hi, *xa_lo, *at_hi, *at_lo, *ac_hi, *ac_lo, *fc_hi, *fc_lo;
+  bf16 *xa, *at, *ac, *fc;            // activation tiles (xstore layout), 2048 elements per 64 k
   int *attn_cnt;
   float4 *amax2;
   unsigned *gbar;
@@ -227,10 +227,10 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->d_eagle = w.take<LayerPtrs>(1);
   x->n_maps = (int)(7 * (L + 1) + 2 + 8);
   x->d_maps = w.take<TensorMap128>(x->n_maps);
-  x->xa_hi = w.take<bf16>(16 * d); x->xa_lo = w.take<bf16>(16 * d);
-  x->at_hi = w.take<bf16>(16 * d); x->at_lo = w.take<bf16>(16 * d);
-  x->ac_hi = w.take<bf16>(16 * F); x->ac_lo = w.take<bf16>(16 * F);
-  x->fc_hi = w.take<bf16>(32 * d); x->fc_lo = w.take<bf16>(32 * d);
+  x->xa = w.take<bf16>(((d + 63) / 64) * 2048);
+  x->at = w.take<bf16>(((d + 63) / 64) * 2048);
+  x->ac = w.take<bf16>(((F + 63) / 64) * 2048);
+  x->fc = w.take<bf16>(((2 * d + 63) / 64) * 2048);
   x->ss_part = w.take<float>(256 * 16);
   x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
   x->attn_cnt = w.take<int>(H);
@@ -398,11 +398,6 @@ bool build_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
   layer(7 * c.n_layers, x->eagle);
   const int m0 = 7 * (c.n_layers + 1);
   ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, b_d) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, b_v);
-  const int pl = m0 + 2;
-  ok = ok && encode_map(fn, &maps[pl + MAPX_XA], x->xa_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_XA + 1], x->xa_lo, 16, d, 16) &&
-       encode_map(fn, &maps[pl + MAPX_AT], x->at_hi, 16, d, 16) && encode_map(fn, &maps[pl + MAPX_AT + 1], x->at_lo, 16, d, 16) &&
-       encode_map(fn, &maps[pl + MAPX_AC], x->ac_hi, 16, F, 16) && encode_map(fn, &maps[pl + MAPX_AC + 1], x->ac_lo, 16, F, 16) &&
-       encode_map(fn, &maps[pl + MAPX_FC], x->fc_hi, 16, 2 * d, 16) && encode_map(fn, &maps[pl + MAPX_FC + 1], x->fc_lo, 16, 2 * d, 16);
   return ok;
 }
 
@@ -435,8 +430,7 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.embed = x->embed; p.lm_head = x->lm_head; p.final_norm = x->final_norm; p.eagle_fc = x->eagle_fc;
   p.mode = mode; p.draft_step = step; p.with_lm = with_lm;
   p.h = x->h; p.qkv = x->qkv; p.ss_part = x->ss_part;
-  p.xa_hi = x->xa_hi; p.xa_lo = x->xa_lo; p.at_hi = x->at_hi; p.at_lo = x->at_lo;
-  p.ac_hi = x->ac_hi; p.ac_lo = x->ac_lo; p.fc_hi = x->fc_hi; p.fc_lo = x->fc_lo;
+  p.xa = x->xa; p.at = x->at; p.ac = x->ac; p.fc = x->fc;
   p.feat = x->feat; p.cap = c.kv_capacity; p.dfeat = x->dfeat; p.nmax = c.n_max;
   p.rope = x->rope;
   p.kpool = mode == 0 ? x->tk : x->dk; p.vpool = mode == 0 ? x->tv : x->dv;
@@ -606,14 +600,10 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       if (e == cudaSuccess) e = cudaMemcpy(x->d_maps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);
       // planes start finite: rows past the live ones are read by the tensor-core tiles
       const size_t dd = cfg->d_model, FF = cfg->d_ffn;
-      if (e == cudaSuccess) e = cudaMemset(x->xa_hi, 0, 32 * dd); 
-      if (e == cudaSuccess) e = cudaMemset(x->xa_lo, 0, 32 * dd);
-      if (e == cudaSuccess) e = cudaMemset(x->at_hi, 0, 32 * dd);
-      if (e == cudaSuccess) e = cudaMemset(x->at_lo, 0, 32 * dd);
-      if (e == cudaSuccess) e = cudaMemset(x->ac_hi, 0, 32 * FF);
-      if (e == cudaSuccess) e = cudaMemset(x->ac_lo, 0, 32 * FF);
-      if (e == cudaSuccess) e = cudaMemset(x->fc_hi, 0, 64 * dd);
-      if (e == cudaSuccess) e = cudaMemset(x->fc_lo, 0, 64 * dd);
+      if (e == cudaSuccess) e = cudaMemset(x->xa, 0, ((dd + 63) / 64) * 4096);
+      if (e == cudaSuccess) e = cudaMemset(x->at, 0, ((dd + 63) / 64) * 4096);
+      if (e == cudaSuccess) e = cudaMemset(x->ac, 0, ((FF + 63) / 64) * 4096);
+      if (e == cudaSuccess) e = cudaMemset(x->fc, 0, ((2 * dd + 63) / 64) * 4096);
       if (e == cudaSuccess) e = cudaMemset(x->attn_cnt, 0, sizeof(int) * cfg->n_heads);
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }

@@ -11,9 +11,10 @@
 // producer runs ahead across phase boundaries: while the other warps sit in a grid barrier or in
 // the attention phase, the ring is already filling with the next GEMM's weights.
 //
-// Every GEMM input lives in global memory already split into two bf16 planes (hi, lo), written by
-// the epilogue that produced it, so activations too are fetched by bulk copies with no conversion
-// on the way.  RMSNorm is folded around the GEMM: the producing epilogue stores split(h * gain) and
+// Every GEMM input lives in global memory already split into two bf16 planes (hi, lo) and already in
+// the swizzled tile layout the tensor core reads, written by the epilogue that produced it, so a
+// whole 256-k chunk of activations is one plain 16 KB bulk copy (tiled TMA loads of 128-byte rows
+// were measured to run out of request rate when activations shared them with the weights).  RMSNorm is folded around the GEMM: the producing epilogue stores split(h * gain) and
 // the per-row sum of squares; the consuming epilogue multiplies its accumulators by 1/rms(row).
 //
 // The contraction runs on the 5th-generation tensor cores: one thread issues tcgen05.mma
@@ -96,10 +97,11 @@ struct PassParams {
   int with_lm;                 // run the LM head
   // activations: fp32 residual stream and qkv; bf16 (hi, lo) planes of every GEMM input
   float *h, *qkv;              // [16][d], [16][3d]
-  __nv_bfloat16 *xa_hi, *xa_lo;   // [16][d]   h * gain of the norm that follows
-  __nv_bfloat16 *at_hi, *at_lo;   // [16][d]   attention output
-  __nv_bfloat16 *ac_hi, *ac_lo;   // [16][F]   SwiGLU output
-  __nv_bfloat16 *fc_hi, *fc_lo;   // [16][2d]  draft-head input [e ; f]
+  // each input is stored as tensor-core-ready tiles (see xstore): per 64 k one 4 KB box of 32 rows
+  __nv_bfloat16 *xa;              // K = d    h * gain of the norm that follows
+  __nv_bfloat16 *at;              // K = d    attention output
+  __nv_bfloat16 *ac;              // K = F    SwiGLU output
+  __nv_bfloat16 *fc;              // K = 2d   draft-head input [e ; f]
   float *ss_part;              // [grid][16] partial sums of squares of h
   float *feat; int cap;        // target features by position [seq][cap][d]
   float *dfeat; int nmax;      // draft features [seq][nmax][d]
@@ -229,6 +231,19 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
   return v;
 }
 
+// Activation tiles in global memory: for every 64 k one box of 32 rows x 128 bytes (rows 0..15 the hi
+// plane of pass rows 0..15, rows 16..31 the lo plane), with the 16-byte chunk index XORed with
+// (row & 7): exactly what a 128-byte-swizzle K-major operand looks like in shared memory, so a box
+// (or four of them) is copied verbatim.
+__device__ __forceinline__ void xstore(__nv_bfloat16 *tiles, int t, int k, float v) {
+  __nv_bfloat16 hi, lo;
+  split_bf16(v, hi, lo);
+  const int kk = k & 63;
+  const size_t o = (size_t)(k >> 6) * 2048 + (size_t)t * 64 + ((((kk >> 3) ^ (t & 7)) << 3) | (kk & 7));
+  tiles[o] = hi;
+  tiles[o + 16 * 64] = lo;   // row 16 + t: same (row & 7)
+}
+
 // ---------------------------------------------------------------------------------- GEMM phases
 
 enum { EPI_STORE_QKV = 0, EPI_RESID_H = 1, EPI_SWIGLU_ACT = 2, EPI_ARGMAX_LM = 3, EPI_STORE_H = 4 };
@@ -236,7 +251,7 @@ enum { EPI_STORE_QKV = 0, EPI_RESID_H = 1, EPI_SWIGLU_ACT = 2, EPI_ARGMAX_LM = 3
 struct GemmDesc {
   int wmap[3];                      // tensor maps of the weight matrices (segments, or gate / up)
   int nseg, Nseg, K, epi;
-  int xmap;                         // tensor map of the input's hi plane (lo plane = xmap + 1)
+  const __nv_bfloat16 *xt;          // input tiles (xstore layout)
   int scale_inv_rms;                // accumulators are multiplied by 1/rms(row) of h (input was h * gain)
   int lm_rows;                      // input rows are pass->lm_row[i] (draft LM head)
   const __nv_bfloat16 *gain_next;   // RESID_H / STORE_H: planes written are split(h * gain_next); null = no gain
@@ -269,29 +284,29 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
   switch (kind) {
     case PH_FC:
       g.wmap[0] = p.map_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H;
-      g.xmap = p.map_planes + MAPX_FC; g.gain_next = L.na;
+      g.xt = p.fc; g.gain_next = L.na;
       return true;
     case PH_QKV:
       g.wmap[0] = lm + MAP_WQ; g.wmap[1] = lm + MAP_WK; g.wmap[2] = lm + MAP_WV; g.nseg = 3; g.Nseg = p.d; g.K = p.d;
-      g.epi = EPI_STORE_QKV; g.xmap = p.map_planes + MAPX_XA; g.scale_inv_rms = 1;
+      g.epi = EPI_STORE_QKV; g.xt = p.xa; g.scale_inv_rms = 1;
       return true;
     case PH_O:
       g.wmap[0] = lm + MAP_WO; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H;
-      g.xmap = p.map_planes + MAPX_AT; g.gain_next = L.nm;
+      g.xt = p.at; g.gain_next = L.nm;
       return true;
     case PH_GATEUP:
       g.wmap[0] = lm + MAP_WG; g.wmap[1] = lm + MAP_WU; g.Nseg = p.F; g.K = p.d; g.epi = EPI_SWIGLU_ACT;
-      g.xmap = p.map_planes + MAPX_XA; g.scale_inv_rms = 1;
+      g.xt = p.xa; g.scale_inv_rms = 1;
       return true;
     case PH_DOWN:
       g.wmap[0] = lm + MAP_WD; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H;
-      g.xmap = p.map_planes + MAPX_AC;
+      g.xt = p.ac;
       // the norm that follows: next layer's, or the final one; the draft head has none after its layer
       g.gain_next = (layer + 1 < p.n_layers) ? p.layers[layer + 1].na : (p.mode == 0 ? p.final_norm : nullptr);
       return true;
     case PH_LM:
       g.wmap[0] = p.map_lm; g.Nseg = p.V; g.K = p.d; g.epi = EPI_ARGMAX_LM;
-      g.xmap = p.map_planes + MAPX_XA;
+      g.xt = p.xa;
       if (p.mode == 0) g.scale_inv_rms = 1; else g.lm_rows = 1;
       return true;
     default:
@@ -580,9 +595,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const float v = __bfloat162float(e[c]);
               p.h[(size_t)t * p.d + c] = v;
               ss += v * v;
-              __nv_bfloat16 hi, lo;
-              split_bf16(v * __bfloat162float(gain[c]), hi, lo);
-              p.xa_hi[(size_t)t * p.d + c] = hi; p.xa_lo[(size_t)t * p.d + c] = lo;
+              xstore(p.xa, t, c, v * __bfloat162float(gain[c]));
             } else {
               float v;
               if (c < p.d) v = __bfloat162float(e[c]);
@@ -591,9 +604,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                                                    : p.dfeat + ((size_t)b * p.nmax + (p.draft_step - 1)) * p.d;
                 v = __ldcg(f + (c - p.d));
               }
-              __nv_bfloat16 hi, lo;
-              split_bf16(v, hi, lo);
-              p.fc_hi[(size_t)t * 2 * p.d + c] = hi; p.fc_lo[(size_t)t * 2 * p.d + c] = lo;
+              xstore(p.fc, t, c, v);
             }
           }
         }
@@ -793,10 +804,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   oo += __ldcg(gp + s2 * sst + c) * e;
                 }
               }
-              __nv_bfloat16 hi, lw;
-              split_bf16(oo / lo, hi, lw);
-              p.at_hi[(size_t)r * d + hh * HD + c] = hi;
-              p.at_lo[(size_t)r * d + hh * HD + c] = lw;
+              xstore(p.at, r, hh * HD + c, oo / lo);
             }
             if (ctid == 0) p.attn_cnt[hh] = 0;
           }
@@ -816,23 +824,18 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     const int nchunk = (g.K + kKc - 1) / kKc;
 
     if (is_xprod) {
-      // ---- activation producer: the input planes of this GEMM, chunk by chunk, by TMA.
-      // Shared-memory layout of a chunk: per 64-k box, 16 hi rows then 16 lo rows (one 32-row B tile).
+      // ---- activation producer: the input tiles of this GEMM, one bulk copy per 256-k chunk
       if (s.rows > 0) {
-        const int plane = lane >> 2, box = lane & 3;           // lanes 0..7: (plane, box)
-        const int y0 = g.lm_rows ? p.pass->lm_row[0] : 0;       // draft LM head: its single row
         for (int c = 0; c < nchunk; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
-          if (xcount >= kXBufs) {
-            if (lane == 0) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
-            __syncwarp();
+          if (lane == 0) {
+            if (xcount >= kXBufs) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
+            const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
+            mbar_expect_tx(&xfull[buf], (unsigned)(nbox * kXBoxBytes));
+            bulk_g2s(xbuf + (size_t)buf * kXBufBytes, g.xt + (size_t)c * (kKc / kBoxK) * (kXBoxBytes / 2),
+                     (unsigned)(nbox * kXBoxBytes), &xfull[buf]);
           }
-          const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
-          if (lane == 0) mbar_expect_tx(&xfull[buf], (unsigned)(nbox * kXBoxBytes));
           __syncwarp();
-          if (lane < 8 && box < nbox)
-            tma_load_2d(xbuf + (size_t)buf * kXBufBytes + (size_t)box * kXBoxBytes + (size_t)plane * (kXBoxBytes / 2),
-                        p.maps + g.xmap + plane, c * kKc + box * kBoxK, y0, &xfull[buf]);
         }
       }
       grid_barrier(p, epoch, tid, abort_s);
@@ -920,7 +923,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         for (int t = 0; t < 16; ++t) {
           if (t < Tg) {
             const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
-            const float y = (v[t] + v[16 + t]) * sc;
+            float yy = v[t] + v[16 + t];   // accumulator column = pass row
+            if (g.lm_rows) {               // draft LM head: output row t is pass row lm_row[t]
+              const int col = p.pass->lm_row[t];
+              yy = 0.f;
+#pragma unroll
+              for (int cc = 0; cc < 16; ++cc) yy = (cc == col) ? v[cc] + v[16 + cc] : yy;
+            }
+            const float y = yy * sc;
             if (g.epi == EPI_STORE_QKV) {
               p.qkv[(size_t)t * 3 * p.d + vrow] = y;
             } else if (has_ss) {
@@ -929,14 +939,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               *hp = hn;
               ssl[t] = hn * hn;
               const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
-              __nv_bfloat16 hi, lo;
-              split_bf16(hn * gn, hi, lo);
-              p.xa_hi[(size_t)t * p.d + vrow] = hi; p.xa_lo[(size_t)t * p.d + vrow] = lo;
+              xstore(p.xa, t, vrow, hn * gn);
             } else if (sw) {
               const float up = (u[t] + u[16 + t]) * sc;
-              __nv_bfloat16 hi, lo;
-              split_bf16((y / (1.f + __expf(-y))) * up, hi, lo);
-              p.ac_hi[(size_t)t * p.F + vrow] = hi; p.ac_lo[(size_t)t * p.F + vrow] = lo;
+              xstore(p.ac, t, vrow, (y / (1.f + __expf(-y))) * up);
             } else {  // EPI_ARGMAX_LM
               if (p.logits) {
                 const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
