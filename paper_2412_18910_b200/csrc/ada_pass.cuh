@@ -202,6 +202,12 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// true in exactly one lane of the (converged) warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.b32 %0, 1, 0, P;\n}" : "=r"(pred));
+  return pred != 0;
+}
 // arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -494,8 +500,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   // alternate stages and accumulate into tensor-memory regions 0 and 1, which the epilogue adds in
   // that order.  Every product of an accumulator is thus issued by one thread, in schedule order.
   if (warp == 2 || warp == 3) {
-    const int me = warp - 2;
-    if (lane == 0) {
+    // The whole warp walks the loop so that descriptors and addresses stay warp-uniform (the compiler
+    // can keep them in uniform registers: issued from inside a one-lane branch each tcgen05.mma cost
+    // about 140 cycles instead of about 55); one elected lane issues.
+    const int me = __shfl_sync(0xffffffffu, warp, 0) - 2;
+    {
       RingPos rp{0, 0};
       int xcount = 0;
       const uint32_t ring_u = smem_u32(ring), xbuf_u = smem_u32(xbuf);
@@ -535,19 +544,22 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   const uint64_t bd = bdesc0 + (uint64_t)(box * (kXBoxBytes >> 4));
                   const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
                   for (int s4 = 0; s4 < nstep; ++s4) {
-                    umma_bf16(dcol, ad + 2 * s4, bd + 2 * s4, idesc, started);   // + 32 bytes per k16 step
+                    if (elect_one()) umma_bf16(dcol, ad + 2 * s4, bd + 2 * s4, idesc, started);   // + 32 bytes per k16 step
                     started = 1;
                   }
                 }
-                umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
+                if (elect_one()) umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
+                __syncwarp();
               }
               rp.advance();
             }
           }
           // both issuers release the chunk (an issuer with no stage in it releases it at once)
-          umma_commit(&xempty[buf]);
+          if (elect_one()) umma_commit(&xempty[buf]);
+          __syncwarp();
         }
-        umma_commit(accfull);
+        if (elect_one()) umma_commit(accfull);
+        __syncwarp();
       }
     }
     __syncwarp();
