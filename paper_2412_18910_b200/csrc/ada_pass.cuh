@@ -56,8 +56,8 @@ constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
-constexpr int kAttnLoopBytes = (3 * 16 * 128 + 8 * 16 * 32) * 4;   // q, k, v rows and softmax weights
-constexpr int kAttnPartBytes = 8 * 16 * 130 * 4;                   // per-warp partial results
+constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 8 * 32 * 4 + 4 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; staged values
+constexpr int kAttnPartBytes = 8 * 8 * 130 * 4;                    // per-warp partial results
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (the + 16 KB: a tensor-core read of 128 tile rows may run past a short last stage; it must stay inside the allocation)
 constexpr int kScratchBytes = ((kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes) + 16 * 1024;
@@ -435,12 +435,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   (void)red;
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
+  uint64_t *attn_bar = accfull + 1;                        // attention: values of a round have landed
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 2); }
     mbar_init(accfull, 2);
+    mbar_init(attn_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(tmem_slot, kTmemCols);
@@ -583,6 +585,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   RingPos rp{0, 0};
   int xcount = 0;   // activation chunks produced so far (buffer = xcount % kXBufs)
   unsigned acc_phase = 0;   // GEMM phases of this CTA whose accumulator has been awaited
+  unsigned attn_uses = 0;   // completed phases of the attention barrier
   (void)g8; (void)q4; (void)rp;
 
   for (int ph = 0; ph < nphase; ++ph) {
@@ -640,18 +643,26 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     // ------------------------------------------------------------- attention
     if (kind == PH_ATTN) {
       if (!is_xprod) {
-        // items (head, split) round-robin over CTAs; one sequence on this path
+        // Items (head, KV split) round-robin over CTAs; one sequence on this path.  Inside an item a
+        // round covers 4 blocks of 32 keys; warp w works on block w/2 for the query rows of parity
+        // w%2, lane = key while scoring, lane = 4 channels while accumulating values.  Values of a
+        // round arrive by one bulk copy per block (a block is contiguous in its cache page); keys are
+        // read straight from the cache, each lane its own row.
         const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
         const int nkeys = pos0 + R, nsp = p.attn_splits;
         int chunk = (nkeys + nsp - 1) / nsp;
         chunk = ((chunk + 31) / 32) * 32;
         const int b = p.pass->row_seq[0];
-        float *q_s = reinterpret_cast<float *>(xbuf);          // [16][128]
-        float *k_s = q_s + 16 * 128;                           // new rows, rotated, bf16-rounded [16][128]
-        float *v_s = k_s + 16 * 128;
-        float *p_s = v_s + 16 * 128;                           // [8][16][32]
-        float *part_s = q_s;                                   // [8][16][130], reuses the loop's scratch
+        float *q_s = reinterpret_cast<float *>(xbuf);                                 // [16][128] fp32
+        __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(q_s + 16 * 128);      // new rows, rotated [16][128]
+        __nv_bfloat16 *v_s = k_s + 16 * 128;
+        float *p_s = reinterpret_cast<float *>(v_s + 16 * 128);                       // [8 warps][8 rows][32 keys]
+        __nv_bfloat16 *vst = reinterpret_cast<__nv_bfloat16 *>(p_s + 8 * 8 * 32);    // [4 blocks][32 keys][HD]
+        float *part_s = q_s;                                                          // [8][8][130], reuses the above
         const int VPL = HD / 32;
+        const int rsel = cw & 1, bw = cw >> 1;
+        const int NR = (R - rsel + 1) >> 1;          // my rows: r = 2 i + rsel, i < NR
+        const size_t head_stride = (size_t)p.page_size * HD;
         for (int item = cta; item < p.H * nsp; item += ncta) {
           const int hh = item / nsp, split = item - hh * nsp;
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
@@ -664,131 +675,160 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const float *qr = p.qkv + (size_t)r * 3 * d + hh * HD;
             const float qa = __ldcg(qr + c), qb = __ldcg(qr + c + half);
             const float ka = __ldcg(qr + d + c), kb = __ldcg(qr + d + c + half);
+            const float va = __ldcg(qr + 2 * d + c), vb = __ldcg(qr + 2 * d + c + half);
             q_s[r * 128 + c] = (qa * cs.x - qb * cs.y) * qscale;
             q_s[r * 128 + c + half] = (qb * cs.x + qa * cs.y) * qscale;
             const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(qr + 2 * d + c));
-            const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(qr + 2 * d + c + half));
-            k_s[r * 128 + c] = __bfloat162float(k0); k_s[r * 128 + c + half] = __bfloat162float(k1);
-            v_s[r * 128 + c] = __bfloat162float(v0); v_s[r * 128 + c + half] = __bfloat162float(v1);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(va), v1 = __float2bfloat16_rn(vb);
+            k_s[r * 128 + c] = k0; k_s[r * 128 + c + half] = k1;
+            v_s[r * 128 + c] = v0; v_s[r * 128 + c + half] = v1;
             if (split == 0) {  // one item per head stores the new rows in the cache
               const int pos = pos0 + r;
               const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
-              const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD;
+              const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
               p.kpool[base + c] = k0; p.kpool[base + c + half] = k1;
               p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
             }
           }
-          named_bar(3, kNumCWarps * 32);
-          float m[16], l[16], o[16][4];
+          float m[8], l[8], o[8][4];
 #pragma unroll
-          for (int r = 0; r < 16; ++r) { m[r] = -INFINITY; l[r] = 0.f; o[r][0] = o[r][1] = o[r][2] = o[r][3] = 0.f; }
-          for (int kb = kbeg + cw * 32; kb < kend; kb += kNumCWarps * 32) {
-            const int key = kb + lane;
-            const bool kv = key < kend;
-            float sc[16];
+          for (int i = 0; i < 8; ++i) { m[i] = -INFINITY; l[i] = 0.f; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+          for (int r0 = kbeg; r0 < kend; r0 += 128) {
+            const int nblk = min(4, (kend - r0 + 31) >> 5);
+            named_bar(3, kNumCWarps * 32);   // staging visible; previous round's values no longer read
+            if (ctid == 0) {                 // values of this round: one bulk copy per 32-key block
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
+              mbar_expect_tx(attn_bar, (unsigned)(nblk * 32 * HD * 2));
+              for (int bb = 0; bb < nblk; ++bb) {
+                const int key0 = r0 + 32 * bb;
+                const int page = p.page_table[b * p.pages_per_seq + key0 / p.page_size], slot = key0 % p.page_size;
+                bulk_g2s(vst + (size_t)bb * 32 * HD,
+                         p.vpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD,
+                         (unsigned)(32 * HD * 2), attn_bar);
+              }
+            }
+            const int kb0 = r0 + 32 * bw;
+            const bool have = bw < nblk;
+            const int key = kb0 + lane;
+            const bool kv = have && key < kend;
+            float sc[8];
 #pragma unroll
-            for (int r = 0; r < 16; ++r) sc[r] = 0.f;
+            for (int i = 0; i < 8; ++i) sc[i] = 0.f;
             if (kv) {
               if (key >= pos0) {
-                const float *kr = k_s + (key - pos0) * 128;
-                for (int c = 0; c < HD; c += 4) {
-                  const float4 kk = *reinterpret_cast<const float4 *>(kr + c);
-#pragma unroll
-                  for (int r = 0; r < 16; ++r)
-                    if (r < R) {
-                      const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c);
-                      sc[r] += qa.x * kk.x + qa.y * kk.y + qa.z * kk.z + qa.w * kk.w;
-                    }
-                }
-              } else {
-                const int page = p.page_table[b * p.pages_per_seq + key / p.page_size], slot = key % p.page_size;
-                const uint4 *kr = reinterpret_cast<const uint4 *>(
-                    p.kpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD);
-                for (int c = 0; c < HD / 8; ++c) {
-                  const uint4 kk = kr[c];
+                const __nv_bfloat16 *kr = k_s + (key - pos0) * 128;
+                for (int c = 0; c < HD; c += 8) {
+                  const uint4 kk = *reinterpret_cast<const uint4 *>(kr + c);
                   float kf[8];
                   kf[0] = bf16_bits_to_float(kk.x & 0xffffu); kf[1] = bf16_bits_to_float(kk.x >> 16);
                   kf[2] = bf16_bits_to_float(kk.y & 0xffffu); kf[3] = bf16_bits_to_float(kk.y >> 16);
                   kf[4] = bf16_bits_to_float(kk.z & 0xffffu); kf[5] = bf16_bits_to_float(kk.z >> 16);
                   kf[6] = bf16_bits_to_float(kk.w & 0xffffu); kf[7] = bf16_bits_to_float(kk.w >> 16);
 #pragma unroll
-                  for (int r = 0; r < 16; ++r)
-                    if (r < R) {
-                      const float4 qa = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8);
-                      const float4 qb = *reinterpret_cast<const float4 *>(q_s + r * 128 + c * 8 + 4);
-                      sc[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                  for (int i = 0; i < 8; ++i)
+                    if (i < NR) {
+                      const float *qq = q_s + (2 * i + rsel) * 128 + c;
+                      const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
+                      sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
                                qb.z * kf[6] + qb.w * kf[7];
                     }
                 }
+              } else {
+                const int page = p.page_table[b * p.pages_per_seq + key / p.page_size], slot = key % p.page_size;
+                const uint4 *kr = reinterpret_cast<const uint4 *>(
+                    p.kpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD);
+                for (int c8 = 0; c8 < HD / 8; c8 += 8) {   // eight 16-byte loads in flight, then the arithmetic
+                  uint4 kq[8];
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) kq[u] = kr[c8 + u];
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) {
+                    float kf[8];
+                    kf[0] = bf16_bits_to_float(kq[u].x & 0xffffu); kf[1] = bf16_bits_to_float(kq[u].x >> 16);
+                    kf[2] = bf16_bits_to_float(kq[u].y & 0xffffu); kf[3] = bf16_bits_to_float(kq[u].y >> 16);
+                    kf[4] = bf16_bits_to_float(kq[u].z & 0xffffu); kf[5] = bf16_bits_to_float(kq[u].z >> 16);
+                    kf[6] = bf16_bits_to_float(kq[u].w & 0xffffu); kf[7] = bf16_bits_to_float(kq[u].w >> 16);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                      if (i < NR) {
+                        const float *qq = q_s + (2 * i + rsel) * 128 + (c8 + u) * 8;
+                        const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
+                        sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                                 qb.z * kf[6] + qb.w * kf[7];
+                      }
+                  }
+                }
               }
             }
+            if (have) {
 #pragma unroll
-            for (int r = 0; r < 16; ++r)
-              if (r < R) {
-                const bool seen = kv && key <= pos0 + r;
-                const float sv = seen ? sc[r] : -INFINITY;
-                const float mx = warp_max(sv);
-                const float mn = fmaxf(m[r], mx);
-                float pe = 0.f, corr = 1.f;
-                if (mn > -INFINITY) { pe = seen ? __expf(sv - mn) : 0.f; corr = __expf(m[r] - mn); }
-                l[r] = l[r] * corr + warp_sum(pe);
-                o[r][0] *= corr; o[r][1] *= corr; o[r][2] *= corr; o[r][3] *= corr;
-                m[r] = mn;
-                p_s[(cw * 16 + r) * 32 + lane] = pe;
-              }
-            __syncwarp();
-            const int nk = min(32, kend - kb);
-            for (int kk = 0; kk < nk; ++kk) {
-              const int key2 = kb + kk;
-              float vf[4] = {0.f, 0.f, 0.f, 0.f};
-              if (key2 >= pos0) {
-                const float *vr = v_s + (key2 - pos0) * 128 + lane * VPL;
-                for (int c = 0; c < VPL; ++c) vf[c] = vr[c];
-              } else {
-                const int page = p.page_table[b * p.pages_per_seq + key2 / p.page_size], slot = key2 % p.page_size;
-                const __nv_bfloat16 *vr =
-                    p.vpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * p.page_size * HD + (size_t)slot * HD;
+              for (int i = 0; i < 8; ++i)
+                if (i < NR) {
+                  const bool seen = kv && key <= pos0 + 2 * i + rsel;
+                  const float sv = seen ? sc[i] : -INFINITY;
+                  const float mx = warp_max(sv);
+                  const float mn = fmaxf(m[i], mx);
+                  float pe = 0.f, corr = 1.f;
+                  if (mn > -INFINITY) { pe = seen ? __expf(sv - mn) : 0.f; corr = __expf(m[i] - mn); }
+                  l[i] = l[i] * corr + warp_sum(pe);
+                  o[i][0] *= corr; o[i][1] *= corr; o[i][2] *= corr; o[i][3] *= corr;
+                  m[i] = mn;
+                  p_s[(cw * 8 + i) * 32 + lane] = pe;
+                }
+              __syncwarp();
+            }
+            // values: wait for this round's copies (every worker keeps the barrier's parity in step)
+            mbar_wait(attn_bar, attn_uses & 1u, p.cnt, abort_s);
+            ++attn_uses;
+            if (have) {
+              const int nk = min(32, kend - kb0);
+              const __nv_bfloat16 *vb = vst + (size_t)bw * 32 * HD;
+              for (int kk = 0; kk < nk; ++kk) {
+                const int key2 = kb0 + kk;
+                const __nv_bfloat16 *vr = (key2 >= pos0 ? v_s + (key2 - pos0) * 128 : vb + kk * HD) + lane * VPL;
+                float vf[4] = {0.f, 0.f, 0.f, 0.f};
                 if (VPL == 4) {
-                  const uint2 vv = *reinterpret_cast<const uint2 *>(vr + lane * 4);
+                  const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
                   vf[0] = bf16_bits_to_float(vv.x & 0xffffu); vf[1] = bf16_bits_to_float(vv.x >> 16);
                   vf[2] = bf16_bits_to_float(vv.y & 0xffffu); vf[3] = bf16_bits_to_float(vv.y >> 16);
                 } else {
-                  const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr + lane * 2);
+                  const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr);
                   vf[0] = bf16_bits_to_float(vv & 0xffffu); vf[1] = bf16_bits_to_float(vv >> 16);
                 }
-              }
 #pragma unroll
-              for (int r = 0; r < 16; ++r)
-                if (r < R) {
-                  const float pe = p_s[(cw * 16 + r) * 32 + kk];
-                  o[r][0] += pe * vf[0]; o[r][1] += pe * vf[1]; o[r][2] += pe * vf[2]; o[r][3] += pe * vf[3];
-                }
+                for (int i = 0; i < 8; ++i)
+                  if (i < NR) {
+                    const float pe = p_s[(cw * 8 + i) * 32 + kk];
+                    o[i][0] += pe * vf[0]; o[i][1] += pe * vf[1]; o[i][2] += pe * vf[2]; o[i][3] += pe * vf[3];
+                  }
+              }
             }
-            __syncwarp();
           }
           // per-warp partials -> shared (over the loop's scratch once every warp has left the loop),
-          // merged in warp order, stored per (head, split)
+          // merged over the four key blocks in block order, stored per (head, split)
           named_bar(3, kNumCWarps * 32);
 #pragma unroll
-          for (int r = 0; r < 16; ++r)
-            if (r < R) {
-              float *pp = part_s + (cw * 16 + r) * 130;
-              for (int c = 0; c < VPL; ++c) pp[lane * VPL + c] = o[r][c];
-              if (lane == 0) { pp[128] = m[r]; pp[129] = l[r]; }
+          for (int i = 0; i < 8; ++i)
+            if (i < NR) {
+              float *pp = part_s + (cw * 8 + i) * 130;
+              if (VPL == 4) { pp[lane * 4] = o[i][0]; pp[lane * 4 + 1] = o[i][1]; pp[lane * 4 + 2] = o[i][2]; pp[lane * 4 + 3] = o[i][3]; }
+              else { pp[lane * 2] = o[i][0]; pp[lane * 2 + 1] = o[i][1]; }
+              if (lane == 0) { pp[128] = m[i]; pp[129] = l[i]; }
             }
           named_bar(3, kNumCWarps * 32);
           for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
             const int r = i / HD, c = i - r * HD;
+            const int ri = r >> 1, rs = r & 1;
             float M = -INFINITY;
-            for (int w = 0; w < kNumCWarps; ++w) M = fmaxf(M, part_s[(w * 16 + r) * 130 + 128]);
+            for (int q = 0; q < 4; ++q) M = fmaxf(M, part_s[((2 * q + rs) * 8 + ri) * 130 + 128]);
             float lo = 0.f, oo = 0.f;
             if (M > -INFINITY)
-              for (int w = 0; w < kNumCWarps; ++w) {
-                const float e = __expf(part_s[(w * 16 + r) * 130 + 128] - M);
-                lo += part_s[(w * 16 + r) * 130 + 129] * e;
-                oo += part_s[(w * 16 + r) * 130 + c] * e;
+              for (int q = 0; q < 4; ++q) {
+                const float *pp = part_s + ((2 * q + rs) * 8 + ri) * 130;
+                const float e = __expf(pp[128] - M);
+                lo += pp[129] * e;
+                oo += pp[c] * e;
               }
             float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
             __stcg(gp + c, oo);
@@ -843,6 +883,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           if (lane == 0) {
             if (xcount >= kXBufs) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
             const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffer doubles as attention scratch
             mbar_expect_tx(&xfull[buf], (unsigned)(nbox * kXBoxBytes));
             bulk_g2s(xbuf + (size_t)buf * kXBufBytes, g.xt + (size_t)c * (kKc / kBoxK) * (kXBoxBytes / 2),
                      (unsigned)(nbox * kXBoxBytes), &xfull[buf]);
