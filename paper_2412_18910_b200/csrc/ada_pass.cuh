@@ -841,22 +841,43 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           named_bar(3, kNumCWarps * 32);
           if (*flag_s) {
             __threadfence();
-            for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
-              const int r = i / HD, c = i - r * HD;
+            // weights of the splits per row first (shared), then every output element is one pass of
+            // independent loads over the splits
+            float *wgt = p_s;   // [8 splits][16 rows]
+            if (ctid < 16 && ctid < R) {
+              const int r = ctid;
               const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2);
               const size_t sst = (size_t)16 * (HD + 2);
-              float M = -INFINITY;
-              for (int s2 = 0; s2 < nsp; ++s2) M = fmaxf(M, __ldcg(gp + s2 * sst + HD));
-              float lo = 0.f, oo = 0.f;
-              for (int s2 = 0; s2 < nsp; ++s2) {
-                const float ms = __ldcg(gp + s2 * sst + HD);
-                if (ms > -INFINITY) {
-                  const float e = __expf(ms - M);
-                  lo += __ldcg(gp + s2 * sst + HD + 1) * e;
-                  oo += __ldcg(gp + s2 * sst + c) * e;
-                }
+              float ms[8], ls[8];
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) {
+                ms[s2] = s2 < nsp ? __ldcg(gp + s2 * sst + HD) : -INFINITY;
+                ls[s2] = s2 < nsp ? __ldcg(gp + s2 * sst + HD + 1) : 0.f;
               }
-              xstore(p.at, r, hh * HD + c, oo / lo);
+              float M = -INFINITY;
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) M = fmaxf(M, ms[s2]);
+              float lo = 0.f;
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) {
+                ms[s2] = ms[s2] > -INFINITY ? __expf(ms[s2] - M) : 0.f;
+                lo += ls[s2] * ms[s2];
+              }
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) wgt[s2 * 16 + r] = ms[s2] / lo;
+            }
+            named_bar(3, kNumCWarps * 32);
+            for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
+              const int r = i / HD, c = i - r * HD;
+              const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2) + c;
+              const size_t sst = (size_t)16 * (HD + 2);
+              float ov[8];
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) ov[s2] = s2 < nsp ? __ldcg(gp + s2 * sst) : 0.f;
+              float oo = 0.f;
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) oo += ov[s2] * wgt[s2 * 16 + r];
+              xstore(p.at, r, hh * HD + c, oo);
             }
             if (ctid == 0) p.attn_cnt[hh] = 0;
           }
