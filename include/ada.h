@@ -124,7 +124,8 @@ int ada_step(ada_ctx *ctx, int32_t *d_emitted, int32_t *d_n_emitted, int32_t *d_
 int ada_force_n(ada_ctx *ctx, const int32_t *n);
 
 /* Teacher forcing: after every draft step the drafted token of sequence seq is replaced by
- * d_tokens[seq][step] (device, [max_batch][n_max]).  NULL switches it off. */
+ * d_tokens[seq][step] (device, [max_batch][n_max]).  The array is copied (stream-ordered) when the call is
+ * made; call again to change the tokens.  NULL switches it off. */
 int ada_force_draft(ada_ctx *ctx, const int32_t *d_tokens);
 
 /* Replace the outcome of the iteration that just ran for sequence `seq`: rewind to its start and

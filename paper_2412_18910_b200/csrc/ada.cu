@@ -54,7 +54,7 @@ struct ada_ctx {
   int ldx, ldx2;
   int *gemm_cnt;
   float4 *amax;
-  int *draft, *target, *force_n_dev, *chunk_tok;
+  int *draft, *target, *force_n_dev, *chunk_tok, *forced_buf;
   float2 *vtop, *dtop;
   float *chunk_logits_unused;
   const int *force_draft;           // user device pointer or null
@@ -216,6 +216,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->draft = w.take<int>(B * c->n_max);
   x->target = w.take<int>(B * (c->n_max + 1));
   x->force_n_dev = w.take<int>(B);
+  x->forced_buf = w.take<int>(B * c->n_max);
   x->chunk_tok = w.take<int>(kMaxRows);
   x->vtop = w.take<float2>(B * (c->n_max + 1) + kMaxRows);
   x->dtop = w.take<float2>(B * c->n_max + kMaxRows);
@@ -757,7 +758,13 @@ extern "C" int ada_force_n(ada_ctx *x, const int32_t *n) {
 
 extern "C" int ada_force_draft(ada_ctx *x, const int32_t *d_tokens) {
   if (!x) return ADA_ERR_NULL;
-  x->force_draft = d_tokens;
+  if (!d_tokens) { x->force_draft = nullptr; return ADA_OK; }
+  // the tokens are copied now (stream-ordered) into a buffer of the context: the step graph keeps reading that
+  // buffer, so the caller may pass a different array on every call
+  if (cudaMemcpyAsync(x->forced_buf, d_tokens, sizeof(int) * x->B * x->c.n_max, cudaMemcpyDeviceToDevice, x->stream) !=
+      cudaSuccess)
+    return fail(x, ADA_ERR_CUDA, "ada_force_draft: copy failed");
+  x->force_draft = x->forced_buf;
   return ADA_OK;
 }
 

@@ -678,9 +678,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const float va = __ldcg(qr + 2 * d + c), vb = __ldcg(qr + 2 * d + c + half);
             q_s[r * 128 + c] = (qa * cs.x - qb * cs.y) * qscale;
             q_s[r * 128 + c + half] = (qb * cs.x + qa * cs.y) * qscale;
-            const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
-            const __nv_bfloat16 k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(va), v1 = __float2bfloat16_rn(vb);
+            const __nv_bfloat16 k0 = kv_store(ka * cs.x - kb * cs.y);   // 16-bit cache elements (see kv_store)
+            const __nv_bfloat16 k1 = kv_store(kb * cs.x + ka * cs.y);
+            const __nv_bfloat16 v0 = kv_store(va), v1 = kv_store(vb);
             k_s[r * 128 + c] = k0; k_s[r * 128 + c + half] = k1;
             v_s[r * 128 + c] = v0; v_s[r * 128 + c + half] = v1;
             if (split == 0) {  // one item per head stores the new rows in the cache
@@ -721,10 +721,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 for (int c = 0; c < HD; c += 8) {
                   const uint4 kk = *reinterpret_cast<const uint4 *>(kr + c);
                   float kf[8];
-                  kf[0] = bf16_bits_to_float(kk.x & 0xffffu); kf[1] = bf16_bits_to_float(kk.x >> 16);
-                  kf[2] = bf16_bits_to_float(kk.y & 0xffffu); kf[3] = bf16_bits_to_float(kk.y >> 16);
-                  kf[4] = bf16_bits_to_float(kk.z & 0xffffu); kf[5] = bf16_bits_to_float(kk.z >> 16);
-                  kf[6] = bf16_bits_to_float(kk.w & 0xffffu); kf[7] = bf16_bits_to_float(kk.w >> 16);
+                  kf[0] = kv_lo(kk.x); kf[1] = kv_hi(kk.x);
+                  kf[2] = kv_lo(kk.y); kf[3] = kv_hi(kk.y);
+                  kf[4] = kv_lo(kk.z); kf[5] = kv_hi(kk.z);
+                  kf[6] = kv_lo(kk.w); kf[7] = kv_hi(kk.w);
 #pragma unroll
                   for (int i = 0; i < 8; ++i)
                     if (i < NR) {
@@ -745,10 +745,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
                   for (int u = 0; u < 8; ++u) {
                     float kf[8];
-                    kf[0] = bf16_bits_to_float(kq[u].x & 0xffffu); kf[1] = bf16_bits_to_float(kq[u].x >> 16);
-                    kf[2] = bf16_bits_to_float(kq[u].y & 0xffffu); kf[3] = bf16_bits_to_float(kq[u].y >> 16);
-                    kf[4] = bf16_bits_to_float(kq[u].z & 0xffffu); kf[5] = bf16_bits_to_float(kq[u].z >> 16);
-                    kf[6] = bf16_bits_to_float(kq[u].w & 0xffffu); kf[7] = bf16_bits_to_float(kq[u].w >> 16);
+                    kf[0] = kv_lo(kq[u].x); kf[1] = kv_hi(kq[u].x);
+                    kf[2] = kv_lo(kq[u].y); kf[3] = kv_hi(kq[u].y);
+                    kf[4] = kv_lo(kq[u].z); kf[5] = kv_hi(kq[u].z);
+                    kf[6] = kv_lo(kq[u].w); kf[7] = kv_hi(kq[u].w);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                       if (i < NR) {
@@ -790,11 +790,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 float vf[4] = {0.f, 0.f, 0.f, 0.f};
                 if (VPL == 4) {
                   const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
-                  vf[0] = bf16_bits_to_float(vv.x & 0xffffu); vf[1] = bf16_bits_to_float(vv.x >> 16);
-                  vf[2] = bf16_bits_to_float(vv.y & 0xffffu); vf[3] = bf16_bits_to_float(vv.y >> 16);
+                  vf[0] = kv_lo(vv.x); vf[1] = kv_hi(vv.x);
+                  vf[2] = kv_lo(vv.y); vf[3] = kv_hi(vv.y);
                 } else {
                   const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr);
-                  vf[0] = bf16_bits_to_float(vv & 0xffffu); vf[1] = bf16_bits_to_float(vv >> 16);
+                  vf[0] = kv_lo(vv); vf[1] = kv_hi(vv);
                 }
 #pragma unroll
                 for (int i = 0; i < 8; ++i)

@@ -81,3 +81,53 @@ def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=
                 em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(dev)
                 engine.ada_force_commit(b, em, len(o["emitted"]))
     return dict(iterations=compared, exempt=exempt, failures=failures)
+
+
+def run_golden(engine, golden, prompts, forced_n_schedule=None, greedy_streams=None, logit_tol=2e-2):
+    """Replays stored oracle iterations (tests/golden/*.json, written by make_goldens.py) in lock step.
+
+    golden: the parsed file; prompts: the same seeded prompts.  forced_n_schedule: per iteration the
+    forced draft length (teacher-forced configuration), else the predictor decides.  greedy_streams:
+    per sequence the oracle's greedy continuation used as forced drafts.
+    Returns dict(iterations, exempt, failures, max_top1_diff).
+    """
+    B, nmax = engine.B, engine.nmax
+    dev = engine.dev
+    draft_buf = engine.ada_debug_buffer(7, torch.int32, (B, nmax))
+    target_buf = engine.ada_debug_buffer(8, torch.int32, (B, nmax + 1))
+    vtop = engine.ada_debug_buffer(5, torch.float32, (B, nmax + 1, 2))
+    n_iters = min(len(s["iters"]) for s in golden["seqs"])
+    emitted_so_far = [1] * B
+    failures, exempt, compared, worst = [], 0, 0, 0.0
+    for r in range(n_iters):
+        if forced_n_schedule is not None:
+            engine.ada_force_n([forced_n_schedule[r]] * B)
+        if greedy_streams is not None:
+            ft = torch.zeros(B, nmax, dtype=torch.int32)
+            for b in range(B):
+                chunk = np.asarray(greedy_streams[b][emitted_so_far[b]: emitted_so_far[b] + nmax], dtype=np.int32)
+                ft[b, : len(chunk)] = torch.from_numpy(chunk)
+            engine.ada_force_draft(ft.to(dev))
+        g = engine.step()
+        gd, gt, gv = draft_buf.cpu().numpy(), target_buf.cpu().numpy(), vtop.cpu().numpy()
+        for b in range(B):
+            o = golden["seqs"][b]["iters"][r]
+            o = dict(o, ldlp_z=np.asarray(o["ldlp_z"]), d_top1=np.asarray(o["d_top1"]), d_top2=np.asarray(o["d_top2"]),
+                     v_top1=np.asarray(o["v_top1"]), v_top2=np.asarray(o["v_top2"]))
+            ok, ex, resync, msg = compare_iteration(o, g["n"][b], gd[b], gt[b], g["k"][b], g["emitted"][b], nmax,
+                                                    forced_n=forced_n_schedule is not None)
+            compared += 1
+            exempt += ex
+            if not ok:
+                failures.append("iter %d seq %d: %s" % (r, b, msg))
+            if ok and ex == 0 and g["n"][b] == o["n"]:
+                # same rows on both sides: the top logit of every verify row must agree within the logit bound
+                diff = float(np.abs(gv[b, : o["n"] + 1, 0] - o["v_top1"]).max())
+                worst = max(worst, diff)
+                if diff > logit_tol:
+                    failures.append("iter %d seq %d: top-1 logit differs by %.4f" % (r, b, diff))
+            if resync:
+                em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(dev)
+                engine.ada_force_commit(b, em, len(o["emitted"]))
+            emitted_so_far[b] += len(o["emitted"])
+    return dict(iterations=compared, exempt=exempt, failures=failures, max_top1_diff=worst)

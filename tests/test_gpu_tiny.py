@@ -192,3 +192,47 @@ def test_cache_full_clips_the_draft_length(tiny):
         assert e.ada_get_counters()["status"] & 1                   # clipped at least once
     finally:
         e.close()
+
+
+@pytest.mark.parametrize("plen", [200, 333, 420, 451, 1500])
+def test_long_context_attention_spans_blocks_and_rounds(tiny, plen):
+    """Contexts of several hundred positions: every KV split holds more than one 32-key block."""
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, m = tiny
+    long_prompt = si.uniform_ids(5, "long%d" % plen, plen, sh.vocab)
+    cap = sh.kv_capacity if plen + 64 < sh.kv_capacity else 2048   # 1500: splits of more than four blocks (two rounds)
+    e = Engine(sh, w, max_batch=1, kv_capacity=cap)
+    try:
+        seq = m.new_seq(cap)
+        t_o = seq.prefill(long_prompt)
+        t_g = e.prefill(0, long_prompt)
+        feat = e.ada_debug_buffer(0, torch.float32, (1, cap, sh.d_model))
+        err = np.abs(feat[0, :plen].cpu().numpy() - seq.features(0, plen)).max(axis=1)
+        assert err.max() < 2e-2, (int(err.argmax()), float(err.max()))
+        if t_o != t_g:      # only inside the oracle's own margin; the two states then differ, stop here
+            lg, _ = m.forward_nocache(long_prompt)
+            top = np.sort(lg)
+            assert top[-1] - top[-2] <= lockstep.TOKEN_MARGIN
+            return
+        logits = torch.zeros(1, sh.n_max + 1, sh.vocab, dtype=torch.float32, device=e.dev)
+        dfeat = e.ada_debug_buffer(4, torch.float32, (1, sh.n_max, sh.d_model))
+        for it in range(4):
+            n = sh.n_max
+            e.d_n.fill_(n)
+            d_o, d1, d2 = seq.draft(n)
+            e.ada_draft(e.d_n, e.d_draft)
+            derr = np.abs(dfeat[0, :n].cpu().numpy() - seq.draft_features(n)).max(axis=1)
+            assert derr.max() < 2e-2, (it, derr)
+            e.d_draft[0, :n] = torch.from_numpy(d_o).to(e.dev)
+            tt_o, v1, v2, lg_o = seq.verify(d_o, want_logits=True)
+            e.ada_verify(e.d_draft, e.d_n, e.d_target, logits)
+            lerr = np.abs(logits[0, : n + 1].cpu().numpy() - lg_o).max(axis=1)
+            assert lerr.max() < 2e-2, (it, lerr)
+            k_o, em_o = seq.accept(d_o, tt_o)
+            e.ada_accept(e.d_accept, e.d_emitted, e.d_nemit)
+            em_g = e.d_emitted.cpu().numpy()[0, : int(e.d_nemit.cpu()[0])]
+            if list(em_g) != list(em_o):
+                e.ada_force_commit(0, torch.from_numpy(em_o).to(e.dev), len(em_o))
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
