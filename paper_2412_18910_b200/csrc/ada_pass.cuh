@@ -56,11 +56,11 @@ constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
-constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 8 * 32 * 4 + 4 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; staged values
+constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 8 * 32 * 4 + 2 * 4 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; staged values and keys
 constexpr int kAttnPartBytes = 8 * 8 * 130 * 4;                    // per-warp partial results
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
-// (the + 16 KB: a tensor-core read of 128 tile rows may run past a short last stage; it must stay inside the allocation)
-constexpr int kScratchBytes = ((kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes) + 16 * 1024;
+// (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
+constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
 constexpr int kPassSmemBytes = 1024 + kStages * kStageBytes + kMiscBytes + kScratchBytes;   // 1 KB to align the ring
 static_assert(kPassSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr int kStatTimeout = 4;
@@ -658,6 +658,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         __nv_bfloat16 *v_s = k_s + 16 * 128;
         float *p_s = reinterpret_cast<float *>(v_s + 16 * 128);                       // [8 warps][8 rows][32 keys]
         __nv_bfloat16 *vst = reinterpret_cast<__nv_bfloat16 *>(p_s + 8 * 8 * 32);    // [4 blocks][32 keys][HD]
+        __nv_bfloat16 *kst = vst + 4 * 32 * 128;                                     // same for keys (chunk-swizzled rows)
         float *part_s = q_s;                                                          // [8][8][130], reuses the above
         const int VPL = HD / 32;
         const int rsel = cw & 1, bw = cw >> 1;
@@ -667,6 +668,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           const int hh = item / nsp, split = item - hh * nsp;
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
           named_bar(3, kNumCWarps * 32);
+          // keys and values of a round: one bulk copy per 32-key block each (a block is contiguous in its page)
+          auto issue_round = [&](int r0, int nblk) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffers come first
+            mbar_expect_tx(attn_bar, (unsigned)(2 * nblk * 32 * HD * 2));
+            for (int bb = 0; bb < nblk; ++bb) {
+              const int key0 = r0 + 32 * bb;
+              const int page = p.page_table[b * p.pages_per_seq + key0 / p.page_size], slot = key0 % p.page_size;
+              const size_t off = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
+              bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), attn_bar);
+              bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), attn_bar);
+            }
+          };
+          if (ctid == 0 && kend > kbeg) issue_round(kbeg, min(4, (kend - kbeg + 31) >> 5));   // first round: under the staging below
           // q (scaled), k, v of the block rows with rotary embedding
           const float qscale = rsqrtf((float)HD);
           for (int i = ctid; i < R * half; i += kNumCWarps * 32) {
@@ -687,7 +701,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const int pos = pos0 + r;
               const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
               const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
-              p.kpool[base + c] = k0; p.kpool[base + c + half] = k1;
+              // key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared
+              // memory, the 32 lanes of a warp (one key each) then read without bank conflicts
+              const int sw = slot & 7;
+              p.kpool[base + ((((c >> 3) ^ sw) << 3) | (c & 7))] = k0;
+              p.kpool[base + (((((c + half) >> 3) ^ sw) << 3) | (c & 7))] = k1;
               p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
             }
           }
@@ -696,18 +714,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           for (int i = 0; i < 8; ++i) { m[i] = -INFINITY; l[i] = 0.f; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
           for (int r0 = kbeg; r0 < kend; r0 += 128) {
             const int nblk = min(4, (kend - r0 + 31) >> 5);
-            named_bar(3, kNumCWarps * 32);   // staging visible; previous round's values no longer read
-            if (ctid == 0) {                 // values of this round: one bulk copy per 32-key block
-              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
-              mbar_expect_tx(attn_bar, (unsigned)(nblk * 32 * HD * 2));
-              for (int bb = 0; bb < nblk; ++bb) {
-                const int key0 = r0 + 32 * bb;
-                const int page = p.page_table[b * p.pages_per_seq + key0 / p.page_size], slot = key0 % p.page_size;
-                bulk_g2s(vst + (size_t)bb * 32 * HD,
-                         p.vpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD,
-                         (unsigned)(32 * HD * 2), attn_bar);
-              }
-            }
+            named_bar(3, kNumCWarps * 32);   // staging visible; previous round's keys and values no longer read
+            if (r0 > kbeg && ctid == 0) issue_round(r0, nblk);
+            // keys and values of this round have landed (every worker keeps the barrier's parity in step)
+            mbar_wait(attn_bar, attn_uses & 1u, p.cnt, abort_s);
+            ++attn_uses;
             const int kb0 = r0 + 32 * bw;
             const bool have = bw < nblk;
             const int key = kb0 + lane;
@@ -735,29 +746,21 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                     }
                 }
               } else {
-                const int page = p.page_table[b * p.pages_per_seq + key / p.page_size], slot = key % p.page_size;
-                const uint4 *kr = reinterpret_cast<const uint4 *>(
-                    p.kpool + (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD);
-                for (int c8 = 0; c8 < HD / 8; c8 += 8) {   // eight 16-byte loads in flight, then the arithmetic
-                  uint4 kq[8];
+                const unsigned char *kr = reinterpret_cast<const unsigned char *>(kst + (size_t)(bw * 32 + lane) * HD);
+                const int sw = lane & 7;   // = slot & 7: blocks start at multiples of 32
+                for (int u = 0; u < HD / 8; ++u) {
+                  const uint4 kq = *reinterpret_cast<const uint4 *>(kr + ((u ^ sw) << 4));
+                  float kf[8];
+                  kf[0] = kv_lo(kq.x); kf[1] = kv_hi(kq.x); kf[2] = kv_lo(kq.y); kf[3] = kv_hi(kq.y);
+                  kf[4] = kv_lo(kq.z); kf[5] = kv_hi(kq.z); kf[6] = kv_lo(kq.w); kf[7] = kv_hi(kq.w);
 #pragma unroll
-                  for (int u = 0; u < 8; ++u) kq[u] = kr[c8 + u];
-#pragma unroll
-                  for (int u = 0; u < 8; ++u) {
-                    float kf[8];
-                    kf[0] = kv_lo(kq[u].x); kf[1] = kv_hi(kq[u].x);
-                    kf[2] = kv_lo(kq[u].y); kf[3] = kv_hi(kq[u].y);
-                    kf[4] = kv_lo(kq[u].z); kf[5] = kv_hi(kq[u].z);
-                    kf[6] = kv_lo(kq[u].w); kf[7] = kv_hi(kq[u].w);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                      if (i < NR) {
-                        const float *qq = q_s + (2 * i + rsel) * 128 + (c8 + u) * 8;
-                        const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
-                        sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                                 qb.z * kf[6] + qb.w * kf[7];
-                      }
-                  }
+                  for (int i = 0; i < 8; ++i)
+                    if (i < NR) {
+                      const float *qq = q_s + (2 * i + rsel) * 128 + u * 8;
+                      const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
+                      sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                               qb.z * kf[6] + qb.w * kf[7];
+                    }
                 }
               }
             }
@@ -778,9 +781,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 }
               __syncwarp();
             }
-            // values: wait for this round's copies (every worker keeps the barrier's parity in step)
-            mbar_wait(attn_bar, attn_uses & 1u, p.cnt, abort_s);
-            ++attn_uses;
             if (have) {
               const int nk = min(32, kend - kb0);
               const __nv_bfloat16 *vb = vst + (size_t)bw * 32 * HD;
