@@ -48,7 +48,7 @@ constexpr int kKc = 256;                         // k elements per activation ch
 constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
 constexpr int kStageBytes = 16 * 1024;           // ring stage: kb boxes of [box_rows x 64 k], kb = 1, 2 or 4
 constexpr int kStages = 8;
-constexpr int kXBufs = 4;
+constexpr int kXBufs = 5;
 constexpr int kXBoxBytes = 32 * 128;             // activation box pair: 16 hi rows then 16 lo rows, 64 k
 constexpr int kXBufBytes = (kKc / kBoxK) * kXBoxBytes;    // 16 KB per chunk
 constexpr int kTmemCols = 64;                    // two accumulators of 32 columns
@@ -387,7 +387,7 @@ __device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoc
     for (unsigned i = 0; i < kSpinLimit && !*abort_flag; ++i) {
       if (ld_acquire(p.gbar) >= target) { ok = true; break; }
       if ((i & 63) == 63 && (ld_acquire(reinterpret_cast<const unsigned *>(&p.cnt->status)) & kStatTimeout)) break;
-      if (i > 32) __nanosleep(64);
+      if (i > 4096) __nanosleep(64);   // a barrier normally completes within a few polls
     }
     if (!ok) { *abort_flag = 1; atomicOr(&p.cnt->status, kStatTimeout); }
     __threadfence();
