@@ -66,7 +66,8 @@ struct ada_ctx {
   LayerPtrs *d_layers, *d_eagle;
   TensorMap128 *d_maps;
   int n_maps;
-  float *ss_part, *attn_part2;
+  float *ss_part, *attn_part2, *kpart;
+  int *kcnt;
   bf16 *xa, *at, *ac, *fc;            // activation tiles (xstore layout), 2048 elements per 64 k
   int *attn_cnt;
   float4 *amax2;
@@ -233,6 +234,8 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->ac = w.take<bf16>(((F + 63) / 64) * 2048);
   x->fc = w.take<bf16>(((2 * d + 63) / 64) * 2048);
   x->ss_part = w.take<float>(256 * 16);
+  x->kpart = w.take<float>(4 * 16 * d);
+  x->kcnt = w.take<int>(256);
   x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
   x->attn_cnt = w.take<int>(H);
   x->amax2 = w.take<float4>(256 * 16);
@@ -386,19 +389,25 @@ bool build_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
   bool ok = true;
   // box height of each matrix = rows of one m tile of its slabs (same arithmetic as the kernel's make_slab)
   const unsigned b_qkv = slab_box_rows(slab_rpc((int)d, 3, x->n_sm), false);
-  const unsigned b_d = slab_box_rows(slab_rpc((int)d, 1, x->n_sm), false);
+  // matrices with d output rows may be cut along K too (see make_slab): their slabs are then taller
+  auto d_rows = [&](size_t K) {
+    const int ks = slab_ksplit((int)d, (int)K, x->n_sm);
+    const int groups = ks > 1 ? x->n_sm / ks : x->n_sm;
+    return (unsigned)slab_box_rows(((int)d + groups - 1) / groups, false);
+  };
+  const unsigned b_wo = d_rows(d), b_wd = d_rows(F), b_fc = d_rows(2 * d);
   const unsigned b_f = slab_box_rows(slab_rpc((int)F, 1, x->n_sm), true);
   const unsigned b_v = slab_box_rows(slab_rpc((int)V, 1, x->n_sm), false);
   auto layer = [&](int base, const LayerW &a) {
     ok = ok && encode_map(fn, &maps[base + MAP_WQ], a.wq, d, d, b_qkv) && encode_map(fn, &maps[base + MAP_WK], a.wk, d, d, b_qkv) &&
-         encode_map(fn, &maps[base + MAP_WV], a.wv, d, d, b_qkv) && encode_map(fn, &maps[base + MAP_WO], a.wo, d, d, b_d) &&
+         encode_map(fn, &maps[base + MAP_WV], a.wv, d, d, b_qkv) && encode_map(fn, &maps[base + MAP_WO], a.wo, d, d, b_wo) &&
          encode_map(fn, &maps[base + MAP_WG], a.wg, F, d, b_f) && encode_map(fn, &maps[base + MAP_WU], a.wu, F, d, b_f) &&
-         encode_map(fn, &maps[base + MAP_WD], a.wd, d, F, b_d);
+         encode_map(fn, &maps[base + MAP_WD], a.wd, d, F, b_wd);
   };
   for (int l = 0; l < c.n_layers; ++l) layer(7 * l, x->layers[l]);
   layer(7 * c.n_layers, x->eagle);
   const int m0 = 7 * (c.n_layers + 1);
-  ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, b_d) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, b_v);
+  ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, b_fc) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, b_v);
   return ok;
 }
 
@@ -438,6 +447,7 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.page_table = x->page_table; p.pages_per_seq = x->pages_per_seq; p.page_size = c.page_size;
   p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
   p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
+  p.kpart = x->kpart; p.kcnt = x->kcnt;
   p.gbar = x->gbar; p.cnt = x->cnt;
   p.phase_ns = (x->prof && mode == 0) ? x->phase_ns : nullptr;
   timed(x, 0, pass_weight_bytes(x, mode, with_lm), [&] {
@@ -606,6 +616,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       if (e == cudaSuccess) e = cudaMemset(x->ac, 0, ((FF + 63) / 64) * 4096);
       if (e == cudaSuccess) e = cudaMemset(x->fc, 0, ((2 * dd + 63) / 64) * 4096);
       if (e == cudaSuccess) e = cudaMemset(x->attn_cnt, 0, sizeof(int) * cfg->n_heads);
+      if (e == cudaSuccess) e = cudaMemset(x->kcnt, 0, sizeof(int) * 256);
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }
   }

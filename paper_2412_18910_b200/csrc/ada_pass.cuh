@@ -117,6 +117,8 @@ struct PassParams {
   float *logits;               // optional [slot][V]
   int *tok_out; float2 *top_out; const int *forced;
   // sync
+  float *kpart;                // [4][16][d] partial sums of K-split groups
+  int *kcnt;                   // [grid] arrival counters of the groups (zero between phases)
   unsigned *gbar;              // grid barrier counter, zero at launch
   Counters *cnt;
   unsigned long long *phase_ns;  // optional [512]: [0] = start, [i+1] = time CTA 0 left barrier i (globaltimer)
@@ -261,6 +263,7 @@ struct GemmDesc {
   int scale_inv_rms;                // accumulators are multiplied by 1/rms(row) of h (input was h * gain)
   int lm_rows;                      // input rows are pass->lm_row[i] (draft LM head)
   const __nv_bfloat16 *gain_next;   // RESID_H / STORE_H: planes written are split(h * gain_next); null = no gain
+  int split_k;                      // this GEMM may be cut along K as well (outputs of d columns: O, down, fc)
 };
 
 // Phase list.  Target: EMBED, then per layer QKV, ATTN, O, GATEUP, DOWN, then LM.
@@ -285,11 +288,11 @@ __device__ __forceinline__ int phase_kind(const PassParams &p, int idx, int &lay
 __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int layer, GemmDesc &g) {
   const LayerPtrs &L = p.layers[layer];
   const int lm = p.map_layer0 + 7 * layer;
-  g.nseg = 1; g.scale_inv_rms = 0; g.lm_rows = 0; g.gain_next = nullptr;
+  g.nseg = 1; g.scale_inv_rms = 0; g.lm_rows = 0; g.gain_next = nullptr; g.split_k = 0;
   g.wmap[1] = g.wmap[2] = -1;
   switch (kind) {
     case PH_FC:
-      g.wmap[0] = p.map_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H;
+      g.wmap[0] = p.map_fc; g.Nseg = p.d; g.K = 2 * p.d; g.epi = EPI_STORE_H; g.split_k = 1;
       g.xt = p.fc; g.gain_next = L.na;
       return true;
     case PH_QKV:
@@ -297,7 +300,7 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
       g.epi = EPI_STORE_QKV; g.xt = p.xa; g.scale_inv_rms = 1;
       return true;
     case PH_O:
-      g.wmap[0] = lm + MAP_WO; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H;
+      g.wmap[0] = lm + MAP_WO; g.Nseg = p.d; g.K = p.d; g.epi = EPI_RESID_H; g.split_k = 1;
       g.xt = p.at; g.gain_next = L.nm;
       return true;
     case PH_GATEUP:
@@ -305,7 +308,7 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
       g.xt = p.xa; g.scale_inv_rms = 1;
       return true;
     case PH_DOWN:
-      g.wmap[0] = lm + MAP_WD; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H;
+      g.wmap[0] = lm + MAP_WD; g.Nseg = p.d; g.K = p.F; g.epi = EPI_RESID_H; g.split_k = 1;
       g.xt = p.ac;
       // the norm that follows: next layer's, or the final one; the draft head has none after its layer
       g.gain_next = (layer + 1 < p.n_layers) ? p.layers[layer + 1].na : (p.mode == 0 ? p.final_norm : nullptr);
@@ -325,6 +328,12 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
 // tiles of box_rows <= 128 rows (the tensor map's box height, fixed per matrix at initialisation
 // from the same arithmetic); SWIGLU: the two m tiles are the same row range of the gate and of the
 // up matrix.  A ring stage holds kb boxes (kb * 64 k) of one m tile.
+//
+// GEMMs with only d output columns (O, down, the draft head's fc) would leave each CTA a slab of ~28
+// rows: the tensor core then spends a whole instruction per 28 x 16 weights and every CTA re-reads the
+// whole activation.  They are cut along K too: ks CTAs share a slab of ~111 rows, each takes a
+// contiguous K range (whole 256-k chunks), writes its partial sums, and the CTA of the group that
+// arrives last adds the ks partials in split order and runs the epilogue.
 struct Slab {
   int seg;          // matrix (segment) of this CTA
   int r0, rows;     // rows [r0, r0 + rows) inside that matrix
@@ -333,6 +342,9 @@ struct Slab {
   int region;       // bytes of one box in shared memory (box_rows rounded up to 8, times 128)
   int kb;           // boxes per stage
   int m64;          // 1: M = 64 products (accumulator row i in lane (i % 16) + 32 * (i / 16))
+  int ks, kj;       // K splits of this GEMM and this CTA's split
+  int c0, c1;       // this CTA's 256-k chunks [c0, c1)
+  int group;        // index of the slab (= group of ks CTAs)
 };
 __host__ __device__ __forceinline__ int slab_rpc(int Nseg, int nseg, int ncta) {
   const int cps = ncta / nseg;
@@ -342,15 +354,47 @@ __host__ __device__ __forceinline__ int slab_box_rows(int rpc, bool swiglu) {
   const int mt = swiglu ? 1 : (rpc + 127) / 128;
   return (rpc + mt - 1) / mt;
 }
+// K splits for a GEMM of N output columns over K: the largest of 4, 3, 2 that leaves every split at least
+// one 256-k chunk and keeps a slab within one m tile (128 rows); else 1
+__host__ __device__ __forceinline__ int slab_ksplit(int N, int K, int ncta) {
+  const int nchunk = (K + kKc - 1) / kKc;
+  for (int ks = 4; ks >= 2; --ks) {
+    const int groups = ncta / ks;
+    if (groups < 1) continue;
+    const int per = (nchunk + ks - 1) / ks;
+    if ((ks - 1) * per >= nchunk) continue;          // some split would get nothing
+    if ((N + groups - 1) / groups > 128) continue;
+    return ks;
+  }
+  return 1;
+}
 __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) {
   Slab s;
   const bool sw = g.epi == EPI_SWIGLU_ACT;
-  const int cps = ncta / g.nseg;                  // CTAs per matrix
-  s.seg = cta / cps;
-  const int li = cta - s.seg * cps;
-  const int rpc = slab_rpc(g.Nseg, g.nseg, ncta);
+  const int nchunk = (g.K + kKc - 1) / kKc;
+  s.ks = g.split_k ? slab_ksplit(g.Nseg, g.K, ncta) : 1;
+  int rpc, li;
+  if (s.ks > 1) {
+    const int groups = ncta / s.ks;
+    s.seg = 0;
+    s.group = cta / s.ks;
+    s.kj = cta - s.group * s.ks;
+    rpc = (g.Nseg + groups - 1) / groups;
+    li = s.group;
+    const int per = (nchunk + s.ks - 1) / s.ks;
+    s.c0 = s.kj * per;
+    s.c1 = min(nchunk, s.c0 + per);
+    if (s.group >= groups) { s.c0 = s.c1 = 0; li = groups; }   // CTAs beyond the last whole group idle
+  } else {
+    const int cps = ncta / g.nseg;                  // CTAs per matrix
+    s.seg = cta / cps;
+    li = cta - s.seg * cps;
+    rpc = slab_rpc(g.Nseg, g.nseg, ncta);
+    s.kj = 0; s.c0 = 0; s.c1 = nchunk; s.group = cta;
+  }
   s.r0 = li * rpc;
   s.rows = (s.seg < g.nseg) ? max(0, min(g.Nseg, s.r0 + rpc) - s.r0) : 0;
+  if (s.c1 <= s.c0) s.rows = 0;
   s.box_rows = slab_box_rows(rpc, sw);
   s.mtiles = sw ? 2 : ((rpc + 127) / 128);
   if (!sw && s.rows <= s.box_rows) s.mtiles = 1;  // a short last slab may not reach the second tile
@@ -470,8 +514,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       if ((g.lm_rows ? lmT : T) <= 0) continue;
       const Slab s = make_slab(g, cta, ncta);
       if (s.rows == 0) continue;
-      const int nchunk = (g.K + kKc - 1) / kKc;
-      for (int c = 0; c < nchunk; ++c) {
+      for (int c = s.c0; c < s.c1; ++c) {
         const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;   // boxes that hold any k < K
         for (int b0 = 0; b0 < nbox; b0 += s.kb) {
           const int nb = min(s.kb, nbox - b0);
@@ -518,12 +561,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         if ((g.lm_rows ? lmT : T) <= 0) continue;
         const Slab s = make_slab(g, cta, ncta);
         if (s.rows == 0) continue;
-        const int nchunk = (g.K + kKc - 1) / kKc;
         const uint32_t idesc = umma_idesc(s.m64 ? 64u : 128u);
         const uint32_t region16 = (uint32_t)s.region >> 4;
         uint32_t started = 0;   // this issuer's accumulator holds a product of this phase
         int sidx = 0;           // stage index inside the phase
-        for (int c = 0; c < nchunk; ++c, ++xcount) {
+        for (int c = s.c0; c < s.c1; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
           const int kleft = min(kKc, g.K - c * kKc);
           const int nbox = (kleft + kBoxK - 1) / kBoxK;
@@ -894,12 +936,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     if (Tg <= 0) { grid_barrier(p, epoch, tid, abort_s); continue; }
     const int nt_act = (Tg + 7) >> 3;
     const Slab s = make_slab(g, cta, ncta);
-    const int nchunk = (g.K + kKc - 1) / kKc;
 
     if (is_xprod) {
       // ---- activation producer: the input tiles of this GEMM, one bulk copy per 256-k chunk
       if (s.rows > 0) {
-        for (int c = 0; c < nchunk; ++c, ++xcount) {
+        for (int c = s.c0; c < s.c1; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
           if (lane == 0) {
             if (xcount >= kXBufs) mbar_wait(&xempty[buf], ((unsigned)(xcount / kXBufs) & 1u) ^ 1u, p.cnt, abort_s);
@@ -955,7 +996,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
     const bool sw = g.epi == EPI_SWIGLU_ACT;
     int nstages_phase = 0;   // ring stages of this phase in this CTA (as the issuers count them)
-    for (int c = 0; c < nchunk; ++c) {
+    for (int c = s.c0; c < s.c1; ++c) {
       const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
       nstages_phase += ((nbox + s.kb - 1) / s.kb) * s.mtiles;
     }
@@ -978,57 +1019,101 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       tc_fence_after();
     }
     stamp(p, ph, 2, stamper);
+    float yy[16], uu[16];   // this thread's weight row against the 16 pass rows (hi + lo columns added)
+#pragma unroll
+    for (int t = 0; t < 16; ++t) { yy[t] = 0.f; uu[t] = 0.f; }
     if (active_warp) {
       float v[32], u[32];
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * 32);
       tmem_ld32(taddr, v);
-      if (sw) tmem_ld32(taddr + 32, u);
-      else if (s.mtiles == 1 && nstages_phase >= 2) {   // one m tile: issuer 1's share sits in region 1
+      if (sw) {
+        tmem_ld32(taddr + 32, u);
+#pragma unroll
+        for (int t = 0; t < 16; ++t) uu[t] = u[t] + u[16 + t];
+      } else if (s.mtiles == 1 && nstages_phase >= 2) {   // one m tile: issuer 1's share sits in region 1
         tmem_ld32(taddr + 32, u);
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] += u[i];
       }
-      if (valid) {
-        float hold[16];
 #pragma unroll
-        for (int t = 0; t < 16; ++t)
-          hold[t] = (g.epi == EPI_RESID_H && t < Tg) ? __ldcg(p.h + (size_t)t * p.d + vrow) : 0.f;
+      for (int t = 0; t < 16; ++t) yy[t] = v[t] + v[16 + t];   // accumulator column = pass row
+      if (g.lm_rows) {               // draft LM head: output row t is pass row lm_row[t]
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           if (t < Tg) {
-            const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
-            float yy = v[t] + v[16 + t];   // accumulator column = pass row
-            if (g.lm_rows) {               // draft LM head: output row t is pass row lm_row[t]
-              const int col = p.pass->lm_row[t];
-              yy = 0.f;
+            const int col = p.pass->lm_row[t];
+            float sel = 0.f;
 #pragma unroll
-              for (int cc = 0; cc < 16; ++cc) yy = (cc == col) ? v[cc] + v[16 + cc] : yy;
-            }
-            const float y = yy * sc;
-            if (g.epi == EPI_STORE_QKV) {
-              p.qkv[(size_t)t * 3 * p.d + vrow] = y;
-            } else if (has_ss) {
-              float *hp = p.h + (size_t)t * p.d + vrow;
-              const float hn = hold[t] + y;
-              *hp = hn;
-              ssl[t] = hn * hn;
-              const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
-              xstore(p.xa, t, vrow, hn * gn);
-            } else if (sw) {
-              const float up = (u[t] + u[16 + t]) * sc;
-              xstore(p.ac, t, vrow, (y / (1.f + __expf(-y))) * up);
-            } else {  // EPI_ARGMAX_LM
-              if (p.logits) {
-                const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
-                p.logits[(size_t)slot_out * p.V + vrow] = y;
-              }
-              tb[t].v1 = y; tb[t].i1 = vrow;
-            }
+            for (int cc = 0; cc < 16; ++cc) sel = (cc == col) ? v[cc] + v[16 + cc] : sel;
+            yy[t] = sel;
           }
         }
       }
     }
     tc_fence_before();
+    bool do_epi = true;
+    if (s.ks > 1 && s.rows > 0) {
+      // K-split group: publish the partial sums; the CTA that arrives last adds the ks partials in split
+      // order (all read back from memory, its own included, so the order never depends on who is last)
+      if (valid)
+#pragma unroll
+        for (int t = 0; t < 16; ++t)
+          if (t < Tg) __stcg(p.kpart + ((size_t)(s.kj * 16 + t)) * p.d + vrow, yy[t]);
+      __threadfence();
+      named_bar(3, kNumCWarps * 32);
+      if (ctid == 0) *flag_s = (atomicAdd(p.kcnt + s.group, 1) == s.ks - 1);
+      named_bar(3, kNumCWarps * 32);
+      do_epi = *flag_s != 0;
+      if (do_epi) {
+        __threadfence();
+        if (valid) {
+#pragma unroll
+          for (int t0 = 0; t0 < 16; t0 += 8) {   // 32 independent loads in flight, then the sums in split order
+            float pv[8][4];
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                pv[t][j] = (t0 + t < Tg && j < s.ks) ? __ldcg(p.kpart + ((size_t)(j * 16 + t0 + t)) * p.d + vrow) : 0.f;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) yy[t0 + t] = ((pv[t][0] + pv[t][1]) + pv[t][2]) + pv[t][3];
+          }
+        }
+        if (ctid == 0) p.kcnt[s.group] = 0;
+      }
+    }
+    if (valid && do_epi) {
+      float hold[16];
+#pragma unroll
+      for (int t = 0; t < 16; ++t)
+        hold[t] = (g.epi == EPI_RESID_H && t < Tg) ? __ldcg(p.h + (size_t)t * p.d + vrow) : 0.f;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        if (t < Tg) {
+          const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
+          const float y = yy[t] * sc;
+          if (g.epi == EPI_STORE_QKV) {
+            p.qkv[(size_t)t * 3 * p.d + vrow] = y;
+          } else if (has_ss) {
+            float *hp = p.h + (size_t)t * p.d + vrow;
+            const float hn = hold[t] + y;
+            *hp = hn;
+            ssl[t] = hn * hn;
+            const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
+            xstore(p.xa, t, vrow, hn * gn);
+          } else if (sw) {
+            const float up = uu[t] * sc;
+            xstore(p.ac, t, vrow, (y / (1.f + __expf(-y))) * up);
+          } else {  // EPI_ARGMAX_LM
+            if (p.logits) {
+              const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
+              p.logits[(size_t)slot_out * p.V + vrow] = y;
+            }
+            tb[t].v1 = y; tb[t].i1 = vrow;
+          }
+        }
+      }
+    }
     if (has_ss) {
       // per pass row: sum over the warp's 32 weight rows, then over the warps in order
 #pragma unroll
