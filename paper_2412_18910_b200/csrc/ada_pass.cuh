@@ -56,8 +56,8 @@ constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
-constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 8 * 32 * 4 + 2 * 4 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; staged values and keys
-constexpr int kAttnPartBytes = 8 * 8 * 130 * 4;                    // per-warp partial results
+constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 4 * 32 * 4 + 2 * 2 * 2 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; two buffers of staged keys and values
+constexpr int kAttnPartBytes = 8 * 4 * 130 * 4;                    // per-warp partial results
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
@@ -468,18 +468,18 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   unsigned char *ring = smem;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
   uint64_t *full = bars, *empty = bars + kStages, *xfull = bars + 2 * kStages, *xempty = bars + 2 * kStages + kXBufs;
-  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs + 2);   // [16] (after accfull)
+  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs + 4);   // [16] (after accfull and the attention barriers)
   float *ssw = inv_rms + 16;                                                       // [8][16]
   Top2 *topw = reinterpret_cast<Top2 *>(ssw + 8 * 16);                             // [8][16]
   int *flag_s = reinterpret_cast<int *>(topw + 8 * 16);
   volatile int *abort_s = flag_s + 1;
   unsigned char *xbuf = smem + kStages * kStageBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
-  static_assert((2 * kStages + 2 * kXBufs + 2) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
+  static_assert((2 * kStages + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
   (void)red;
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
-  uint64_t *attn_bar = accfull + 1;                        // attention: values of a round have landed
+  uint64_t *attn_bar = accfull + 1;                        // attention: keys and values of a round have landed (two buffers)
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
   if (tid == 0) {
     *abort_s = 0;
@@ -487,6 +487,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 2); }
     mbar_init(accfull, 2);
     mbar_init(attn_bar, 1);
+    mbar_init(attn_bar + 1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(tmem_slot, kTmemCols);
@@ -627,7 +628,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   RingPos rp{0, 0};
   int xcount = 0;   // activation chunks produced so far (buffer = xcount % kXBufs)
   unsigned acc_phase = 0;   // GEMM phases of this CTA whose accumulator has been awaited
-  unsigned attn_uses = 0;   // completed phases of the attention barrier
+  unsigned attn_uses[2] = {0, 0};   // completed phases of the two attention barriers
   (void)g8; (void)q4; (void)rp;
 
   for (int ph = 0; ph < nphase; ++ph) {
@@ -686,10 +687,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     if (kind == PH_ATTN) {
       if (!is_xprod) {
         // Items (head, KV split) round-robin over CTAs; one sequence on this path.  Inside an item a
-        // round covers 4 blocks of 32 keys; warp w works on block w/2 for the query rows of parity
-        // w%2, lane = key while scoring, lane = 4 channels while accumulating values.  Values of a
-        // round arrive by one bulk copy per block (a block is contiguous in its cache page); keys are
-        // read straight from the cache, each lane its own row.
+        // round covers two blocks of 32 keys; warp w works on block w/4 for the query rows r with
+        // r % 4 == w % 4, lane = key while scoring, lane = 4 channels while accumulating values.  Keys
+        // and values of a round arrive by one bulk copy per block each (a block is contiguous in its cache
+        // page) into one of two buffers, so the copies of the next round fly while this one is computed.
         const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
         const int nkeys = pos0 + R, nsp = p.attn_splits;
         int chunk = (nkeys + nsp - 1) / nsp;
@@ -698,31 +699,38 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         float *q_s = reinterpret_cast<float *>(xbuf);                                 // [16][128] fp32
         __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(q_s + 16 * 128);      // new rows, rotated [16][128]
         __nv_bfloat16 *v_s = k_s + 16 * 128;
-        float *p_s = reinterpret_cast<float *>(v_s + 16 * 128);                       // [8 warps][8 rows][32 keys]
-        __nv_bfloat16 *vst = reinterpret_cast<__nv_bfloat16 *>(p_s + 8 * 8 * 32);    // [4 blocks][32 keys][HD]
-        __nv_bfloat16 *kst = vst + 4 * 32 * 128;                                     // same for keys (chunk-swizzled rows)
-        float *part_s = q_s;                                                          // [8][8][130], reuses the above
+        float *p_s = reinterpret_cast<float *>(v_s + 16 * 128);                       // [8 warps][4 rows][32 keys]
+        __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(p_s + 8 * 4 * 32);    // [2 buffers][K, V][2 blocks][32 keys][128]
+        float *part_s = q_s;                                                          // [8][4][130], reuses the above
         const int VPL = HD / 32;
-        const int rsel = cw & 1, bw = cw >> 1;
-        const int NR = (R - rsel + 1) >> 1;          // my rows: r = 2 i + rsel, i < NR
+        const int rq = cw & 3, bw = cw >> 2;
+        const int NR = (R - rq + 3) >> 2;            // my rows: r = 4 i + rq, i < NR
         const size_t head_stride = (size_t)p.page_size * HD;
         for (int item = cta; item < p.H * nsp; item += ncta) {
           const int hh = item / nsp, split = item - hh * nsp;
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
+          const int nround = kend > kbeg ? (kend - kbeg + 63) >> 6 : 0;
           named_bar(3, kNumCWarps * 32);
-          // keys and values of a round: one bulk copy per 32-key block each (a block is contiguous in its page)
-          auto issue_round = [&](int r0, int nblk) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffers come first
-            mbar_expect_tx(attn_bar, (unsigned)(2 * nblk * 32 * HD * 2));
+          // round rd -> buffer rd & 1: keys then values, two blocks each
+          auto issue_round = [&](int rd) {
+            const int r0 = kbeg + 64 * rd;
+            const int nblk = min(2, (kend - r0 + 31) >> 5);
+            uint64_t *bar = attn_bar + (rd & 1);
+            __nv_bfloat16 *kst = stg + (size_t)(rd & 1) * 4 * 32 * 128, *vst = kst + 2 * 32 * 128;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
+            mbar_expect_tx(bar, (unsigned)(2 * nblk * 32 * HD * 2));
             for (int bb = 0; bb < nblk; ++bb) {
               const int key0 = r0 + 32 * bb;
               const int page = p.page_table[b * p.pages_per_seq + key0 / p.page_size], slot = key0 % p.page_size;
               const size_t off = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
-              bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), attn_bar);
-              bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), attn_bar);
+              bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), bar);
+              bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), bar);
             }
           };
-          if (ctid == 0 && kend > kbeg) issue_round(kbeg, min(4, (kend - kbeg + 31) >> 5));   // first round: under the staging below
+          if (ctid == 0) {   // the first two rounds fly under the staging below
+            if (nround > 0) issue_round(0);
+            if (nround > 1) issue_round(1);
+          }
           // q (scaled), k, v of the block rows with rotary embedding
           const float qscale = rsqrtf((float)HD);
           for (int i = ctid; i < R * half; i += kNumCWarps * 32) {
@@ -751,66 +759,48 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
             }
           }
-          float m[8], l[8], o[8][4];
+          float m[4], l[4], o[4][4];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { m[i] = -INFINITY; l[i] = 0.f; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-          for (int r0 = kbeg; r0 < kend; r0 += 128) {
-            const int nblk = min(4, (kend - r0 + 31) >> 5);
-            named_bar(3, kNumCWarps * 32);   // staging visible; previous round's keys and values no longer read
-            if (r0 > kbeg && ctid == 0) issue_round(r0, nblk);
-            // keys and values of this round have landed (every worker keeps the barrier's parity in step)
-            mbar_wait(attn_bar, attn_uses & 1u, p.cnt, abort_s);
-            ++attn_uses;
+          for (int i = 0; i < 4; ++i) { m[i] = -INFINITY; l[i] = 0.f; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+          named_bar(3, kNumCWarps * 32);   // staging visible
+          for (int rd = 0; rd < nround; ++rd) {
+            const int r0 = kbeg + 64 * rd;
+            const int nblk = min(2, (kend - r0 + 31) >> 5);
+            const __nv_bfloat16 *kst = stg + (size_t)(rd & 1) * 4 * 32 * 128, *vst = kst + 2 * 32 * 128;
+            // keys and values of this round have landed (every worker keeps the barriers' parity in step)
+            mbar_wait(attn_bar + (rd & 1), (attn_uses[rd & 1]++) & 1u, p.cnt, abort_s);
             const int kb0 = r0 + 32 * bw;
             const bool have = bw < nblk;
             const int key = kb0 + lane;
             const bool kv = have && key < kend;
-            float sc[8];
+            float sc[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) sc[i] = 0.f;
+            for (int i = 0; i < 4; ++i) sc[i] = 0.f;
             if (kv) {
-              if (key >= pos0) {
-                const __nv_bfloat16 *kr = k_s + (key - pos0) * 128;
-                for (int c = 0; c < HD; c += 8) {
-                  const uint4 kk = *reinterpret_cast<const uint4 *>(kr + c);
-                  float kf[8];
-                  kf[0] = kv_lo(kk.x); kf[1] = kv_hi(kk.x);
-                  kf[2] = kv_lo(kk.y); kf[3] = kv_hi(kk.y);
-                  kf[4] = kv_lo(kk.z); kf[5] = kv_hi(kk.z);
-                  kf[6] = kv_lo(kk.w); kf[7] = kv_hi(kk.w);
+              const bool fresh = key >= pos0;   // a row of this pass: from the staged new rows, natural layout
+              const unsigned char *kr = fresh ? reinterpret_cast<const unsigned char *>(k_s + (key - pos0) * 128)
+                                              : reinterpret_cast<const unsigned char *>(kst + (size_t)(bw * 32 + lane) * HD);
+              const int sw = fresh ? 0 : (lane & 7);   // = slot & 7: blocks start at multiples of 32
+              for (int u = 0; u < HD / 8; ++u) {
+                const uint4 kq = *reinterpret_cast<const uint4 *>(kr + ((u ^ sw) << 4));
+                float kf[8];
+                kf[0] = kv_lo(kq.x); kf[1] = kv_hi(kq.x); kf[2] = kv_lo(kq.y); kf[3] = kv_hi(kq.y);
+                kf[4] = kv_lo(kq.z); kf[5] = kv_hi(kq.z); kf[6] = kv_lo(kq.w); kf[7] = kv_hi(kq.w);
 #pragma unroll
-                  for (int i = 0; i < 8; ++i)
-                    if (i < NR) {
-                      const float *qq = q_s + (2 * i + rsel) * 128 + c;
-                      const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
-                      sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                               qb.z * kf[6] + qb.w * kf[7];
-                    }
-                }
-              } else {
-                const unsigned char *kr = reinterpret_cast<const unsigned char *>(kst + (size_t)(bw * 32 + lane) * HD);
-                const int sw = lane & 7;   // = slot & 7: blocks start at multiples of 32
-                for (int u = 0; u < HD / 8; ++u) {
-                  const uint4 kq = *reinterpret_cast<const uint4 *>(kr + ((u ^ sw) << 4));
-                  float kf[8];
-                  kf[0] = kv_lo(kq.x); kf[1] = kv_hi(kq.x); kf[2] = kv_lo(kq.y); kf[3] = kv_hi(kq.y);
-                  kf[4] = kv_lo(kq.z); kf[5] = kv_hi(kq.z); kf[6] = kv_lo(kq.w); kf[7] = kv_hi(kq.w);
-#pragma unroll
-                  for (int i = 0; i < 8; ++i)
-                    if (i < NR) {
-                      const float *qq = q_s + (2 * i + rsel) * 128 + u * 8;
-                      const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
-                      sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                               qb.z * kf[6] + qb.w * kf[7];
-                    }
-                }
+                for (int i = 0; i < 4; ++i)
+                  if (i < NR) {
+                    const float *qq = q_s + (4 * i + rq) * 128 + u * 8;
+                    const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
+                    sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                             qb.z * kf[6] + qb.w * kf[7];
+                  }
               }
             }
             if (have) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
+              for (int i = 0; i < 4; ++i)
                 if (i < NR) {
-                  const bool seen = kv && key <= pos0 + 2 * i + rsel;
+                  const bool seen = kv && key <= pos0 + 4 * i + rq;
                   const float sv = seen ? sc[i] : -INFINITY;
                   const float mx = warp_max(sv);
                   const float mn = fmaxf(m[i], mx);
@@ -819,11 +809,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   l[i] = l[i] * corr + warp_sum(pe);
                   o[i][0] *= corr; o[i][1] *= corr; o[i][2] *= corr; o[i][3] *= corr;
                   m[i] = mn;
-                  p_s[(cw * 8 + i) * 32 + lane] = pe;
+                  p_s[(cw * 4 + i) * 32 + lane] = pe;
                 }
               __syncwarp();
-            }
-            if (have) {
               const int nk = min(32, kend - kb0);
               const __nv_bfloat16 *vb = vst + (size_t)bw * 32 * HD;
               for (int kk = 0; kk < nk; ++kk) {
@@ -832,28 +820,28 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 float vf[4] = {0.f, 0.f, 0.f, 0.f};
                 if (VPL == 4) {
                   const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
-                  vf[0] = kv_lo(vv.x); vf[1] = kv_hi(vv.x);
-                  vf[2] = kv_lo(vv.y); vf[3] = kv_hi(vv.y);
+                  vf[0] = kv_lo(vv.x); vf[1] = kv_hi(vv.x); vf[2] = kv_lo(vv.y); vf[3] = kv_hi(vv.y);
                 } else {
                   const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr);
                   vf[0] = kv_lo(vv); vf[1] = kv_hi(vv);
                 }
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
+                for (int i = 0; i < 4; ++i)
                   if (i < NR) {
-                    const float pe = p_s[(cw * 8 + i) * 32 + kk];
+                    const float pe = p_s[(cw * 4 + i) * 32 + kk];
                     o[i][0] += pe * vf[0]; o[i][1] += pe * vf[1]; o[i][2] += pe * vf[2]; o[i][3] += pe * vf[3];
                   }
               }
             }
+            named_bar(3, kNumCWarps * 32);   // every warp is done with this buffer
+            if (ctid == 0 && rd + 2 < nround) issue_round(rd + 2);
           }
-          // per-warp partials -> shared (over the loop's scratch once every warp has left the loop),
-          // merged over the four key blocks in block order, stored per (head, split)
-          named_bar(3, kNumCWarps * 32);
+          // per-warp partials -> shared (over the staging areas, which every warp has left), merged over
+          // the two key blocks in block order, stored per (head, split)
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < 4; ++i)
             if (i < NR) {
-              float *pp = part_s + (cw * 8 + i) * 130;
+              float *pp = part_s + (cw * 4 + i) * 130;
               if (VPL == 4) { pp[lane * 4] = o[i][0]; pp[lane * 4 + 1] = o[i][1]; pp[lane * 4 + 2] = o[i][2]; pp[lane * 4 + 3] = o[i][3]; }
               else { pp[lane * 2] = o[i][0]; pp[lane * 2 + 1] = o[i][1]; }
               if (lane == 0) { pp[128] = m[i]; pp[129] = l[i]; }
@@ -861,17 +849,15 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           named_bar(3, kNumCWarps * 32);
           for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
             const int r = i / HD, c = i - r * HD;
-            const int ri = r >> 1, rs = r & 1;
-            float M = -INFINITY;
-            for (int q = 0; q < 4; ++q) M = fmaxf(M, part_s[((2 * q + rs) * 8 + ri) * 130 + 128]);
+            const int ri = r >> 2, rs = r & 3;
+            const float *pa = part_s + ((0 * 4 + rs) * 4 + ri) * 130, *pb = part_s + ((1 * 4 + rs) * 4 + ri) * 130;
+            const float M = fmaxf(pa[128], pb[128]);
             float lo = 0.f, oo = 0.f;
-            if (M > -INFINITY)
-              for (int q = 0; q < 4; ++q) {
-                const float *pp = part_s + ((2 * q + rs) * 8 + ri) * 130;
-                const float e = __expf(pp[128] - M);
-                lo += pp[129] * e;
-                oo += pp[c] * e;
-              }
+            if (M > -INFINITY) {
+              const float ea = __expf(pa[128] - M), eb = __expf(pb[128] - M);
+              lo = pa[129] * ea + pb[129] * eb;
+              oo = pa[c] * ea + pb[c] * eb;
+            }
             float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
             __stcg(gp + c, oo);
             if (c == 0) { __stcg(gp + HD, M); __stcg(gp + HD + 1, lo); }
