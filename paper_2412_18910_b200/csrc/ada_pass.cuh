@@ -46,8 +46,9 @@ constexpr int kNumCWarps = 8;                    // workers
 constexpr int kFirstWorker = 4;                  // warp index of worker 0
 constexpr int kKc = 256;                         // k elements per activation chunk = 4 boxes of 64
 constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
-constexpr int kStageBytes = 16 * 1024;           // ring stage: kb boxes of [box_rows x 64 k], kb = 1, 2 or 4
-constexpr int kStages = 8;
+constexpr int kStageBytes = 32 * 1024;           // largest ring stage: kb boxes of [box_rows x 64 k], kb = 2 or 4
+constexpr int kRingBytes = 128 * 1024;           // weight ring; stages take exactly the bytes of their boxes
+constexpr int kSlots = 16;                       // barrier pairs of the ring = most stages in flight
 constexpr int kXBufs = 5;
 constexpr int kXBoxBytes = 32 * 128;             // activation box pair: 16 hi rows then 16 lo rows, 64 k
 constexpr int kXBufBytes = (kKc / kBoxK) * kXBoxBytes;    // 16 KB per chunk
@@ -61,7 +62,7 @@ constexpr int kAttnPartBytes = 8 * 4 * 130 * 4;                    // per-warp p
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
-constexpr int kPassSmemBytes = 1024 + kStages * kStageBytes + kMiscBytes + kScratchBytes;   // 1 KB to align the ring
+constexpr int kPassSmemBytes = 1024 + kRingBytes + kMiscBytes + kScratchBytes;   // 1 KB to align the ring
 static_assert(kPassSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr int kStatTimeout = 4;
 constexpr unsigned kSpinLimit = 1u << 22;
@@ -399,7 +400,7 @@ __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) 
   s.mtiles = sw ? 2 : ((rpc + 127) / 128);
   if (!sw && s.rows <= s.box_rows) s.mtiles = 1;  // a short last slab may not reach the second tile
   s.region = ((s.box_rows + 7) & ~7) * 128;
-  s.kb = s.region <= 4096 ? 4 : (s.region <= 8192 ? 2 : 1);
+  s.kb = s.region <= 8192 ? 4 : 2;   // a stage is at most 32 KB
   s.m64 = s.box_rows <= 64;
   return s;
 }
@@ -409,11 +410,19 @@ __device__ __forceinline__ void tile_source(const GemmDesc &g, const Slab &s, in
   else { map = g.wmap[s.seg]; row0 = s.r0 + mi * s.box_rows; }
 }
 
-struct RingPos {
-  int stage;
-  unsigned parity;
-  __device__ __forceinline__ void advance() {
-    if (++stage == kStages) { stage = 0; parity ^= 1u; }
+// Walk over the weight ring.  A stage takes exactly the bytes of its boxes (a multiple of 1 KB), at the
+// head of the ring, or at offset 0 if it would run past the end; stage j uses barrier pair j % kSlots in
+// its (j / kSlots)-th phase.  The walk depends on the static schedule only, so the producer and both
+// issuers compute the same offsets without talking to each other.
+struct RingCursor {
+  uint32_t head;
+  unsigned n;     // stages taken so far
+  __device__ __forceinline__ uint32_t take(uint32_t bytes) {
+    if (head + bytes > (uint32_t)kRingBytes) head = 0;
+    const uint32_t off = head;
+    head += bytes;
+    ++n;
+    return off;
   }
 };
 
@@ -466,24 +475,25 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   // swizzled TMA boxes need 1024-byte aligned bases
   unsigned char *const smem = pass_smem + ((1024u - (smem_u32(pass_smem) & 1023u)) & 1023u);
   unsigned char *ring = smem;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
-  uint64_t *full = bars, *empty = bars + kStages, *xfull = bars + 2 * kStages, *xempty = bars + 2 * kStages + kXBufs;
-  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kStages + 2 * kXBufs + 4);   // [16] (after accfull and the attention barriers)
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kRingBytes);
+  uint64_t *full = bars, *empty = bars + kSlots, *xfull = bars + 2 * kSlots, *xempty = bars + 2 * kSlots + kXBufs;
+  float *inv_rms = reinterpret_cast<float *>(bars + 2 * kSlots + 2 * kXBufs + 4);   // [16] (after accfull and the attention barriers)
   float *ssw = inv_rms + 16;                                                       // [8][16]
   Top2 *topw = reinterpret_cast<Top2 *>(ssw + 8 * 16);                             // [8][16]
   int *flag_s = reinterpret_cast<int *>(topw + 8 * 16);
   volatile int *abort_s = flag_s + 1;
-  unsigned char *xbuf = smem + kStages * kStageBytes + kMiscBytes;
+  unsigned char *xbuf = smem + kRingBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
-  static_assert((2 * kStages + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 <= kMiscBytes, "misc area");
+  static_assert((2 * kSlots + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 + 2 * kSlots * 4 <= kMiscBytes, "misc area");
   (void)red;
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
   uint64_t *attn_bar = accfull + 1;                        // attention: keys and values of a round have landed (two buffers)
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
+  uint32_t *st_off = tmem_slot + 1, *st_end = st_off + kSlots;   // producer's record of the stages in flight
   if (tid == 0) {
     *abort_s = 0;
-    for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 2); }
     mbar_init(accfull, 2);
     mbar_init(attn_bar, 1);
@@ -505,8 +515,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 
   // ================================================================= weight producer
   if (warp == 0) {
-    RingPos rp{0, 0};
-    unsigned filled = 0;  // stages issued so far; the first kStages need no wait
+    RingCursor cur{0, 0};
+    unsigned tail = 0;   // stages [tail, cur.n) may still be unread
+    uint32_t t_off = 0, t_end = 0;
     for (int ph = 0; ph < nphase; ++ph) {
       int layer;
       const int kind = phase_kind(p, ph, layer);
@@ -515,24 +526,44 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       if ((g.lm_rows ? lmT : T) <= 0) continue;
       const Slab s = make_slab(g, cta, ncta);
       if (s.rows == 0) continue;
-      for (int c = s.c0; c < s.c1; ++c) {
-        const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;   // boxes that hold any k < K
-        for (int b0 = 0; b0 < nbox; b0 += s.kb) {
-          const int nb = min(s.kb, nbox - b0);
-          for (int mi = 0; mi < s.mtiles; ++mi) {
-            if (filled >= (unsigned)kStages) {
-              if (lane == 0) mbar_wait(&empty[rp.stage], rp.parity ^ 1u, p.cnt, abort_s);
-              __syncwarp();
+      if (lane != 0) continue;   // one thread produces: no warp synchronisation on the per-stage path
+      // per-phase constants in registers (tensor map and first row of each m tile)
+      int map0, map1, row0, row1;
+      tile_source(g, s, 0, map0, row0);
+      tile_source(g, s, s.mtiles - 1, map1, row1);
+      const unsigned long long m0 = reinterpret_cast<unsigned long long>(p.maps + map0);
+      const unsigned long long m1 = reinterpret_cast<unsigned long long>(p.maps + map1);
+      const int region = s.region, kb = s.kb, mtiles = s.mtiles, K = g.K, c1 = s.c1;
+      const unsigned tx_box = (unsigned)(s.box_rows * 128);
+      for (int c = s.c0; c < c1; ++c) {
+        const int nbox = (min(kKc, K - c * kKc) + kBoxK - 1) / kBoxK;   // boxes that hold any k < K
+        for (int b0 = 0; b0 < nbox; b0 += kb) {
+          const int nb = min(kb, nbox - b0);
+          for (int mi = 0; mi < mtiles; ++mi) {
+            const uint32_t bytes = (uint32_t)(nb * region);
+            const uint32_t off = cur.take(bytes);
+            const unsigned j = cur.n - 1, slot = j % kSlots;
+            // The oldest stages in flight are the first ones a new stage can run into: retire them until a
+            // barrier pair is free and no unread stage overlaps the new one.  (t_off, t_end) is the record
+            // of stage `tail`, read ahead so that the usual check needs no shared-memory access.
+            while (tail < j && (j - tail >= (unsigned)kSlots || (t_off < off + bytes && off < t_end))) {
+              mbar_wait(&empty[tail % kSlots], (tail / kSlots) & 1u, p.cnt, abort_s);
+              ++tail;
+              t_off = st_off[tail % kSlots];   // (stale if tail == j: replaced below)
+              t_end = st_end[tail % kSlots];
             }
-            int map, row0;
-            tile_source(g, s, mi, map, row0);
-            if (lane == 0) mbar_expect_tx(&full[rp.stage], (unsigned)(nb * s.box_rows * 128));
-            __syncwarp();
-            if (lane < nb)   // one box per lane; rows past the matrix and k past K read as zero
-              tma_load_2d(ring + (size_t)rp.stage * kStageBytes + (size_t)lane * s.region, p.maps + map,
-                          c * kKc + (b0 + lane) * kBoxK, row0, &full[rp.stage]);
-            ++filled;
-            rp.advance();
+            st_off[slot] = off; st_end[slot] = off + bytes;
+            if (tail == j) { t_off = off; t_end = off + bytes; }
+            mbar_expect_tx(&full[slot], (unsigned)nb * tx_box);
+            const uint32_t dst = smem_u32(ring) + off, bar = smem_u32(&full[slot]);
+            const unsigned long long mp = mi ? m1 : m0;
+            const int y = mi ? row1 : row0;
+            for (int b = 0; b < nb; ++b)   // rows past the matrix and k past K read as zero
+              asm volatile(
+                  "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                      dst + (uint32_t)(b * region)),
+                  "l"(mp), "r"(c * kKc + (b0 + b) * kBoxK), "r"(y), "r"(bar)
+                  : "memory");
           }
         }
       }
@@ -551,7 +582,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     // about 140 cycles instead of about 55); one elected lane issues.
     const int me = __shfl_sync(0xffffffffu, warp, 0) - 2;
     {
-      RingPos rp{0, 0};
+      RingCursor cur{0, 0};
       int xcount = 0;
       const uint32_t ring_u = smem_u32(ring), xbuf_u = smem_u32(xbuf);
       for (int ph = 0; ph < nphase; ++ph) {
@@ -578,10 +609,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const int nb = min(s.kb, nbox - b0);
             for (int mi = 0; mi < s.mtiles; ++mi, ++sidx) {
               const bool mine = (s.mtiles == 2 ? mi : (sidx & 1)) == me;
+              const uint32_t off = cur.take((uint32_t)(nb * s.region));
+              const unsigned slot = (cur.n - 1) % kSlots, parity = ((cur.n - 1) / kSlots) & 1u;
               if (mine) {
-                const uint64_t adesc0 = umma_desc(ring_u + (uint32_t)rp.stage * kStageBytes);
+                const uint64_t adesc0 = umma_desc(ring_u + off);
                 const uint32_t dcol = tmem_base + (uint32_t)(s.mtiles == 2 ? mi : me) * 32;
-                mbar_wait(&full[rp.stage], rp.parity, p.cnt, abort_s);
+                mbar_wait(&full[slot], parity, p.cnt, abort_s);
                 tc_fence_after();
                 for (int bi = 0; bi < nb; ++bi) {
                   const int box = b0 + bi;
@@ -593,10 +626,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                     started = 1;
                   }
                 }
-                if (elect_one()) umma_commit(&empty[rp.stage]);   // the stage is free once these products have read it
+                if (elect_one()) umma_commit(&empty[slot]);   // the stage is free once these products have read it
                 __syncwarp();
               }
-              rp.advance();
             }
           }
           // both issuers release the chunk (an issuer with no stage in it releases it at once)
@@ -625,11 +657,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   const int nnth = (kNumXWarps + kNumCWarps) * 32;
   const int ctid = tid - kFirstWorker * 32;   // index among the 256 worker threads
   unsigned epoch = 0;
-  RingPos rp{0, 0};
   int xcount = 0;   // activation chunks produced so far (buffer = xcount % kXBufs)
   unsigned acc_phase = 0;   // GEMM phases of this CTA whose accumulator has been awaited
   unsigned attn_uses[2] = {0, 0};   // completed phases of the two attention barriers
-  (void)g8; (void)q4; (void)rp;
+  (void)g8; (void)q4;
 
   for (int ph = 0; ph < nphase; ++ph) {
     int layer;
