@@ -151,7 +151,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, unsigned parity) {
 }
 // bounded wait; on give-up records a status bit and returns
 // (*abort_flag is a per-CTA shared word: once any wait of the CTA has given up, later waits do not spin)
+// non-blocking test of the same condition (cheaper than try_wait when the phase is already complete)
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
+  if (mbar_test(bar, parity)) return;
   for (unsigned i = 0; i < kSpinLimit; ++i) {
     if (mbar_try(bar, parity)) return;
     if (*abort_flag) return;
@@ -616,17 +627,26 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 const uint32_t dcol = tmem_base + (uint32_t)(s.mtiles == 2 ? mi : me) * 32;
                 mbar_wait(&full[slot], parity, p.cnt, abort_s);
                 tc_fence_after();
-                for (int bi = 0; bi < nb; ++bi) {
-                  const int box = b0 + bi;
-                  const uint64_t ad = adesc0 + (uint64_t)(bi * region16);
-                  const uint64_t bd = bdesc0 + (uint64_t)(box * (kXBoxBytes >> 4));
-                  const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
-                  for (int s4 = 0; s4 < nstep; ++s4) {
-                    if (elect_one()) umma_bf16(dcol, ad + 2 * s4, bd + 2 * s4, idesc, started);   // + 32 bytes per k16 step
-                    started = 1;
+                if (elect_one()) {   // one thread issues the stage's products and the commit that frees it
+                  uint32_t acc = started;
+                  for (int bi = 0; bi < nb; ++bi) {
+                    const int box = b0 + bi;
+                    const uint64_t ad = adesc0 + (uint64_t)(bi * region16);
+                    const uint64_t bd = bdesc0 + (uint64_t)(box * (kXBoxBytes >> 4));
+                    const int nstep = min(4, (kleft - box * kBoxK + 15) >> 4);   // k16 steps holding any k < K
+                    if (nstep == 4) {
+                      umma_bf16(dcol, ad, bd, idesc, acc);            // + 32 bytes per k16 step
+                      umma_bf16(dcol, ad + 2, bd + 2, idesc, 1);
+                      umma_bf16(dcol, ad + 4, bd + 4, idesc, 1);
+                      umma_bf16(dcol, ad + 6, bd + 6, idesc, 1);
+                    } else {
+                      for (int s4 = 0; s4 < nstep; ++s4) umma_bf16(dcol, ad + 2 * s4, bd + 2 * s4, idesc, s4 ? 1u : acc);
+                    }
+                    acc = 1;
                   }
+                  umma_commit(&empty[slot]);   // the stage is free once these products have read it
                 }
-                if (elect_one()) umma_commit(&empty[slot]);   // the stage is free once these products have read it
+                started = 1;
                 __syncwarp();
               }
             }
