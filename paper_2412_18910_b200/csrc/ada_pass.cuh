@@ -495,18 +495,18 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   volatile int *abort_s = flag_s + 1;
   unsigned char *xbuf = smem + kRingBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
-  static_assert((2 * kSlots + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 + 2 * kSlots * 4 <= kMiscBytes, "misc area");
+  static_assert((2 * kSlots + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 + 4 * kSlots * 4 <= kMiscBytes, "misc area");
   (void)red;
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
   uint64_t *attn_bar = accfull + 1;                        // attention: keys and values of a round have landed (two buffers)
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
-  uint32_t *st_off = tmem_slot + 1, *st_end = st_off + kSlots;   // producer's record of the stages in flight
+  uint32_t *st_rec = tmem_slot + 1;   // [2 producers][offsets, ends][kSlots]: records of the stages in flight
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kSlots; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 2); }
-    mbar_init(accfull, 2);
+    for (int i = 0; i < kXBufs; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
+    mbar_init(accfull, 1);
     mbar_init(attn_bar, 1);
     mbar_init(attn_bar + 1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -525,7 +525,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   }
 
   // ================================================================= weight producer
-  if (warp == 0) {
+  if (warp == 0 || warp == 3) {
+    const unsigned pidx = warp == 0 ? 0u : 1u;   // producer 0 loads the even stages, producer 1 the odd ones
+    uint32_t *st_off = st_rec + pidx * 2 * kSlots, *st_end = st_off + kSlots;   // this producer's own record of the stages
     RingCursor cur{0, 0};
     unsigned tail = 0;   // stages [tail, cur.n) may still be unread
     uint32_t t_off = 0, t_end = 0;
@@ -554,17 +556,23 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const uint32_t bytes = (uint32_t)(nb * region);
             const uint32_t off = cur.take(bytes);
             const unsigned j = cur.n - 1, slot = j % kSlots;
-            // The oldest stages in flight are the first ones a new stage can run into: retire them until a
-            // barrier pair is free and no unread stage overlaps the new one.  (t_off, t_end) is the record
-            // of stage `tail`, read ahead so that the usual check needs no shared-memory access.
-            while (tail < j && (j - tail >= (unsigned)kSlots || (t_off < off + bytes && off < t_end))) {
-              mbar_wait(&empty[tail % kSlots], (tail / kSlots) & 1u, p.cnt, abort_s);
-              ++tail;
-              t_off = st_off[tail % kSlots];   // (stale if tail == j: replaced below)
-              t_end = st_end[tail % kSlots];
-            }
             st_off[slot] = off; st_end[slot] = off + bytes;
             if (tail == j) { t_off = off; t_end = off + bytes; }
+            if ((j & 1u) != pidx) continue;   // the other producer's stage
+            // The oldest stages in flight are the first ones a new stage can run into: they are retired until a
+            // barrier pair is free and no unread stage overlaps the new one.  One thread issues all products,
+            // so stages are read in order and waiting for the newest retired one covers the older ones.
+            // (t_off, t_end) is the record of stage `tail`, read ahead of its use.
+            {
+              unsigned last = 0xffffffffu;
+              while (tail < j && (j - tail >= (unsigned)kSlots || (t_off < off + bytes && off < t_end))) {
+                last = tail;
+                ++tail;
+                t_off = st_off[tail % kSlots];
+                t_end = st_end[tail % kSlots];
+              }
+              if (last != 0xffffffffu) mbar_wait(&empty[last % kSlots], (last / kSlots) & 1u, p.cnt, abort_s);
+            }
             mbar_expect_tx(&full[slot], (unsigned)nb * tx_box);
             const uint32_t dst = smem_u32(ring) + off, bar = smem_u32(&full[slot]);
             const unsigned long long mp = mi ? m1 : m0;
@@ -582,16 +590,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     return;
   }
 
-  // ================================================================= tensor-core issuers (warps 2 and 3)
-  // One thread's tcgen05.mma issue rate (about 55 cycles each) is below what a 28-row slab needs, so
-  // two threads issue.  With two m tiles issuer i owns m tile i; with one m tile the issuers take
-  // alternate stages and accumulate into tensor-memory regions 0 and 1, which the epilogue adds in
-  // that order.  Every product of an accumulator is thus issued by one thread, in schedule order.
-  if (warp == 2 || warp == 3) {
-    // The whole warp walks the loop so that descriptors and addresses stay warp-uniform (the compiler
-    // can keep them in uniform registers: issued from inside a one-lane branch each tcgen05.mma cost
-    // about 140 cycles instead of about 55); one elected lane issues.
-    const int me = __shfl_sync(0xffffffffu, warp, 0) - 2;
+  // ================================================================= tensor-core issuer (warp 2)
+  // One elected thread issues every product, in schedule order (about 58 cycles per tcgen05.mma when the
+  // products of a stage are issued back to back), so stages are also released in order.  M tile mi
+  // accumulates in tensor-memory columns [32 mi, 32 mi + 32).
+  if (warp == 2) {
     {
       RingCursor cur{0, 0};
       int xcount = 0;
@@ -606,29 +609,25 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         if (s.rows == 0) continue;
         const uint32_t idesc = umma_idesc(s.m64 ? 64u : 128u);
         const uint32_t region16 = (uint32_t)s.region >> 4;
-        uint32_t started = 0;   // this issuer's accumulator holds a product of this phase
-        int sidx = 0;           // stage index inside the phase
+        uint32_t started = 0;   // bit mi: the accumulator of m tile mi holds a product of this phase
         for (int c = s.c0; c < s.c1; ++c, ++xcount) {
           const int buf = xcount % kXBufs;
           const int kleft = min(kKc, g.K - c * kKc);
           const int nbox = (kleft + kBoxK - 1) / kBoxK;
           const uint64_t bdesc0 = umma_desc(xbuf_u + (uint32_t)buf * kXBufBytes);
-          // both issuers wait for the chunk even if only one has a stage in it: an issuer can then never
-          // release a buffer twice before the other has released it once
           mbar_wait(&xfull[buf], (unsigned)(xcount / kXBufs) & 1u, p.cnt, abort_s);
           for (int b0 = 0; b0 < nbox; b0 += s.kb) {
             const int nb = min(s.kb, nbox - b0);
-            for (int mi = 0; mi < s.mtiles; ++mi, ++sidx) {
-              const bool mine = (s.mtiles == 2 ? mi : (sidx & 1)) == me;
+            for (int mi = 0; mi < s.mtiles; ++mi) {
               const uint32_t off = cur.take((uint32_t)(nb * s.region));
               const unsigned slot = (cur.n - 1) % kSlots, parity = ((cur.n - 1) / kSlots) & 1u;
-              if (mine) {
+              {
                 const uint64_t adesc0 = umma_desc(ring_u + off);
-                const uint32_t dcol = tmem_base + (uint32_t)(s.mtiles == 2 ? mi : me) * 32;
+                const uint32_t dcol = tmem_base + (uint32_t)mi * 32;
                 mbar_wait(&full[slot], parity, p.cnt, abort_s);
                 tc_fence_after();
                 if (elect_one()) {   // one thread issues the stage's products and the commit that frees it
-                  uint32_t acc = started;
+                  uint32_t acc = (started >> mi) & 1u;
                   for (int bi = 0; bi < nb; ++bi) {
                     const int box = b0 + bi;
                     const uint64_t ad = adesc0 + (uint64_t)(bi * region16);
@@ -646,12 +645,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                   }
                   umma_commit(&empty[slot]);   // the stage is free once these products have read it
                 }
-                started = 1;
+                started |= 1u << mi;
                 __syncwarp();
               }
             }
           }
-          // both issuers release the chunk (an issuer with no stage in it releases it at once)
           if (elect_one()) umma_commit(&xempty[buf]);
           __syncwarp();
         }
@@ -660,7 +658,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       }
     }
     __syncwarp();
-    if (warp == 3) return;
     // the workers signal when their last read of tensor memory is done
     tc_fence_before();
     named_bar(5, 32 + kNumCWarps * 32);
@@ -971,7 +968,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     make_gemm(p, kind, layer, g);
     const int Tg = g.lm_rows ? lmT : T;
     if (Tg <= 0) { grid_barrier(p, epoch, tid, abort_s); continue; }
-    const int nt_act = (Tg + 7) >> 3;
     const Slab s = make_slab(g, cta, ncta);
 
     if (is_xprod) {
@@ -1032,11 +1028,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     stamp(p, ph, 1, stamper);
     const bool has_ss = g.epi == EPI_RESID_H || g.epi == EPI_STORE_H;
     const bool sw = g.epi == EPI_SWIGLU_ACT;
-    int nstages_phase = 0;   // ring stages of this phase in this CTA (as the issuers count them)
-    for (int c = s.c0; c < s.c1; ++c) {
-      const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
-      nstages_phase += ((nbox + s.kb - 1) / s.kb) * s.mtiles;
-    }
     // thread <-> weight row: quarter = warp index mod 4 (the tensor-memory lanes this warp may read),
     // m tile = worker index / 4 (SWIGLU: the first four workers read both accumulators)
     const int quarter = warp & 3, mi = sw ? 0 : (cw >> 2);
@@ -1067,10 +1058,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         tmem_ld32(taddr + 32, u);
 #pragma unroll
         for (int t = 0; t < 16; ++t) uu[t] = u[t] + u[16 + t];
-      } else if (s.mtiles == 1 && nstages_phase >= 2) {   // one m tile: issuer 1's share sits in region 1
-        tmem_ld32(taddr + 32, u);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] += u[i];
       }
 #pragma unroll
       for (int t = 0; t < 16; ++t) yy[t] = v[t] + v[16 + t];   // accumulator column = pass row
