@@ -57,8 +57,8 @@ constexpr int kRedBytes = kNumCWarps * 32 * 8 * 4;
 constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA arrays
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
-constexpr int kAttnLoopBytes = 16 * 128 * 4 + 2 * 16 * 128 * 2 + 8 * 4 * 32 * 4 + 2 * 2 * 2 * 32 * 128 * 2;   // q; new k, v rows; softmax weights; two buffers of staged keys and values
-constexpr int kAttnPartBytes = 8 * 4 * 130 * 4;                    // per-warp partial results
+constexpr int kAttnLoopBytes = 4 * 16 * 128 * 2 + 2 * 2 * 2 * 32 * 128 * 2;   // q hi, q lo, new k, v rows; two buffers of staged keys and values
+constexpr int kAttnPartBytes = 8 * 16 * 130 * 4 + 2 * 8 * 16 * 4;   // per-warp partial results, merge weights
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
@@ -188,6 +188,23 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// warp-level products on 16-bit halves with fp32 sums (attention): c[16 x 8] += a[16 x 16] b[16 x 8], and k = 8
+__device__ __forceinline__ void mma_f16_k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                            uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16_k8(float *c, uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(b0));
 }
 // ---- tcgen05 (5th generation tensor cores, accumulators in tensor memory)
 __device__ __forceinline__ void tmem_alloc(uint32_t *smem_slot, uint32_t ncols) {   // whole warp
@@ -734,26 +751,31 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     // ------------------------------------------------------------- attention
     if (kind == PH_ATTN) {
       if (!is_xprod) {
-        // Items (head, KV split) round-robin over CTAs; one sequence on this path.  Inside an item a
-        // round covers two blocks of 32 keys; warp w works on block w/4 for the query rows r with
-        // r % 4 == w % 4, lane = key while scoring, lane = 4 channels while accumulating values.  Keys
-        // and values of a round arrive by one bulk copy per block each (a block is contiguous in its cache
-        // page) into one of two buffers, so the copies of the next round fly while this one is computed.
+        // Items (head, KV split) round-robin over CTAs; one sequence on this path.  Inside an item a round
+        // covers two blocks of 32 keys; warp w works on 8 keys (block w / 4, keys 8 (w % 4) .. + 8 of it) for
+        // all 16 query rows with mma.sync: scores = q k^T (m16n8k16 per 16 channels), then the weighted
+        // values (m16n8k8 per 8 channels).  Cache elements are 16-bit halves and enter the products as they
+        // are; q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, so each product is
+        // issued twice and the sums are fp32.  Keys and values of a round arrive by one bulk copy per block
+        // each (a block is contiguous in its cache page) into one of two buffers, so the copies of the next
+        // round fly while this one is computed.
         const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
         const int nkeys = pos0 + R, nsp = p.attn_splits;
         int chunk = (nkeys + nsp - 1) / nsp;
         chunk = ((chunk + 31) / 32) * 32;
         const int b = p.pass->row_seq[0];
-        float *q_s = reinterpret_cast<float *>(xbuf);                                 // [16][128] fp32
-        __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(q_s + 16 * 128);      // new rows, rotated [16][128]
+        __half *qh_s = reinterpret_cast<__half *>(xbuf);                              // q hi [16][128], 16-byte chunks XORed with row & 7
+        __half *ql_s = qh_s + 16 * 128;                                              // q lo, same layout
+        __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(ql_s + 16 * 128);    // new rows, rotated [16][128]
         __nv_bfloat16 *v_s = k_s + 16 * 128;
-        float *p_s = reinterpret_cast<float *>(v_s + 16 * 128);                       // [8 warps][4 rows][32 keys]
-        __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(p_s + 8 * 4 * 32);    // [2 buffers][K, V][2 blocks][32 keys][128]
-        float *part_s = q_s;                                                          // [8][4][130], reuses the above
-        const int VPL = HD / 32;
-        const int rq = cw & 3, bw = cw >> 2;
-        const int NR = (R - rq + 3) >> 2;            // my rows: r = 4 i + rq, i < NR
+        __nv_bfloat16 *stg = v_s + 16 * 128;                                         // [2 buffers][K, V][2 blocks][32 keys][128]
+        float *part_s = reinterpret_cast<float *>(xbuf);                              // [8 warps][16 rows][130], reuses the above
+        float *lw_s = part_s + 8 * 16 * 130;                                          // [8 warps][16 rows] merge weights
+        float *wgt = lw_s + 8 * 16;                                                   // [8 splits][16 rows] (cross-CTA merge)
+        const int g8r = lane >> 2, t4 = lane & 3;
+        const int bw = cw >> 2, kq = cw & 3;
         const size_t head_stride = (size_t)p.page_size * HD;
+        const uint32_t qh_u = smem_u32(qh_s), ql_u = smem_u32(ql_s);
         for (int item = cta; item < p.H * nsp; item += ncta) {
           const int hh = item / nsp, split = item - hh * nsp;
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
@@ -779,37 +801,59 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             if (nround > 0) issue_round(0);
             if (nround > 1) issue_round(1);
           }
-          // q (scaled), k, v of the block rows with rotary embedding
+          // q (scaled), k, v of the block rows with rotary embedding; rows past R are zero
           const float qscale = rsqrtf((float)HD);
-          for (int i = ctid; i < R * half; i += kNumCWarps * 32) {
-            const int r = i / half, c = i - r * half;
-            const float2 cs = p.rope[(size_t)(pos0 + r) * half + c];
-            const float *qr = p.qkv + (size_t)r * 3 * d + hh * HD;
-            const float qa = __ldcg(qr + c), qb = __ldcg(qr + c + half);
-            const float ka = __ldcg(qr + d + c), kb = __ldcg(qr + d + c + half);
-            const float va = __ldcg(qr + 2 * d + c), vb = __ldcg(qr + 2 * d + c + half);
-            q_s[r * 128 + c] = (qa * cs.x - qb * cs.y) * qscale;
-            q_s[r * 128 + c + half] = (qb * cs.x + qa * cs.y) * qscale;
-            const __nv_bfloat16 k0 = kv_store(ka * cs.x - kb * cs.y);   // 16-bit cache elements (see kv_store)
-            const __nv_bfloat16 k1 = kv_store(kb * cs.x + ka * cs.y);
-            const __nv_bfloat16 v0 = kv_store(va), v1 = kv_store(vb);
-            k_s[r * 128 + c] = k0; k_s[r * 128 + c + half] = k1;
-            v_s[r * 128 + c] = v0; v_s[r * 128 + c + half] = v1;
-            if (split == 0) {  // one item per head stores the new rows in the cache
-              const int pos = pos0 + r;
-              const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
-              const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
-              // key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared
-              // memory, the 32 lanes of a warp (one key each) then read without bank conflicts
-              const int sw = slot & 7;
-              p.kpool[base + ((((c >> 3) ^ sw) << 3) | (c & 7))] = k0;
-              p.kpool[base + (((((c + half) >> 3) ^ sw) << 3) | (c & 7))] = k1;
-              p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
+          for (int i0 = 0; i0 < 16 * half; i0 += 2 * kNumCWarps * 32) {
+            float qa[2], qb[2], ka[2], kb[2], va[2], vb[2];
+            float2 cs[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {   // all loads of two elements first
+              const int i = i0 + u * kNumCWarps * 32 + ctid;
+              const int r = i / half, c = i - r * half;
+              qa[u] = qb[u] = ka[u] = kb[u] = va[u] = vb[u] = 0.f;
+              cs[u] = make_float2(1.f, 0.f);
+              if (i < R * half) {
+                cs[u] = p.rope[(size_t)(pos0 + r) * half + c];
+                const float *qr = p.qkv + (size_t)r * 3 * d + hh * HD;
+                qa[u] = __ldcg(qr + c); qb[u] = __ldcg(qr + c + half);
+                ka[u] = __ldcg(qr + d + c); kb[u] = __ldcg(qr + d + c + half);
+                va[u] = __ldcg(qr + 2 * d + c); vb[u] = __ldcg(qr + 2 * d + c + half);
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int i = i0 + u * kNumCWarps * 32 + ctid;
+              if (i >= 16 * half) continue;
+              const int r = i / half, c = i - r * half;
+              const float q0 = (qa[u] * cs[u].x - qb[u] * cs[u].y) * qscale, q1 = (qb[u] * cs[u].x + qa[u] * cs[u].y) * qscale;
+              const __half h0 = __float2half_rn(q0), h1 = __float2half_rn(q1);
+              const int o0 = r * 128 + ((((c >> 3) ^ (r & 7)) << 3) | (c & 7));
+              const int o1 = r * 128 + (((((c + half) >> 3) ^ (r & 7)) << 3) | (c & 7));
+              qh_s[o0] = h0; qh_s[o1] = h1;
+              ql_s[o0] = __float2half_rn(q0 - __half2float(h0)); ql_s[o1] = __float2half_rn(q1 - __half2float(h1));
+              const __nv_bfloat16 k0 = kv_store(ka[u] * cs[u].x - kb[u] * cs[u].y);   // 16-bit cache elements (see kv_store)
+              const __nv_bfloat16 k1 = kv_store(kb[u] * cs[u].x + ka[u] * cs[u].y);
+              const __nv_bfloat16 v0 = kv_store(va[u]), v1 = kv_store(vb[u]);
+              k_s[r * 128 + c] = k0; k_s[r * 128 + c + half] = k1;
+              v_s[r * 128 + c] = v0; v_s[r * 128 + c + half] = v1;
+              if (split == 0 && r < R) {  // one item per head stores the new rows in the cache
+                const int pos = pos0 + r;
+                const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
+                const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
+                // key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared
+                // memory, eight consecutive keys then sit in eight different bank groups
+                const int sw = slot & 7;
+                p.kpool[base + ((((c >> 3) ^ sw) << 3) | (c & 7))] = k0;
+                p.kpool[base + (((((c + half) >> 3) ^ sw) << 3) | (c & 7))] = k1;
+                p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
+              }
             }
           }
-          float m[4], l[4], o[4][4];
+          // running maxima, sums and outputs of rows g8r and g8r + 8 over this warp's keys
+          float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+          float o[16][4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) { m[i] = -INFINITY; l[i] = 0.f; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+          for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
           named_bar(3, kNumCWarps * 32);   // staging visible
           for (int rd = 0; rd < nround; ++rd) {
             const int r0 = kbeg + 64 * rd;
@@ -817,98 +861,114 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const __nv_bfloat16 *kst = stg + (size_t)(rd & 1) * 4 * 32 * 128, *vst = kst + 2 * 32 * 128;
             // keys and values of this round have landed (every worker keeps the barriers' parity in step)
             mbar_wait(attn_bar + (rd & 1), (attn_uses[rd & 1]++) & 1u, p.cnt, abort_s);
-            const int kb0 = r0 + 32 * bw;
-            const bool have = bw < nblk;
-            const int key = kb0 + lane;
-            const bool kv = have && key < kend;
-            float sc[4];
+            const int key0 = r0 + 32 * bw + 8 * kq;     // first of this warp's 8 keys
+            if (bw < nblk && key0 < kend) {
+              // ---- scores: 16 rows x 8 keys
+              float sc[4] = {0.f, 0.f, 0.f, 0.f};
+              const int myk = key0 + (lane & 7);          // key whose row address this lane supplies
+              const bool fresh = myk >= pos0;             // a row of this pass: from the staged new rows, natural layout
+              const uint32_t krow = fresh ? smem_u32(k_s + (size_t)min(myk - pos0, 15) * 128)
+                                          : smem_u32(kst + (size_t)(bw * 32 + 8 * kq + (lane & 7)) * HD);
+              const int ksw = fresh ? 0 : (lane & 7);     // = slot & 7: blocks start at multiples of 32
+              const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) sc[i] = 0.f;
-            if (kv) {
-              const bool fresh = key >= pos0;   // a row of this pass: from the staged new rows, natural layout
-              const unsigned char *kr = fresh ? reinterpret_cast<const unsigned char *>(k_s + (key - pos0) * 128)
-                                              : reinterpret_cast<const unsigned char *>(kst + (size_t)(bw * 32 + lane) * HD);
-              const int sw = fresh ? 0 : (lane & 7);   // = slot & 7: blocks start at multiples of 32
-              for (int u = 0; u < HD / 8; ++u) {
-                const uint4 kq = *reinterpret_cast<const uint4 *>(kr + ((u ^ sw) << 4));
-                float kf[8];
-                kf[0] = kv_lo(kq.x); kf[1] = kv_hi(kq.x); kf[2] = kv_lo(kq.y); kf[3] = kv_hi(kq.y);
-                kf[4] = kv_lo(kq.z); kf[5] = kv_hi(kq.z); kf[6] = kv_lo(kq.w); kf[7] = kv_hi(kq.w);
+              for (int kp = 0; kp < 4; ++kp) {            // pairs of 16-channel steps
+                if (kp * 32 < HD) {
+                  uint32_t kb0, kb1, kb2, kb3;
+                  ldmatrix_x4(krow + ((((kp * 4 + (lane >> 3)) ^ ksw)) << 4), kb0, kb1, kb2, kb3);
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  if (i < NR) {
-                    const float *qq = q_s + (4 * i + rq) * 128 + u * 8;
-                    const float4 qa = *reinterpret_cast<const float4 *>(qq), qb = *reinterpret_cast<const float4 *>(qq + 4);
-                    sc[i] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                             qb.z * kf[6] + qb.w * kf[7];
+                  for (int h2 = 0; h2 < 2; ++h2) {
+                    const int ks = kp * 2 + h2;
+                    const uint32_t aoff = (uint32_t)(arow * 256 + (((ks * 2 + (lane >> 4)) ^ (arow & 7)) << 4));
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(qh_u + aoff, a0, a1, a2, a3);
+                    mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+                    ldmatrix_x4(ql_u + aoff, a0, a1, a2, a3);
+                    mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
                   }
+                }
               }
-            }
-            if (have) {
+              // ---- online softmax: this thread holds keys kc, kc + 1 of rows g8r and g8r + 8
+              const int kc = key0 + 2 * t4;
+              const bool s00 = kc < kend && kc <= pos0 + g8r, s01 = kc + 1 < kend && kc + 1 <= pos0 + g8r;
+              const bool s10 = kc < kend && kc <= pos0 + g8r + 8, s11 = kc + 1 < kend && kc + 1 <= pos0 + g8r + 8;
+              float mx0 = fmaxf(s00 ? sc[0] : -INFINITY, s01 ? sc[1] : -INFINITY);
+              float mx1 = fmaxf(s10 ? sc[2] : -INFINITY, s11 ? sc[3] : -INFINITY);
+              mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+              mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+              const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+              float p00 = 0.f, p01 = 0.f, p10 = 0.f, p11 = 0.f, c0 = 1.f, c1 = 1.f;
+              if (mn0 > -INFINITY) { p00 = s00 ? __expf(sc[0] - mn0) : 0.f; p01 = s01 ? __expf(sc[1] - mn0) : 0.f; c0 = __expf(m0 - mn0); }
+              if (mn1 > -INFINITY) { p10 = s10 ? __expf(sc[2] - mn1) : 0.f; p11 = s11 ? __expf(sc[3] - mn1) : 0.f; c1 = __expf(m1 - mn1); }
+              float ps0 = p00 + p01, ps1 = p10 + p11;
+              ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1); ps1 += __shfl_xor_sync(0xffffffffu, ps1, 1);
+              ps0 += __shfl_xor_sync(0xffffffffu, ps0, 2); ps1 += __shfl_xor_sync(0xffffffffu, ps1, 2);
+              l0 = l0 * c0 + ps0; l1 = l1 * c1 + ps1;
+              m0 = mn0; m1 = mn1;
+              // weights as (hi, lo) halves: A operand rows g8r, g8r + 8, k = keys 2 t4, 2 t4 + 1
+              const __half2 ph0 = __floats2half2_rn(p00, p01), ph1 = __floats2half2_rn(p10, p11);
+              const float2 pf0 = __half22float2(ph0), pf1 = __half22float2(ph1);
+              const __half2 pl0 = __floats2half2_rn(p00 - pf0.x, p01 - pf0.y), pl1 = __floats2half2_rn(p10 - pf1.x, p11 - pf1.y);
+              const uint32_t ah0 = *reinterpret_cast<const uint32_t *>(&ph0), ah1 = *reinterpret_cast<const uint32_t *>(&ph1);
+              const uint32_t al0 = *reinterpret_cast<const uint32_t *>(&pl0), al1 = *reinterpret_cast<const uint32_t *>(&pl1);
+              // ---- values: out[16 rows][HD] += w[16 x 8 keys] v[8 keys x HD]
+              const uint32_t vrow = fresh ? smem_u32(v_s + (size_t)min(myk - pos0, 15) * 128)
+                                          : smem_u32(vst + (size_t)(bw * 32 + 8 * kq + (lane & 7)) * HD);
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                if (i < NR) {
-                  const bool seen = kv && key <= pos0 + 4 * i + rq;
-                  const float sv = seen ? sc[i] : -INFINITY;
-                  const float mx = warp_max(sv);
-                  const float mn = fmaxf(m[i], mx);
-                  float pe = 0.f, corr = 1.f;
-                  if (mn > -INFINITY) { pe = seen ? __expf(sv - mn) : 0.f; corr = __expf(m[i] - mn); }
-                  l[i] = l[i] * corr + warp_sum(pe);
-                  o[i][0] *= corr; o[i][1] *= corr; o[i][2] *= corr; o[i][3] *= corr;
-                  m[i] = mn;
-                  p_s[(cw * 4 + i) * 32 + lane] = pe;
-                }
-              __syncwarp();
-              const int nk = min(32, kend - kb0);
-              const __nv_bfloat16 *vb = vst + (size_t)bw * 32 * HD;
-              for (int kk = 0; kk < nk; ++kk) {
-                const int key2 = kb0 + kk;
-                const __nv_bfloat16 *vr = (key2 >= pos0 ? v_s + (key2 - pos0) * 128 : vb + kk * HD) + lane * VPL;
-                float vf[4] = {0.f, 0.f, 0.f, 0.f};
-                if (VPL == 4) {
-                  const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
-                  vf[0] = kv_lo(vv.x); vf[1] = kv_hi(vv.x); vf[2] = kv_lo(vv.y); vf[3] = kv_hi(vv.y);
-                } else {
-                  const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr);
-                  vf[0] = kv_lo(vv); vf[1] = kv_hi(vv);
-                }
+              for (int nq = 0; nq < 4; ++nq) {            // four 8-channel tiles per load
+                if (nq * 32 < HD) {
+                  uint32_t v0, v1, v2, v3;
+                  ldmatrix_x4_trans(vrow + ((nq * 4 + (lane >> 3)) << 4), v0, v1, v2, v3);
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  if (i < NR) {
-                    const float pe = p_s[(cw * 4 + i) * 32 + kk];
-                    o[i][0] += pe * vf[0]; o[i][1] += pe * vf[1]; o[i][2] += pe * vf[2]; o[i][3] += pe * vf[3];
+                  for (int j = 0; j < 4; ++j) {
+                    float *oo = o[nq * 4 + j];
+                    oo[0] *= c0; oo[1] *= c0; oo[2] *= c1; oo[3] *= c1;
+                    const uint32_t vb = j == 0 ? v0 : j == 1 ? v1 : j == 2 ? v2 : v3;
+                    mma_f16_k8(oo, ah0, ah1, vb);
+                    mma_f16_k8(oo, al0, al1, vb);
                   }
+                }
               }
             }
             named_bar(3, kNumCWarps * 32);   // every warp is done with this buffer
             if (ctid == 0 && rd + 2 < nround) issue_round(rd + 2);
           }
           // per-warp partials -> shared (over the staging areas, which every warp has left), merged over
-          // the two key blocks in block order, stored per (head, split)
+          // the eight warps in warp order, stored per (head, split)
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            if (i < NR) {
-              float *pp = part_s + (cw * 4 + i) * 130;
-              if (VPL == 4) { pp[lane * 4] = o[i][0]; pp[lane * 4 + 1] = o[i][1]; pp[lane * 4 + 2] = o[i][2]; pp[lane * 4 + 3] = o[i][3]; }
-              else { pp[lane * 2] = o[i][0]; pp[lane * 2 + 1] = o[i][1]; }
-              if (lane == 0) { pp[128] = m[i]; pp[129] = l[i]; }
+          for (int nt = 0; nt < 16; ++nt)
+            if (nt * 8 < HD) {
+              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r) * 130 + nt * 8 + 2 * t4) = make_float2(o[nt][0], o[nt][1]);
+              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r + 8) * 130 + nt * 8 + 2 * t4) = make_float2(o[nt][2], o[nt][3]);
             }
+          if (t4 == 0) {
+            part_s[(cw * 16 + g8r) * 130 + 128] = m0; part_s[(cw * 16 + g8r) * 130 + 129] = l0;
+            part_s[(cw * 16 + g8r + 8) * 130 + 128] = m1; part_s[(cw * 16 + g8r + 8) * 130 + 129] = l1;
+          }
+          named_bar(3, kNumCWarps * 32);
+          if (ctid < 16) {   // per row: maximum over the warps, each warp's weight, the merged sum
+            const int r = ctid;
+            float M = -INFINITY;
+            for (int w8 = 0; w8 < kNumCWarps; ++w8) M = fmaxf(M, part_s[(w8 * 16 + r) * 130 + 128]);
+            float lo = 0.f;
+            for (int w8 = 0; w8 < kNumCWarps; ++w8) {
+              const float mw = part_s[(w8 * 16 + r) * 130 + 128];
+              const float e = mw > -INFINITY ? __expf(mw - M) : 0.f;
+              lw_s[w8 * 16 + r] = e;
+              lo += part_s[(w8 * 16 + r) * 130 + 129] * e;
+            }
+            if (r < R) {
+              float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
+              __stcg(gp + HD, M); __stcg(gp + HD + 1, lo);
+            }
+          }
           named_bar(3, kNumCWarps * 32);
           for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
             const int r = i / HD, c = i - r * HD;
-            const int ri = r >> 2, rs = r & 3;
-            const float *pa = part_s + ((0 * 4 + rs) * 4 + ri) * 130, *pb = part_s + ((1 * 4 + rs) * 4 + ri) * 130;
-            const float M = fmaxf(pa[128], pb[128]);
-            float lo = 0.f, oo = 0.f;
-            if (M > -INFINITY) {
-              const float ea = __expf(pa[128] - M), eb = __expf(pb[128] - M);
-              lo = pa[129] * ea + pb[129] * eb;
-              oo = pa[c] * ea + pb[c] * eb;
-            }
-            float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
-            __stcg(gp + c, oo);
-            if (c == 0) { __stcg(gp + HD, M); __stcg(gp + HD + 1, lo); }
+            float oo = 0.f;
+#pragma unroll
+            for (int w8 = 0; w8 < kNumCWarps; ++w8) oo += part_s[(w8 * 16 + r) * 130 + c] * lw_s[w8 * 16 + r];
+            __stcg(p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2) + c, oo);
           }
           // the item that arrives last for this head merges the splits in split order
           __threadfence();
@@ -919,7 +979,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             __threadfence();
             // weights of the splits per row first (shared), then every output element is one pass of
             // independent loads over the splits
-            float *wgt = p_s;   // [8 splits][16 rows]
             if (ctid < 16 && ctid < R) {
               const int r = ctid;
               const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2);
