@@ -48,7 +48,9 @@ constexpr int kKc = 256;                         // k elements per activation ch
 constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
 constexpr int kStageBytes = 32 * 1024;           // largest ring stage: kb boxes of [box_rows x 64 k], kb = 2 or 4
 constexpr int kRingBytes = 128 * 1024;           // weight ring; stages take exactly the bytes of their boxes
-constexpr int kSlots = 16;                       // barrier pairs of the ring = most stages in flight
+constexpr int kFlight = 16;                      // most stages in flight
+constexpr int kSlots = 32;                       // barrier pairs of the ring: twice kFlight, so that a pair is not
+                                                 // reused before both producers have passed its previous use
 constexpr int kXBufs = 5;
 constexpr int kXBoxBytes = 32 * 128;             // activation box pair: 16 hi rows then 16 lo rows, 64 k
 constexpr int kXBufBytes = (kKc / kBoxK) * kXBoxBytes;    // 16 KB per chunk
@@ -512,13 +514,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   volatile int *abort_s = flag_s + 1;
   unsigned char *xbuf = smem + kRingBytes + kMiscBytes;
   float *red = reinterpret_cast<float *>(xbuf + kXBufs * kXBufBytes);
-  static_assert((2 * kSlots + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 + 4 * kSlots * 4 <= kMiscBytes, "misc area");
+  static_assert((2 * kSlots + 2 * kXBufs + 4) * 8 + (16 + 128) * 4 + 128 * 12 + 16 + 4 * kFlight * 4 <= kMiscBytes, "misc area");
   (void)red;
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
   uint64_t *attn_bar = accfull + 1;                        // attention: keys and values of a round have landed (two buffers)
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
-  uint32_t *st_rec = tmem_slot + 1;   // [2 producers][offsets, ends][kSlots]: records of the stages in flight
+  uint32_t *st_rec = tmem_slot + 1;   // [2 producers][offsets, ends][kFlight]: records of the stages in flight
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kSlots; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -544,10 +546,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   // ================================================================= weight producer
   if (warp == 0 || warp == 3) {
     const unsigned pidx = warp == 0 ? 0u : 1u;   // producer 0 loads the even stages, producer 1 the odd ones
-    uint32_t *st_off = st_rec + pidx * 2 * kSlots, *st_end = st_off + kSlots;   // this producer's own record of the stages
+    uint32_t *st_off = st_rec + pidx * 2 * kFlight, *st_end = st_off + kFlight;   // this producer's own record of the stages
     RingCursor cur{0, 0};
     unsigned tail = 0;   // stages [tail, cur.n) may still be unread
     uint32_t t_off = 0, t_end = 0;
+    unsigned pending = 0xffffffffu;   // newest retired stage not yet waited for
     for (int ph = 0; ph < nphase; ++ph) {
       int layer;
       const int kind = phase_kind(p, ph, layer);
@@ -573,22 +576,24 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const uint32_t bytes = (uint32_t)(nb * region);
             const uint32_t off = cur.take(bytes);
             const unsigned j = cur.n - 1, slot = j % kSlots;
-            st_off[slot] = off; st_end[slot] = off + bytes;
+            st_off[j % kFlight] = off; st_end[j % kFlight] = off + bytes;
             if (tail == j) { t_off = off; t_end = off + bytes; }
-            if ((j & 1u) != pidx) continue;   // the other producer's stage
             // The oldest stages in flight are the first ones a new stage can run into: they are retired until a
-            // barrier pair is free and no unread stage overlaps the new one.  One thread issues all products,
-            // so stages are read in order and waiting for the newest retired one covers the older ones.
-            // (t_off, t_end) is the record of stage `tail`, read ahead of its use.
-            {
-              unsigned last = 0xffffffffu;
-              while (tail < j && (j - tail >= (unsigned)kSlots || (t_off < off + bytes && off < t_end))) {
-                last = tail;
-                ++tail;
-                t_off = st_off[tail % kSlots];
-                t_end = st_end[tail % kSlots];
-              }
-              if (last != 0xffffffffu) mbar_wait(&empty[last % kSlots], (last / kSlots) & 1u, p.cnt, abort_s);
+            // barrier pair is free and no unread stage overlaps the new one.  Both producers retire for every
+            // stage, so that `tail` is always the oldest stage the ring still holds, but wait only before a
+            // stage of their own.  One thread issues all products, so stages are read in order and waiting
+            // for the newest retired one covers the older ones.  (t_off, t_end) is the record of stage
+            // `tail`, read ahead of its use.
+            while (tail < j && (j - tail >= (unsigned)kFlight || (t_off < off + bytes && off < t_end))) {
+              pending = tail;
+              ++tail;
+              t_off = st_off[tail % kFlight];
+              t_end = st_end[tail % kFlight];
+            }
+            if ((j & 1u) != pidx) continue;   // the other producer's stage
+            if (pending != 0xffffffffu) {
+              mbar_wait(&empty[pending % kSlots], (pending / kSlots) & 1u, p.cnt, abort_s);
+              pending = 0xffffffffu;
             }
             mbar_expect_tx(&full[slot], (unsigned)nb * tx_box);
             const uint32_t dst = smem_u32(ring) + off, bar = smem_u32(&full[slot]);
