@@ -545,6 +545,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 
   // ================================================================= weight producer
   if (warp == 0 || warp == 3) {
+    if (lane != 0) return;   // one thread produces (idle lanes walking the schedule would only steal its issue slots)
     const unsigned pidx = warp == 0 ? 0u : 1u;   // producer 0 loads the even stages, producer 1 the odd ones
     uint32_t *st_off = st_rec + pidx * 2 * kFlight, *st_end = st_off + kFlight;   // this producer's own record of the stages
     RingCursor cur{0, 0};
@@ -559,7 +560,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       if ((g.lm_rows ? lmT : T) <= 0) continue;
       const Slab s = make_slab(g, cta, ncta);
       if (s.rows == 0) continue;
-      if (lane != 0) continue;   // one thread produces: no warp synchronisation on the per-stage path
       // per-phase constants in registers (tensor map and first row of each m tile)
       int map0, map1, row0, row1;
       tile_source(g, s, 0, map0, row0);
