@@ -163,8 +163,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
-  if (mbar_test(bar, parity)) return;
+// (the spin is kept out of line: the kernel's phases together exceed the instruction cache, so every
+// copy of cold code that is not inlined into them makes the hot part smaller)
+__device__ __noinline__ void mbar_spin(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
   for (unsigned i = 0; i < kSpinLimit; ++i) {
     if (mbar_try(bar, parity)) return;
     if (*abort_flag) return;
@@ -172,6 +173,10 @@ __device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counte
   }
   *abort_flag = 1;
   atomicOr(&cnt->status, kStatTimeout);
+}
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
+  if (mbar_test(bar, parity)) return;
+  mbar_spin(bar, parity, cnt, abort_flag);
 }
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -459,28 +464,32 @@ struct RingCursor {
 // ---------------------------------------------------------------------------------- grid barrier
 
 // Warp 1 and the eight worker warps (288 threads) take part; the producers' and the issuer's warps do not.
-__device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoch, int tid, volatile int *abort_flag) {
+__device__ __noinline__ void grid_barrier_body(unsigned *gbar, Counters *cnt, unsigned long long *phase_ns, unsigned epoch, int tid,
+                                              volatile int *abort_flag) {
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
-  ++epoch;
   if (tid == 32) {
     __threadfence();
-    atomicAdd(p.gbar, 1u);
+    atomicAdd(gbar, 1u);
     const unsigned target = epoch * gridDim.x;
     bool ok = false;
     for (unsigned i = 0; i < kSpinLimit && !*abort_flag; ++i) {
-      if (ld_acquire(p.gbar) >= target) { ok = true; break; }
-      if ((i & 63) == 63 && (ld_acquire(reinterpret_cast<const unsigned *>(&p.cnt->status)) & kStatTimeout)) break;
+      if (ld_acquire(gbar) >= target) { ok = true; break; }
+      if ((i & 63) == 63 && (ld_acquire(reinterpret_cast<const unsigned *>(&cnt->status)) & kStatTimeout)) break;
       if (i > 4096) __nanosleep(64);   // a barrier normally completes within a few polls
     }
-    if (!ok) { *abort_flag = 1; atomicOr(&p.cnt->status, kStatTimeout); }
+    if (!ok) { *abort_flag = 1; atomicOr(&cnt->status, kStatTimeout); }
     __threadfence();
-    if (p.phase_ns && blockIdx.x == 0 && epoch < 511) {
+    if (phase_ns && blockIdx.x == 0 && epoch < 511) {
       unsigned long long t;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-      p.phase_ns[epoch] = t;
+      phase_ns[epoch] = t;
     }
   }
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
+}
+__device__ __forceinline__ void grid_barrier(const PassParams &p, unsigned &epoch, int tid, volatile int *abort_flag) {
+  ++epoch;
+  grid_barrier_body(p.gbar, p.cnt, p.phase_ns, epoch, tid, abort_flag);
 }
 
 // optional fine-grained clock of CTA 0's first consumer lane: 4 stamps per phase after the 512 barrier stamps
@@ -1100,11 +1109,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     const int rslab = mi * s.box_rows + rloc;                   // row inside the slab
     const bool valid = active_warp && rloc < s.box_rows && rslab < s.rows;
     const int vrow = s.seg * g.Nseg + s.r0 + rslab;             // output column
-    float ssl[16];
-    Top2 tb[16];
-#pragma unroll
-    for (int t = 0; t < 16; ++t) { ssl[t] = 0.f; tb[t].v1 = -INFINITY; tb[t].i1 = 0x7fffffff; tb[t].v2 = -INFINITY; }
 
+    // the CTA that runs the epilogue of a K-split group is the one of the last split
+    const bool reducer = s.ks > 1 && s.kj == s.ks - 1;
+    // old residual values, fetched while the products run
+    float hold[16];
+#pragma unroll
+    for (int t = 0; t < 16; ++t)
+      hold[t] = (valid && (s.ks == 1 || reducer) && g.epi == EPI_RESID_H && t < Tg) ? __ldcg(p.h + (size_t)t * p.d + vrow) : 0.f;
     if (s.rows > 0) {
       mbar_wait(accfull, acc_phase & 1u, p.cnt, abort_s);
       ++acc_phase;
@@ -1141,89 +1153,111 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     tc_fence_before();
     bool do_epi = true;
     if (s.ks > 1 && s.rows > 0) {
-      // K-split group: publish the partial sums; the CTA that arrives last adds the ks partials in split
-      // order (all read back from memory, its own included, so the order never depends on who is last)
-      if (valid)
+      // K-split group: the CTA of the last split adds the partial sums in split order, its own last; the
+      // others publish theirs and go on to the barrier.
+      if (!reducer) {
+        if (valid)
 #pragma unroll
-        for (int t = 0; t < 16; ++t)
-          if (t < Tg) __stcg(p.kpart + ((size_t)(s.kj * 16 + t)) * p.d + vrow, yy[t]);
-      __threadfence();
-      named_bar(3, kNumCWarps * 32);
-      if (ctid == 0) *flag_s = (atomicAdd(p.kcnt + s.group, 1) == s.ks - 1);
-      named_bar(3, kNumCWarps * 32);
-      do_epi = *flag_s != 0;
-      if (do_epi) {
+          for (int t = 0; t < 16; ++t)
+            if (t < Tg) __stcg(p.kpart + ((size_t)(s.kj * 16 + t)) * p.d + vrow, yy[t]);
         __threadfence();
+        named_bar(3, kNumCWarps * 32);
+        if (ctid == 0) atomicAdd(p.kcnt + s.group, 1);
+        do_epi = false;
+      } else {
+        if (lane == 0) {   // every warp waits for the ks - 1 other partials by itself (bounded)
+          const unsigned *cntp = reinterpret_cast<const unsigned *>(p.kcnt + s.group);
+          bool ok = false;
+          for (unsigned i = 0; i < kSpinLimit && !*abort_s; ++i) {
+            if (ld_acquire(cntp) >= (unsigned)(s.ks - 1)) { ok = true; break; }
+            if (i > 4096) __nanosleep(64);
+          }
+          if (!ok) { *abort_s = 1; atomicOr(&p.cnt->status, kStatTimeout); }
+        }
+        __syncwarp();
         if (valid) {
+          float pv[16][3];   // 48 independent loads in flight, then the sums in split order
 #pragma unroll
-          for (int t0 = 0; t0 < 16; t0 += 8) {   // 32 independent loads in flight, then the sums in split order
-            float pv[8][4];
+          for (int t = 0; t < 16; ++t)
 #pragma unroll
-            for (int t = 0; t < 8; ++t)
+            for (int j = 0; j < 3; ++j)
+              pv[t][j] = (t < Tg && j < s.ks - 1) ? __ldcg(p.kpart + ((size_t)(j * 16 + t)) * p.d + vrow) : 0.f;
 #pragma unroll
-              for (int j = 0; j < 4; ++j)
-                pv[t][j] = (t0 + t < Tg && j < s.ks) ? __ldcg(p.kpart + ((size_t)(j * 16 + t0 + t)) * p.d + vrow) : 0.f;
-#pragma unroll
-            for (int t = 0; t < 8; ++t) yy[t0 + t] = ((pv[t][0] + pv[t][1]) + pv[t][2]) + pv[t][3];
+          for (int t = 0; t < 16; ++t) {
+            float a = pv[t][0];
+            if (s.ks > 2) a += pv[t][1];
+            if (s.ks > 3) a += pv[t][2];
+            yy[t] = a + yy[t];
           }
         }
-        if (ctid == 0) p.kcnt[s.group] = 0;
       }
     }
-    if (valid && do_epi) {
-      float hold[16];
+    // The loop over the pass rows is not unrolled (the unrolled epilogues were a sixth of the kernel's code,
+    // which as a whole no longer fitted the instruction cache): each thread first parks its values in a
+    // column of shared memory that only it touches (the activation buffers are idle once the accumulator
+    // is complete), then walks the rows.
+    float *ys = reinterpret_cast<float *>(xbuf) + ctid;   // [16][256] accumulator values
+    float *us = ys + 16 * 256;                            // [16][256] up-projection values (SwiGLU)
+    float *hs = us + 16 * 256;                            // [16][256] old residual values
 #pragma unroll
-      for (int t = 0; t < 16; ++t)
-        hold[t] = (g.epi == EPI_RESID_H && t < Tg) ? __ldcg(p.h + (size_t)t * p.d + vrow) : 0.f;
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
-        if (t < Tg) {
-          const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
-          const float y = yy[t] * sc;
-          if (g.epi == EPI_STORE_QKV) {
-            p.qkv[(size_t)t * 3 * p.d + vrow] = y;
-          } else if (has_ss) {
-            float *hp = p.h + (size_t)t * p.d + vrow;
-            const float hn = hold[t] + y;
-            *hp = hn;
-            ssl[t] = hn * hn;
-            const float gn = g.gain_next ? __bfloat162float(g.gain_next[vrow]) : 1.f;
-            xstore(p.xa, t, vrow, hn * gn);
-          } else if (sw) {
-            const float up = uu[t] * sc;
-            xstore(p.ac, t, vrow, (y / (1.f + __expf(-y))) * up);
-          } else {  // EPI_ARGMAX_LM
-            if (p.logits) {
-              const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
-              p.logits[(size_t)slot_out * p.V + vrow] = y;
-            }
-            tb[t].v1 = y; tb[t].i1 = vrow;
-          }
+    for (int t = 0; t < 16; ++t) {
+      ys[t * 256] = yy[t];
+      if (sw) us[t * 256] = uu[t];
+      if (g.epi == EPI_RESID_H) hs[t * 256] = hold[t];
+    }
+    const bool act = valid && do_epi;
+    const float gn = (act && has_ss && g.gain_next) ? __bfloat162float(g.gain_next[vrow]) : 1.f;
+    const int epi = g.epi;
+#pragma unroll 1
+    for (int t = 0; t < Tg; ++t) {
+      const float sc = g.scale_inv_rms ? inv_rms[t] : 1.f;
+      const float y = ys[t * 256] * sc;
+      if (epi == EPI_STORE_QKV) {
+        if (act) p.qkv[(size_t)t * 3 * p.d + vrow] = y;
+      } else if (has_ss) {
+        float hn = 0.f;
+        if (act) {
+          hn = (epi == EPI_RESID_H ? hs[t * 256] : 0.f) + y;
+          p.h[(size_t)t * p.d + vrow] = hn;
+          xstore(p.xa, t, vrow, hn * gn);
         }
+        // sum of squares per pass row: over the warp's 32 weight rows, then over the warps in order (below)
+        const float r = warp_sum(hn * hn);
+        if (lane == 0) ssw[cw * 16 + t] = r;
+      } else if (sw) {
+        if (act) {
+          const float up = us[t * 256] * sc;
+          xstore(p.ac, t, vrow, (y / (1.f + __expf(-y))) * up);
+        }
+      } else {  // EPI_ARGMAX_LM: the warp's two largest logits of this pass row
+        Top2 b;
+        b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+        if (act) {
+          if (p.logits) {
+            const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
+            p.logits[(size_t)slot_out * p.V + vrow] = y;
+          }
+          b.v1 = y; b.i1 = vrow;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+        if (lane == 0) topw[cw * 16 + t] = b;
       }
     }
     if (has_ss) {
-      // per pass row: sum over the warp's 32 weight rows, then over the warps in order
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
-        const float r = warp_sum(ssl[t]);
-        if (lane == 0) ssw[cw * 16 + t] = r;
-      }
+      if (lane >= Tg && lane < 16) ssw[cw * 16 + lane] = 0.f;
       named_bar(3, kNumCWarps * 32);
       if (cw == 0 && lane < 16) {
         float r = 0.f;
         for (int w = 0; w < kNumCWarps; ++w) r += ssw[w * 16 + lane];
         p.ss_part[(size_t)cta * 16 + lane] = r;
       }
-    } else if (g.epi == EPI_ARGMAX_LM) {
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
-        Top2 b = tb[t];
-        if (t < Tg) {
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
-        }
-        if (lane == 0) topw[cw * 16 + t] = b;
+      if (reducer && do_epi && ctid == 0) p.kcnt[s.group] = 0;   // every warp has seen the count (barrier above)
+    } else if (epi == EPI_ARGMAX_LM) {
+      if (lane >= Tg && lane < 16) {
+        Top2 b;
+        b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+        topw[cw * 16 + lane] = b;
       }
       named_bar(3, kNumCWarps * 32);
       if (cw == 0 && lane < 16) {
