@@ -51,10 +51,13 @@ typedef struct {
   float rope_theta, rms_eps;
   int32_t ldlp_hidden;  /* hidden width of the predictor MLP */
   int32_t n_max;        /* largest draft length (k_max of Eq. 3), 1..15 */
-  int32_t ldlp_mode;    /* 0: class logits, n = argmax + 1 (the classification variant of Section 4.3.2) */
+  int32_t ldlp_mode;    /* 0: class logits, n = argmax + 1 (the classification variant of Section 4.3.2);
+                         * 1: one scalar, n = clip(round(z), k_min, n_max) (Eq. 3; ties round to even)      */
   int32_t max_batch;    /* sequences decoded together, 1..8 */
   int32_t kv_capacity;  /* positions per sequence, multiple of page_size */
   int32_t page_size;    /* KV page length in positions: 64 */
+  int32_t ldlp_blocks;  /* ldlp_mode 1: residual blocks h += ReLU(W_r h + b_r) between the two linear maps, 0..8 */
+  int32_t k_min;        /* ldlp_mode 1: smallest draft length (k_min of Eq. 3), 1..n_max                         */
 } ada_config;
 
 /* Device pointers to bf16 tensors.  Per-layer members are HOST arrays of n_layers device pointers. */
@@ -69,7 +72,8 @@ typedef struct {
   const void *eagle_fc;   /* [d][2d], input [embedding ; feature]                           */
   const void *e_wq, *e_wk, *e_wv, *e_wo, *e_gate, *e_up, *e_down, *e_norm_attn, *e_norm_mlp;
   const void *ldlp_w1, *ldlp_b1; /* [hid][2d], [hid]   input [embedding ; feature] (Section 3.3) */
-  const void *ldlp_w2, *ldlp_b2; /* [n_max][hid], [n_max]                                   */
+  const void *ldlp_w2, *ldlp_b2; /* [n_max][hid], [n_max]   (ldlp_mode 1 reads row 0 and entry 0 only) */
+  const void *ldlp_wr, *ldlp_br; /* ldlp_mode 1: [ldlp_blocks][hid][hid], [ldlp_blocks][hid]; else unused (may be NULL) */
 } ada_weights;
 
 /* Bytes of device workspace (KV pools, feature rows, scratch) ada_init needs for this config;

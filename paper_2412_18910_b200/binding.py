@@ -28,19 +28,21 @@ class AdaError(RuntimeError):
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
-               [(n, C.c_int32) for n in ("ldlp_hidden", "n_max", "ldlp_mode", "max_batch", "kv_capacity", "page_size")]
+               [(n, C.c_int32) for n in ("ldlp_hidden", "n_max", "ldlp_mode", "max_batch", "kv_capacity", "page_size",
+                                         "ldlp_blocks", "k_min")]
 
 
 _PER_LAYER = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm_attn", "norm_mlp")
 _SINGLE_A = ("embed", "lm_head", "final_norm")
 _SINGLE_B = ("eagle_fc", "e_wq", "e_wk", "e_wv", "e_wo", "e_gate", "e_up", "e_down", "e_norm_attn", "e_norm_mlp",
              "ldlp_w1", "ldlp_b1", "ldlp_w2", "ldlp_b2")
+_OPTIONAL = ("ldlp_wr", "ldlp_br")   # scalar-form predictor only
 _ALIAS = {"e_gate": "e_w_gate", "e_up": "e_w_up", "e_down": "e_w_down"}
 
 
 class Weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in _SINGLE_A] + [(n, C.POINTER(C.c_void_p)) for n in _PER_LAYER] + \
-               [(n, C.c_void_p) for n in _SINGLE_B]
+               [(n, C.c_void_p) for n in _SINGLE_B + _OPTIONAL]
 
 
 _lib = None
@@ -105,7 +107,7 @@ class Engine:
     """
 
     def __init__(self, shape, weights: dict, max_batch: int = 1, kv_capacity: int = 4096, device: str = "cuda:0",
-                 stream=None):
+                 stream=None, ldlp_mode: int = 0, ldlp_blocks: int = 2, k_min: int = 1):
         import numpy as np
         import torch
 
@@ -118,8 +120,8 @@ class Engine:
         torch.cuda.set_device(self.dev)
         self.B, self.nmax, self.cap = max_batch, shape.n_max, kv_capacity
         self.cfg = Config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
-                          shape.rope_theta, shape.rms_eps, shape.ldlp_hidden, shape.n_max, 0, max_batch, kv_capacity,
-                          64)
+                          shape.rope_theta, shape.rms_eps, shape.ldlp_hidden, shape.n_max, ldlp_mode, max_batch,
+                          kv_capacity, 64, ldlp_blocks, k_min)
         need = self.L.ada_workspace_bytes(C.byref(self.cfg))
         if need == 0:
             raise AdaError("invalid configuration")
@@ -135,6 +137,11 @@ class Engine:
             t = up(weights[_ALIAS.get(n, n)])
             self.w[n] = t
             setattr(cw, n, t.data_ptr())
+        for n in _OPTIONAL:
+            if ldlp_mode == 1 and ldlp_blocks > 0:
+                t = up(weights[n][:ldlp_blocks])
+                self.w[n] = t
+                setattr(cw, n, t.data_ptr())
         for n in _PER_LAYER:
             ts = [up(a) for a in weights[n]]
             self.w[n] = ts

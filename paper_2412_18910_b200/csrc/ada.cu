@@ -38,7 +38,7 @@ struct ada_ctx {
   int pages_per_seq, n_pages;
   std::vector<LayerW> layers;
   LayerW eagle;
-  const bf16 *embed, *lm_head, *final_norm, *eagle_fc, *ldlp_w1, *ldlp_b1, *ldlp_w2, *ldlp_b2;
+  const bf16 *embed, *lm_head, *final_norm, *eagle_fc, *ldlp_w1, *ldlp_b1, *ldlp_w2, *ldlp_b2, *ldlp_wr, *ldlp_br;
   // workspace pieces (device)
   bf16 *tk, *tv, *dk, *dv;          // KV pools: target [page][L][H][ps][hd], draft [page][1][H][ps][hd]
   int *page_table;                  // [B][pages_per_seq]
@@ -49,7 +49,7 @@ struct ada_ctx {
   SeqState *st;                     // [B]
   Counters *cnt;
   Pass *pass;
-  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_z;
+  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z;
   bf16 *xhi, *xlo, *x2hi, *x2lo;    // [TP][ldx], [TP][ldx2]
   int ldx, ldx2;
   int *gemm_cnt;
@@ -132,7 +132,8 @@ bool config_ok(const ada_config *c) {
   if (c->n_heads < 1 || c->d_model != c->n_heads * c->head_dim) return false;
   if (c->d_model % 64 || c->d_ffn % 16 || c->d_ffn < 16 || c->vocab % 16 || c->vocab < 16) return false;
   if (c->ldlp_hidden < 1 || c->n_max < 1 || c->n_max > ADA_MAX_NMAX) return false;
-  if (c->ldlp_mode != 0) return false;
+  if (c->ldlp_mode != 0 && c->ldlp_mode != 1) return false;
+  if (c->ldlp_mode == 1 && (c->ldlp_blocks < 0 || c->ldlp_blocks > 8 || c->k_min < 1 || c->k_min > c->n_max)) return false;
   if (c->max_batch < 1 || c->max_batch > ADA_MAX_BATCH) return false;
   if (c->max_batch * (c->n_max + 1) > 88) return false;
   if (c->page_size != 64 || c->kv_capacity < 64 || c->kv_capacity % c->page_size) return false;
@@ -213,6 +214,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->gemm_cnt = w.take<int>(4096);
   x->amax = w.take<float4>(((V + 63) / 64) * TP);
   x->ldlp_h = w.take<float>(B * c->ldlp_hidden);
+  x->ldlp_h2 = w.take<float>(B * c->ldlp_hidden);
   x->ldlp_z = w.take<float>(B * 16);
   x->draft = w.take<int>(B * c->n_max);
   x->target = w.take<int>(B * (c->n_max + 1));
@@ -464,8 +466,15 @@ void enqueue_ldlp(ada_ctx *x, int *d_n) {
   dim3 g((c.ldlp_hidden + 7) / 8, x->B);
   LAUNCH(x, k_ldlp_hidden, g, 256, 0, x->st, x->tok, x->feat, c.kv_capacity, x->embed, x->ldlp_w1, x->ldlp_b1,
          c.d_model, c.ldlp_hidden, x->ldlp_h);
-  LAUNCH(x, k_ldlp_out, x->B, 32, 0, x->st, x->ldlp_h, x->ldlp_w2, x->ldlp_b2, c.ldlp_hidden, c.n_max, c.kv_capacity,
-         x->force_n_dev, x->has_force_n, x->ldlp_z, d_n, x->cnt);
+  float *hin = x->ldlp_h, *hout = x->ldlp_h2;
+  if (c.ldlp_mode == 1)
+    for (int blk = 0; blk < c.ldlp_blocks; ++blk) {   // residual blocks of the scalar form, ping-pong buffers
+      LAUNCH(x, k_ldlp_block, g, 256, 0, x->st, hin, hout, x->ldlp_wr + (size_t)blk * c.ldlp_hidden * c.ldlp_hidden,
+             x->ldlp_br + (size_t)blk * c.ldlp_hidden, c.ldlp_hidden);
+      float *t = hin; hin = hout; hout = t;
+    }
+  LAUNCH(x, k_ldlp_out, x->B, 32, 0, x->st, hin, x->ldlp_w2, x->ldlp_b2, c.ldlp_hidden, c.n_max, c.ldlp_mode, c.k_min,
+         c.kv_capacity, x->force_n_dev, x->has_force_n, x->ldlp_z, d_n, x->cnt);
 }
 
 void enqueue_draft(ada_ctx *x) {
@@ -518,6 +527,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
                            w->ldlp_w2, w->ldlp_b2};
   for (const void *p : singles)
     if (!p || ((uintptr_t)p & 15)) return ADA_ERR_NULL;
+  if (cfg->ldlp_mode == 1 && cfg->ldlp_blocks > 0 && (!w->ldlp_wr || !w->ldlp_br)) return ADA_ERR_NULL;
   const void *const *per[] = {w->wq, w->wk, w->wv, w->wo, w->w_gate, w->w_up, w->w_down, w->norm_attn, w->norm_mlp};
   for (auto arr : per) {
     if (!arr) return ADA_ERR_NULL;
@@ -544,6 +554,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   x->eagle_fc = (const bf16 *)w->eagle_fc;
   x->ldlp_w1 = (const bf16 *)w->ldlp_w1; x->ldlp_b1 = (const bf16 *)w->ldlp_b1;
   x->ldlp_w2 = (const bf16 *)w->ldlp_w2; x->ldlp_b2 = (const bf16 *)w->ldlp_b2;
+  x->ldlp_wr = (const bf16 *)w->ldlp_wr; x->ldlp_br = (const bf16 *)w->ldlp_br;
   x->force_draft = nullptr; x->has_force_n = 0; x->launches = 0; x->graph = nullptr; x->graph_launches = 0;
   x->graph_key = -1;
   x->capture_stream = nullptr;

@@ -707,17 +707,34 @@ __global__ void k_ldlp_hidden(const SeqState *st, const int *tok, const float *f
   if (lane == 0) hbuf[(size_t)b * hid + u] = fmaxf(s + __bfloat162float(b1[u]), 0.f);
 }
 
-// Stage 2: z = W2 h + b2, n = argmax + 1 (lowest index among equals), then the override and the
-// clip to the cache capacity.  One warp per sequence.
+// Scalar form (Eq. 3), one residual block: hout = hin + ReLU(W_r hin + b_r).  One warp per unit.
+__global__ void k_ldlp_block(const SeqState *st, const float *hin, float *hout, const __nv_bfloat16 *wr,
+                             const __nv_bfloat16 *br, int hid) {
+  const int b = blockIdx.y;
+  const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (u >= hid || st[b].len < 2) return;
+  const __nv_bfloat16 *w = wr + (size_t)u * hid;
+  const float *h = hin + (size_t)b * hid;
+  float s = 0.f;
+  for (int i = lane; i < hid; i += 32) s += __bfloat162float(w[i]) * h[i];
+  s = warp_sum(s);
+  if (lane == 0) hout[(size_t)b * hid + u] = h[u] + fmaxf(s + __bfloat162float(br[u]), 0.f);
+}
+
+// Stage 2: z = W2 h + b2, then n = argmax + 1 (class form, lowest index among equals) or
+// n = clip(round-half-even(z_0), k_min, n_max) (scalar form, Eq. 3), then the override and the clip to the
+// cache capacity.  One warp per sequence.
 __global__ void k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 *w2, const __nv_bfloat16 *b2,
-                           int hid, int nmax, int cap, const int *force_n, int has_force, float *zbuf,
+                           int hid, int nmax, int mode, int kmin, int cap, const int *force_n, int has_force, float *zbuf,
                            int *n_out, Counters *cnt) {
   const int b = blockIdx.x, lane = threadIdx.x;
   const int len = st[b].len;
   if (len < 2) { if (lane == 0) { st[b].n = 0; if (n_out) n_out[b] = 0; } return; }
   float best = -INFINITY;
   int bi = 0;
-  for (int c = 0; c < nmax; ++c) {
+  const int nz = mode == 0 ? nmax : 1;
+  for (int c = 0; c < nz; ++c) {
     float s = 0.f;
     for (int i = lane; i < hid; i += 32) s += __bfloat162float(w2[(size_t)c * hid + i]) * hbuf[(size_t)b * hid + i];
     s = warp_sum(s) + __bfloat162float(b2[c]);
@@ -726,6 +743,7 @@ __global__ void k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 
   }
   if (lane == 0) {
     int n = bi + 1;
+    if (mode != 0) n = (int)fminf(fmaxf(rintf(best), (float)kmin), (float)nmax);   // best = z_0
     if (has_force) n = force_n[b];
     const int room = cap - len - 1;  // the n + 1 tokens this iteration may commit must fit: len + n + 1 <= cap
     if (n > room) { n = room < 0 ? 0 : room; atomicOr(&cnt->status, kStatKvFull); }

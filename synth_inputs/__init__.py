@@ -121,6 +121,9 @@ def scaled(shape: Shape, **kw) -> Shape:
 TARGET_LAYER_TENSORS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")
 
 
+LDLP_BLOCKS = 2   # residual blocks generated for the scalar-form predictor
+
+
 def make_weights(shape: Shape, seed: int = DEFAULT_SEED) -> dict:
     """All model tensors as uint16 bf16 bit patterns, row-major [out][in].
 
@@ -146,6 +149,9 @@ def make_weights(shape: Shape, seed: int = DEFAULT_SEED) -> dict:
     w["ldlp_b1"] = normal_bf16(seed, "ldlp.b1", (hid,))
     w["ldlp_w2"] = normal_bf16(seed, "ldlp.w2", (nmax, hid))
     w["ldlp_b2"] = normal_bf16(seed, "ldlp.b2", (nmax,))
+    # scalar-form predictor (Eq. 3): residual blocks between the two linear maps
+    w["ldlp_wr"] = normal_bf16(seed, "ldlp.wr", (LDLP_BLOCKS, hid, hid))
+    w["ldlp_br"] = normal_bf16(seed, "ldlp.br", (LDLP_BLOCKS, hid))
     return w
 
 

@@ -19,12 +19,20 @@ def _top2_gap(z):
     return float(s[-1] - s[-2]) if len(s) > 1 else float("inf")
 
 
-def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n=False):
-    """o: dict from oracle Seq.step().  Returns (ok, exempt, needs_resync, message)."""
+def _round_gap(z):
+    """Distance of a scalar from the nearest point where rounding to an integer changes."""
+    return abs((float(z) - np.floor(float(z))) - 0.5)
+
+
+def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n=False, ldlp_scalar=False):
+    """o: dict from oracle Seq.step().  Returns (ok, exempt, needs_resync, message).
+
+    ldlp_scalar: the predictor is the scalar form (Eq. 3): its decision flips where z crosses k + 1/2."""
     exempt = 0
     n = o["n"]
     if g_n != n:
-        if forced_n or _top2_gap(o["ldlp_z"][:n_max]) > LDLP_MARGIN:
+        gap = _round_gap(o["ldlp_z"][0]) if ldlp_scalar else _top2_gap(o["ldlp_z"][:n_max])
+        if forced_n or gap > LDLP_MARGIN:
             return False, 0, True, "draft length %d != oracle %d" % (g_n, n)
         return True, 1, list(g_emitted) != list(o["emitted"]), "n flipped inside the predictor margin"
     for i in range(n):
@@ -49,7 +57,7 @@ def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n
     return True, exempt, False, ""
 
 
-def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=None):
+def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=None, ldlp_scalar=False):
     """Runs `iters` ada_step iterations against oracle sequences (one per batch slot).
 
     Returns dict(iterations, exempt, failures[list of str], tokens[list per seq]).
@@ -76,7 +84,7 @@ def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=
         gd, gt = draft_buf.cpu().numpy(), target_buf.cpu().numpy()
         for b, o in enumerate(olist):
             ok, ex, resync, msg = compare_iteration(o, g["n"][b], gd[b], gt[b], g["k"][b], g["emitted"][b], nmax,
-                                                    forced_n=n_forced >= 0)
+                                                    forced_n=n_forced >= 0, ldlp_scalar=ldlp_scalar)
             compared += 1
             exempt += ex
             if not ok:

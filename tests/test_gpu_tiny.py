@@ -87,6 +87,50 @@ def test_step_lockstep(tiny, eng, n_forced):
     assert res["exempt"] <= res["iterations"] // 2
 
 
+def test_scalar_form_predictor_lockstep(tiny):
+    """Eq. 3 in its scalar form: residual blocks, one output, round (ties to even) and clip to [k_min, n_max].
+    The predictor's weights are rescaled so that the scalar really moves over the whole range."""
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, _ = tiny
+    hid = sh.ldlp_hidden
+    w2 = dict(w)
+    w2["ldlp_w1"] = si.normal_bf16(7, "t.ldlp.w1", (hid, 2 * sh.d_model), std=0.08)
+    w2["ldlp_wr"] = si.normal_bf16(7, "t.ldlp.wr", (2, hid, hid), std=0.08)
+    w2["ldlp_w2"] = si.normal_bf16(7, "t.ldlp.w2", (sh.n_max, hid), std=0.1)
+    b2 = si.normal_bf16(7, "t.ldlp.b2", (sh.n_max,))
+    b2[0] = np.frombuffer(np.float32(9.0).tobytes(), dtype=np.uint16)[1]   # bf16 bits of 9.0
+    w2["ldlp_b2"] = b2
+    seen = set()
+    for k_min in (1, 6):
+        m = oracle.Model(sh, w2, ldlp_mode=1, ldlp_blocks=2, k_min=k_min)
+        e = Engine(sh, w2, max_batch=1, kv_capacity=sh.kv_capacity, ldlp_mode=1, ldlp_blocks=2, k_min=k_min)
+        try:
+            seq, t_o, t_g = _prefill_both(e, m, prompt)
+            assert t_o == t_g
+            zbuf = e.ada_debug_buffer(1, torch.float32, (1, 16))
+            for it in range(10):   # the scalar itself, before any decision
+                o = seq.step()
+                g = e.step()
+                assert abs(float(zbuf[0, 0]) - float(o["ldlp_z"][0])) < 2e-2
+                ok, ex, resync, msg = lockstep.compare_iteration(o, g["n"][0], *_bufs(e), g["k"][0], g["emitted"][0],
+                                                                 sh.n_max, ldlp_scalar=True)
+                assert ok, msg
+                assert k_min <= g["n"][0] <= sh.n_max
+                seen.add(int(g["n"][0]))
+                if resync:
+                    em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(e.dev)
+                    e.ada_force_commit(0, em, len(o["emitted"]))
+        finally:
+            e.close()
+    assert len(seen) >= 3, "the test's predictor should produce several different lengths, saw %s" % sorted(seen)
+
+
+def _bufs(e):
+    d = e.ada_debug_buffer(7, torch.int32, (e.B, e.nmax)).cpu().numpy()[0]
+    t = e.ada_debug_buffer(8, torch.int32, (e.B, e.nmax + 1)).cpu().numpy()[0]
+    return d, t
+
+
 def test_teacher_forced_drafts_accept_everything(tiny, eng):
     sh, w, prompt, m = tiny
     ar = oracle.decode(m, prompt, 120, n_policy=0)["tokens"]

@@ -25,3 +25,15 @@ def test_workspace_size_is_reported_without_a_gpu():
     assert 2 * 2 * 32 * 4096 * 4096 < n < 8 * 2**30          # at least the KV pool, well under 8 GiB
     bad = pkg.Config(32, 4096, 32, 128, 11008, 32000, 1e4, 1e-6, 512, 16, 0, 1, 4096, 64)   # n_max too large
     assert L.ada_workspace_bytes(C.byref(bad)) == 0
+
+
+def test_scalar_predictor_configuration_is_validated():
+    import ctypes as C
+    import paper_2412_18910_b200 as pkg
+    L = pkg.lib()
+    base = (32, 4096, 32, 128, 11008, 32000, 1e4, 1e-6, 512, 10)
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 1, 1, 4096, 64, 2, 1))) > 0      # Eq. 3, k_min = 1
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 1, 1, 4096, 64, 2, 0))) == 0     # k_min below 1
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 1, 1, 4096, 64, 2, 11))) == 0    # k_min above n_max
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 1, 1, 4096, 64, 9, 1))) == 0     # too many blocks
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 2, 1, 4096, 64, 2, 1))) == 0     # unknown mode
