@@ -4,8 +4,8 @@
 //
 // Why: a 7B verify pass streams 13.2 GB of weights in about 2 ms at HBM speed; one layer is ~60 us.
 // Nine separate launches per layer lose a large share of that to launch gaps, ramp-up and tails.
-// Here each CTA owns a fixed slab of rows of every weight matrix (N / gridDim rows), and a
-// producer warp streams those slabs through a shared-memory ring with TMA tiled loads
+// Here each CTA owns a fixed slab of rows of every weight matrix (N / gridDim rows), and two
+// producer threads stream those slabs through a shared-memory ring with TMA tiled loads
 // (cp.async.bulk.tensor.2d, 128-byte swizzle, mbarrier transaction counts; one 4 KB box per
 // instruction -- separate 512-byte bulk copies were measured to cap a CTA near 12 GB/s).  Weights do not depend on activations, so the
 // producer runs ahead across phase boundaries: while the other warps sit in a grid barrier or in
@@ -25,13 +25,15 @@
 // 40 % of the streaming rate.)
 //
 // Roles inside a CTA (12 warps):
-//   warp 0        weight producer: walks the static schedule of (phase, k chunk, k boxes, m tile) stages
+//   warps 0, 3    weight producers, one thread each: both walk the static schedule of (phase, k chunk,
+//                 k boxes, m tile) stages; warp 0 loads the even stages, warp 3 the odd ones (a single
+//                 thread's mbarrier / TMA issue latency, about 700 cycles per stage, was the limit of the loops)
 //   warp 1        activation producer: per GEMM phase (after the grid barrier that makes its input
 //                 visible) copies the input planes chunk by chunk into shared memory
-//   warps 2, 3    lane 0 of each issues tcgen05.mma and commit (two issuers: one thread's issue
-//                 rate is too low for short slabs); warp 2 also owns the tensor-memory allocation
+//   warp 2        one elected thread issues every tcgen05.mma and commit, in schedule order; the warp
+//                 also owns the tensor-memory allocation
 //   warps 4..11   workers: epilogues out of tensor memory (tcgen05.ld: one weight row per thread),
-//                 attention, row-wise phases
+//                 attention (mma.sync on the 16-bit cache elements), row-wise phases
 //
 // Every wait (mbarrier, grid barrier) is bounded; when a bound is hit the kernel sets a status bit
 // and carries on as if the wait had succeeded, so it always terminates.
