@@ -1271,18 +1271,38 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     stamp(p, ph, 3, stamper);
     grid_barrier(p, epoch, tid, abort_s);
 
-    if (g.epi == EPI_ARGMAX_LM && cta == 0 && cw == 0 && lane < 16 && lane < Tg) {
-      // greedy choice per row: candidates of all CTAs merged in CTA order
+    if (g.epi == EPI_ARGMAX_LM && cta == 0) {
+      // greedy choice per row: the candidates of all CTAs merged (largest value, lowest index among equals, so
+      // any merge order gives the same result).  Warp w takes rows 2w and 2w + 1, 16 lanes per row, each lane
+      // the CTAs congruent to it mod 16 with all its loads in flight at once.
+      const int row = 2 * cw + (lane >> 4), l16 = lane & 15;
       Top2 b;
       b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
-      for (int i = 0; i < ncta; ++i) {
-        const float4 c4 = __ldcg(p.amax + (size_t)i * 16 + lane);
-        Top2 x; x.v1 = c4.x; x.i1 = __float_as_int(c4.y); x.v2 = c4.z;
-        b = top2_merge(b, x);
+      if (row < Tg) {
+        float4 c4[10];
+#pragma unroll
+        for (int k = 0; k < 10; ++k) {
+          const int i = l16 + 16 * k;
+          c4[k] = i < ncta ? __ldcg(p.amax + (size_t)i * 16 + row) : make_float4(-INFINITY, __int_as_float(0x7fffffff), -INFINITY, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < 10; ++k) {
+          Top2 x; x.v1 = c4[k].x; x.i1 = __float_as_int(c4[k].y); x.v2 = c4[k].z;
+          b = top2_merge(b, x);
+        }
+        for (int i = l16 + 160; i < ncta; i += 16) {   // grids beyond 160 CTAs
+          const float4 c = __ldcg(p.amax + (size_t)i * 16 + row);
+          Top2 x; x.v1 = c.x; x.i1 = __float_as_int(c.y); x.v2 = c.z;
+          b = top2_merge(b, x);
+        }
       }
-      const int slot_out = g.lm_rows ? p.pass->lm_out[lane] : p.pass->row_out[lane];
-      p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
-      if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+      if (row < Tg && l16 == 0) {
+        const int slot_out = g.lm_rows ? p.pass->lm_out[row] : p.pass->row_out[row];
+        p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
+        if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
+      }
     }
   }
   // let warp 2 free the tensor memory once every worker has made its last read
