@@ -449,14 +449,19 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.page_table = x->page_table; p.pages_per_seq = x->pages_per_seq; p.page_size = c.page_size;
   p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
   p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
-  p.kpart = x->kpart; p.kcnt = x->kcnt;
   p.gbar = x->gbar; p.cnt = x->cnt;
   p.phase_ns = (x->prof && mode == 0) ? x->phase_ns : nullptr;
   timed(x, 0, pass_weight_bytes(x, mode, with_lm), [&] {
     cudaMemsetAsync(x->gbar, 0, sizeof(unsigned), x->stream);
-    void *args[] = {&p};
-    cudaLaunchCooperativeKernel((const void *)k_pass, dim3(x->n_sm), dim3(kPassThreads), args, kPassSmemBytes,
-                                x->stream);
+    // cooperative (all CTAs resident: they meet at grid barriers) in clusters of two (K-split pairs)
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(x->n_sm); lc.blockDim = dim3(kPassThreads); lc.dynamicSmemBytes = kPassSmemBytes; lc.stream = x->stream;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeCooperative; at[1].val.cooperative = 1;
+    lc.attrs = at; lc.numAttrs = 2;
+    cudaLaunchKernelEx(&lc, k_pass, p);
     x->launches++;
   });
 }
@@ -601,11 +606,23 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
     if (e == cudaSuccess)
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pass, kPassThreads, kPassSmemBytes);
     // slabs must fit the tensor-memory accumulators: one m tile (128 rows) for gate/up, two otherwise
-    const bool fits = sms >= 3 && slab_rpc(cfg->d_ffn, 1, sms) <= 128 && slab_rpc(cfg->vocab, 1, sms) <= 256 &&
+    const bool fits = sms >= 4 && slab_rpc(cfg->d_ffn, 1, sms) <= 128 && slab_rpc(cfg->vocab, 1, sms) <= 256 &&
                       slab_rpc(cfg->d_model, 3, sms) <= 256;
-    if (e == cudaSuccess && per_sm >= 1 && sms <= 256 && fits) {
+    // the kernel runs as clusters of two CTAs, one CTA per SM: an even grid, all clusters resident at once
+    const int grid = sms & ~1;
+    int max_clusters = 0;
+    if (e == cudaSuccess && per_sm >= 1) {
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(grid); lc.blockDim = dim3(kPassThreads); lc.dynamicSmemBytes = kPassSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at; lc.numAttrs = 1;
+      if (cudaOccupancyMaxActiveClusters(&max_clusters, k_pass, &lc) != cudaSuccess) { max_clusters = 0; cudaGetLastError(); }
+    }
+    if (e == cudaSuccess && per_sm >= 1 && sms <= 256 && fits && max_clusters >= grid / 2) {
       x->use_pass = 1;
-      x->n_sm = sms;
+      x->n_sm = grid;
       int sp = sms / cfg->n_heads;
       x->attn_splits = sp < 1 ? 1 : (sp > 8 ? 8 : sp);
       std::vector<LayerPtrs> lp(cfg->n_layers);

@@ -39,6 +39,7 @@
 // and carries on as if the wait had succeeded, so it always terminates.
 #pragma once
 #include "ada_kernels.cuh"
+#include "ada_ring.h"
 
 namespace ada {
 
@@ -49,10 +50,6 @@ constexpr int kFirstWorker = 4;                  // warp index of worker 0
 constexpr int kKc = 256;                         // k elements per activation chunk = 4 boxes of 64
 constexpr int kBoxK = 64;                        // box width: 64 bf16 = 128 bytes = one swizzle row
 constexpr int kStageBytes = 32 * 1024;           // largest ring stage: kb boxes of [box_rows x 64 k], kb = 2 or 4
-constexpr int kRingBytes = 128 * 1024;           // weight ring; stages take exactly the bytes of their boxes
-constexpr int kFlight = 16;                      // most stages in flight
-constexpr int kSlots = 32;                       // barrier pairs of the ring: twice kFlight, so that a pair is not
-                                                 // reused before both producers have passed its previous use
 constexpr int kXBufs = 5;
 constexpr int kXBoxBytes = 32 * 128;             // activation box pair: 16 hi rows then 16 lo rows, 64 k
 constexpr int kXBufBytes = (kKc / kBoxK) * kXBoxBytes;    // 16 KB per chunk
@@ -122,8 +119,6 @@ struct PassParams {
   float *logits;               // optional [slot][V]
   int *tok_out; float2 *top_out; const int *forced;
   // sync
-  float *kpart;                // [4][16][d] partial sums of K-split groups
-  int *kcnt;                   // [grid] arrival counters of the groups (zero between phases)
   unsigned *gbar;              // grid barrier counter, zero at launch
   Counters *cnt;
   unsigned long long *phase_ns;  // optional [512]: [0] = start, [i+1] = time CTA 0 left barrier i (globaltimer)
@@ -271,6 +266,37 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 __device__ __forceinline__ void named_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
+// ---- thread-block cluster of two CTAs: the peer's shared memory and its mbarriers are addressable
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t peer_addr(const void *own_smem, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(own_smem)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_peer_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t addr) {   // releases this CTA's earlier writes to the peer
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint64_t *bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void cluster_sync_all() {   // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -392,19 +418,15 @@ __host__ __device__ __forceinline__ int slab_box_rows(int rpc, bool swiglu) {
   const int mt = swiglu ? 1 : (rpc + 127) / 128;
   return (rpc + mt - 1) / mt;
 }
-// K splits for a GEMM of N output columns over K: the largest of 4, 3, 2 that leaves every split at least
-// one 256-k chunk and keeps a slab within one m tile (128 rows); else 1
+// K splits for a GEMM of N output columns over K: 2 (the two CTAs of a cluster, which exchange their partial
+// sums through distributed shared memory) if each split gets at least one 256-k chunk and a slab stays within
+// one m tile (128 rows); else 1
 __host__ __device__ __forceinline__ int slab_ksplit(int N, int K, int ncta) {
   const int nchunk = (K + kKc - 1) / kKc;
-  for (int ks = 4; ks >= 2; --ks) {
-    const int groups = ncta / ks;
-    if (groups < 1) continue;
-    const int per = (nchunk + ks - 1) / ks;
-    if ((ks - 1) * per >= nchunk) continue;          // some split would get nothing
-    if ((N + groups - 1) / groups > 128) continue;
-    return ks;
-  }
-  return 1;
+  const int groups = ncta / 2;
+  if (groups < 1 || nchunk < 2) return 1;
+  if ((N + groups - 1) / groups > 128) return 1;
+  return 2;
 }
 __device__ __forceinline__ Slab make_slab(const GemmDesc &g, int cta, int ncta) {
   Slab s;
@@ -446,22 +468,6 @@ __device__ __forceinline__ void tile_source(const GemmDesc &g, const Slab &s, in
   if (g.epi == EPI_SWIGLU_ACT) { map = g.wmap[mi]; row0 = s.r0; }
   else { map = g.wmap[s.seg]; row0 = s.r0 + mi * s.box_rows; }
 }
-
-// Walk over the weight ring.  A stage takes exactly the bytes of its boxes (a multiple of 1 KB), at the
-// head of the ring, or at offset 0 if it would run past the end; stage j uses barrier pair j % kSlots in
-// its (j / kSlots)-th phase.  The walk depends on the static schedule only, so the producer and both
-// issuers compute the same offsets without talking to each other.
-struct RingCursor {
-  uint32_t head;
-  unsigned n;     // stages taken so far
-  __device__ __forceinline__ uint32_t take(uint32_t bytes) {
-    if (head + bytes > (uint32_t)kRingBytes) head = 0;
-    const uint32_t off = head;
-    head += bytes;
-    ++n;
-    return off;
-  }
-};
 
 // ---------------------------------------------------------------------------------- grid barrier
 
@@ -530,6 +536,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 
   uint64_t *accfull = xempty + kXBufs;                     // accumulator of the phase complete
   uint64_t *attn_bar = accfull + 1;                        // attention: keys and values of a round have landed (two buffers)
+  uint64_t *kbar = attn_bar + 2;                           // K-split pair: the peer's partial sums are parked in its shared memory
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_s) + 1);
   uint32_t *st_rec = tmem_slot + 1;   // [2 producers][offsets, ends][kFlight]: records of the stages in flight
   if (tid == 0) {
@@ -539,6 +546,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     mbar_init(accfull, 1);
     mbar_init(attn_bar, 1);
     mbar_init(attn_bar + 1, 1);
+    mbar_init(kbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(tmem_slot, kTmemCols);
@@ -546,6 +554,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // the two CTAs of a cluster arrive on each other's barriers later on: both must have initialised them
+  cluster_sync_all();
 
   const int nphase = phase_count(p);
   if (p.phase_ns && cta == 0 && tid == 32) {
@@ -559,10 +569,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     if (lane != 0) return;   // one thread produces (idle lanes walking the schedule would only steal its issue slots)
     const unsigned pidx = warp == 0 ? 0u : 1u;   // producer 0 loads the even stages, producer 1 the odd ones
     uint32_t *st_off = st_rec + pidx * 2 * kFlight, *st_end = st_off + kFlight;   // this producer's own record of the stages
-    RingCursor cur{0, 0};
-    unsigned tail = 0;   // stages [tail, cur.n) may still be unread
-    uint32_t t_off = 0, t_end = 0;
-    unsigned pending = 0xffffffffu;   // newest retired stage not yet waited for
+    RingRetire rr;   // both producers place and retire every stage of the schedule (see ada_ring.h)
+    rr.init();
     for (int ph = 0; ph < nphase; ++ph) {
       int layer;
       const int kind = phase_kind(p, ph, layer);
@@ -585,26 +593,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           const int nb = min(kb, nbox - b0);
           for (int mi = 0; mi < mtiles; ++mi) {
             const uint32_t bytes = (uint32_t)(nb * region);
-            const uint32_t off = cur.take(bytes);
-            const unsigned j = cur.n - 1, slot = j % kSlots;
-            st_off[j % kFlight] = off; st_end[j % kFlight] = off + bytes;
-            if (tail == j) { t_off = off; t_end = off + bytes; }
-            // The oldest stages in flight are the first ones a new stage can run into: they are retired until a
-            // barrier pair is free and no unread stage overlaps the new one.  Both producers retire for every
-            // stage, so that `tail` is always the oldest stage the ring still holds, but wait only before a
-            // stage of their own.  One thread issues all products, so stages are read in order and waiting
-            // for the newest retired one covers the older ones.  (t_off, t_end) is the record of stage
-            // `tail`, read ahead of its use.
-            while (tail < j && (j - tail >= (unsigned)kFlight || (t_off < off + bytes && off < t_end))) {
-              pending = tail;
-              ++tail;
-              t_off = st_off[tail % kFlight];
-              t_end = st_end[tail % kFlight];
-            }
+            const uint32_t off = rr.place(bytes, st_off, st_end);
+            const unsigned j = rr.cur.n - 1, slot = j % kSlots;
             if ((j & 1u) != pidx) continue;   // the other producer's stage
-            if (pending != 0xffffffffu) {
-              mbar_wait(&empty[pending % kSlots], (pending / kSlots) & 1u, p.cnt, abort_s);
-              pending = 0xffffffffu;
+            if (rr.pending != RingRetire::kNone) {   // stages are read in order: the newest retired one covers the rest
+              mbar_wait(&empty[rr.pending % kSlots], (rr.pending / kSlots) & 1u, p.cnt, abort_s);
+              rr.pending = RingRetire::kNone;
             }
             mbar_expect_tx(&full[slot], (unsigned)nb * tx_box);
             const uint32_t dst = smem_u32(ring) + off, bar = smem_u32(&full[slot]);
@@ -710,6 +704,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   int xcount = 0;   // activation chunks produced so far (buffer = xcount % kXBufs)
   unsigned acc_phase = 0;   // GEMM phases of this CTA whose accumulator has been awaited
   unsigned attn_uses[2] = {0, 0};   // completed phases of the two attention barriers
+  unsigned kuses = 0;               // completed phases of the K-split pair barrier
   (void)g8; (void)q4;
 
   for (int ph = 0; ph < nphase; ++ph) {
@@ -1155,42 +1150,31 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     tc_fence_before();
     bool do_epi = true;
     if (s.ks > 1 && s.rows > 0) {
-      // K-split group: the CTA of the last split adds the partial sums in split order, its own last; the
-      // others publish theirs and go on to the barrier.
+      // K-split pair = the two CTAs of a cluster (same slab, same thread <-> row mapping).  The CTA of the first
+      // split parks its partial sums in its own shared memory and arrives on the peer's barrier; the CTA of
+      // the second split waits for that, reads them through distributed shared memory, adds its own and runs
+      // the epilogue: first split + second split, the same order whoever is faster.  The parked values stay
+      // untouched until the next grid barrier, which the reader passes only after it has read them.
       if (!reducer) {
-        if (valid)
+        float *pk = reinterpret_cast<float *>(xbuf) + ctid;
 #pragma unroll
-          for (int t = 0; t < 16; ++t)
-            if (t < Tg) __stcg(p.kpart + ((size_t)(s.kj * 16 + t)) * p.d + vrow, yy[t]);
-        __threadfence();
+        for (int t = 0; t < 16; ++t) pk[t * 256] = yy[t];
         named_bar(3, kNumCWarps * 32);
-        if (ctid == 0) atomicAdd(p.kcnt + s.group, 1);
+        if (ctid == 0) mbar_arrive_peer(peer_addr(kbar, 1));
         do_epi = false;
       } else {
-        if (lane == 0) {   // every warp waits for the ks - 1 other partials by itself (bounded)
-          const unsigned *cntp = reinterpret_cast<const unsigned *>(p.kcnt + s.group);
-          bool ok = false;
-          for (unsigned i = 0; i < kSpinLimit && !*abort_s; ++i) {
-            if (ld_acquire(cntp) >= (unsigned)(s.ks - 1)) { ok = true; break; }
-            if (i > 4096) __nanosleep(64);
-          }
-          if (!ok) { *abort_s = 1; atomicOr(&p.cnt->status, kStatTimeout); }
+        bool ok = false;
+        for (unsigned i = 0; i < kSpinLimit; ++i) {
+          if (mbar_try_cluster(kbar, kuses & 1u)) { ok = true; break; }
+          if (*abort_s) break;
+          if (i > 64) __nanosleep(40);
         }
-        __syncwarp();
+        if (!ok) { *abort_s = 1; atomicOr(&p.cnt->status, kStatTimeout); }
+        ++kuses;
+        const uint32_t pk = peer_addr(reinterpret_cast<float *>(xbuf) + ctid, 0);
         if (valid) {
-          float pv[16][3];   // 48 independent loads in flight, then the sums in split order
 #pragma unroll
-          for (int t = 0; t < 16; ++t)
-#pragma unroll
-            for (int j = 0; j < 3; ++j)
-              pv[t][j] = (t < Tg && j < s.ks - 1) ? __ldcg(p.kpart + ((size_t)(j * 16 + t)) * p.d + vrow) : 0.f;
-#pragma unroll
-          for (int t = 0; t < 16; ++t) {
-            float a = pv[t][0];
-            if (s.ks > 2) a += pv[t][1];
-            if (s.ks > 3) a += pv[t][2];
-            yy[t] = a + yy[t];
-          }
+          for (int t = 0; t < 16; ++t) yy[t] = (t < Tg ? ld_peer_f32(pk + (uint32_t)t * 1024u) : 0.f) + yy[t];
         }
       }
     }
@@ -1254,7 +1238,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         for (int w = 0; w < kNumCWarps; ++w) r += ssw[w * 16 + lane];
         p.ss_part[(size_t)cta * 16 + lane] = r;
       }
-      if (reducer && do_epi && ctid == 0) p.kcnt[s.group] = 0;   // every warp has seen the count (barrier above)
     } else if (epi == EPI_ARGMAX_LM) {
       if (lane >= Tg && lane < 16) {
         Top2 b;
