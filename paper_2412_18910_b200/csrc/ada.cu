@@ -460,7 +460,12 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     at[1].id = cudaLaunchAttributeCooperative; at[1].val.cooperative = 1;
-    lc.attrs = at; lc.numAttrs = 2;
+    // ADA_PASS_NONCOOP=1 drops the cooperative attribute (same kernel, grid and clusters): Nsight Compute refuses
+    // the launch with both attributes.  Residency of all clusters was checked at initialisation, and every
+    // wait in the kernel is bounded, so without the attribute a grid that is not resident ends with a status
+    // bit instead of the launch error.
+    static const bool noncoop = getenv("ADA_PASS_NONCOOP") != nullptr;
+    lc.attrs = at; lc.numAttrs = noncoop ? 1 : 2;
     cudaLaunchKernelEx(&lc, k_pass, p);
     x->launches++;
   });
