@@ -395,9 +395,9 @@ __device__ __forceinline__ bool make_gemm(const PassParams &p, int kind, int lay
 //
 // GEMMs with only d output columns (O, down, the draft head's fc) would leave each CTA a slab of ~28
 // rows: the tensor core then spends a whole instruction per 28 x 16 weights and every CTA re-reads the
-// whole activation.  They are cut along K too: ks CTAs share a slab of ~111 rows, each takes a
-// contiguous K range (whole 256-k chunks), writes its partial sums, and the CTA of the group that
-// arrives last adds the ks partials in split order and runs the epilogue.
+// whole activation.  They are cut along K too: the two CTAs of a thread-block cluster share a slab of
+// twice the rows, each takes one half of K (whole 256-k chunks), and the CTA of the second half adds the
+// first half's partial sums, read through distributed shared memory, to its own and runs the epilogue.
 struct Slab {
   int seg;          // matrix (segment) of this CTA
   int r0, rows;     // rows [r0, r0 + rows) inside that matrix
