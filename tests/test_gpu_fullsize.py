@@ -71,3 +71,34 @@ def test_13b_predictor_lengths():
 def test_7b_batch8_ragged(w7b):
     g = _golden("7b_b8")
     _run(si.SHAPES["7b_b8"], w7b, g, 8)
+
+
+@pytest.mark.parametrize("name", ["7b", "13b"])
+def test_full_width_two_layers_against_the_live_oracle(name):
+    """Full matrix widths (slab heights, K-split pairs, ring stage sizes of the real shapes) with two layers, so that
+    the oracle runs live: prefill with a ragged last chunk, lock-step iterations, and the same pass twice in two
+    engines must give bit-identical features (no schedule-dependent result)."""
+    import oracle
+    from paper_2412_18910_b200 import Engine
+    sh = si.scaled(si.SHAPES[name], n_layers=2)
+    w = si.make_weights(sh)
+    prompt = si.make_prompts(sh)[0][:40]
+    m = oracle.Model(sh, w)
+    feats = []
+    for rep in range(2):
+        e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
+        try:
+            seq = m.new_seq(512)
+            t_o = seq.prefill(prompt)
+            t_g = e.prefill(0, prompt)
+            f = e.ada_debug_buffer(0, torch.float32, (1, sh.kv_capacity, sh.d_model))[0, :len(prompt)].cpu().numpy()
+            assert np.abs(f - seq.features(0, len(prompt))).max() < 2e-2
+            assert t_o == t_g
+            feats.append(f)
+            res = lockstep.run_lockstep(e, [seq], 8)
+            assert e.ada_get_counters()["status"] == 0
+        finally:
+            e.close()
+        assert not res["failures"], res["failures"]
+        assert res["exempt"] <= 2
+    assert np.array_equal(feats[0], feats[1])
