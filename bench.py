@@ -319,6 +319,19 @@ def main():
     verify_ms = va.elapsed_time(vb) / reps
     ctx_len = sh.prompt_len + 1
     vbytes = verify_weight_bytes(sh) + ctx_len * kv_bytes_per_token(sh)
+    # verify latency as a function of the number of rows (draft length n forced, same context)
+    by_n = []
+    for n_f in range(1, sh.n_max + 1):
+        eng.d_n.fill_(n_f)
+        eng.ada_draft(eng.d_n, eng.d_draft)
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+        va.record(eng.stream)
+        for _ in range(4):
+            eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+        vb.record(eng.stream)
+        torch.cuda.synchronize(dev)
+        ms_n = va.elapsed_time(vb) / 4
+        by_n.append({"n": n_f, "rows": n_f + 1, "ms": round(ms_n, 4), "gbs": round(vbytes / (ms_n * 1e-3) / 1e9, 1)})
     # the dominant kernel: the persistent pass kernel, one launch per verify pass (weights + KV read once)
     launch_ms = prof["gemm_ms"] / max(1, prof["gemm_launches"])
     pass_gbs = vbytes / (launch_ms * 1e-3) / 1e9 if launch_ms > 0 else None
@@ -334,7 +347,8 @@ def main():
                                 "weight_bytes": verify_weight_bytes(sh), "kv_bytes": ctx_len * kv_bytes_per_token(sh),
                                 "gbs": vbytes / (verify_ms * 1e-3) / 1e9,
                                 "frac_of_measured": vbytes / (verify_ms * 1e-3) / 1e9 / peak,
-                                "frac_of_8000": vbytes / (verify_ms * 1e-3) / 1e9 / 8000.0}}
+                                "frac_of_8000": vbytes / (verify_ms * 1e-3) / 1e9 / 8000.0},
+                "verify_by_n": by_n}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
             "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
