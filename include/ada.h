@@ -81,7 +81,11 @@ typedef struct {
 size_t ada_workspace_bytes(const ada_config *cfg);
 
 /* Validates cfg, carves d_workspace (256-byte aligned, >= ada_workspace_bytes) and builds the
- * rotary table.  cuda_stream is a cudaStream_t (NULL = default stream). */
+ * rotary table.  cuda_stream is a cudaStream_t (NULL = default stream).
+ * With max_batch = 1 every pass is one persistent kernel launched cooperatively in thread-block
+ * clusters of two, one CTA per SM; ada_init checks that the whole grid can be resident and falls
+ * back to the multi-kernel path otherwise.  The environment variable ADA_PASS_NONCOOP (any value)
+ * drops the cooperative launch attribute, for profilers that refuse it together with clusters. */
 int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights *w, void *d_workspace,
              size_t workspace_bytes, void *cuda_stream);
 

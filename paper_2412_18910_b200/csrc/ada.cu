@@ -66,8 +66,7 @@ struct ada_ctx {
   LayerPtrs *d_layers, *d_eagle;
   TensorMap128 *d_maps;
   int n_maps;
-  float *ss_part, *attn_part2, *kpart;
-  int *kcnt;
+  float *ss_part, *attn_part2;
   bf16 *xa, *at, *ac, *fc;            // activation tiles (xstore layout), 2048 elements per 64 k
   int *attn_cnt;
   float4 *amax2;
@@ -236,8 +235,6 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->ac = w.take<bf16>(((F + 63) / 64) * 2048);
   x->fc = w.take<bf16>(((2 * d + 63) / 64) * 2048);
   x->ss_part = w.take<float>(256 * 16);
-  x->kpart = w.take<float>(4 * 16 * d);
-  x->kcnt = w.take<int>(256);
   x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
   x->attn_cnt = w.take<int>(H);
   x->amax2 = w.take<float4>(256 * 16);
@@ -649,7 +646,6 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       if (e == cudaSuccess) e = cudaMemset(x->ac, 0, ((FF + 63) / 64) * 4096);
       if (e == cudaSuccess) e = cudaMemset(x->fc, 0, ((2 * dd + 63) / 64) * 4096);
       if (e == cudaSuccess) e = cudaMemset(x->attn_cnt, 0, sizeof(int) * cfg->n_heads);
-      if (e == cudaSuccess) e = cudaMemset(x->kcnt, 0, sizeof(int) * 256);
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }
   }
