@@ -32,7 +32,7 @@ class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
                [(n, C.c_int32) for n in ("ldlp_hidden", "n_max", "ldlp_mode", "ldlp_embed_shift",
-                                         "ldlp_blocks", "k_min")]
+                                         "ldlp_blocks", "k_min")] + [("ddd_threshold", C.c_float)]
 
 
 _PER_LAYER = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm_attn", "norm_mlp")
@@ -70,7 +70,8 @@ def _load():
     L.orc_draft.argtypes = [vp, vp, C.c_int, i32p, i32p, f32p, f32p]
     L.orc_verify.argtypes = [vp, vp, i32p, C.c_int, i32p, f32p, f32p, f32p]
     L.orc_accept.argtypes = [vp, vp, i32p, i32p, C.c_int, i32p, i32p]
-    L.orc_step.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, f32p, f32p]
+    L.orc_step.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, f32p, f32p, f32p]
+    L.orc_draft_dyn.argtypes = [vp, vp, C.c_int, i32p, i32p, f32p, f32p, f32p, i32p]
     L.orc_force_commit.argtypes = [vp, vp, C.c_int, i32p, C.c_int]
     L.orc_forward_nocache.argtypes = [vp, i32p, C.c_int, f32p, f32p]
     L.orc_draft_rows.argtypes = [vp, i32p, f32p, C.c_int, C.c_int, f32p, f32p, f32p]
@@ -103,13 +104,13 @@ class Model:
     """The oracle's view of one set of weights (bf16 bit patterns as uint16 numpy arrays)."""
 
     def __init__(self, shape, weights: dict, ldlp_mode: int = 0, ldlp_embed_shift: int = 0,
-                 ldlp_blocks: int = 2, k_min: int = 1):
+                 ldlp_blocks: int = 2, k_min: int = 1, ddd_threshold: float = 0.0):
         self.lib = _load()
         self.shape = shape
         self.weights = weights  # keeps the arrays alive
         c = _Config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                     shape.rope_theta, shape.rms_eps, shape.ldlp_hidden, shape.n_max, ldlp_mode,
-                    ldlp_embed_shift, ldlp_blocks, k_min)
+                    ldlp_embed_shift, ldlp_blocks, k_min, ddd_threshold)
         w = _Weights()
         self._arrays = []
         for n in _SINGLE_A + _SINGLE_B:
@@ -222,6 +223,20 @@ class Seq:
         assert rc == 0, "draft failed rc=%d" % rc
         return out, t1, t2
 
+    def draft_dyn(self, n: int, forced=None):
+        """Draft with the model's stopping rule (AdaEAGLE-DDD when its threshold is negative).
+        Returns (draft tokens [n_used], top1, top2, running log-probability of the draft sequence)."""
+        nm = self.m.shape.n_max
+        out = np.zeros(nm, dtype=np.int32)
+        t1, t2, lp = (np.zeros(nm, dtype=np.float32) for _ in range(3))
+        nu = C.c_int32(0)
+        f = None if forced is None else np.ascontiguousarray(forced, dtype=np.int32)
+        rc = self.lib.orc_draft_dyn(self.m.h, self.h, n, _ptr(f), out.ctypes.data, t1.ctypes.data, t2.ctypes.data,
+                                    lp.ctypes.data, C.addressof(nu))
+        assert rc == 0, "draft failed rc=%d" % rc
+        k = nu.value
+        return out[:k].copy(), t1[:k].copy(), t2[:k].copy(), lp[:k].copy()
+
     def verify(self, draft, want_logits: bool = False):
         """Returns (target tokens [n+1], top1, top2, logits or None)."""
         d = np.ascontiguousarray(draft, dtype=np.int32)
@@ -255,16 +270,17 @@ class Seq:
         v1, v2 = np.zeros(nm + 1, dtype=np.float32), np.zeros(nm + 1, dtype=np.float32)
         d1, d2 = np.zeros(nm, dtype=np.float32), np.zeros(nm, dtype=np.float32)
         z = np.zeros(nm, dtype=np.float32)
+        lp = np.zeros(nm, dtype=np.float32)
         f = None if forced_draft is None else np.ascontiguousarray(forced_draft, dtype=np.int32)
         j = self.len - 1
         k = self.lib.orc_step(self.m.h, self.h, n_forced, _ptr(f), em.ctypes.data, C.addressof(ne),
                               C.addressof(nu), dr.ctypes.data, tg.ctypes.data, v1.ctypes.data, v2.ctypes.data,
-                              d1.ctypes.data, d2.ctypes.data, z.ctypes.data)
+                              d1.ctypes.data, d2.ctypes.data, z.ctypes.data, lp.ctypes.data)
         assert k >= 0, "step failed rc=%d" % k
         n = nu.value
         return dict(j=j, n=n, k=k, emitted=em[: ne.value].copy(), draft=dr[:n].copy(), target=tg[: n + 1].copy(),
                     v_top1=v1[: n + 1].copy(), v_top2=v2[: n + 1].copy(), d_top1=d1[:n].copy(),
-                    d_top2=d2[:n].copy(), ldlp_z=z.copy())
+                    d_top2=d2[:n].copy(), ldlp_z=z.copy(), d_logp=lp[:n].copy())
 
     def force_commit(self, j_start: int, tokens) -> None:
         t = np.ascontiguousarray(tokens, dtype=np.int32)

@@ -60,6 +60,7 @@ typedef struct {
   int32_t ldlp_embed_shift; /* 0: e of the token whose hidden state is f (paper); 1: e of the bonus token */
   int32_t ldlp_blocks;      /* scalar form: number of residual blocks */
   int32_t k_min;            /* lower clamp of the scalar form (Eq. 3 prints 0; the loop needs >= 1) */
+  float ddd_threshold;      /* < 0: AdaEAGLE-DDD (Section 4): log-probability threshold of the draft sequence; else off */
 } orc_config;
 
 typedef struct {
@@ -403,11 +404,32 @@ int orc_ldlp(const orc_model *m, const orc_seq *s, float *z_out) {
  * forced (optional, n entries) replaces each drafted token after it is computed
  * (teacher forcing); draft_out receives the n tokens that enter the verify;
  * top1/top2 (optional, n entries) the two largest draft logits of each step. */
-int orc_draft(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int32_t *draft_out,
-              float *top1, float *top2v) {
+/* log of the softmax probability of logit `t` among the V logits (sums in double) */
+static float log_prob_of(const float *logits, int V, int t) {
+  float mx = logits[0];
+  for (int i = 1; i < V; ++i) mx = logits[i] > mx ? logits[i] : mx;
+  double sum = 0.0;
+  for (int i = 0; i < V; ++i) sum += exp((double)logits[i] - (double)mx);
+  return (float)((double)logits[t] - ((double)mx + log(sum)));
+}
+
+/* Draft with the combined stopping rule of Section 4 (AdaEAGLE-DDD): the head keeps drafting past the
+ * predicted length n while the log-probability of the draft sequence so far (the sum of the log softmax
+ * probabilities of its tokens) has not fallen below the threshold; it stops as soon as both hold, step >= n and
+ * log-probability < threshold, and in any case at n_max tokens or at the cache capacity.  With ddd = 0
+ * exactly n tokens are drafted.  logp_out (optional) receives the running log-probability after each token,
+ * n_used the number of tokens drafted. */
+static int draft_impl(const orc_model *m, orc_seq *s, int n, int ddd, const int32_t *forced, int32_t *draft_out,
+                      float *top1, float *top2v, float *logp_out, int32_t *n_used) {
   const int d = m->c.d_model, V = m->c.vocab;
   const int j = s->len - 1; /* index of the pending token */
   if (n < 1 || n > m->c.n_max || j + n + 2 > s->cap) return -1;
+  int n_lim = n;
+  if (ddd) {
+    n_lim = m->c.n_max;
+    if (j + n_lim + 2 > s->cap) n_lim = s->cap - j - 2;
+  }
+  float seq_logp = 0.0f;
   float *logits = (float *)malloc(sizeof(float) * (size_t)V);
   const int R = j - s->dlen; /* catch-up rows: positions dlen .. j-1 */
   if (R < 1) { free(logits); return -2; }
@@ -416,7 +438,8 @@ int orc_draft(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int3
   s->dlen = j;
   memcpy(s->dfeat, out + (size_t)(R - 1) * d, sizeof(float) * (size_t)d);
   free(out);
-  for (int step = 1; step <= n; ++step) {
+  int made = 0;
+  for (int step = 1; step <= n_lim; ++step) {
     float *fh = s->dfeat + (size_t)(step - 1) * d; /* estimate of the feature of position j+step-1 */
     if (step > 1) {
       /* position j+step-2: own feature of that position + embedding of draft token step-1 */
@@ -427,9 +450,27 @@ int orc_draft(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int3
     int t = argmax_low(logits, V);
     if (top1 && top2v) top2(logits, V, &top1[step - 1], &top2v[step - 1]);
     draft_out[step - 1] = forced ? forced[step - 1] : t;
+    made = step;
+    if (ddd || logp_out) {
+      seq_logp += log_prob_of(logits, V, draft_out[step - 1]);
+      if (logp_out) logp_out[step - 1] = seq_logp;
+    }
+    if (ddd && step >= n && seq_logp < m->c.ddd_threshold) break;
   }
+  if (n_used) *n_used = made;
   free(logits);
   return 0;
+}
+
+int orc_draft(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int32_t *draft_out,
+              float *top1, float *top2v) {
+  return draft_impl(m, s, n, 0, forced, draft_out, top1, top2v, NULL, NULL);
+}
+
+/* as orc_draft, with the stopping rule of the model's configuration (ddd_threshold < 0: AdaEAGLE-DDD) */
+int orc_draft_dyn(const orc_model *m, orc_seq *s, int n, const int32_t *forced, int32_t *draft_out,
+                  float *top1, float *top2v, float *logp_out, int32_t *n_used) {
+  return draft_impl(m, s, n, m->c.ddd_threshold < 0.0f, forced, draft_out, top1, top2v, logp_out, n_used);
 }
 
 /* Eq. 1, forward part.  Rows: the pending token then the n draft tokens, at
@@ -489,7 +530,7 @@ int orc_accept(const orc_model *m, orc_seq *s, const int32_t *draft, const int32
 int orc_step(const orc_model *m, orc_seq *s, int n_forced, const int32_t *forced_draft,
              int32_t *emitted, int32_t *n_emitted, int32_t *n_used, int32_t *draft_out,
              int32_t *target_out, float *v_top1, float *v_top2, float *d_top1, float *d_top2,
-             float *ldlp_z) {
+             float *ldlp_z, float *d_logp) {
   int32_t draft[64], target[65];
   int n = n_forced;
   if (n < 0) n = orc_ldlp(m, s, ldlp_z);
@@ -497,7 +538,11 @@ int orc_step(const orc_model *m, orc_seq *s, int n_forced, const int32_t *forced
   const int j = s->len - 1;
   if (j + 2 > s->cap) return -2;
   if (j + n + 2 > s->cap) n = s->cap - j - 2;
-  if (n >= 1 && orc_draft(m, s, n, forced_draft, draft, d_top1, d_top2)) return -3;
+  if (n >= 1) {
+    int32_t made = n;
+    if (orc_draft_dyn(m, s, n, forced_draft, draft, d_top1, d_top2, d_logp, &made)) return -3;
+    n = made;
+  }
   if (orc_verify(m, s, draft, n, target, NULL, v_top1, v_top2)) return -4;
   int k = orc_accept(m, s, draft, target, n, emitted, n_emitted);
   if (n_used) *n_used = n;

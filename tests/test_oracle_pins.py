@@ -339,3 +339,71 @@ def test_drafting_exactly_the_accept_length_wastes_nothing(tiny):
     assert np.array_equal(run["tokens"], ar[:32])
     assert run["counters"]["n_waste"] == 0
     assert run["counters"]["n_target"] <= probe["counters"]["n_target"]
+
+
+# ----------------------------------------------------------------- AdaEAGLE-DDD stopping rule (Section 4)
+
+def _ddd_seq(sh, w, prompt, thr, cap=512):
+    m = oracle.Model(sh, w, ddd_threshold=thr)
+    seq = m.new_seq(cap)
+    seq.prefill(prompt)
+    return m, seq
+
+
+def test_ddd_off_drafts_exactly_n(tiny):
+    sh, w, prompt, m0 = tiny
+    _, seq = _ddd_seq(sh, w, prompt, 0.0)
+    ref = m0.new_seq(512)
+    ref.prefill(prompt)
+    for n in (1, 3, sh.n_max):
+        a = seq.step(n_forced=n)
+        b = ref.step(n_forced=n)
+        assert a["n"] == n and list(a["draft"]) == list(b["draft"]) and list(a["emitted"]) == list(b["emitted"])
+
+
+def test_ddd_log_probability_is_log_softmax_of_the_draft_logits(tiny):
+    """The running log-probability against float64 log-softmax of (draft feature x LM head), built from stock ops."""
+    sh, w, prompt, _ = tiny
+    _, seq = _ddd_seq(sh, w, prompt, -1e30)                 # never stops early: n_max tokens
+    toks, _, _, lp = seq.draft_dyn(1)
+    assert len(toks) == sh.n_max
+    feats = seq.draft_features(sh.n_max).astype(np.float64)
+    W = si.bf16_bits_to_f32(w["lm_head"]).astype(np.float64)
+    logits = feats @ W.T
+    ls = logits - logits.max(1, keepdims=True)
+    logsm = ls - np.log(np.exp(ls).sum(1, keepdims=True))
+    assert list(toks) == list(logits.argmax(1))
+    expect = np.cumsum(logsm[np.arange(sh.n_max), toks])
+    assert np.abs(lp - expect).max() < 1e-3
+    assert np.all(np.diff(lp) < 0)                           # a product of probabilities only shrinks
+
+
+@pytest.mark.parametrize("n", [1, 2, 5])
+@pytest.mark.parametrize("thr", [-4.0, -12.5, -17.0, -26.0, -41.0, -1e30])
+def test_ddd_length_is_first_step_past_n_below_the_threshold(tiny, n, thr):
+    """Brute force on the log-probabilities of a full-length draft: stop at the first s >= n with S_s < thr."""
+    sh, w, prompt, _ = tiny
+    _, full = _ddd_seq(sh, w, prompt, -1e30)
+    _, _, _, lp = full.draft_dyn(1)
+    expect = next((s for s in range(n, sh.n_max + 1) if lp[s - 1] < thr), sh.n_max)
+    _, seq = _ddd_seq(sh, w, prompt, thr)
+    toks, _, _, lp2 = seq.draft_dyn(n)
+    assert len(toks) == expect
+    assert np.array_equal(lp2, lp[:expect])
+
+
+def test_ddd_respects_the_cache_capacity(tiny):
+    sh, w, prompt, _ = tiny
+    cap = len(prompt) + 4                                     # j = len(prompt): room for j + n + 2 <= cap -> n <= 2
+    _, seq = _ddd_seq(sh, w, prompt, -1e30, cap=cap)
+    o = seq.step(n_forced=1)
+    assert o["n"] == 2
+
+
+def test_ddd_output_is_still_greedy_decoding(tiny):
+    sh, w, prompt, m0 = tiny
+    ar = oracle.decode(m0, prompt, 24, n_policy=0)["tokens"]
+    m = oracle.Model(sh, w, ddd_threshold=-17.0)
+    sd = oracle.decode(m, prompt, 24, n_policy=1)
+    assert list(sd["tokens"]) == list(ar)
+    assert sd["counters"]["n_draft"] > sd["counters"]["n_target"]   # the rule did extend drafts past n = 1
