@@ -58,6 +58,10 @@ typedef struct {
   int32_t page_size;    /* KV page length in positions: 64 */
   int32_t ldlp_blocks;  /* ldlp_mode 1: residual blocks h += ReLU(W_r h + b_r) between the two linear maps, 0..8 */
   int32_t k_min;        /* ldlp_mode 1: smallest draft length (k_min of Eq. 3), 1..n_max                         */
+  float ddd_threshold;  /* < 0: the combined stopping rule of Section 4 (AdaEAGLE-DDD): the head keeps drafting past
+                         * the predicted length while the log-probability of the draft sequence (sum of the log
+                         * softmax probabilities of its tokens) is at or above this value, up to n_max; it stops as
+                         * soon as step >= n and log-probability < threshold.  >= 0: off.  Needs max_batch = 1.   */
 } ada_config;
 
 /* Device pointers to bf16 tensors.  Per-layer members are HOST arrays of n_layers device pointers. */
@@ -104,6 +108,10 @@ int ada_ldlp_predict(ada_ctx *ctx, int32_t *d_n);
  * up to date with the target features of the positions accepted last time).
  * d_draft: [max_batch][n_max], entries beyond n are left untouched. */
 int ada_draft(ada_ctx *ctx, const int32_t *d_n, int32_t *d_draft);
+
+/* The draft lengths in force after ada_draft: d_n itself, or, with ddd_threshold < 0 (Section 4), the lengths
+ * the stopping rule settled on; these are the lengths to hand to ada_verify.  d_n: [max_batch]. */
+int ada_draft_lengths(ada_ctx *ctx, int32_t *d_n);
 
 /* Eq. 1, forward part: the target runs over the pending token and the n draft tokens of every
  * sequence (n may be 0: plain autoregressive step) and returns its greedy choice after each row.

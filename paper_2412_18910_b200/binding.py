@@ -15,7 +15,8 @@ ADA_ERRORS = {0: "ADA_OK", -1: "ADA_ERR_BAD_CONFIG", -2: "ADA_ERR_NULL", -3: "AD
               -5: "ADA_ERR_CUDA", -6: "ADA_ERR_WORKSPACE", -7: "ADA_ERR_STATE",
               -8: "ADA_ERR_TOO_LARGE (a size exceeds a fixed maximum of the library)"}
 
-exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_verify",
+exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_draft_lengths",
+                    "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
                     "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
                     "ada_destroy", "ada_ldlp_eval_static")
@@ -29,7 +30,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
                [(n, C.c_int32) for n in ("ldlp_hidden", "n_max", "ldlp_mode", "max_batch", "kv_capacity", "page_size",
-                                         "ldlp_blocks", "k_min")]
+                                         "ldlp_blocks", "k_min")] + [("ddd_threshold", C.c_float)]
 
 
 _PER_LAYER = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm_attn", "norm_mlp")
@@ -62,6 +63,7 @@ def lib():
     L.ada_prefill.argtypes = [vp, C.c_int, vp, i32, vp]
     L.ada_ldlp_predict.argtypes = [vp, vp]
     L.ada_draft.argtypes = [vp, vp, vp]
+    L.ada_draft_lengths.argtypes = [vp, vp]
     L.ada_verify.argtypes = [vp, vp, vp, vp, vp]
     L.ada_accept.argtypes = [vp, vp, vp, vp]
     L.ada_step.argtypes = [vp, vp, vp, vp, vp]
@@ -107,7 +109,7 @@ class Engine:
     """
 
     def __init__(self, shape, weights: dict, max_batch: int = 1, kv_capacity: int = 4096, device: str = "cuda:0",
-                 stream=None, ldlp_mode: int = 0, ldlp_blocks: int = 2, k_min: int = 1):
+                 stream=None, ldlp_mode: int = 0, ldlp_blocks: int = 2, k_min: int = 1, ddd_threshold: float = 0.0):
         import numpy as np
         import torch
 
@@ -121,7 +123,7 @@ class Engine:
         self.B, self.nmax, self.cap = max_batch, shape.n_max, kv_capacity
         self.cfg = Config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                           shape.rope_theta, shape.rms_eps, shape.ldlp_hidden, shape.n_max, ldlp_mode, max_batch,
-                          kv_capacity, 64, ldlp_blocks, k_min)
+                          kv_capacity, 64, ldlp_blocks, k_min, ddd_threshold)
         need = self.L.ada_workspace_bytes(C.byref(self.cfg))
         if need == 0:
             raise AdaError("invalid configuration")
@@ -192,6 +194,9 @@ class Engine:
 
     def ada_draft(self, d_n, d_draft):
         self._check(self.L.ada_draft(self.h, _dp(d_n), _dp(d_draft)), "ada_draft")
+
+    def ada_draft_lengths(self, d_n):
+        self._check(self.L.ada_draft_lengths(self.h, _dp(d_n)), "ada_draft_lengths")
 
     def ada_verify(self, d_draft, d_n, d_target, d_logits=None):
         self._check(self.L.ada_verify(self.h, _dp(d_draft), _dp(d_n), _dp(d_target), _dp(d_logits)), "ada_verify")

@@ -49,7 +49,7 @@ struct ada_ctx {
   SeqState *st;                     // [B]
   Counters *cnt;
   Pass *pass;
-  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z;
+  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z, *dlp, *dfl, *dcum;
   bf16 *xhi, *xlo, *x2hi, *x2lo;    // [TP][ldx], [TP][ldx2]
   int ldx, ldx2;
   int *gemm_cnt;
@@ -132,6 +132,7 @@ bool config_ok(const ada_config *c) {
   if (c->d_model % 64 || c->d_ffn % 16 || c->d_ffn < 16 || c->vocab % 16 || c->vocab < 16) return false;
   if (c->ldlp_hidden < 1 || c->n_max < 1 || c->n_max > ADA_MAX_NMAX) return false;
   if (c->ldlp_mode != 0 && c->ldlp_mode != 1) return false;
+  if (c->ddd_threshold < 0.f && c->max_batch != 1) return false;
   if (c->ldlp_mode == 1 && (c->ldlp_blocks < 0 || c->ldlp_blocks > 8 || c->k_min < 1 || c->k_min > c->n_max)) return false;
   if (c->max_batch < 1 || c->max_batch > ADA_MAX_BATCH) return false;
   if (c->max_batch * (c->n_max + 1) > 88) return false;
@@ -219,6 +220,9 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->target = w.take<int>(B * (c->n_max + 1));
   x->force_n_dev = w.take<int>(B);
   x->forced_buf = w.take<int>(B * c->n_max);
+  x->dlp = w.take<float>(B * c->n_max);
+  x->dfl = w.take<float>(B * c->n_max);
+  x->dcum = w.take<float>(B);
   x->chunk_tok = w.take<int>(kMaxRows);
   x->vtop = w.take<float2>(B * (c->n_max + 1) + kMaxRows);
   x->dtop = w.take<float2>(B * c->n_max + kMaxRows);
@@ -447,6 +451,7 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
   p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
   p.gbar = x->gbar; p.cnt = x->cnt;
+  p.lp_out = (mode == 1 && with_lm && x->c.ddd_threshold < 0.f) ? x->dlp : nullptr; p.tok_logit = x->dfl;
   p.phase_ns = (x->prof && mode == 0) ? x->phase_ns : nullptr;
   timed(x, 0, pass_weight_bytes(x, mode, with_lm), [&] {
     cudaMemsetAsync(x->gbar, 0, sizeof(unsigned), x->stream);
@@ -491,6 +496,8 @@ void enqueue_draft(ada_ctx *x) {
            x->cnt);
     if (x->use_pass) run_pass(x, 1, step, 1, nullptr, x->draft, x->dtop, x->force_draft);
     else draft_rows(x, step, true);
+    if (c.ddd_threshold < 0.f)   // Section 4: the draft may grow past the predicted length
+      LAUNCH(x, k_ddd_update, 1, 32, 0, x->st, x->dlp, x->dcum, c.ddd_threshold, c.n_max, c.kv_capacity, x->B, step);
   }
 }
 
@@ -659,6 +666,10 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
     delete x;
     return ADA_ERR_CUDA;
   }
+  if (cfg->ddd_threshold < 0.f && !x->use_pass) {   // the log-probabilities come from the persistent pass kernel
+    delete x;
+    return ADA_ERR_BAD_CONFIG;
+  }
   *out = x;
   return ADA_OK;
 }
@@ -712,6 +723,12 @@ extern "C" int ada_draft(ada_ctx *x, const int32_t *d_n, int32_t *d_draft) {
   return cuda_ok(x, "ada_draft") ? ADA_OK : ADA_ERR_CUDA;
 }
 
+extern "C" int ada_draft_lengths(ada_ctx *x, int32_t *d_n) {
+  if (!x || !d_n) return ADA_ERR_NULL;
+  LAUNCH(x, k_gather_n, 1, 32, 0, x->st, d_n, x->B);
+  return cuda_ok(x, "ada_draft_lengths") ? ADA_OK : ADA_ERR_CUDA;
+}
+
 extern "C" int ada_verify(ada_ctx *x, const int32_t *d_draft, const int32_t *d_n, int32_t *d_target_tok,
                           float *d_logits) {
   if (!x || !d_n || !d_target_tok) return ADA_ERR_NULL;
@@ -759,6 +776,8 @@ extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, in
     }
     enqueue_ldlp(x, x->out_nused);
     if (!all_ar) enqueue_draft(x);
+    if (!all_ar && c.ddd_threshold < 0.f)   // report the lengths the stopping rule settled on
+      LAUNCH(x, k_gather_n, 1, 32, 0, x->st, x->out_nused, x->B);
     enqueue_verify(x, -1, nullptr);
     LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, -1,
            (const int *)nullptr, 0, x->out_acc, x->out_emit, x->out_nemit, (int *)nullptr);
@@ -845,6 +864,7 @@ extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *byt
     case 6: *d_ptr = x->dtop; *bytes = B * c.n_max * sizeof(float2); break;
     case 7: *d_ptr = x->draft; *bytes = B * c.n_max * sizeof(int); break;
     case 8: *d_ptr = x->target; *bytes = B * (c.n_max + 1) * sizeof(int); break;
+    case 10: *d_ptr = x->dlp; *bytes = B * c.n_max * sizeof(float); break;
     case 9: *d_ptr = x->phase_ns; *bytes = (512 + 4 * 512) * sizeof(unsigned long long); break;
     default: return fail(x, ADA_ERR_RANGE, "ada_debug_buffer: unknown buffer");
   }

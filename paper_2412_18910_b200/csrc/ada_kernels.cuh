@@ -928,6 +928,22 @@ __global__ void k_rewind(SeqState *st, int b, int count, const int *forced_tok, 
 __global__ void k_copy_i32(int *dst, const int *src, int n) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = src[i];
 }
+// Stopping rule of Section 4 (AdaEAGLE-DDD), after draft step `step` (0-based: it produced token step + 1):
+// the running log-probability of the draft sequence takes the new token's log-probability; if the predicted
+// length is reached (step + 1 >= n) and the sequence is still at or above the threshold, the draft grows by one
+// token, within n_max and the cache capacity.  One thread per sequence.
+__global__ void k_ddd_update(SeqState *st, const float *lp, float *cum, float thr, int nmax, int cap, int B, int step) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  const int n = st[b].n;
+  if (n <= step) return;                       // this step did not run for the sequence
+  const float c = (step == 0 ? 0.f : cum[b]) + lp[b * nmax + step];
+  cum[b] = c;
+  const int made = step + 1;
+  const int room = cap - st[b].len - 1;        // len + n + 1 <= cap
+  if (made >= n && made < nmax && made < room && !(c < thr)) st[b].n = made + 1;
+}
+
 __global__ void k_gather_n(const SeqState *st, int *out, int B) {
   if (threadIdx.x < B) out[threadIdx.x] = st[threadIdx.x].n;
 }

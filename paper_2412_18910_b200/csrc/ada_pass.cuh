@@ -118,6 +118,8 @@ struct PassParams {
   float4 *amax;                // [grid][16]
   float *logits;               // optional [slot][V]
   int *tok_out; float2 *top_out; const int *forced;
+  float *lp_out;               // optional [slot]: log softmax probability of the token written to tok_out
+  float *tok_logit;            // scratch [slot]: logit of a forced token (lp_out with forced tokens)
   // sync
   unsigned *gbar;              // grid barrier counter, zero at launch
   Counters *cnt;
@@ -1228,6 +1230,16 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
         if (lane == 0) topw[cw * 16 + t] = b;
+        if (p.lp_out) {
+          // for the log-probability of the chosen token: sum of exp(logit - warp maximum), and the logit of a
+          // forced token where one is given
+          const float e = warp_sum(act ? __expf(y - b.v1) : 0.f);
+          if (lane == 0) ssw[cw * 16 + t] = e;
+          if (act && p.forced) {
+            const int slot_out = g.lm_rows ? p.pass->lm_out[t] : p.pass->row_out[t];
+            if (p.forced[slot_out] == vrow) p.tok_logit[slot_out] = y;
+          }
+        }
       }
     }
     if (has_ss) {
@@ -1248,7 +1260,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       if (cw == 0 && lane < 16) {
         Top2 b = topw[lane];
         for (int w = 1; w < kNumCWarps; ++w) b = top2_merge(b, topw[w * 16 + lane]);
-        p.amax[(size_t)cta * 16 + lane] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+        float se = 0.f;   // sum of exp(logit - this CTA's maximum) over the CTA's vocabulary rows
+        if (p.lp_out && lane < Tg)
+          for (int w = 0; w < kNumCWarps; ++w) {
+            const float mw = topw[w * 16 + lane].v1;
+            if (mw > -INFINITY) se += ssw[w * 16 + lane] * __expf(mw - b.v1);
+          }
+        p.amax[(size_t)cta * 16 + lane] = make_float4(b.v1, __int_as_float(b.i1), b.v2, se);
       }
     }
     stamp(p, ph, 3, stamper);
@@ -1281,10 +1299,22 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       }
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+      float se = 0.f;   // sum over the vocabulary of exp(logit - maximum): the CTAs' sums rescaled to the global maximum
+      if (p.lp_out) {
+        if (row < Tg)
+          for (int i = l16; i < ncta; i += 16) {
+            const float4 c = __ldcg(p.amax + (size_t)i * 16 + row);
+            if (c.x > -INFINITY) se += c.w * __expf(c.x - b.v1);
+          }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+      }
       if (row < Tg && l16 == 0) {
         const int slot_out = g.lm_rows ? p.pass->lm_out[row] : p.pass->row_out[row];
         p.tok_out[slot_out] = p.forced ? p.forced[slot_out] : b.i1;
         if (p.top_out) p.top_out[slot_out] = make_float2(b.v1, b.v2);
+        // log softmax of the token that goes out: its logit minus (maximum + log of the sum)
+        if (p.lp_out) p.lp_out[slot_out] = (p.forced ? __ldcg(p.tok_logit + slot_out) - b.v1 : 0.f) - __logf(se);
       }
     }
   }

@@ -10,6 +10,7 @@ import numpy as np
 import torch
 
 TOKEN_MARGIN = 0.05   # logits: positions with a smaller oracle margin may flip (bf16 cache vs fp32)
+DDD_MARGIN = 0.1      # log-probabilities inherit the logits' 2e-2 bound, summed over up to n_max draft tokens
 LDLP_MARGIN = 2e-3    # predictor logits are fp32 on both sides; only features differ
 DRAFT_CHAIN_GROWTH = 1.5   # per-step growth of a deviation inside the draft chain (see compare_iteration)
 
@@ -24,12 +25,20 @@ def _round_gap(z):
     return abs((float(z) - np.floor(float(z))) - 0.5)
 
 
-def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n=False, ldlp_scalar=False):
+def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n=False, ldlp_scalar=False, ddd=None):
     """o: dict from oracle Seq.step().  Returns (ok, exempt, needs_resync, message).
 
     ldlp_scalar: the predictor is the scalar form (Eq. 3): its decision flips where z crosses k + 1/2."""
     exempt = 0
     n = o["n"]
+    if g_n != n and ddd is not None:
+        # Section 4 rule: the length is decided by comparing the running log-probability of the draft sequence with
+        # the threshold; the two sides may differ only where the oracle's value at a deciding step is that close
+        lp = np.asarray(o["d_logp"], dtype=np.float64)
+        close = any(abs(lp[s - 1] - ddd) < DDD_MARGIN for s in range(1, len(lp) + 1))
+        if not close:
+            return False, 0, True, "draft length %d != oracle %d (log-probabilities %s, threshold %g)" % (g_n, n, lp, ddd)
+        return True, 1, True, "draft length flipped inside the threshold margin"
     if g_n != n:
         gap = _round_gap(o["ldlp_z"][0]) if ldlp_scalar else _top2_gap(o["ldlp_z"][:n_max])
         if forced_n or gap > LDLP_MARGIN:
@@ -57,7 +66,7 @@ def compare_iteration(o, g_n, g_draft, g_target, g_k, g_emitted, n_max, forced_n
     return True, exempt, False, ""
 
 
-def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=None, ldlp_scalar=False):
+def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=None, ldlp_scalar=False, ddd=None):
     """Runs `iters` ada_step iterations against oracle sequences (one per batch slot).
 
     Returns dict(iterations, exempt, failures[list of str], tokens[list per seq]).
@@ -84,7 +93,7 @@ def run_lockstep(engine, oseqs, iters, n_forced=-1, forced_stream=None, prompts=
         gd, gt = draft_buf.cpu().numpy(), target_buf.cpu().numpy()
         for b, o in enumerate(olist):
             ok, ex, resync, msg = compare_iteration(o, g["n"][b], gd[b], gt[b], g["k"][b], g["emitted"][b], nmax,
-                                                    forced_n=n_forced >= 0, ldlp_scalar=ldlp_scalar)
+                                                    forced_n=n_forced >= 0 and ddd is None, ldlp_scalar=ldlp_scalar, ddd=ddd)
             compared += 1
             exempt += ex
             if not ok:

@@ -102,3 +102,28 @@ def test_full_width_two_layers_against_the_live_oracle(name):
         assert not res["failures"], res["failures"]
         assert res["exempt"] <= 2
     assert np.array_equal(feats[0], feats[1])
+
+
+def test_full_width_ddd_stopping_rule_against_the_live_oracle():
+    """Section 4 (AdaEAGLE-DDD) at the 7B widths and vocabulary (two layers): the log-probabilities come from the
+    LM-head phase of the draft pass, the length from the device-side rule."""
+    import oracle
+    from paper_2412_18910_b200 import Engine
+    sh = si.scaled(si.SHAPES["7b"], n_layers=2)
+    w = si.make_weights(sh)
+    prompt = si.make_prompts(sh)[0][:40]
+    thr = -22.0
+    m = oracle.Model(sh, w, ddd_threshold=thr)
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity, ddd_threshold=thr)
+    try:
+        seq = m.new_seq(512)
+        assert seq.prefill(prompt) == e.prefill(0, prompt)
+        e.ada_force_n([1])
+        res = lockstep.run_lockstep(e, [seq], 8, n_forced=1, ddd=thr)
+        assert e.ada_get_counters()["status"] == 0
+        c = e.ada_get_counters()
+    finally:
+        e.close()
+    assert not res["failures"], res["failures"]
+    assert res["exempt"] <= 2
+    assert c["n_draft"] > c["n_target"]          # drafts did grow past n = 1

@@ -280,3 +280,38 @@ def test_long_context_attention_spans_blocks_and_rounds(tiny, plen):
         assert e.ada_get_counters()["status"] == 0
     finally:
         e.close()
+
+
+@pytest.mark.parametrize("thr,n_forced", [(-17.0, 1), (-26.0, 2), (-12.5, 1), (-1e30, 3), (-4.0, 2)])
+def test_ddd_stopping_rule_lockstep(tiny, thr, n_forced):
+    """Section 4 (AdaEAGLE-DDD): drafts grow past the predicted length while the sequence log-probability holds."""
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, _ = tiny
+    m = oracle.Model(sh, w, ddd_threshold=thr)
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity, ddd_threshold=thr)
+    try:
+        seq, t_o, t_g = _prefill_both(e, m, prompt)
+        assert t_o == t_g
+        e.ada_force_n([n_forced])
+        lens = set()
+        lpbuf = e.ada_debug_buffer(10, torch.float32, (1, sh.n_max))
+        for it in range(10):
+            o = seq.step(n_forced=n_forced)
+            g = e.step()
+            ok, ex, resync, msg = lockstep.compare_iteration(o, g["n"][0], *_bufs(e), g["k"][0], g["emitted"][0],
+                                                             sh.n_max, ddd=thr)
+            assert ok, msg
+            if g["n"][0] == o["n"]:   # per-token log-probabilities: differences of the running sums
+                glp = np.cumsum(lpbuf[0, : o["n"]].cpu().numpy().astype(np.float64))
+                assert np.abs(glp - o["d_logp"]).max() < 0.1
+            lens.add(int(g["n"][0]))
+            if resync:
+                em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(e.dev)
+                e.ada_force_commit(0, em, len(o["emitted"]))
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
+    if thr == -1e30:
+        assert lens == {sh.n_max}
+    if thr == -4.0:
+        assert lens == {n_forced}
