@@ -109,6 +109,13 @@ int ada_ldlp_predict(ada_ctx *ctx, int32_t *d_n);
  * d_draft: [max_batch][n_max], entries beyond n are left untouched. */
 int ada_draft(ada_ctx *ctx, const int32_t *d_n, int32_t *d_draft);
 
+/* Label of Section 3.3 (the optimal draft length that the predictor is trained on; the draft-length oracle of
+ * Section 2.3 is a decoder that is told it): for every sequence drafts as many tokens as allowed (n_max, or what
+ * the cache still holds), verifies them and writes to d_k[seq] the length of the longest prefix of the draft that
+ * the target confirms.  Nothing is committed: a following ada_step or ada_draft starts from the same state (the
+ * draft head recomputes the row of the last verified position).  d_k: [max_batch]. */
+int ada_label(ada_ctx *ctx, int32_t *d_k);
+
 /* The draft lengths in force after ada_draft: d_n itself, or, with ddd_threshold < 0 (Section 4), the lengths
  * the stopping rule settled on; these are the lengths to hand to ada_verify.  d_n: [max_batch]. */
 int ada_draft_lengths(ada_ctx *ctx, int32_t *d_n);

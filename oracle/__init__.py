@@ -72,6 +72,7 @@ def _load():
     L.orc_accept.argtypes = [vp, vp, i32p, i32p, C.c_int, i32p, i32p]
     L.orc_step.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, f32p, f32p, f32p]
     L.orc_draft_dyn.argtypes = [vp, vp, C.c_int, i32p, i32p, f32p, f32p, f32p, i32p]
+    L.orc_label.argtypes = [vp, vp]
     L.orc_force_commit.argtypes = [vp, vp, C.c_int, i32p, C.c_int]
     L.orc_forward_nocache.argtypes = [vp, i32p, C.c_int, f32p, f32p]
     L.orc_draft_rows.argtypes = [vp, i32p, f32p, C.c_int, C.c_int, f32p, f32p, f32p]
@@ -281,6 +282,13 @@ class Seq:
         return dict(j=j, n=n, k=k, emitted=em[: ne.value].copy(), draft=dr[:n].copy(), target=tg[: n + 1].copy(),
                     v_top1=v1[: n + 1].copy(), v_top2=v2[: n + 1].copy(), d_top1=d1[:n].copy(),
                     d_top2=d2[:n].copy(), ldlp_z=z.copy(), d_logp=lp[:n].copy())
+
+    def label(self) -> int:
+        """The optimal draft length for the current state (longest confirmed prefix of a full-length draft);
+        the sequence is left unchanged."""
+        k = self.lib.orc_label(self.m.h, self.h)
+        assert k >= 0, "label failed rc=%d" % k
+        return k
 
     def force_commit(self, j_start: int, tokens) -> None:
         t = np.ascontiguousarray(tokens, dtype=np.int32)

@@ -551,6 +551,26 @@ int orc_step(const orc_model *m, orc_seq *s, int n_forced, const int32_t *forced
   return k;
 }
 
+/* Label of Section 3.3 / the draft-length oracle of Section 2.3 for the current state: draft as many tokens as
+ * allowed (n_max, or what the cache still holds), verify them, and return the length of the longest prefix of the
+ * draft that the target confirms -- the optimal draft length for this iteration.  Nothing is committed: the
+ * sequence is left as it was (the draft head's rows of true features are recomputed identically by the next
+ * draft, the target's rows are overwritten by the next verify). */
+int orc_label(const orc_model *m, orc_seq *s) {
+  int32_t draft[64], target[65];
+  const int j = s->len - 1;
+  int n = m->c.n_max;
+  if (j + n + 2 > s->cap) n = s->cap - j - 2;
+  if (n < 1) return 0;
+  const int dlen0 = s->dlen;
+  if (draft_impl(m, s, n, 0, NULL, draft, NULL, NULL, NULL, NULL)) return -1;
+  if (orc_verify(m, s, draft, n, target, NULL, NULL, NULL)) return -2;
+  s->dlen = dlen0;
+  int k = 0;
+  while (k < n && draft[k] == target[k]) ++k;
+  return k;
+}
+
 /* Replace the outcome of the iteration that just ran: rewind to its start
  * (pending index j_start), and commit `count` given tokens instead (count-1
  * accepted drafts and a bonus), recomputing cache rows and features for them. */

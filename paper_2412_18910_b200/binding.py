@@ -15,7 +15,7 @@ ADA_ERRORS = {0: "ADA_OK", -1: "ADA_ERR_BAD_CONFIG", -2: "ADA_ERR_NULL", -3: "AD
               -5: "ADA_ERR_CUDA", -6: "ADA_ERR_WORKSPACE", -7: "ADA_ERR_STATE",
               -8: "ADA_ERR_TOO_LARGE (a size exceeds a fixed maximum of the library)"}
 
-exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_draft_lengths",
+exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_draft_lengths", "ada_label",
                     "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
                     "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
@@ -64,6 +64,7 @@ def lib():
     L.ada_ldlp_predict.argtypes = [vp, vp]
     L.ada_draft.argtypes = [vp, vp, vp]
     L.ada_draft_lengths.argtypes = [vp, vp]
+    L.ada_label.argtypes = [vp, vp]
     L.ada_verify.argtypes = [vp, vp, vp, vp, vp]
     L.ada_accept.argtypes = [vp, vp, vp, vp]
     L.ada_step.argtypes = [vp, vp, vp, vp, vp]
@@ -194,6 +195,9 @@ class Engine:
 
     def ada_draft(self, d_n, d_draft):
         self._check(self.L.ada_draft(self.h, _dp(d_n), _dp(d_draft)), "ada_draft")
+
+    def ada_label(self, d_k):
+        self._check(self.L.ada_label(self.h, _dp(d_k)), "ada_label")
 
     def ada_draft_lengths(self, d_n):
         self._check(self.L.ada_draft_lengths(self.h, _dp(d_n)), "ada_draft_lengths")

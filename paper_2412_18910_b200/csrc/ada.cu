@@ -723,6 +723,16 @@ extern "C" int ada_draft(ada_ctx *x, const int32_t *d_n, int32_t *d_draft) {
   return cuda_ok(x, "ada_draft") ? ADA_OK : ADA_ERR_CUDA;
 }
 
+extern "C" int ada_label(ada_ctx *x, int32_t *d_k) {
+  if (!x || !d_k) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  LAUNCH(x, k_set_n_full, 1, 32, 0, x->st, x->B, c.n_max, c.kv_capacity);
+  enqueue_draft(x);
+  enqueue_verify(x, -1, nullptr);
+  LAUNCH(x, k_label, 1, 32, 0, x->st, x->draft, x->target, c.n_max, x->B, d_k);
+  return cuda_ok(x, "ada_label") ? ADA_OK : ADA_ERR_CUDA;
+}
+
 extern "C" int ada_draft_lengths(ada_ctx *x, int32_t *d_n) {
   if (!x || !d_n) return ADA_ERR_NULL;
   LAUNCH(x, k_gather_n, 1, 32, 0, x->st, d_n, x->B);

@@ -823,10 +823,13 @@ __global__ void k_rows_draft(Pass *pass, SeqState *st, const int *tok, int cap, 
     const int n = st[b].n, j = st[b].len - 1;
     if (n <= step || j < 1) continue;
     if (step == 0) {
-      const int R = j - st[b].dlen;
+      int R = j - st[b].dlen, p0 = st[b].dlen;
+      // already up to date (a second draft from the same state, e.g. after a label pass): the row of position
+      // j - 1 is computed again -- same inputs, same cache row -- because its output yields the first draft token
+      if (R == 0) { R = 1; p0 = j - 1; }
       if (R < 1 || T + R > max_rows || st[b].stale) { st[b].n = 0; atomicOr(&cnt->status, kStatStale); continue; }
       for (int i = 0; i < R; ++i) {
-        const int p = st[b].dlen + i;
+        const int p = p0 + i;
         pass->row_seq[T] = b;
         pass->row_pos[T] = p;
         pass->row_tok[T] = tok[(size_t)b * cap + p + 1];
@@ -942,6 +945,23 @@ __global__ void k_ddd_update(SeqState *st, const float *lp, float *cum, float th
   const int made = step + 1;
   const int room = cap - st[b].len - 1;        // len + n + 1 <= cap
   if (made >= n && made < nmax && made < room && !(c < thr)) st[b].n = made + 1;
+}
+
+// Label pass (Section 3.3 / the draft-length oracle of Section 2.3): full-length drafts for every sequence ...
+__global__ void k_set_n_full(SeqState *st, int B, int nmax, int cap) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  const int room = cap - st[b].len - 1;
+  st[b].n = st[b].len < 2 ? 0 : max(0, min(nmax, room));
+}
+// ... and, after the verify pass, the length of the longest draft prefix the target confirms.  Nothing is committed.
+__global__ void k_label(const SeqState *st, const int *draft, const int *target, int nmax, int B, int *k_out) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  const int n = st[b].n;
+  int k = 0;
+  while (k < n && draft[b * nmax + k] == target[b * (nmax + 1) + k]) ++k;
+  k_out[b] = k;
 }
 
 __global__ void k_gather_n(const SeqState *st, int *out, int B) {

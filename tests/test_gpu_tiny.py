@@ -315,3 +315,55 @@ def test_ddd_stopping_rule_lockstep(tiny, thr, n_forced):
         assert lens == {sh.n_max}
     if thr == -4.0:
         assert lens == {n_forced}
+
+
+def test_label_pass_and_told_the_label_nothing_is_wasted(tiny, eng):
+    """Sections 2.3 / 3.3: ada_label = accept length of a full-length draft, state untouched; forcing n = label
+    gives N_waste = 0 (EAGLE-Oracle).  Teacher-forced drafts with planted mistakes make the labels non-trivial."""
+    sh, w, prompt, m = tiny
+    ar = oracle.decode(m, prompt, 48, n_policy=0)["tokens"]
+    bad = ar.copy()
+    bad[3::4] = (bad[3::4] + 1) % sh.vocab
+    seq, t_o, t_g = _prefill_both(eng, m, prompt)
+    assert t_o == t_g
+    d_k = torch.zeros(1, dtype=torch.int32, device=eng.dev)
+    before = eng.ada_get_counters()
+    labels = []
+    for it in range(8):
+        off = seq.len - len(prompt)
+        forced = np.asarray(bad[off: off + sh.n_max], dtype=np.int32)
+        ft = torch.zeros(1, sh.n_max, dtype=torch.int32)
+        ft[0, : len(forced)] = torch.from_numpy(forced)
+        eng.ada_force_draft(ft.to(eng.dev))
+        eng.ada_label(d_k)
+        k = int(d_k.cpu()[0])
+        # the label against the planted pattern; that the state is untouched shows in the step below
+        expect = 0
+        while expect < sh.n_max and (off + expect) % 4 != 3:
+            expect += 1
+        assert k == expect, (it, off, k, expect)
+        labels.append(k)
+        eng.ada_force_n([k])
+        o = seq.step(n_forced=k, forced_draft=forced)
+        g = eng.step()
+        assert g["n"][0] == k and g["k"][0] == o["k"] == k and list(g["emitted"][0]) == list(o["emitted"])
+    eng.ada_force_n(None)
+    eng.ada_force_draft(None)
+    after = eng.ada_get_counters()
+    assert after["n_waste"] == before["n_waste"]
+    assert max(labels) >= 3
+    assert after["status"] == 0
+
+
+def test_label_pass_matches_the_oracle_label_on_own_drafts(tiny, eng):
+    """Without forced drafts: the head's own full-length draft (random weights: labels are almost always 0)."""
+    sh, w, prompt, m = tiny
+    seq, t_o, t_g = _prefill_both(eng, m, prompt)
+    assert t_o == t_g
+    eng.ada_force_draft(None)
+    d_k = torch.zeros(1, dtype=torch.int32, device=eng.dev)
+    for it in range(4):
+        eng.ada_label(d_k)
+        assert int(d_k.cpu()[0]) == seq.label()
+        res = lockstep.run_lockstep(eng, [seq], 1)
+        assert not res["failures"], res["failures"]

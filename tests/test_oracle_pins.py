@@ -407,3 +407,38 @@ def test_ddd_output_is_still_greedy_decoding(tiny):
     sd = oracle.decode(m, prompt, 24, n_policy=1)
     assert list(sd["tokens"]) == list(ar)
     assert sd["counters"]["n_draft"] > sd["counters"]["n_target"]   # the rule did extend drafts past n = 1
+
+
+# ----------------------------------------------------------------- draft-length labels / EAGLE-Oracle (Sections 2.3, 3.3)
+
+def test_label_is_the_accept_length_of_a_full_draft_and_leaves_the_state_alone(tiny):
+    sh, w, prompt, m = tiny
+    ar = oracle.decode(m, prompt, 40, n_policy=0)["tokens"]
+    a, b = m.new_seq(512), m.new_seq(512)
+    a.prefill(prompt)
+    b.prefill(prompt)
+    bad = ar.copy()
+    bad[2::3] = (bad[2::3] + 1) % sh.vocab
+    for it in range(6):
+        k = a.label()
+        o = b.step(n_forced=sh.n_max)                   # same state: a full-length draft, verified and accepted
+        assert k == o["k"]
+        o2 = a.step(n_forced=sh.n_max)                  # the labelled sequence continues exactly like the other
+        assert list(o2["emitted"]) == list(o["emitted"]) and list(o2["draft"]) == list(o["draft"])
+    # with teacher-forced drafts corrupted at known places the label is the distance to the next corruption
+    c = m.new_seq(512)
+    c.prefill(prompt)
+    # (label() drafts with the head's own tokens, so here the corrupted stream is checked through step())
+    o = c.step(n_forced=sh.n_max, forced_draft=bad[1:1 + sh.n_max])
+    assert o["k"] == 1                                   # bad[2] is the first corrupted token: drafts 0..0 confirmed
+
+
+def test_told_the_label_no_draft_is_wasted(tiny):
+    """EAGLE-Oracle of Section 2.3: N_waste = 0, output unchanged, no more target passes than any fixed length."""
+    sh, w, prompt, m = tiny
+    ar = oracle.decode(m, prompt, 32, n_policy=0)["tokens"]
+    run = oracle.decode(m, prompt, 32, n_policy=lambda r, seq: seq.label())
+    assert np.array_equal(run["tokens"], ar)
+    assert run["counters"]["n_waste"] == 0
+    for n in (1, 4, sh.n_max):
+        assert run["counters"]["n_target"] <= oracle.decode(m, prompt, 32, n_policy=n)["counters"]["n_target"]
