@@ -478,8 +478,9 @@ __device__ __noinline__ void grid_barrier_body(unsigned *gbar, Counters *cnt, un
                                               volatile int *abort_flag) {
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
   if (tid == 32) {
-    __threadfence();
-    atomicAdd(gbar, 1u);
+    // arrive with release semantics (the named barrier above ordered the other threads' writes before this
+    // thread; the release makes them visible with the count), poll with acquire loads
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(gbar) : "memory");
     const unsigned target = epoch * gridDim.x;
     bool ok = false;
     for (unsigned i = 0; i < kSpinLimit && !*abort_flag; ++i) {
@@ -488,7 +489,6 @@ __device__ __noinline__ void grid_barrier_body(unsigned *gbar, Counters *cnt, un
       if (i > 4096) __nanosleep(64);   // a barrier normally completes within a few polls
     }
     if (!ok) { *abort_flag = 1; atomicOr(&cnt->status, kStatTimeout); }
-    __threadfence();
     if (phase_ns && blockIdx.x == 0 && epoch < 511) {
       unsigned long long t;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
