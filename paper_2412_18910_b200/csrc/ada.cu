@@ -14,6 +14,9 @@
 
 #include "ada_kernels.cuh"
 #include "ada_pass.cuh"
+#include "ada_gemm_tc.cuh"
+
+#include <unordered_map>
 
 using namespace ada;
 typedef __nv_bfloat16 bf16;
@@ -63,6 +66,12 @@ struct ada_ctx {
   size_t part_floats;
   // persistent pass kernel (batch 1): device copies of the layer pointer tables and its scratch
   int use_pass, n_sm, attn_splits;
+  // tensor-core GEMM of the multi-row path (passes of up to 88 rows): tensor maps of every weight matrix and of
+  // the activation planes, found by base pointer
+  int use_tc;
+  TensorMap128 *d_tcmaps;
+  int n_tcmaps;
+  std::unordered_map<const void *, int> tcmap_of;
   LayerPtrs *d_layers, *d_eagle;
   TensorMap128 *d_maps;
   int n_maps;
@@ -165,9 +174,30 @@ GemmPlan plan_gemm(int NT, int K, int tiles) {
   return p;
 }
 
+// K splits of the tensor-core GEMM: the smallest count that fills whole waves of one CTA per SM well (each split
+// costs a round trip of partial sums), with at least four 64-k boxes per split.
+int plan_tc_splits(int tiles, int K) {
+  const int sms = 148;   // B200; the split is part of the arithmetic (summation order), so it follows the shape alone
+  const int kboxes = (K + 63) / 64;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int S = 1; S <= 16 && S * 4 <= (kboxes > 4 ? kboxes : 4); ++S) {
+    const int ctas = tiles * S, waves = (ctas + sms - 1) / sms;
+    const double cost = (double)waves * sms / ctas + 0.03 * (S - 1);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = S; }
+  }
+  return best;
+}
+int tc_tiles(int epi, int nseg, int Nseg) { return epi == EPI_SWIGLU ? (Nseg + 127) / 128 : nseg * ((Nseg + 255) / 256); }
+
 size_t part_need(int NT, int Ntot, int K, int tiles) {
   GemmPlan p = plan_gemm(NT, K, tiles);
   return p.S > 1 ? (size_t)p.S * NT * 8 * Ntot : 0;
+}
+size_t part_need_tc(int epi, int nseg, int Nseg, int K) {
+  const int S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tc_tiles(epi, nseg, Nseg), K);
+  const size_t Ntot = epi == EPI_SWIGLU ? 2 * (size_t)Nseg : (size_t)nseg * Nseg;
+  return S > 1 ? (size_t)S * kTcRows * Ntot : 0;
 }
 
 // Lays the workspace out; with base == nullptr only measures it.
@@ -176,7 +206,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   const size_t d = c->d_model, F = c->d_ffn, V = c->vocab, L = c->n_layers, H = c->n_heads, hd = c->head_dim;
   const size_t B = c->max_batch, cap = c->kv_capacity, ps = c->page_size;
   const int TM = rows_per_pass(c), NT = TM / 8 > 2 ? 11 : 2;
-  const size_t TP = (size_t)NT * 8;
+  const size_t TP = kTcRows;   // row scratch holds the largest pass of any engine: prompts go through 88-row chunks
   const size_t pps = cap / ps, pages = pps * B;
   x->B = (int)B; x->TM = TM; x->NT = NT; x->pages_per_seq = (int)pps; x->n_pages = (int)pages;
   x->tk = w.take<bf16>(pages * L * H * ps * hd);
@@ -209,10 +239,18 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   upd(part_need(NT, (int)d, (int)F, (int)((d + 63) / 64)));
   upd(part_need(NT, (int)V, (int)d, (int)((V + 63) / 64)));
   upd(part_need(NT, (int)d, (int)(2 * d), (int)((d + 63) / 64)));
+  {
+    upd(part_need_tc(EPI_STORE, 3, (int)d, (int)d));
+    upd(part_need_tc(EPI_RESID, 1, (int)d, (int)d));
+    upd(part_need_tc(EPI_SWIGLU, 1, (int)F, (int)d));
+    upd(part_need_tc(EPI_RESID, 1, (int)d, (int)F));
+    upd(part_need_tc(EPI_ARGMAX, 1, (int)V, (int)d));
+    upd(part_need_tc(EPI_STORE, 1, (int)d, (int)(2 * d)));
+  }
   x->part_floats = pf;
   x->gemm_part = w.take<float>(pf ? pf : 1);
   x->gemm_cnt = w.take<int>(4096);
-  x->amax = w.take<float4>(((V + 63) / 64) * TP);
+  x->amax = w.take<float4>(((V + 63) / 64) * TP);   // (at least as many tiles as either GEMM uses)
   x->ldlp_h = w.take<float>(B * c->ldlp_hidden);
   x->ldlp_h2 = w.take<float>(B * c->ldlp_hidden);
   x->ldlp_z = w.take<float>(B * 16);
@@ -234,6 +272,8 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->d_eagle = w.take<LayerPtrs>(1);
   x->n_maps = (int)(7 * (L + 1) + 2 + 8);
   x->d_maps = w.take<TensorMap128>(x->n_maps);
+  x->n_tcmaps = (int)(7 * (L + 1) + 2 + 4);
+  x->d_tcmaps = w.take<TensorMap128>(x->n_tcmaps);
   x->xa = w.take<bf16>(((d + 63) / 64) * 2048);
   x->at = w.take<bf16>(((d + 63) / 64) * 2048);
   x->ac = w.take<bf16>(((F + 63) / 64) * 2048);
@@ -274,6 +314,32 @@ cudaError_t gemm_attr_nt(int bytes) {
 void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, int nseg, int Nseg, int K,
           const bf16 *Xhi, const bf16 *Xlo, int ldx, float *Y, int ldy, bf16 *Ohi, bf16 *Olo, int ldo,
           float *logits, int use_lm_rows) {
+  if (x->NT != 2) {
+    GemmTcArgs t;
+    memset(&t, 0, sizeof(t));
+    const bf16 *Ws[3] = {W0, W1, W2};
+    for (int i = 0; i < 3; ++i)
+      if (Ws[i]) t.wmap[i] = x->d_tcmaps + x->tcmap_of.at(Ws[i]);
+    t.xhi_map = x->d_tcmaps + x->tcmap_of.at(Xhi);
+    t.xlo_map = x->d_tcmaps + x->tcmap_of.at(Xlo);
+    t.epi = epi; t.nseg = nseg; t.Nseg = Nseg; t.K = K;
+    const int tiles = tc_tiles(epi, nseg, Nseg);
+    t.S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tiles, K);
+    t.Y = Y; t.ldy = ldy; t.Ohi = Ohi; t.Olo = Olo; t.ldo = ldo;
+    t.part = x->gemm_part;
+    t.logits = logits; t.ldl = x->c.vocab; t.amax = x->amax;
+    t.pass = x->pass; t.use_lm_rows = use_lm_rows; t.cnts = x->cnt;
+    const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
+    timed(x, 0, wb, [&] {
+      LAUNCH(x, k_gemm_tc, dim3(tiles, t.S), kTcThreads, kTcSmemBytes, t);
+      if (t.S > 1) {   // the splits' partial sums, added in split order, then the epilogue
+        const int ncol = epi == EPI_SWIGLU ? Nseg : nseg * Nseg;
+        const int blocks = (kTcRows * (ncol / 4) + 255) / 256;
+        LAUNCH(x, k_tc_reduce, blocks < 1184 ? blocks : 1184, 256, 0, t);
+      }
+    });
+    return;
+  }
   GemmArgs a;
   memset(&a, 0, sizeof(a));
   a.W[0] = W0; a.W[1] = W1; a.W[2] = W2;
@@ -290,24 +356,23 @@ void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   const size_t smem = (size_t)2 * x->NT * 8 * (p.KC * 2 + 64);
   dim3 grid(tiles, p.S);
   const double wbytes = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
-  timed(x, 0, wbytes, [&] {
-    if (x->NT == 2) launch_gemm_nt<2>(x, epi, a, grid, smem);
-    else launch_gemm_nt<11>(x, epi, a, grid, smem);
-  });
+  timed(x, 0, wbytes, [&] { launch_gemm_nt<2>(x, epi, a, grid, smem); });   // (16-row passes without the persistent kernel)
 }
 
 void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   const ada_config &c = x->c;
-  dim3 g1(c.n_heads, kAttnSplits, x->B);
+  // query rows of a sequence in groups of 16 across grid.z (a prompt chunk is one sequence with up to 88 rows)
+  const int nrg = (x->TM / x->B + kRowGroup - 1) / kRowGroup;
+  dim3 g1(c.n_heads, kAttnSplits, x->B * nrg);
   dim3 g2(c.n_heads, x->TM);
   timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
     LAUNCH(x, k_attn_partial<128>, g1, 128, attn_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
     LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   } else {
     LAUNCH(x, k_attn_partial<64>, g1, 128, attn_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
     LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   }
   });
@@ -320,7 +385,7 @@ void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L,
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.na, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
   gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->ldx, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rope_kv, x->TM, 256, 0, x->pass, x->qkv, x->rope, x->qrot, kpool, vpool, x->page_table,
-         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim));
+         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim), x->use_pass);
   attention(x, kpool, vpool, L, layer);
   gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->ldx, x->h, d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.nm, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
@@ -344,8 +409,8 @@ void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int ldx, int use_lm_r
   const ada_config &c = x->c;
   gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, ldx, nullptr, 0, nullptr, nullptr,
        0, logits, use_lm_rows);
-  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 63) / 64, x->NT * 8, x->pass, use_lm_rows, tok_out,
-         top_out, forced);
+  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, x->NT != 2 ? (c.vocab + 255) / 256 : (c.vocab + 63) / 64, x->NT * 8,
+         x->pass, use_lm_rows, tok_out, top_out, forced);
 }
 
 // Draft head over the rows of x->pass (already built for `step`).
@@ -411,6 +476,37 @@ bool build_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
   layer(7 * c.n_layers, x->eagle);
   const int m0 = 7 * (c.n_layers + 1);
   ok = ok && encode_map(fn, &maps[m0], x->eagle_fc, d, 2 * d, b_fc) && encode_map(fn, &maps[m0 + 1], x->lm_head, V, d, b_v);
+  return ok;
+}
+
+// Tensor maps of the multi-row tensor-core GEMM: every weight matrix with a box of 64 k x 128 rows, the four
+// activation planes with a box of 64 k x 88 rows; tcmap_of finds a map by the base pointer of its tensor.
+bool build_tc_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
+  void *sym = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym) return false;
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(sym);
+  const ada_config &c = x->c;
+  const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+  maps.assign(x->n_tcmaps, TensorMap128());
+  x->tcmap_of.clear();
+  bool ok = true;
+  int next = 0;
+  auto add = [&](const void *base, size_t rows, size_t cols, unsigned box_rows) {
+    if (x->tcmap_of.count(base)) return;   // a tensor is looked up by its base pointer
+    ok = ok && next < x->n_tcmaps && encode_map(fn, &maps[next], base, rows, cols, box_rows);
+    x->tcmap_of[base] = next++;
+  };
+  auto layer = [&](const LayerW &a) {
+    add(a.wq, d, d, 128); add(a.wk, d, d, 128); add(a.wv, d, d, 128); add(a.wo, d, d, 128);
+    add(a.wg, F, d, 128); add(a.wu, F, d, 128); add(a.wd, d, F, 128);
+  };
+  for (int l = 0; l < c.n_layers; ++l) layer(x->layers[l]);
+  layer(x->eagle);
+  add(x->eagle_fc, d, 2 * d, 128);
+  add(x->lm_head, V, d, 128);
+  add(x->xhi, kTcRows, x->ldx, kTcRows); add(x->xlo, kTcRows, x->ldx, kTcRows);
+  add(x->x2hi, kTcRows, x->ldx2, kTcRows); add(x->x2lo, kTcRows, x->ldx2, kTcRows);
   return ok;
 }
 
@@ -600,10 +696,10 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess) e = cudaMemsetAsync(x->target, 0, sizeof(int) * x->B * (cfg->n_max + 1), x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->force_n_dev, 0, sizeof(int) * x->B, x->stream);
   // activation staging rows beyond the live ones are read by the tensor-core tiles: keep them finite
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->xhi, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->xlo, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)x->NT * 8 * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xhi, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xlo, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);  // host vectors go out of scope
   // persistent pass kernel: used when a pass never has more than 16 rows (batch 1)
   x->use_pass = 0;
@@ -656,8 +752,19 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }
   }
+  // passes of more than 16 rows: the tensor-core GEMM
+  x->use_tc = 0;
+  const bool tc_fits = cfg->d_model >= 128 && cfg->d_ffn >= 128 && cfg->vocab >= 128;   // boxes are 128 rows high
+  if (e == cudaSuccess && !tc_fits && x->NT != 2) e = cudaErrorInvalidValue;
+  if (e == cudaSuccess && tc_fits) {
+    e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    std::vector<TensorMap128> maps;
+    if (e == cudaSuccess && !build_tc_maps(x, maps)) e = cudaErrorUnknown;
+    if (e == cudaSuccess) e = cudaMemcpy(x->d_tcmaps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) x->use_tc = 1;
+  }
   const int gemm_smem = 2 * x->NT * 8 * ((x->NT == 2 ? 1024 : 256) * 2 + 64);
-  if (e == cudaSuccess) e = x->NT == 2 ? gemm_attr_nt<2>(gemm_smem) : gemm_attr_nt<11>(gemm_smem);
+  if (e == cudaSuccess && x->NT == 2) e = gemm_attr_nt<2>(gemm_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_attn_partial<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<128>());
   if (e == cudaSuccess)
@@ -682,10 +789,16 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
   LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
   int last_rows = 0;
+  // A prompt is a many-row pass: an engine whose decode passes have 16 rows takes it through the multi-row kernels
+  // (tensor-core GEMM, 88 rows per chunk: a sixth of the weight passes) when their tensor maps exist.
+  const bool wide = x->NT == 2 && x->use_tc;
+  const bool by_pass = x->use_pass && !wide;
+  const int TM0 = x->TM, NT0 = x->NT;
+  if (wide) { x->TM = kTcRows; x->NT = kTcRows / 8; }
   for (int p0 = 0; p0 < m; p0 += x->TM) {
     const int R = (m - p0 < x->TM) ? m - p0 : x->TM;
     LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
-    if (x->use_pass) {  // the LM phase also writes the features; its choices matter only in the last chunk
+    if (by_pass) {  // the LM phase also writes the features; its choices matter only in the last chunk
       run_pass(x, 0, 0, 1, nullptr, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr);
       if (p0 + R == m) last_rows = R;
     } else {
@@ -699,10 +812,11 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
     const int Rd = (p0 + R <= m - 1) ? R : (m - 1 - p0);
     if (Rd > 0) {
       LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
-      if (x->use_pass) run_pass(x, 1, 0, 0, nullptr, nullptr, nullptr, nullptr);
+      if (by_pass) run_pass(x, 1, 0, 0, nullptr, nullptr, nullptr, nullptr);
       else draft_rows(x, 0, false);
     }
   }
+  x->TM = TM0; x->NT = NT0;
   LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),
          d_first_token);
   return cuda_ok(x, "ada_prefill") ? ADA_OK : ADA_ERR_CUDA;

@@ -1,0 +1,295 @@
+// Multi-row GEMM on the 5th-generation tensor cores for passes of up to 88 rows (ragged batches, prompt chunks):
+//   Y[t][n] = sum_k X[t][k] * W[n][k],  t < T <= 88,  W bf16 [N][K] streamed once from HBM.
+//
+// With this many rows the activation operand is no longer small next to the weights (88 rows x {hi, lo} = 22 KB per
+// 64 k against 16 KB for 128 weight rows), so a CTA takes a tall tile -- two m tiles of 128 weight rows that share
+// every activation box (SwiGLU: 128 rows of the gate and the same 128 rows of the up matrix) -- and a range of K
+// (grid.y splits); level-2 to shared-memory traffic then stays below 1.7 times the weight bytes.
+//
+//   warp 0   producer, one thread: per 64 k one stage = weight boxes (TMA tiled loads, 128-byte swizzle, box 64 k x 128
+//            rows) + the hi plane box and the lo plane box of the activations (64 k x 88 rows each, stacked so that they
+//            form one K-major operand of 176 rows); 4 stages of 54 KB, mbarrier transaction counts
+//   warp 1   one elected thread issues tcgen05.mma (M = 128, N = 176, K = 16) per m tile and 16 k straight from the
+//            TMA-written tiles; accumulators in tensor memory (m tile i in columns [256 i, 256 i + 176));
+//            tcgen05.commit frees the stage and, at the end, signals the accumulators
+//   warp 2   owns the tensor-memory allocation (512 columns)
+//   warps 4..11  epilogue: thread = one weight row (tensor-memory lane), tcgen05.ld eight pass rows at a time,
+//            column t (hi) + column 88 + t (lo)
+//
+// K splits leave their partial sums in a scratch buffer and k_tc_reduce, launched next, adds them in split order
+// and runs the epilogue over the whole grid (a last-arriving CTA per tile doing this alone was measured to take
+// longer than the products: 16 CTAs walking 9 x 88 x 256 values each).  Every output element depends only on its
+// own input row and on the fixed split of K.  Every wait is bounded.
+#pragma once
+#include "ada_pass.cuh"
+
+namespace ada {
+
+constexpr int kTcRows = 88;                          // rows of a pass at most = box height of the plane maps
+constexpr int kTcN = 2 * kTcRows;                    // MMA N: hi rows then lo rows
+constexpr int kTcABytes = 128 * 128;                 // one weight box: 128 rows x 64 k bf16
+constexpr int kTcBBytes = kTcRows * 128;             // one plane box
+constexpr int kTcStageBytes = 2 * kTcABytes + 2 * kTcBBytes;   // 55296
+constexpr int kTcStages = 4;
+constexpr int kTcThreads = 12 * 32;
+constexpr int kTcSmemBytes = 1024 + kTcStages * kTcStageBytes + 256;
+constexpr int kTcTmemCols = 512;
+static_assert(kTcBBytes % 1024 == 0, "the lo plane must start on a swizzle-atom boundary");
+static_assert(kTcSmemBytes <= 227 * 1024, "shared memory budget");
+
+struct GemmTcArgs {
+  const TensorMap128 *wmap[3];   // box {64 k, 128 rows}; STORE: up to 3 row segments; SWIGLU: gate, up
+  const TensorMap128 *xhi_map, *xlo_map;   // planes [88][ld]: box {64 k, 88 rows}
+  int epi;                    // EPI_STORE / EPI_RESID / EPI_SWIGLU / EPI_ARGMAX
+  int nseg, Nseg, K;
+  int S;                      // K splits (grid.y)
+  float *Y; int ldy;          // STORE / RESID target
+  __nv_bfloat16 *Ohi, *Olo; int ldo;   // SWIGLU target planes
+  float *part;                // [S][88][Ntot] partial sums (S > 1; ARGMAX is never split)
+  float *logits; int ldl;     // ARGMAX: optional logits [slot][ldl]
+  float4 *amax;               // ARGMAX: [tiles][88] (v1, i1, v2)
+  const Pass *pass;
+  int use_lm_rows;            // ARGMAX in the draft: T = pass->lmT, slots = pass->lm_out
+  Counters *cnts;             // status word for waits that gave up
+};
+
+// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = 128, N = 176, K = 16
+__host__ __device__ constexpr uint32_t umma_idesc_mn(uint32_t m, uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
+}
+// 8 consecutive accumulator columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
+  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
+  if (T <= 0) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool sw = a.epi == EPI_SWIGLU;
+
+  extern __shared__ __align__(128) unsigned char tc_smem[];
+  unsigned char *const smem = tc_smem + ((1024u - (smem_u32(tc_smem) & 1023u)) & 1023u);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kTcStages * kTcStageBytes);
+  uint64_t *full = bars, *empty = bars + kTcStages, *accfull = bars + 2 * kTcStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kTcStages + 1);
+  int *flag_s = reinterpret_cast<int *>(tmem_slot + 1);
+  volatile int *abort_s = flag_s + 1;
+
+  // tile -> segment (matrix), first weight row of each m tile
+  const int tiles_per_seg = sw ? (a.Nseg + 127) / 128 : (a.Nseg + 255) / 256;
+  const int seg = sw ? 0 : blockIdx.x / tiles_per_seg;
+  const int tile = sw ? blockIdx.x : blockIdx.x - seg * tiles_per_seg;
+  const int row0 = sw ? tile * 128 : tile * 256;                    // m tile 0
+  const int row1 = sw ? row0 : row0 + 128;                          // m tile 1
+  const int mtiles = sw ? 2 : (row1 < a.Nseg ? 2 : 1);
+  const int kboxes = (a.K + 63) >> 6;
+  const int kb0 = (int)(((long long)blockIdx.y * kboxes) / a.S), kb1 = (int)(((long long)(blockIdx.y + 1) * kboxes) / a.S);
+
+  if (tid == 0) {
+    *abort_s = 0;
+    for (int i = 0; i < kTcStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(accfull, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) tmem_alloc(tmem_slot, kTcTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- producer
+    if (lane == 0) {
+      const TensorMap128 *m0 = sw ? a.wmap[0] : a.wmap[seg];
+      const TensorMap128 *m1 = sw ? a.wmap[1] : a.wmap[seg];
+      const unsigned tx = (unsigned)(mtiles * kTcABytes + 2 * kTcBBytes);
+      for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
+        const int s = i % kTcStages;
+        if (i >= kTcStages) mbar_wait(&empty[s], ((unsigned)(i / kTcStages) & 1u) ^ 1u, a.cnts, abort_s);
+        unsigned char *st = smem + (size_t)s * kTcStageBytes;
+        mbar_expect_tx(&full[s], tx);
+        tma_load_2d(st, m0, kb * 64, row0, &full[s]);                 // rows past the matrix and k past K read as zero
+        if (mtiles > 1) tma_load_2d(st + kTcABytes, m1, kb * 64, row1, &full[s]);
+        tma_load_2d(st + 2 * kTcABytes, a.xhi_map, kb * 64, 0, &full[s]);
+        tma_load_2d(st + 2 * kTcABytes + kTcBBytes, a.xlo_map, kb * 64, 0, &full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- tensor-core issuer
+    const uint32_t idesc = umma_idesc_mn(128u, (uint32_t)kTcN);
+    for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
+      const int s = i % kTcStages;
+      mbar_wait(&full[s], (unsigned)(i / kTcStages) & 1u, a.cnts, abort_s);
+      tc_fence_after();
+      if (elect_one()) {
+        const uint32_t st = smem_u32(smem + (size_t)s * kTcStageBytes);
+        const uint64_t bd = umma_desc(st + 2 * kTcABytes);
+        const int nstep = min(4, (a.K - kb * 64 + 15) >> 4);          // k16 steps holding any k < K
+        for (int mi = 0; mi < mtiles; ++mi) {
+          const uint64_t ad = umma_desc(st + (uint32_t)mi * kTcABytes);
+          const uint32_t dcol = tmem_base + (uint32_t)mi * 256;
+          for (int k4 = 0; k4 < nstep; ++k4) umma_bf16(dcol, ad + 2 * k4, bd + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty[s]);
+      }
+      __syncwarp();
+    }
+    if (elect_one()) umma_commit(accfull);
+    __syncwarp();
+  }
+
+  if (warp >= 4) {
+    // ------------------------------------------------------------- epilogue
+    const int cw = warp - 4, quarter = warp & 3;
+    const int ctid = tid - 128;
+    const int mi = sw ? 0 : (cw >> 2);
+    const bool active_warp = sw ? cw < 4 : mi < mtiles;
+    const int n = (mi ? row1 : row0) + quarter * 32 + lane;         // weight row inside the segment
+    const bool valid = active_warp && n < a.Nseg;
+    const int Ntot = sw ? 2 * a.Nseg : a.nseg * a.Nseg;
+    const int col = seg * a.Nseg + n;                                  // output column (SWIGLU: gate column)
+    const int nblk = (T + 7) >> 3;
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * 256);
+
+    if (kb1 > kb0) mbar_wait(accfull, 0u, a.cnts, abort_s);
+    tc_fence_after();
+
+    // pass rows 8 j .. 8 j + 7 of this thread's weight row: y (and u, the up projection, for SWIGLU)
+    auto from_tmem = [&](int j, float (&y)[8], float (&u)[8]) {
+      float hi[8], lo[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { y[i] = 0.f; u[i] = 0.f; }
+      if (!active_warp || kb1 <= kb0) return;     // (warp-uniform)
+      tmem_ld8(taddr + (uint32_t)(8 * j), hi);
+      tmem_ld8(taddr + (uint32_t)(kTcRows + 8 * j), lo);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) y[i] = hi[i] + lo[i];
+      if (sw) {
+        tmem_ld8(taddr + 256u + (uint32_t)(8 * j), hi);
+        tmem_ld8(taddr + 256u + (uint32_t)(kTcRows + 8 * j), lo);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = hi[i] + lo[i];
+      }
+    };
+
+    if (a.S > 1) {
+      for (int j = 0; j < nblk; ++j) {
+        float y[8], u[8];
+        from_tmem(j, y, u);
+        if (valid) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int t = 8 * j + i;
+            if (t < T) {
+              float *pp = a.part + ((size_t)blockIdx.y * kTcRows + t) * Ntot;
+              __stcg(pp + col, y[i]);
+              if (sw) __stcg(pp + a.Nseg + n, u[i]);
+            }
+          }
+        }
+      }
+    } else {
+      Top2 *s_top = reinterpret_cast<Top2 *>(smem);   // [8 warps][88]: the stages are idle by now
+      if (a.epi == EPI_ARGMAX) named_bar(3, 256);
+      for (int j = 0; j < nblk; ++j) {
+        float y[8], u[8];
+        from_tmem(j, y, u);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int t = 8 * j + i;
+          if (t >= T) continue;     // (uniform over the CTA)
+          if (a.epi == EPI_STORE) {
+            if (valid) a.Y[(size_t)t * a.ldy + col] = y[i];
+          } else if (a.epi == EPI_RESID) {
+            if (valid) a.Y[(size_t)t * a.ldy + col] += y[i];
+          } else if (sw) {
+            if (valid) {
+              const float o = (y[i] / (1.f + __expf(-y[i]))) * u[i];
+              __nv_bfloat16 hi, lo;
+              split_bf16(o, hi, lo);
+              a.Ohi[(size_t)t * a.ldo + n] = hi;
+              a.Olo[(size_t)t * a.ldo + n] = lo;
+            }
+          } else {   // EPI_ARGMAX: the warp's two largest logits of this pass row
+            Top2 b;
+            b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+            if (valid) {
+              if (a.logits) {
+                const int slot = a.use_lm_rows ? a.pass->lm_out[t] : a.pass->row_out[t];
+                a.logits[(size_t)slot * a.ldl + n] = y[i];
+              }
+              b.v1 = y[i]; b.i1 = n;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+            if (lane == 0) s_top[cw * kTcRows + t] = b;
+          }
+        }
+      }
+      if (a.epi == EPI_ARGMAX) {
+        named_bar(3, 256);
+        if (ctid < T) {
+          Top2 b = s_top[ctid];
+          for (int w = 1; w < 8; ++w) b = top2_merge(b, s_top[w * kTcRows + ctid]);
+          a.amax[(size_t)blockIdx.x * kTcRows + ctid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+        }
+      }
+    }
+  }
+
+  // every read of tensor memory is done: free it
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 2) tmem_dealloc(tmem_base, kTcTmemCols);
+}
+
+// Sum of the K splits' partial sums in split order, then the epilogue; one thread per (pass row, 4 output columns).
+__global__ void __launch_bounds__(256) k_tc_reduce(const GemmTcArgs a) {
+  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
+  const bool sw = a.epi == EPI_SWIGLU;
+  const int Ntot = sw ? 2 * a.Nseg : a.nseg * a.Nseg;
+  const int ncol = sw ? a.Nseg : Ntot;           // output columns
+  const int c4 = ncol >> 2;                       // (column counts are multiples of 16)
+  for (int idx = blockIdx.x * 256 + threadIdx.x; idx < T * c4; idx += gridDim.x * 256) {
+    const int t = idx / c4, col = (idx - t * c4) << 2;
+    float4 y = make_float4(0.f, 0.f, 0.f, 0.f), u = y;
+    for (int sp = 0; sp < a.S; ++sp) {
+      const float *pp = a.part + ((size_t)sp * kTcRows + t) * Ntot + col;
+      const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp));
+      y.x += v.x; y.y += v.y; y.z += v.z; y.w += v.w;
+      if (sw) {
+        const float4 w = __ldcg(reinterpret_cast<const float4 *>(pp + a.Nseg));
+        u.x += w.x; u.y += w.y; u.z += w.z; u.w += w.w;
+      }
+    }
+    if (a.epi == EPI_STORE) {
+      *reinterpret_cast<float4 *>(a.Y + (size_t)t * a.ldy + col) = y;
+    } else if (a.epi == EPI_RESID) {
+      float4 *yp = reinterpret_cast<float4 *>(a.Y + (size_t)t * a.ldy + col);
+      float4 h = *yp;
+      h.x += y.x; h.y += y.y; h.z += y.z; h.w += y.w;
+      *yp = h;
+    } else if (sw) {
+      const float yy[4] = {y.x, y.y, y.z, y.w}, uu[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float o = (yy[i] / (1.f + __expf(-yy[i]))) * uu[i];
+        __nv_bfloat16 hi, lo;
+        split_bf16(o, hi, lo);
+        a.Ohi[(size_t)t * a.ldo + col + i] = hi;
+        a.Olo[(size_t)t * a.ldo + col + i] = lo;
+      }
+    }
+  }
+}
+
+}  // namespace ada

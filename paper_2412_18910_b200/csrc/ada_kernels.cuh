@@ -460,9 +460,11 @@ __global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bf
 // Rotary embedding (rotate-half pairing) of q and k, scaling of q by 1/sqrt(hd), and the write of
 // k, v (bf16) into the paged cache.  qkv: [T][3d] fp32.  rope: [cap][hd/2] (cos, sin).
 // Cache element (page, layer, head, slot, i): ((page*L + layer)*H + head)*page_size*hd + slot*hd + i.
+// kswz: key rows are stored with their 16-byte chunks XORed by (slot & 7), the layout the persistent pass kernel
+// keeps its caches in (an engine that decodes with that kernel and takes prompts through this one).
 __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope, float *qout,
                           __nv_bfloat16 *kpool, __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
-                          int page_size, int L, int layer, int H, int hd, float qscale) {
+                          int page_size, int L, int layer, int H, int hd, float qscale, int kswz) {
   const int t = blockIdx.x;
   if (t >= pass->T) return;
   const int d = H * hd, half = hd >> 1;
@@ -477,8 +479,9 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
     qout[(size_t)t * d + o] = (qa * cs.x - qb * cs.y) * qscale;
     qout[(size_t)t * d + o + half] = (qb * cs.x + qa * cs.y) * qscale;
     const size_t base = (((size_t)page * L + layer) * H + hh) * page_size * hd + (size_t)slot * hd;
-    kpool[base + i] = kv_store(ka * cs.x - kb * cs.y);
-    kpool[base + i + half] = kv_store(kb * cs.x + ka * cs.y);
+    const int sw = kswz ? (slot & 7) : 0;
+    kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(ka * cs.x - kb * cs.y);
+    kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(kb * cs.x + ka * cs.y);
     vpool[base + i] = kv_store(v[o]);
     vpool[base + i + half] = kv_store(v[o + half]);
   }
@@ -493,9 +496,10 @@ template <int HD>
 __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
                                                       const __nv_bfloat16 *vpool, const int *page_table,
                                                       int pages_per_seq, int page_size, int L, int layer, int H,
-                                                      float *part) {
+                                                      float *part, int kswz, int nrg) {
   constexpr int VPL = HD / 32;  // value channels per lane
-  const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
+  // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
+  const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / nrg, rgi = blockIdx.z - b * nrg;
   const int R = pass->seq_rows[b];
   if (pass->T <= 0 || R <= 0) return;
   const int row0 = pass->seq_row0[b];
@@ -515,7 +519,7 @@ __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const fl
   float (*o_s)[kRowGroup][HD] =
       reinterpret_cast<float (*)[kRowGroup][HD]>(attn_smem + kRowGroup * HD + 4 * kRowGroup * 32 + 8 * kRowGroup);
 
-  for (int rg = 0; rg < R; rg += kRowGroup) {
+  for (int rg = rgi * kRowGroup; rg < R; rg += nrg * kRowGroup) {
     const int nr = min(kRowGroup, R - rg);
     __syncthreads();
     for (int i = threadIdx.x; i < nr * HD; i += 128) {
@@ -540,9 +544,10 @@ __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const fl
         const int page = page_table[b * pages_per_seq + key / page_size], slot = key % page_size;
         const uint4 *kr = reinterpret_cast<const uint4 *>(
             kpool + (((size_t)page * L + layer) * H + hh) * page_size * HD + (size_t)slot * HD);
+        const int ksw = kswz ? (slot & 7) : 0;   // chunk-swizzled key rows (see k_rope_kv)
 #pragma unroll 4
         for (int c = 0; c < HD / 8; ++c) {
-          const uint4 kk = kr[c];
+          const uint4 kk = kr[c ^ ksw];
           float kf[8];
           kf[0] = kv_lo(kk.x); kf[1] = kv_hi(kk.x);
           kf[2] = kv_lo(kk.y); kf[3] = kv_hi(kk.y);
