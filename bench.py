@@ -291,6 +291,19 @@ def main():
            "d2h_bytes_per_step": h_out.numel() * 4, "steps": Ke,
            "note": "request latency: pinned-host prompt copy + prefill + steps with a host read-back each"}
 
+    # ---- prompt pass (Algorithm 1's first verify, k = 0): device time of ada_prefill on the resident prompt
+    pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pre_ms = []
+    for _ in range(3):
+        torch.cuda.synchronize(dev)
+        pa.record(eng.stream)
+        eng.ada_prefill(0, d_prompt, None)
+        pb.record(eng.stream)
+        torch.cuda.synchronize(dev)
+        pre_ms.append(pa.elapsed_time(pb))
+    prefill = {"prompt_len": int(sh.prompt_len), "ms": min(pre_ms), "prompt_tokens_per_s": sh.prompt_len / (min(pre_ms) * 1e-3),
+               "note": "88-row chunks through the multi-row tensor-core GEMM; not part of the decode metric"}
+
     # ---- roofline leg: the dominant kernel (skinny GEMM) and the whole verify pass, timed with
     # events on the library's stream at the context length the timed region ended at
     peak, peak_kind = load_peaks()
@@ -354,7 +367,7 @@ def main():
             "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights and KV cache, f32 accumulate", "data": "synthetic", "config": config,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "tau": tokens / max(1, n_target), "mean_draft_len": n_draft / max(1, n_target)}
+            "tau": tokens / max(1, n_target), "mean_draft_len": n_draft / max(1, n_target), "prefill": prefill}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         tps, ms, threads, desc = oracle_sample(sh, weights, prompt, 10 if sh.name != "tiny" else 64, 1)

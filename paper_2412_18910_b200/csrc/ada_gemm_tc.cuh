@@ -93,11 +93,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   const int kboxes = (a.K + 63) >> 6;
   const int kb0 = (int)(((long long)blockIdx.y * kboxes) / a.S), kb1 = (int)(((long long)(blockIdx.y + 1) * kboxes) / a.S);
 
+  // The producing thread initialises the barriers and fills the first stages at once: the loads fly while the
+  // tensor memory is allocated and the CTA meets at the barrier below.
+  const TensorMap128 *m0 = sw ? a.wmap[0] : a.wmap[seg];
+  const TensorMap128 *m1 = sw ? a.wmap[1] : a.wmap[seg];
+  const unsigned tx = (unsigned)(mtiles * kTcABytes + 2 * kTcBBytes);
+  auto load_stage = [&](int kb, int s) {
+    unsigned char *st = smem + (size_t)s * kTcStageBytes;
+    mbar_expect_tx(&full[s], tx);
+    tma_load_2d(st, m0, kb * 64, row0, &full[s]);                 // rows past the matrix and k past K read as zero
+    if (mtiles > 1) tma_load_2d(st + kTcABytes, m1, kb * 64, row1, &full[s]);
+    tma_load_2d(st + 2 * kTcABytes, a.xhi_map, kb * 64, 0, &full[s]);
+    tma_load_2d(st + 2 * kTcABytes + kTcBBytes, a.xlo_map, kb * 64, 0, &full[s]);
+  };
+  const int nfirst = min(kTcStages, kb1 - kb0);
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kTcStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(accfull, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int i = 0; i < nfirst; ++i) load_stage(kb0 + i, i);
   }
   if (warp == 2) tmem_alloc(tmem_slot, kTcTmemCols);
   tc_fence_before();
@@ -108,18 +123,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   if (warp == 0) {
     // ------------------------------------------------------------- producer
     if (lane == 0) {
-      const TensorMap128 *m0 = sw ? a.wmap[0] : a.wmap[seg];
-      const TensorMap128 *m1 = sw ? a.wmap[1] : a.wmap[seg];
-      const unsigned tx = (unsigned)(mtiles * kTcABytes + 2 * kTcBBytes);
-      for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
+      for (int kb = kb0 + nfirst, i = nfirst; kb < kb1; ++kb, ++i) {
         const int s = i % kTcStages;
-        if (i >= kTcStages) mbar_wait(&empty[s], ((unsigned)(i / kTcStages) & 1u) ^ 1u, a.cnts, abort_s);
-        unsigned char *st = smem + (size_t)s * kTcStageBytes;
-        mbar_expect_tx(&full[s], tx);
-        tma_load_2d(st, m0, kb * 64, row0, &full[s]);                 // rows past the matrix and k past K read as zero
-        if (mtiles > 1) tma_load_2d(st + kTcABytes, m1, kb * 64, row1, &full[s]);
-        tma_load_2d(st + 2 * kTcABytes, a.xhi_map, kb * 64, 0, &full[s]);
-        tma_load_2d(st + 2 * kTcABytes + kTcBBytes, a.xlo_map, kb * 64, 0, &full[s]);
+        mbar_wait(&empty[s], ((unsigned)(i / kTcStages) & 1u) ^ 1u, a.cnts, abort_s);
+        load_stage(kb, s);
       }
     }
   } else if (warp == 1) {

@@ -410,8 +410,10 @@ __global__ void k_argmax_final(const float4 *amax, int tiles, int TP, const Pass
 __global__ void k_embed(const Pass *pass, const __nv_bfloat16 *embed, float *h, int d) {
   const int t = blockIdx.x;
   if (t >= pass->T) return;
-  const __nv_bfloat16 *e = embed + (size_t)pass->row_tok[t] * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)t * d + i] = __bfloat162float(e[i]);
+  const __nv_bfloat16 *__restrict__ e = embed + (size_t)pass->row_tok[t] * d;
+  float *__restrict__ hr = h + (size_t)t * d;
+#pragma unroll 8
+  for (int i = threadIdx.x; i < d; i += blockDim.x) hr[i] = __bfloat162float(e[i]);   // (loads of a row in flight together)
 }
 
 // x = h / sqrt(mean(h^2) + eps) * gain  ->  hi/lo halves; optionally also fp32 rows to
@@ -421,18 +423,41 @@ __global__ void k_rmsnorm(const Pass *pass, const float *h, const __nv_bfloat16 
   __shared__ float sh[32];
   const int t = blockIdx.x;
   if (t >= pass->T) return;
-  const float *hr = h + (size_t)t * d;
+  // four elements per thread and step (d is a multiple of 64), the steps unrolled so that a row's loads are in
+  // flight together: one element per step ran at one level-2 round trip per step
+  const float4 *__restrict__ h4 = reinterpret_cast<const float4 *>(h + (size_t)t * d);
+  const int d4 = d >> 2;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += hr[i] * hr[i];
+#pragma unroll 4
+  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
+    const float4 v = h4[i];
+    ss += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+  }
   ss = block_sum(ss, sh);
   const float inv = rsqrtf(ss / (float)d + eps);
-  float *fr = feat ? feat + ((size_t)pass->row_seq[t] * cap + pass->row_pos[t]) * d : nullptr;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float x = (hr[i] * inv) * __bfloat162float(gain[i]);
-    __nv_bfloat16 hi, lo;
-    split_bf16(x, hi, lo);
-    xhi[(size_t)t * ldx + i] = hi;
-    xlo[(size_t)t * ldx + i] = lo;
+  float4 *__restrict__ fr =
+      feat ? reinterpret_cast<float4 *>(feat + ((size_t)pass->row_seq[t] * cap + pass->row_pos[t]) * d) : nullptr;
+  const uint2 *__restrict__ g4 = reinterpret_cast<const uint2 *>(gain);
+  uint2 *__restrict__ oh = reinterpret_cast<uint2 *>(xhi + (size_t)t * ldx);
+  uint2 *__restrict__ ol = reinterpret_cast<uint2 *>(xlo + (size_t)t * ldx);
+#pragma unroll 4
+  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
+    const float4 v = h4[i];
+    const uint2 gg = g4[i];
+    const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x), g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
+    float4 x;
+    x.x = (v.x * inv) * __bfloat162float(g01.x); x.y = (v.y * inv) * __bfloat162float(g01.y);
+    x.z = (v.z * inv) * __bfloat162float(g23.x); x.w = (v.w * inv) * __bfloat162float(g23.y);
+    __nv_bfloat16 hi[4], lo[4];
+    split_bf16(x.x, hi[0], lo[0]); split_bf16(x.y, hi[1], lo[1]);
+    split_bf16(x.z, hi[2], lo[2]); split_bf16(x.w, hi[3], lo[3]);
+    uint2 ph, pl;
+    ph.x = (uint32_t)__bfloat16_as_ushort(hi[0]) | ((uint32_t)__bfloat16_as_ushort(hi[1]) << 16);
+    ph.y = (uint32_t)__bfloat16_as_ushort(hi[2]) | ((uint32_t)__bfloat16_as_ushort(hi[3]) << 16);
+    pl.x = (uint32_t)__bfloat16_as_ushort(lo[0]) | ((uint32_t)__bfloat16_as_ushort(lo[1]) << 16);
+    pl.y = (uint32_t)__bfloat16_as_ushort(lo[2]) | ((uint32_t)__bfloat16_as_ushort(lo[3]) << 16);
+    oh[i] = ph;
+    ol[i] = pl;
     if (fr) fr[i] = x;
   }
 }
@@ -470,20 +495,39 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
   const int d = H * hd, half = hd >> 1;
   const int pos = pass->row_pos[t], b = pass->row_seq[t];
   const int page = page_table[b * pages_per_seq + pos / page_size], slot = pos % page_size;
-  const float *q = qkv + (size_t)t * 3 * d, *k = q + d, *v = k + d;
-  for (int idx = threadIdx.x; idx < H * half; idx += blockDim.x) {
-    const int hh = idx / half, i = idx - hh * half;
-    const float2 cs = rope[(size_t)pos * half + i];
-    const int o = hh * hd + i;
-    const float qa = q[o], qb = q[o + half], ka = k[o], kb = k[o + half];
-    qout[(size_t)t * d + o] = (qa * cs.x - qb * cs.y) * qscale;
-    qout[(size_t)t * d + o + half] = (qb * cs.x + qa * cs.y) * qscale;
-    const size_t base = (((size_t)page * L + layer) * H + hh) * page_size * hd + (size_t)slot * hd;
-    const int sw = kswz ? (slot & 7) : 0;
-    kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(ka * cs.x - kb * cs.y);
-    kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(kb * cs.x + ka * cs.y);
-    vpool[base + i] = kv_store(v[o]);
-    vpool[base + i + half] = kv_store(v[o + half]);
+  const float *__restrict__ q = qkv + (size_t)t * 3 * d;
+  const float *__restrict__ k = q + d, *__restrict__ v = k + d;
+  const int sw = kswz ? (slot & 7) : 0;
+  for (int idx0 = threadIdx.x; idx0 < H * half; idx0 += 4 * blockDim.x) {
+    // the loads of four steps first, so that they are in flight together
+    float qa[4], qb[4], ka[4], kb[4], va[4], vb[4];
+    float2 cs[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = idx0 + u * blockDim.x;
+      qa[u] = qb[u] = ka[u] = kb[u] = va[u] = vb[u] = 0.f;
+      cs[u] = make_float2(1.f, 0.f);
+      if (idx < H * half) {
+        const int hh = idx / half, i = idx - hh * half;
+        const int o = hh * hd + i;
+        cs[u] = rope[(size_t)pos * half + i];
+        qa[u] = q[o]; qb[u] = q[o + half]; ka[u] = k[o]; kb[u] = k[o + half]; va[u] = v[o]; vb[u] = v[o + half];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = idx0 + u * blockDim.x;
+      if (idx >= H * half) continue;
+      const int hh = idx / half, i = idx - hh * half;
+      const int o = hh * hd + i;
+      qout[(size_t)t * d + o] = (qa[u] * cs[u].x - qb[u] * cs[u].y) * qscale;
+      qout[(size_t)t * d + o + half] = (qb[u] * cs[u].x + qa[u] * cs[u].y) * qscale;
+      const size_t base = (((size_t)page * L + layer) * H + hh) * page_size * hd + (size_t)slot * hd;
+      kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(ka[u] * cs[u].x - kb[u] * cs[u].y);
+      kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(kb[u] * cs[u].x + ka[u] * cs[u].y);
+      vpool[base + i] = kv_store(va[u]);
+      vpool[base + i + half] = kv_store(vb[u]);
+    }
   }
 }
 
@@ -535,18 +579,21 @@ __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const fl
       for (int c = 0; c < VPL; ++c) o[r][c] = 0.f;
     }
     for (int kb = kbeg + warp * 32; kb < kend; kb += 128) {
+      if (kb > pos0 + rg + nr - 1) break;   // no row of this group sees the block (nor any later one)
       const int key = kb + lane;
       const bool kv = key < kend;
       float s[kRowGroup];
 #pragma unroll
       for (int r = 0; r < kRowGroup; ++r) s[r] = 0.f;
+      // a block of 32 keys starts at a multiple of 32 and lies in one cache page: one lookup per block
+      const int blk_page = page_table[b * pages_per_seq + kb / page_size];
+      const size_t blk_off = (((size_t)blk_page * L + layer) * H + hh) * page_size * HD + (size_t)(kb % page_size) * HD;
       if (kv) {
-        const int page = page_table[b * pages_per_seq + key / page_size], slot = key % page_size;
-        const uint4 *kr = reinterpret_cast<const uint4 *>(
-            kpool + (((size_t)page * L + layer) * H + hh) * page_size * HD + (size_t)slot * HD);
+        const int slot = key % page_size;
+        const uint4 *__restrict__ kr = reinterpret_cast<const uint4 *>(kpool + blk_off + (size_t)lane * HD);
         const int ksw = kswz ? (slot & 7) : 0;   // chunk-swizzled key rows (see k_rope_kv)
-#pragma unroll 4
-        for (int c = 0; c < HD / 8; ++c) {
+#pragma unroll 8
+        for (int c = 0; c < HD / 8; ++c) {   // (eight 16-byte pieces of the key row in flight)
           const uint4 kk = kr[c ^ ksw];
           float kf[8];
           kf[0] = kv_lo(kk.x); kf[1] = kv_hi(kk.x);
@@ -586,25 +633,31 @@ __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const fl
       }
       __syncwarp();
       const int nk = min(32, kend - kb);
-      for (int kk = 0; kk < nk; ++kk) {
-        const int key2 = kb + kk;
-        const int page = page_table[b * pages_per_seq + key2 / page_size], slot = key2 % page_size;
-        const __nv_bfloat16 *vr = vpool + (((size_t)page * L + layer) * H + hh) * page_size * HD + (size_t)slot * HD;
-        float vf[VPL];
-        if (VPL == 4) {
-          const uint2 vv = *reinterpret_cast<const uint2 *>(vr + lane * 4);
-          vf[0] = kv_lo(vv.x); vf[1] = kv_hi(vv.x);
-          vf[VPL - 2] = kv_lo(vv.y); vf[VPL - 1] = kv_hi(vv.y);
-        } else {
-          const uint32_t vv = *reinterpret_cast<const uint32_t *>(vr + lane * 2);
-          vf[0] = kv_lo(vv); vf[VPL - 1] = kv_hi(vv);
+      const __nv_bfloat16 *__restrict__ vblk = vpool + blk_off;   // the block's value rows are contiguous
+      for (int kk0 = 0; kk0 < nk; kk0 += 8) {   // eight value rows loaded together, then used in key order
+        uint2 vv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          vv[u] = make_uint2(0u, 0u);
+          if (kk0 + u < nk) {
+            if (VPL == 4) vv[u] = *reinterpret_cast<const uint2 *>(vblk + (size_t)(kk0 + u) * HD + lane * 4);
+            else vv[u].x = *reinterpret_cast<const uint32_t *>(vblk + (size_t)(kk0 + u) * HD + lane * 2);
+          }
         }
 #pragma unroll
-        for (int r = 0; r < kRowGroup; ++r) {
-          if (r < nr) {
-            const float p = p_s[warp][r][kk];
+        for (int u = 0; u < 8; ++u) {
+          if (kk0 + u < nk) {
+            float vf[VPL];
+            vf[0] = kv_lo(vv[u].x); vf[1] = kv_hi(vv[u].x);
+            if (VPL == 4) { vf[VPL - 2] = kv_lo(vv[u].y); vf[VPL - 1] = kv_hi(vv[u].y); }
 #pragma unroll
-            for (int c = 0; c < VPL; ++c) o[r][c] += p * vf[c];
+            for (int r = 0; r < kRowGroup; ++r) {
+              if (r < nr) {
+                const float p = p_s[warp][r][kk0 + u];
+#pragma unroll
+                for (int c = 0; c < VPL; ++c) o[r][c] += p * vf[c];
+              }
+            }
           }
         }
       }
@@ -681,13 +734,19 @@ __global__ void k_eagle_input(const Pass *pass, const __nv_bfloat16 *embed, cons
   const __nv_bfloat16 *e = embed + (size_t)pass->row_tok[t] * d;
   const float *f = step == 0 ? feat + ((size_t)b * cap + pass->row_pos[t]) * d
                              : dfeat + ((size_t)b * nmax + (step - 1)) * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    xhi[(size_t)t * ldx + i] = e[i];
-    xlo[(size_t)t * ldx + i] = __float2bfloat16_rn(0.f);
+  __nv_bfloat16 *__restrict__ oh = xhi + (size_t)t * ldx, *__restrict__ ol = xlo + (size_t)t * ldx;
+  const __nv_bfloat16 *__restrict__ er = e;
+  const float *__restrict__ fr = f;
+#pragma unroll 8
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {   // (loads of eight steps in flight together)
+    const __nv_bfloat16 ev = er[i];
+    const float fv = fr[i];
+    oh[i] = ev;
+    ol[i] = __float2bfloat16_rn(0.f);
     __nv_bfloat16 hi, lo;
-    split_bf16(f[i], hi, lo);
-    xhi[(size_t)t * ldx + d + i] = hi;
-    xlo[(size_t)t * ldx + d + i] = lo;
+    split_bf16(fv, hi, lo);
+    oh[d + i] = hi;
+    ol[d + i] = lo;
   }
 }
 
