@@ -140,6 +140,41 @@ def aggregate(dist, local_ms: float, local_units: float, device=None):
     return float(t.item()), float(u.item())
 
 
+# ----------------------------------------------------------------------------- ragged batch of 8 (context)
+
+def batch8_sample(weights, dev, iters: int = 30):
+    """The 7B shape with 8 sequences of ragged prompt lengths (uniform in [128, 2048]) and per-sequence draft
+    lengths: device time of `iters` iterations through the multi-row path.  Reported beside the batch-1 metric,
+    not part of it."""
+    import torch
+    import synth_inputs as si
+    from paper_2412_18910_b200 import Engine
+    sh8 = si.SHAPES["7b_b8"]
+    eng = Engine(sh8, weights, max_batch=sh8.batch, kv_capacity=sh8.kv_capacity, device=str(dev))
+    prompts = si.make_prompts(sh8)
+    for b, pr in enumerate(prompts):
+        eng.ada_prefill(b, torch.from_numpy(pr).to(dev), None)
+    for _ in range(5):
+        eng.ada_step()
+    c0 = eng.ada_get_counters()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    e0.record(eng.stream)
+    for _ in range(iters):
+        eng.ada_step()
+    e1.record(eng.stream)
+    torch.cuda.synchronize(dev)
+    c1 = eng.ada_get_counters()
+    ms = e0.elapsed_time(e1)
+    out = {"workload": "7b shape, 8 sequences, prompts %s, predictor-chosen draft lengths" % [len(p) for p in prompts],
+           "iterations": iters, "ms_per_iteration": ms / iters,
+           "tokens_per_s": (c1["n_tokens"] - c0["n_tokens"]) / (ms * 1e-3),
+           "mean_draft_len": (c1["n_draft"] - c0["n_draft"]) / max(1, c1["n_target"] - c0["n_target"]),
+           "status": c1["status"]}
+    eng.close()
+    return out
+
+
 # ----------------------------------------------------------------------------- the CPU oracle arm
 
 def oracle_sample(sh, weights, prompt, iters: int, warm: int, prefill_tokens: int = 32):
@@ -169,6 +204,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=["tiny", "7b", "13b"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-batch8", action="store_true", help="skip the ragged batch-of-8 sample (7b workload only)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (a reduced case for profiler captures)")
     ap.add_argument("--profile-only", action="store_true", help="prefill, a few verify passes, exit (for ncu)")
     args = ap.parse_args()
@@ -345,6 +381,26 @@ def main():
         torch.cuda.synchronize(dev)
         ms_n = va.elapsed_time(vb) / 4
         by_n.append({"n": n_f, "rows": n_f + 1, "ms": round(ms_n, 4), "gbs": round(vbytes / (ms_n * 1e-3) / 1e9, 1)})
+    # verify latency as a function of the context length (cache bytes grow with it): 9 rows after prompts of
+    # 1024, 2048 and 4000 tokens
+    by_ctx = []
+    for ctx in (1024, 2048, 4000):
+        if ctx + sh.n_max + 2 > sh.kv_capacity:
+            continue
+        d_long = torch.from_numpy(si.uniform_ids(si.DEFAULT_SEED + rank, "ctx%d" % ctx, ctx, sh.vocab)).to(dev)
+        eng.ada_prefill(0, d_long, None)
+        eng.d_n.fill_(min(8, sh.n_max))
+        eng.ada_draft(eng.d_n, eng.d_draft)
+        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+        va.record(eng.stream)
+        for _ in range(4):
+            eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+        vb.record(eng.stream)
+        torch.cuda.synchronize(dev)
+        ms_c = va.elapsed_time(vb) / 4
+        cb = verify_weight_bytes(sh) + (ctx + 1) * kv_bytes_per_token(sh)
+        by_ctx.append({"ctx": ctx + 1, "rows": min(8, sh.n_max) + 1, "ms": round(ms_c, 4), "bytes": cb,
+                       "gbs": round(cb / (ms_c * 1e-3) / 1e9, 1), "frac_of_measured": round(cb / (ms_c * 1e-3) / 1e9 / peak, 4)})
     # the dominant kernel: the persistent pass kernel, one launch per verify pass (weights + KV read once)
     launch_ms = prof["gemm_ms"] / max(1, prof["gemm_launches"])
     pass_gbs = vbytes / (launch_ms * 1e-3) / 1e9 if launch_ms > 0 else None
@@ -361,7 +417,7 @@ def main():
                                 "gbs": vbytes / (verify_ms * 1e-3) / 1e9,
                                 "frac_of_measured": vbytes / (verify_ms * 1e-3) / 1e9 / peak,
                                 "frac_of_8000": vbytes / (verify_ms * 1e-3) / 1e9 / 8000.0},
-                "verify_by_n": by_n}
+                "verify_by_n": by_n, "verify_by_ctx": by_ctx}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
             "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -373,6 +429,8 @@ def main():
         tps, ms, threads, desc = oracle_sample(sh, weights, prompt, 10 if sh.name != "tiny" else 64, 1)
         line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
     eng.close()
+    if rank == 0 and world == 1 and sh.name == "7b" and not args.layers and not args.no_batch8:
+        line["batch8"] = batch8_sample(weights, dev)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

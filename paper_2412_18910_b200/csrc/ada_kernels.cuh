@@ -566,9 +566,20 @@ __global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const fl
   for (int rg = rgi * kRowGroup; rg < R; rg += nrg * kRowGroup) {
     const int nr = min(kRowGroup, R - rg);
     __syncthreads();
-    for (int i = threadIdx.x; i < nr * HD; i += 128) {
-      const int r = i / HD, c = i - r * HD;
-      q_s[r][c] = q[(size_t)(row0 + rg + r) * d + hh * HD + c];
+    {   // the group's query rows, 16 bytes per load, all of a thread's loads in flight together
+      constexpr int PER = kRowGroup * HD / 4 / 128;
+      float4 qv[PER];
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        const int i = threadIdx.x + u * 128, r = i / (HD / 4), c4 = i - r * (HD / 4);
+        qv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nr) qv[u] = *reinterpret_cast<const float4 *>(q + (size_t)(row0 + rg + r) * d + hh * HD + 4 * c4);
+      }
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        const int i = threadIdx.x + u * 128, r = i / (HD / 4), c4 = i - r * (HD / 4);
+        *reinterpret_cast<float4 *>(&q_s[r][4 * c4]) = qv[u];
+      }
     }
     __syncthreads();
     float m[kRowGroup], l[kRowGroup], o[kRowGroup][VPL];
