@@ -9,7 +9,7 @@ _ROOT = os.path.dirname(_HERE)
 LIB = os.path.join(_HERE, "libada.so")
 SOURCES = [os.path.join(_HERE, "csrc", "ada.cu"), os.path.join(_HERE, "csrc", "ada_static.cu")]
 DEPS = SOURCES + [os.path.join(_HERE, "csrc", "ada_kernels.cuh"), os.path.join(_HERE, "csrc", "ada_pass.cuh"),
-                  os.path.join(_HERE, "csrc", "ada_ring.h"), os.path.join(_HERE, "csrc", "ada_gemm_tc.cuh"), os.path.join(_ROOT, "include", "ada.h")]
+                  os.path.join(_HERE, "csrc", "ada_ring.h"), os.path.join(_HERE, "csrc", "ada_gemm_tc.cuh"), os.path.join(_HERE, "csrc", "ada_attn_rows.cuh"), os.path.join(_ROOT, "include", "ada.h")]
 
 
 def stale() -> bool:

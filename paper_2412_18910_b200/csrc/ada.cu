@@ -15,6 +15,7 @@
 #include "ada_kernels.cuh"
 #include "ada_pass.cuh"
 #include "ada_gemm_tc.cuh"
+#include "ada_attn_rows.cuh"
 
 #include <unordered_map>
 
@@ -367,11 +368,11 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   dim3 g2(c.n_heads, x->TM);
   timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
-    LAUNCH(x, k_attn_partial<128>, g1, 128, attn_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+    LAUNCH(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
     LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   } else {
-    LAUNCH(x, k_attn_partial<64>, g1, 128, attn_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+    LAUNCH(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
     LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   }
@@ -766,9 +767,9 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   const int gemm_smem = 2 * x->NT * 8 * ((x->NT == 2 ? 1024 : 256) * 2 + 64);
   if (e == cudaSuccess && x->NT == 2) e = gemm_attr_nt<2>(gemm_smem);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_attn_partial<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<128>());
+    e = cudaFuncSetAttribute(k_attn_rows<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<128>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_attn_partial<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<64>());
+    e = cudaFuncSetAttribute(k_attn_rows<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<64>());
   if (e != cudaSuccess) {
     delete x;
     return ADA_ERR_CUDA;
