@@ -19,9 +19,7 @@ namespace ada {
 constexpr int kMaxBatch = 8;
 constexpr int kMaxRows = 128;   // rows of one pass (all sequences together)
 constexpr int kAttnSplits = 8;  // KV splits per (sequence, head)
-constexpr int kRowGroup = 16;   // query rows an attention warp keeps in registers
-template <int HD>
-constexpr int attn_smem_bytes() { return (kRowGroup * HD + 4 * kRowGroup * 32 + 8 * kRowGroup + 4 * kRowGroup * HD) * 4; }
+constexpr int kRowGroup = 16;   // query rows of one attention CTA (one m16 tile)
 
 // status bits (device status word)
 constexpr int kStatKvFull = 1;
@@ -527,178 +525,6 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
       kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(kb[u] * cs[u].x + ka[u] * cs[u].y);
       vpool[base + i] = kv_store(va[u]);
       vpool[base + i + half] = kv_store(vb[u]);
-    }
-  }
-}
-
-// Attention of the rows of one sequence for one head over one split of the cache.
-// Row r (absolute position pos0 + r) sees cache positions 0..pos0+r: the whole history and the
-// earlier rows of its own block.  Lane = key in the score phase, lane = 4 channels in the
-// value phase.  Partial (m, l, o[hd]) per (head, split, row) goes to `part`.
-// HD must be 64 or 128.
-template <int HD>
-__global__ void __launch_bounds__(128) k_attn_partial(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
-                                                      const __nv_bfloat16 *vpool, const int *page_table,
-                                                      int pages_per_seq, int page_size, int L, int layer, int H,
-                                                      float *part, int kswz, int nrg) {
-  constexpr int VPL = HD / 32;  // value channels per lane
-  // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
-  const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / nrg, rgi = blockIdx.z - b * nrg;
-  const int R = pass->seq_rows[b];
-  if (pass->T <= 0 || R <= 0) return;
-  const int row0 = pass->seq_row0[b];
-  const int pos0 = pass->row_pos[row0];
-  const int nkeys = pos0 + R;
-  int chunk = (nkeys + kAttnSplits - 1) / kAttnSplits;
-  chunk = ((chunk + 31) / 32) * 32;
-  const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int d = H * HD;
-
-  extern __shared__ __align__(16) float attn_smem[];
-  float (*q_s)[HD] = reinterpret_cast<float (*)[HD]>(attn_smem);
-  float (*p_s)[kRowGroup][32] = reinterpret_cast<float (*)[kRowGroup][32]>(attn_smem + kRowGroup * HD);
-  float (*m_s)[kRowGroup] = reinterpret_cast<float (*)[kRowGroup]>(attn_smem + kRowGroup * HD + 4 * kRowGroup * 32);
-  float (*l_s)[kRowGroup] = m_s + 4;
-  float (*o_s)[kRowGroup][HD] =
-      reinterpret_cast<float (*)[kRowGroup][HD]>(attn_smem + kRowGroup * HD + 4 * kRowGroup * 32 + 8 * kRowGroup);
-
-  for (int rg = rgi * kRowGroup; rg < R; rg += nrg * kRowGroup) {
-    const int nr = min(kRowGroup, R - rg);
-    __syncthreads();
-    {   // the group's query rows, 16 bytes per load, all of a thread's loads in flight together
-      constexpr int PER = kRowGroup * HD / 4 / 128;
-      float4 qv[PER];
-#pragma unroll
-      for (int u = 0; u < PER; ++u) {
-        const int i = threadIdx.x + u * 128, r = i / (HD / 4), c4 = i - r * (HD / 4);
-        qv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r < nr) qv[u] = *reinterpret_cast<const float4 *>(q + (size_t)(row0 + rg + r) * d + hh * HD + 4 * c4);
-      }
-#pragma unroll
-      for (int u = 0; u < PER; ++u) {
-        const int i = threadIdx.x + u * 128, r = i / (HD / 4), c4 = i - r * (HD / 4);
-        *reinterpret_cast<float4 *>(&q_s[r][4 * c4]) = qv[u];
-      }
-    }
-    __syncthreads();
-    float m[kRowGroup], l[kRowGroup], o[kRowGroup][VPL];
-#pragma unroll
-    for (int r = 0; r < kRowGroup; ++r) {
-      m[r] = -INFINITY; l[r] = 0.f;
-#pragma unroll
-      for (int c = 0; c < VPL; ++c) o[r][c] = 0.f;
-    }
-    for (int kb = kbeg + warp * 32; kb < kend; kb += 128) {
-      if (kb > pos0 + rg + nr - 1) break;   // no row of this group sees the block (nor any later one)
-      const int key = kb + lane;
-      const bool kv = key < kend;
-      float s[kRowGroup];
-#pragma unroll
-      for (int r = 0; r < kRowGroup; ++r) s[r] = 0.f;
-      // a block of 32 keys starts at a multiple of 32 and lies in one cache page: one lookup per block
-      const int blk_page = page_table[b * pages_per_seq + kb / page_size];
-      const size_t blk_off = (((size_t)blk_page * L + layer) * H + hh) * page_size * HD + (size_t)(kb % page_size) * HD;
-      if (kv) {
-        const int slot = key % page_size;
-        const uint4 *__restrict__ kr = reinterpret_cast<const uint4 *>(kpool + blk_off + (size_t)lane * HD);
-        const int ksw = kswz ? (slot & 7) : 0;   // chunk-swizzled key rows (see k_rope_kv)
-#pragma unroll 8
-        for (int c = 0; c < HD / 8; ++c) {   // (eight 16-byte pieces of the key row in flight)
-          const uint4 kk = kr[c ^ ksw];
-          float kf[8];
-          kf[0] = kv_lo(kk.x); kf[1] = kv_hi(kk.x);
-          kf[2] = kv_lo(kk.y); kf[3] = kv_hi(kk.y);
-          kf[4] = kv_lo(kk.z); kf[5] = kv_hi(kk.z);
-          kf[6] = kv_lo(kk.w); kf[7] = kv_hi(kk.w);
-#pragma unroll
-          for (int r = 0; r < kRowGroup; ++r) {
-            if (r < nr) {
-              const float4 qa = *reinterpret_cast<const float4 *>(&q_s[r][c * 8]);
-              const float4 qb = *reinterpret_cast<const float4 *>(&q_s[r][c * 8 + 4]);
-              s[r] += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
-                      qb.z * kf[6] + qb.w * kf[7];
-            }
-          }
-        }
-      }
-      // online softmax per row over this block of 32 keys
-#pragma unroll
-      for (int r = 0; r < kRowGroup; ++r) {
-        if (r < nr) {
-          const bool seen = kv && key <= pos0 + rg + r;
-          const float sv = seen ? s[r] : -INFINITY;
-          const float mx = warp_max(sv);
-          const float mn = fmaxf(m[r], mx);
-          float p = 0.f, corr = 1.f;
-          if (mn > -INFINITY) {
-            p = seen ? __expf(sv - mn) : 0.f;
-            corr = __expf(m[r] - mn);  // m = -inf gives 0
-          }
-          l[r] = l[r] * corr + warp_sum(p);
-#pragma unroll
-          for (int c = 0; c < VPL; ++c) o[r][c] *= corr;
-          m[r] = mn;
-          p_s[warp][r][lane] = p;
-        }
-      }
-      __syncwarp();
-      const int nk = min(32, kend - kb);
-      const __nv_bfloat16 *__restrict__ vblk = vpool + blk_off;   // the block's value rows are contiguous
-      for (int kk0 = 0; kk0 < nk; kk0 += 8) {   // eight value rows loaded together, then used in key order
-        uint2 vv[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          vv[u] = make_uint2(0u, 0u);
-          if (kk0 + u < nk) {
-            if (VPL == 4) vv[u] = *reinterpret_cast<const uint2 *>(vblk + (size_t)(kk0 + u) * HD + lane * 4);
-            else vv[u].x = *reinterpret_cast<const uint32_t *>(vblk + (size_t)(kk0 + u) * HD + lane * 2);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (kk0 + u < nk) {
-            float vf[VPL];
-            vf[0] = kv_lo(vv[u].x); vf[1] = kv_hi(vv[u].x);
-            if (VPL == 4) { vf[VPL - 2] = kv_lo(vv[u].y); vf[VPL - 1] = kv_hi(vv[u].y); }
-#pragma unroll
-            for (int r = 0; r < kRowGroup; ++r) {
-              if (r < nr) {
-                const float p = p_s[warp][r][kk0 + u];
-#pragma unroll
-                for (int c = 0; c < VPL; ++c) o[r][c] += p * vf[c];
-              }
-            }
-          }
-        }
-      }
-      __syncwarp();
-    }
-    // combine the 4 warps in warp order
-#pragma unroll
-    for (int r = 0; r < kRowGroup; ++r) {
-      if (r < nr) {
-        if (lane == 0) { m_s[warp][r] = m[r]; l_s[warp][r] = l[r]; }
-#pragma unroll
-        for (int c = 0; c < VPL; ++c) o_s[warp][r][lane * VPL + c] = o[r][c];
-      }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < nr * HD; i += 128) {
-      const int r = i / HD, c = i - r * HD;
-      float M = m_s[0][r];
-      for (int w = 1; w < 4; ++w) M = fmaxf(M, m_s[w][r]);
-      float lo = 0.f, oo = 0.f;
-      if (M > -INFINITY) {
-        for (int w = 0; w < 4; ++w) {
-          const float e = __expf(m_s[w][r] - M);
-          lo += l_s[w][r] * e;
-          oo += o_s[w][r][c] * e;
-        }
-      }
-      float *pp = part + (((size_t)hh * kAttnSplits + split) * kMaxRows + (row0 + rg + r)) * (HD + 2);
-      pp[c] = oo;
-      if (c == 0) { pp[HD] = M; pp[HD + 1] = lo; }
     }
   }
 }
