@@ -319,10 +319,18 @@ void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
     GemmTcArgs t;
     memset(&t, 0, sizeof(t));
     const bf16 *Ws[3] = {W0, W1, W2};
+    auto map_of = [&](const void *base) -> const TensorMap128 * {
+      auto it = x->tcmap_of.find(base);
+      return it == x->tcmap_of.end() ? nullptr : x->d_tcmaps + it->second;
+    };
     for (int i = 0; i < 3; ++i)
-      if (Ws[i]) t.wmap[i] = x->d_tcmaps + x->tcmap_of.at(Ws[i]);
-    t.xhi_map = x->d_tcmaps + x->tcmap_of.at(Xhi);
-    t.xlo_map = x->d_tcmaps + x->tcmap_of.at(Xlo);
+      if (Ws[i]) t.wmap[i] = map_of(Ws[i]);
+    t.xhi_map = map_of(Xhi);
+    t.xlo_map = map_of(Xlo);
+    if (!t.wmap[0] || (W1 && !t.wmap[1]) || (W2 && !t.wmap[2]) || !t.xhi_map || !t.xlo_map) {
+      x->err = "gemm: operand without a tensor map";   // (every operand of the path is registered at initialisation)
+      return;
+    }
     t.epi = epi; t.nseg = nseg; t.Nseg = Nseg; t.K = K;
     const int tiles = tc_tiles(epi, nseg, Nseg);
     t.S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tiles, K);
