@@ -146,6 +146,8 @@ bool config_ok(const ada_config *c) {
   if (c->ldlp_mode == 1 && (c->ldlp_blocks < 0 || c->ldlp_blocks > 8 || c->k_min < 1 || c->k_min > c->n_max)) return false;
   if (c->max_batch < 1 || c->max_batch > ADA_MAX_BATCH) return false;
   if (c->max_batch * (c->n_max + 1) > 88) return false;
+  // passes of more than 16 rows run the tensor-core GEMM, whose weight boxes are 128 rows high
+  if (c->max_batch * (c->n_max + 1) > 16 && (c->d_model < 128 || c->d_ffn < 128 || c->vocab < 128)) return false;
   if (c->page_size != 64 || c->kv_capacity < 64 || c->kv_capacity % c->page_size) return false;
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
   return true;
