@@ -73,7 +73,7 @@ def _load():
     L.orc_step.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, f32p, f32p, f32p]
     L.orc_draft_dyn.argtypes = [vp, vp, C.c_int, i32p, i32p, f32p, f32p, f32p, i32p]
     L.orc_label.argtypes = [vp, vp]
-    L.orc_force_commit.argtypes = [vp, vp, C.c_int, i32p, C.c_int]
+    L.orc_rewind.argtypes = [vp, C.c_int, C.c_int]
     L.orc_forward_nocache.argtypes = [vp, i32p, C.c_int, f32p, f32p]
     L.orc_draft_rows.argtypes = [vp, i32p, f32p, C.c_int, C.c_int, f32p, f32p, f32p]
     L.orc_seq_len.argtypes = [vp]
@@ -290,10 +290,11 @@ class Seq:
         assert k >= 0, "label failed rc=%d" % k
         return k
 
-    def force_commit(self, j_start: int, tokens) -> None:
-        t = np.ascontiguousarray(tokens, dtype=np.int32)
-        rc = self.lib.orc_force_commit(self.m.h, self.h, j_start, t.ctypes.data, len(t))
-        assert rc == 0
+    def rewind(self, length: int, dlen: int) -> None:
+        """Back to an earlier state of this sequence: `length` committed tokens (the last one pending), `dlen`
+        draft-head rows of true features; counters restart."""
+        rc = self.lib.orc_rewind(self.h, length, dlen)
+        assert rc == 0, "rewind out of range"
 
 
 def decode(model: Model, prompt, max_new: int, n_policy=-1, capacity=None, forced_stream=None) -> dict:

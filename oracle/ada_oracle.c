@@ -571,18 +571,16 @@ int orc_label(const orc_model *m, orc_seq *s) {
   return k;
 }
 
-/* Replace the outcome of the iteration that just ran: rewind to its start
- * (pending index j_start), and commit `count` given tokens instead (count-1
- * accepted drafts and a bonus), recomputing cache rows and features for them. */
-int orc_force_commit(const orc_model *m, orc_seq *s, int j_start, const int32_t *tokens, int count) {
-  int32_t target[65];
-  if (count < 1 || j_start + count + 1 > s->cap) return -1;
-  const int n_emitted_before = s->len - 1 - j_start;
-  s->n_tokens += count - n_emitted_before;
-  s->len = j_start + 1;
-  if (orc_verify(m, s, tokens, count - 1, target, NULL, NULL, NULL)) return -2;
-  for (int i = 0; i < count; ++i) s->tok[j_start + 1 + i] = tokens[i];
-  s->len = j_start + count + 1;
+/* Roll a sequence back to an earlier state of itself: the first `len` committed tokens stay (the last of them
+ * pending again) and the draft head keeps its first `dlen` true-feature rows.  Cache rows, features and tokens past
+ * those lengths are left in place as garbage; every later pass overwrites the rows it reads (dlen <= len - 2: the
+ * row of position len - 2 yields the first draft token, so the next draft computes it).  Counters restart at
+ * zero.  Used to run several continuations from one prefilled prompt. */
+int orc_rewind(orc_seq *s, int len, int dlen) {
+  if (len < 1 || len > s->len || dlen < 0 || dlen > s->dlen || dlen > len - 2) return -1;
+  s->len = len;
+  s->dlen = dlen;
+  s->n_target = s->n_draft = s->n_waste = s->n_tokens = 0;
   return 0;
 }
 

@@ -144,6 +144,57 @@ def test_state_after_accept_equals_fresh_prefill(tiny):
         assert np.array_equal(x["v_top1"], y["v_top1"])
 
 
+def test_rewound_sequence_continues_like_a_fresh_prefill(tiny):
+    """orc_rewind: a sequence rolled back to its prefilled state (with or without the draft head's prompt rows)
+    repeats, bit for bit, what a freshly prefilled sequence does; counters restart."""
+    sh, w, prompt, m = tiny
+    fresh = m.new_seq(256)
+    fresh.prefill(prompt)
+    a = [fresh.step(n) for n in (-1, 3, 8, -1)]
+    for keep_draft_rows in (True, False):
+        seq = m.new_seq(256)
+        seq.prefill(prompt)
+        for n in (5, -1, 2):
+            seq.step(n)
+        seq.rewind(len(prompt) + 1, len(prompt) - 1 if keep_draft_rows else 0)
+        assert seq.len == len(prompt) + 1 and seq.counters()["n_target"] == 0
+        b = [seq.step(n) for n in (-1, 3, 8, -1)]
+        for x, y in zip(a, b):
+            assert x["n"] == y["n"] and x["k"] == y["k"]
+            assert np.array_equal(x["emitted"], y["emitted"]) and np.array_equal(x["draft"], y["draft"])
+            assert np.array_equal(x["v_top1"], y["v_top1"]) and np.array_equal(x["d_top1"], y["d_top1"])
+        assert seq.counters() == fresh.counters()
+    with pytest.raises(AssertionError):
+        seq.rewind(seq.len + 1, 0)
+
+
+def test_golden_writer_step_equals_the_oracle_step(tiny):
+    """tests/golden/make_goldens.py keeps complete logit rows by composing predict, draft, verify and accept
+    itself: that composition must be the iteration Seq.step runs, and its logits must carry the stored top-2."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_goldens", os.path.join(GOLDEN, "make_goldens.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    sh, w, prompt, m = tiny
+    a, b = m.new_seq(256), m.new_seq(256)
+    assert a.prefill(prompt) == b.prefill(prompt)
+    ar = oracle.decode(m, prompt, 40, n_policy=0)["tokens"]
+    for n, teacher in ((-1, False), (0, False), (4, False), (-1, False), (3, True)):
+        forced = np.asarray(ar[a.len - len(prompt): a.len - len(prompt) + sh.n_max], dtype=np.int32) if teacher else None
+        x = a.step(n, forced)
+        y, lg = mg.step_with_logits(b, n, forced)
+        assert x["n"] == y["n"] and x["k"] == y["k"] and x["j"] == y["j"]
+        for key in ("emitted", "draft", "target", "v_top1", "v_top2", "d_top1", "d_top2"):
+            assert np.array_equal(x[key], y[key]), key
+        if n < 0:
+            assert np.array_equal(x["ldlp_z"][: sh.n_max], y["ldlp_z"][: sh.n_max])
+        assert lg.shape == (x["n"] + 1, sh.vocab)
+        assert np.array_equal(lg.argmax(axis=1), x["target"]) and np.array_equal(lg.max(axis=1), x["v_top1"])
+        if teacher:
+            assert x["k"] == 3
+    assert a.counters() == b.counters()
+
+
 # ----------------------------------------------------------------- draft head
 
 def test_draft_head_block_matches_stock_op_restatement(tiny):
