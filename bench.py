@@ -142,10 +142,11 @@ def aggregate(dist, local_ms: float, local_units: float, device=None):
 
 # ----------------------------------------------------------------------------- ragged batch of 8 (context)
 
-def batch8_sample(weights, dev, iters: int = 30):
+def batch8_sample(weights, dev, peak, iters: int = 30):
     """The 7B shape with 8 sequences of ragged prompt lengths (uniform in [128, 2048]) and per-sequence draft
-    lengths: device time of `iters` iterations through the multi-row path.  Reported beside the batch-1 metric,
-    not part of it."""
+    lengths: device time of `iters` iterations through the multi-row path, with the algorithmic bytes of an iteration
+    (verify weights once + the cached positions of all sequences + one draft-head weight pass per draft step that
+    any sequence takes) against the HBM peak.  Reported beside the batch-1 metric, not part of it."""
     import torch
     import synth_inputs as si
     from paper_2412_18910_b200 import Engine
@@ -157,22 +158,119 @@ def batch8_sample(weights, dev, iters: int = 30):
     for _ in range(5):
         eng.ada_step()
     c0 = eng.ada_get_counters()
+    lens = eng.ada_debug_buffer(3, torch.int32, (sh8.batch, 8))
+    # per iteration, on the device and in stream order: cached positions read by the verify pass (len - 1 per sequence)
+    # and the number of draft steps that ran (the longest draft length of the iteration)
+    ctx_acc = torch.zeros(1, dtype=torch.int64, device=dev)
+    steps_acc = torch.zeros(1, dtype=torch.int64, device=dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(dev)
     e0.record(eng.stream)
     for _ in range(iters):
-        eng.ada_step()
+        ctx_acc += (lens[:, 0].to(torch.int64) - 1).sum()
+        eng.ada_step(None, None, eng.d_nused, None)
+        steps_acc += eng.d_nused.max().to(torch.int64)
     e1.record(eng.stream)
     torch.cuda.synchronize(dev)
     c1 = eng.ada_get_counters()
     ms = e0.elapsed_time(e1)
+    kv = int(ctx_acc.item()) * kv_bytes_per_token(sh8)
+    dkv = int(ctx_acc.item()) * 2 * 2 * sh8.d_model          # the draft head's one-layer cache, read by its first step
+    bytes_total = iters * verify_weight_bytes(sh8) + kv + int(steps_acc.item()) * draft_step_bytes(sh8) + dkv
+    gbs = bytes_total / (ms * 1e-3) / 1e9
     out = {"workload": "7b shape, 8 sequences, prompts %s, predictor-chosen draft lengths" % [len(p) for p in prompts],
            "iterations": iters, "ms_per_iteration": ms / iters,
            "tokens_per_s": (c1["n_tokens"] - c0["n_tokens"]) / (ms * 1e-3),
            "mean_draft_len": (c1["n_draft"] - c0["n_draft"]) / max(1, c1["n_target"] - c0["n_target"]),
+           "bytes_per_iteration": bytes_total / iters, "kv_bytes_per_iteration": kv / iters,
+           "draft_steps_per_iteration": int(steps_acc.item()) / iters, "gbs": gbs, "frac_of_measured": gbs / peak,
            "status": c1["status"]}
     eng.close()
     return out
+
+
+# ----------------------------------------------------------------------------- teacher-forced sweep (context)
+
+def teacher_forced_sweep(weights, dev, peak, iters: int = 64, verify_samples: int = 16):
+    """The 7B shape after a 1024-token prompt with drafts forced to the model's own greedy continuation, so that every
+    draft is accepted (tau = n + 1), for each forced draft length n = 1..n_max, every sweep from the same prefilled
+    state: `iters` whole iterations (ada_step) timed on the device, then `verify_samples` iterations through the
+    separate calls with events around the verify launch (latency and bytes per second against n)."""
+    import torch
+    import synth_inputs as si
+    from paper_2412_18910_b200 import Engine
+    sh = si.SHAPES["7b_tf"]
+    eng = Engine(sh, weights, max_batch=1, kv_capacity=sh.kv_capacity, device=str(dev))
+    d_prompt = torch.from_numpy(si.make_prompts(sh)[0]).to(dev)
+    nmax = sh.n_max
+    need = iters * (nmax + 1) + nmax + 2
+    # the greedy continuation, by plain autoregressive steps of the library itself (bit-identical to what it accepts)
+    eng.ada_prefill(0, d_prompt, eng.d_first)
+    eng.ada_force_n([0])
+    stream = torch.zeros(need + nmax + 1, dtype=torch.int32, device=dev)
+    stream[0:1] = eng.d_first
+    for i in range(1, need):
+        eng.ada_step(eng.d_emitted, None, None, None)
+        stream[i: i + 1] = eng.d_emitted[0, 0:1]
+    rows = []
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for n in range(1, nmax + 1):
+        eng.ada_prefill(0, d_prompt, None)
+        eng.ada_force_n([n])
+        c0 = eng.ada_get_counters()
+        off = 1
+        for w in range(2):      # warm-up iterations (graph capture for this configuration)
+            eng.ada_force_draft(stream[off: off + nmax].view(1, nmax))
+            eng.ada_step()
+            off += n + 1
+        eng.ada_prefill(0, d_prompt, None)
+        off = 1
+        c0 = eng.ada_get_counters()
+        torch.cuda.synchronize(dev)
+        ea.record(eng.stream)
+        for _ in range(iters):
+            eng.ada_force_draft(stream[off: off + nmax].view(1, nmax))
+            eng.ada_step()
+            off += n + 1
+        eb.record(eng.stream)
+        torch.cuda.synchronize(dev)
+        c1 = eng.ada_get_counters()
+        ms = ea.elapsed_time(eb)
+        tokens = c1["n_tokens"] - c0["n_tokens"]
+        accepted_all = tokens == iters * (n + 1) and (c1["n_waste"] - c0["n_waste"]) == 0
+        # verify launch alone, at the contexts the sweep starts from
+        eng.ada_prefill(0, d_prompt, None)
+        off = 1
+        vms, ctxs = [], []
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(verify_samples)]
+        ctx = len(d_prompt)
+        for i in range(verify_samples):
+            eng.ada_force_draft(stream[off: off + nmax].view(1, nmax))
+            eng.ada_ldlp_predict(eng.d_n)
+            eng.ada_draft(eng.d_n, eng.d_draft)
+            evs[i][0].record(eng.stream)
+            eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+            evs[i][1].record(eng.stream)
+            eng.ada_accept()
+            ctxs.append(ctx + 1)
+            ctx += n + 1
+            off += n + 1
+        torch.cuda.synchronize(dev)
+        vms = sorted(a.elapsed_time(b) for a, b in evs)
+        v_ms = vms[len(vms) // 2]
+        vb = verify_weight_bytes(sh) + (sum(ctxs) / len(ctxs)) * kv_bytes_per_token(sh)
+        rows.append({"n": n, "rows": n + 1, "tau": tokens / iters, "all_accepted": bool(accepted_all),
+                     "ms_per_iteration": round(ms / iters, 4), "tokens_per_s": round(tokens / (ms * 1e-3), 1),
+                     "verify_ms": round(v_ms, 4), "verify_gbs": round(vb / (v_ms * 1e-3) / 1e9, 1),
+                     "verify_frac_of_measured": round(vb / (v_ms * 1e-3) / 1e9 / peak, 4)})
+    status = eng.ada_get_counters()["status"]
+    eng.ada_force_n(None)
+    eng.ada_force_draft(None)
+    eng.close()
+    return {"workload": "7b shape, prompt 1024, drafts teacher-forced to the greedy continuation, draft length forced to n, "
+                        "%d iterations per n from the same prefilled state" % iters,
+            "verify_timing": "median of %d verify launches (CUDA events) at contexts from 1025 on" % verify_samples,
+            "by_n": rows, "status": status}
 
 
 # ----------------------------------------------------------------------------- the CPU oracle arm
@@ -205,6 +303,7 @@ def main():
     ap.add_argument("--workload", default="7b", choices=["tiny", "7b", "13b"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch8", action="store_true", help="skip the ragged batch-of-8 sample (7b workload only)")
+    ap.add_argument("--no-teacher-forced", action="store_true", help="skip the teacher-forced sweep n = 1..n_max (7b workload only)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (a reduced case for profiler captures)")
     ap.add_argument("--profile-only", action="store_true", help="prefill, a few verify passes, exit (for ncu)")
     args = ap.parse_args()
@@ -233,6 +332,7 @@ def main():
         iters = min(K, 12 if sh.name != "tiny" else 256)
         warm = min(W, 2)
         tps, ms, threads, desc = oracle_sample(sh, weights, prompt, iters, warm)
+        config = dict(config, sample="this arm runs a bounded sample of the workload: " + desc)
         line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": iters,
                 "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic", "config": config,
@@ -297,6 +397,8 @@ def main():
         used_in_episode += todo
     c1 = eng.ada_get_counters()
     clocks = sampler.stop()
+    if c1["status"] != 0:     # a device-side error (a wait that gave up, a full cache) invalidates the timing
+        raise RuntimeError("device status word %d after the timed region" % c1["status"])
     tokens = c1["n_tokens"] - c0["n_tokens"]
     launches = c1["launches"] - c0["launches"]
     n_draft = c1["n_draft"] - c0["n_draft"]
@@ -322,10 +424,14 @@ def main():
         torch.cuda.synchronize(dev)
         e_tokens += int(h_out[sh.n_max + 1])
     e2e_ms = (time.perf_counter() - t0) * 1e3
+    status_e2e = eng.ada_get_counters()["status"]
+    if status_e2e != 0:
+        raise RuntimeError("device status word %d after the end-to-end leg" % status_e2e)
     e_ms, e_tok = aggregate(dist, e2e_ms, float(e_tokens), dev)
     e2e = {"value": e_tok / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": prompt.nbytes / Ke,
            "d2h_bytes_per_step": h_out.numel() * 4, "steps": Ke,
-           "note": "request latency: pinned-host prompt copy + prefill + steps with a host read-back each"}
+           "note": "request latency: pinned-host prompt copy + prompt pass + steps with a host read-back each; with few "
+                   "steps the prompt pass (see prefill.ms) is a large share of it"}
 
     # ---- prompt pass (Algorithm 1's first verify, k = 0): device time of ada_prefill on the resident prompt
     pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -368,21 +474,8 @@ def main():
     verify_ms = va.elapsed_time(vb) / reps
     ctx_len = sh.prompt_len + 1
     vbytes = verify_weight_bytes(sh) + ctx_len * kv_bytes_per_token(sh)
-    # verify latency as a function of the number of rows (draft length n forced, same context)
-    by_n = []
-    for n_f in range(1, sh.n_max + 1):
-        eng.d_n.fill_(n_f)
-        eng.ada_draft(eng.d_n, eng.d_draft)
-        eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
-        va.record(eng.stream)
-        for _ in range(4):
-            eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
-        vb.record(eng.stream)
-        torch.cuda.synchronize(dev)
-        ms_n = va.elapsed_time(vb) / 4
-        by_n.append({"n": n_f, "rows": n_f + 1, "ms": round(ms_n, 4), "gbs": round(vbytes / (ms_n * 1e-3) / 1e9, 1)})
     # verify latency as a function of the context length (cache bytes grow with it): 9 rows after prompts of
-    # 1024, 2048 and 4000 tokens
+    # 1024, 2048 and 4000 tokens, median of 9 ada_verify calls each
     by_ctx = []
     for ctx in (1024, 2048, 4000):
         if ctx + sh.n_max + 2 > sh.kv_capacity:
@@ -392,12 +485,13 @@ def main():
         eng.d_n.fill_(min(8, sh.n_max))
         eng.ada_draft(eng.d_n, eng.d_draft)
         eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
-        va.record(eng.stream)
-        for _ in range(4):
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(9)]
+        for a_, b_ in pairs:
+            a_.record(eng.stream)
             eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
-        vb.record(eng.stream)
+            b_.record(eng.stream)
         torch.cuda.synchronize(dev)
-        ms_c = va.elapsed_time(vb) / 4
+        ms_c = statistics.median(a_.elapsed_time(b_) for a_, b_ in pairs)
         cb = verify_weight_bytes(sh) + (ctx + 1) * kv_bytes_per_token(sh)
         by_ctx.append({"ctx": ctx + 1, "rows": min(8, sh.n_max) + 1, "ms": round(ms_c, 4), "bytes": cb,
                        "gbs": round(cb / (ms_c * 1e-3) / 1e9, 1), "frac_of_measured": round(cb / (ms_c * 1e-3) / 1e9 / peak, 4)})
@@ -407,9 +501,10 @@ def main():
     roofline = {"bound": "hbm", "kernel": "k_pass (target verify pass: embedding, all layers, LM head and greedy choice in one persistent launch)",
                 "achieved": pass_gbs, "peak": peak, "unit": "GB/s",
                 "frac": (pass_gbs / peak) if pass_gbs else None, "peak_kind": "of " + peak_kind,
-                # dram bytes of one launch: ncu capture of the 4-layer case of the same shape (1.934 GB for 1.915 GB
-                # algorithmic), scaled by the bytes processed; see profiles/k_pass_7b_4layers_ncu.md
+                # dram bytes of one launch: not counted in this run; the counters of an ncu capture of the 4-layer case
+                # of the same shape, scaled by the bytes processed (traffic grows in proportion to the layers)
                 "traffic": (vbytes * TRAFFIC_PER_ALGORITHMIC_BYTE) if (sh.name == "7b" and TRAFFIC_PER_ALGORITHMIC_BYTE) else None,
+                "traffic_kind": "scaled from an ncu capture of the 4-layer case" if (sh.name == "7b" and TRAFFIC_PER_ALGORITHMIC_BYTE) else None,
                 "launches_timed": prof["gemm_launches"], "avg_launch_us": 1e3 * launch_ms,
                 "bytes_per_launch": vbytes, "frac_of_8000": (pass_gbs / 8000.0) if pass_gbs else None,
                 "verify_pass": {"rows": n_now + 1, "ctx": ctx_len, "ms": verify_ms, "bytes": vbytes,
@@ -417,11 +512,28 @@ def main():
                                 "gbs": vbytes / (verify_ms * 1e-3) / 1e9,
                                 "frac_of_measured": vbytes / (verify_ms * 1e-3) / 1e9 / peak,
                                 "frac_of_8000": vbytes / (verify_ms * 1e-3) / 1e9 / 8000.0},
-                "verify_by_n": by_n, "verify_by_ctx": by_ctx}
+                "verify_by_ctx": by_ctx}
+    # one draft-head step (fc, its layer, the LM head; a persistent launch each): a full-length draft at the same context
+    eng.ada_prefill(0, d_prompt, None)
+    eng.d_n.fill_(sh.n_max)
+    eng.ada_draft(eng.d_n, eng.d_draft)
+    eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)      # rows are not committed: the next draft starts from the same state
+    eng.ada_profile(True)
+    eng.ada_draft(eng.d_n, eng.d_draft)
+    dprof = eng.ada_get_profile()
+    eng.ada_profile(False)
+    if dprof["gemm_launches"] > 0:
+        d_us = 1e3 * dprof["gemm_ms"] / dprof["gemm_launches"]
+        dbytes = draft_step_bytes(sh) + ctx_len * 2 * 2 * sh.d_model
+        roofline["draft_step"] = {"launches_timed": dprof["gemm_launches"], "avg_launch_us": d_us, "bytes_per_launch": dbytes,
+                                  "gbs": dbytes / (d_us * 1e-6) / 1e9, "frac_of_measured": dbytes / (d_us * 1e-6) / 1e9 / peak}
+    status_roof = eng.ada_get_counters()["status"]
+    if status_roof != 0:
+        raise RuntimeError("device status word %d after the roofline leg" % status_roof)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
             "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 weights and KV cache, f32 accumulate", "data": "synthetic", "config": config,
+            "dtype": "bf16 weights, fp16 KV cache, f32 accumulate", "data": "synthetic", "config": config, "status": 0,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "tau": tokens / max(1, n_target), "mean_draft_len": n_draft / max(1, n_target), "prefill": prefill}
 
@@ -430,7 +542,9 @@ def main():
         line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
     eng.close()
     if rank == 0 and world == 1 and sh.name == "7b" and not args.layers and not args.no_batch8:
-        line["batch8"] = batch8_sample(weights, dev)
+        line["batch8"] = batch8_sample(weights, dev, peak)
+        if not args.no_teacher_forced:
+            line["teacher_forced"] = teacher_forced_sweep(weights, dev, peak)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

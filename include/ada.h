@@ -37,7 +37,7 @@ extern "C" {
 #define ADA_ERR_KV_FULL (-4)
 #define ADA_ERR_CUDA (-5)
 #define ADA_ERR_WORKSPACE (-6)
-#define ADA_ERR_STATE (-7)
+#define ADA_ERR_STATE (-7)     /* the call cannot run in the context's present state (ada_last_error says why) */
 #define ADA_ERR_TOO_LARGE (-8) /* a size exceeds a fixed maximum of the library (see ada_ldlp_eval_static) */
 
 #define ADA_MAX_LAYERS 128
@@ -88,11 +88,12 @@ size_t ada_workspace_bytes(const ada_config *cfg);
  * rotary table.  cuda_stream is a cudaStream_t (NULL = default stream).
  * With max_batch = 1 every decode pass (draft step, verify) is one persistent kernel launched
  * cooperatively in thread-block clusters of two, one CTA per SM; ada_init checks that the whole grid
- * can be resident and falls back to the multi-kernel path otherwise.  Passes of more than 16 rows
- * (ragged batches, and the prompt of every engine, 88 rows at a time) run the multi-kernel path with
- * its tensor-core GEMM; a configuration with max_batch * (n_max + 1) > 16 therefore needs d_model,
- * d_ffn and vocab of at least 128 (ADA_ERR_BAD_CONFIG otherwise).  The environment variable ADA_PASS_NONCOOP (any value)
- * drops the cooperative launch attribute, for profilers that refuse it together with clusters. */
+ * can be resident and uses the multi-kernel path otherwise.  Batches (max_batch > 1: that kernel's
+ * attention reads one sequence's cache) and the prompt of every engine, 88 rows at a time, run the
+ * multi-kernel path with its tensor-core GEMM, whose weight boxes are 128 rows high: d_model, d_ffn and
+ * vocab must be at least 128 (ADA_ERR_BAD_CONFIG otherwise).  The environment variable ADA_PASS_NONCOOP
+ * (any value) drops the cooperative launch attribute, for profilers that refuse it together with
+ * clusters. */
 int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights *w, void *d_workspace,
              size_t workspace_bytes, void *cuda_stream);
 
@@ -145,8 +146,10 @@ int ada_step(ada_ctx *ctx, int32_t *d_emitted, int32_t *d_n_emitted, int32_t *d_
 /* Test and measurement hooks ------------------------------------------------------------- */
 
 /* Fixed draft lengths instead of the predictor: n[seq] (host array of max_batch entries, each
- * 0..n_max; 0 = plain autoregressive decoding, after which the draft head is out of date and
- * ada_draft refuses to run).  NULL restores the predictor. */
+ * 0..n_max; 0 = plain autoregressive decoding: the draft head is then not kept up to date, and
+ * while every length is forced to 0 ada_draft returns ADA_ERR_STATE; a sequence whose head fell behind by
+ * more rows than one pass holds drafts nothing from then on and the status word gets its "stale" bit).
+ * NULL restores the predictor. */
 int ada_force_n(ada_ctx *ctx, const int32_t *n);
 
 /* Teacher forcing: after every draft step the drafted token of sequence seq is replaced by
@@ -165,6 +168,20 @@ int ada_force_commit(ada_ctx *ctx, int seq, const int32_t *d_tokens, int32_t cou
  * (Table 2's counters), out[4] device status word (0 = no device-side error),
  * out[5] kernels launched by this context so far, out[6..7] 0. */
 int ada_get_counters(ada_ctx *ctx, int64_t out[8]);
+
+/* Clears the device status word (stream-ordered).  After a device-side error (out[4] of ada_get_counters non-zero)
+ * the results of the calls since the last clear are not to be trusted; bit 4 (a bounded wait inside a kernel gave
+ * up) also makes every later pass give up its waits at once, so clear it before going on. */
+int ada_reset_status(ada_ctx *ctx);
+
+/* Failure detection (no passage of the paper: every wait inside the kernels -- on an mbarrier, on the grid barrier,
+ * on the K-split pair's barrier -- is bounded, and gives up by setting bit 4 of the status word and carrying on).
+ * This call runs the kernels' own wait routines on a barrier that nothing ever completes, with a limit of
+ * spin_limit polls (1 .. 2^22), so that the give-up path can be seen to run: mode 0 waits on an mbarrier phase
+ * nobody arrives at, mode 1 on a grid-barrier count that is never reached.  d_result[mode] (device, 2 x int32) is
+ * set to 1 when the wait has returned; ada_get_counters then reports status bit 4.  The context stays usable:
+ * clear the word with ada_reset_status. */
+int ada_selftest_bounded_wait(ada_ctx *ctx, int32_t mode, uint32_t spin_limit, int32_t *d_result);
 
 /* Device pointer and byte size of an internal buffer, for inspection by tests:
  * which = 0 features f [max_batch][kv_capacity][d] fp32 (row = position),

@@ -19,7 +19,7 @@ exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_
                     "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
                     "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
-                    "ada_destroy", "ada_ldlp_eval_static")
+                    "ada_destroy", "ada_ldlp_eval_static", "ada_reset_status", "ada_selftest_bounded_wait")
 
 
 class AdaError(RuntimeError):
@@ -73,6 +73,8 @@ def lib():
     L.ada_force_commit.argtypes = [vp, C.c_int, vp, i32]
     L.ada_get_counters.argtypes = [vp, C.POINTER(C.c_int64)]
     L.ada_debug_buffer.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t)]
+    L.ada_reset_status.argtypes = [vp]
+    L.ada_selftest_bounded_wait.argtypes = [vp, i32, C.c_uint32, vp]
     L.ada_profile.argtypes = [vp, C.c_int]
     L.ada_get_profile.argtypes = [vp, C.POINTER(C.c_double)]
     L.ada_ldlp_eval_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
@@ -229,6 +231,12 @@ class Engine:
         out = (C.c_int64 * 8)()
         self._check(self.L.ada_get_counters(self.h, out), "ada_get_counters")
         return dict(n_target=out[0], n_draft=out[1], n_waste=out[2], n_tokens=out[3], status=out[4], launches=out[5])
+
+    def ada_reset_status(self):
+        self._check(self.L.ada_reset_status(self.h), "ada_reset_status")
+
+    def ada_selftest_bounded_wait(self, mode: int, spin_limit: int, d_result):
+        self._check(self.L.ada_selftest_bounded_wait(self.h, mode, spin_limit, _dp(d_result)), "ada_selftest_bounded_wait")
 
     def ada_profile(self, enable: bool):
         self._check(self.L.ada_profile(self.h, 1 if enable else 0), "ada_profile")

@@ -28,17 +28,13 @@ struct LayerW {
   const bf16 *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nm;
 };
 
-struct GemmPlan {
-  int KC, KS, S;
-};
-
 }  // namespace
 
 struct ada_ctx {
   ada_config c;
   cudaStream_t stream;
   cudaStream_t capture_stream;  // private, only ever used to record the step graph (nothing executes on it)
-  int B, TM, NT;          // batch, rows per pass, n8 tiles
+  int B, TM;              // batch, rows of a decode pass of the multi-kernel path
   int pages_per_seq, n_pages;
   std::vector<LayerW> layers;
   LayerW eagle;
@@ -56,11 +52,9 @@ struct ada_ctx {
   float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z, *dlp, *dfl, *dcum;
   bf16 *xhi, *xlo, *x2hi, *x2lo;    // [TP][ldx], [TP][ldx2]
   int ldx, ldx2;
-  int *gemm_cnt;
   float4 *amax;
   int *draft, *target, *force_n_dev, *chunk_tok, *forced_buf;
   float2 *vtop, *dtop;
-  float *chunk_logits_unused;
   const int *force_draft;           // user device pointer or null
   int has_force_n;
   int host_force_n[ADA_MAX_BATCH];
@@ -69,7 +63,6 @@ struct ada_ctx {
   int use_pass, n_sm, attn_splits;
   // tensor-core GEMM of the multi-row path (passes of up to 88 rows): tensor maps of every weight matrix and of
   // the activation planes, found by base pointer
-  int use_tc;
   TensorMap128 *d_tcmaps;
   int n_tcmaps;
   std::unordered_map<const void *, int> tcmap_of;
@@ -95,6 +88,7 @@ struct ada_ctx {
   std::vector<ProfRec> prof_recs;
   int ev_used;
   std::string err;
+  int enqueue_failed;               // a helper could not enqueue part of a call (its text is in err)
 };
 
 namespace {
@@ -146,8 +140,8 @@ bool config_ok(const ada_config *c) {
   if (c->ldlp_mode == 1 && (c->ldlp_blocks < 0 || c->ldlp_blocks > 8 || c->k_min < 1 || c->k_min > c->n_max)) return false;
   if (c->max_batch < 1 || c->max_batch > ADA_MAX_BATCH) return false;
   if (c->max_batch * (c->n_max + 1) > 88) return false;
-  // passes of more than 16 rows run the tensor-core GEMM, whose weight boxes are 128 rows high
-  if (c->max_batch * (c->n_max + 1) > 16 && (c->d_model < 128 || c->d_ffn < 128 || c->vocab < 128)) return false;
+  // prompts and batches run the multi-row tensor-core GEMM, whose weight boxes are 128 rows high
+  if (c->d_model < 128 || c->d_ffn < 128 || c->vocab < 128) return false;
   if (c->page_size != 64 || c->kv_capacity < 64 || c->kv_capacity % c->page_size) return false;
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
   return true;
@@ -156,25 +150,6 @@ bool config_ok(const ada_config *c) {
 int rows_per_pass(const ada_config *c) {
   int t = c->max_batch * (c->n_max + 1);
   return t < 16 ? 16 : ((t + 7) / 8) * 8;
-}
-
-GemmPlan plan_gemm(int NT, int K, int tiles) {
-  GemmPlan p;
-  const int Kr = ((K + 63) / 64) * 64;
-  if (NT <= 2) {
-    p.KC = Kr < 1024 ? Kr : 1024;
-    p.KS = p.KC;
-  } else {
-    p.KC = Kr < 256 ? Kr : 256;
-    int chunks = (K + p.KC - 1) / p.KC;
-    int want = (592 + tiles - 1) / tiles;  // about four CTAs per SM in total
-    if (want < 1) want = 1;
-    if (want > chunks) want = chunks;
-    int per = (chunks + want - 1) / want;
-    p.KS = per * p.KC;
-  }
-  p.S = (K + p.KS - 1) / p.KS;
-  return p;
 }
 
 // K splits of the tensor-core GEMM: the smallest count that fills whole waves of one CTA per SM well (each split
@@ -193,10 +168,6 @@ int plan_tc_splits(int tiles, int K) {
 }
 int tc_tiles(int epi, int nseg, int Nseg) { return epi == EPI_SWIGLU ? (Nseg + 127) / 128 : nseg * ((Nseg + 255) / 256); }
 
-size_t part_need(int NT, int Ntot, int K, int tiles) {
-  GemmPlan p = plan_gemm(NT, K, tiles);
-  return p.S > 1 ? (size_t)p.S * NT * 8 * Ntot : 0;
-}
 size_t part_need_tc(int epi, int nseg, int Nseg, int K) {
   const int S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tc_tiles(epi, nseg, Nseg), K);
   const size_t Ntot = epi == EPI_SWIGLU ? 2 * (size_t)Nseg : (size_t)nseg * Nseg;
@@ -208,10 +179,10 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   Carver w{base, 0};
   const size_t d = c->d_model, F = c->d_ffn, V = c->vocab, L = c->n_layers, H = c->n_heads, hd = c->head_dim;
   const size_t B = c->max_batch, cap = c->kv_capacity, ps = c->page_size;
-  const int TM = rows_per_pass(c), NT = TM / 8 > 2 ? 11 : 2;
+  const int TM = rows_per_pass(c);
   const size_t TP = kTcRows;   // row scratch holds the largest pass of any engine: prompts go through 88-row chunks
   const size_t pps = cap / ps, pages = pps * B;
-  x->B = (int)B; x->TM = TM; x->NT = NT; x->pages_per_seq = (int)pps; x->n_pages = (int)pages;
+  x->B = (int)B; x->TM = TM; x->pages_per_seq = (int)pps; x->n_pages = (int)pages;
   x->tk = w.take<bf16>(pages * L * H * ps * hd);
   x->tv = w.take<bf16>(pages * L * H * ps * hd);
   x->dk = w.take<bf16>(pages * H * ps * hd);
@@ -236,12 +207,6 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->x2lo = w.take<bf16>(TP * ldx2);
   size_t pf = 0;
   auto upd = [&](size_t v) { if (v > pf) pf = v; };
-  upd(part_need(NT, (int)(3 * d), (int)d, (int)(3 * ((d + 63) / 64))));
-  upd(part_need(NT, (int)d, (int)d, (int)((d + 63) / 64)));
-  upd(part_need(NT, (int)(2 * F), (int)d, (int)((F + 63) / 64)));
-  upd(part_need(NT, (int)d, (int)F, (int)((d + 63) / 64)));
-  upd(part_need(NT, (int)V, (int)d, (int)((V + 63) / 64)));
-  upd(part_need(NT, (int)d, (int)(2 * d), (int)((d + 63) / 64)));
   {
     upd(part_need_tc(EPI_STORE, 3, (int)d, (int)d));
     upd(part_need_tc(EPI_RESID, 1, (int)d, (int)d));
@@ -252,8 +217,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   }
   x->part_floats = pf;
   x->gemm_part = w.take<float>(pf ? pf : 1);
-  x->gemm_cnt = w.take<int>(4096);
-  x->amax = w.take<float4>(((V + 63) / 64) * TP);   // (at least as many tiles as either GEMM uses)
+  x->amax = w.take<float4>(((V + 255) / 256) * TP);
   x->ldlp_h = w.take<float>(B * c->ldlp_hidden);
   x->ldlp_h2 = w.take<float>(B * c->ldlp_hidden);
   x->ldlp_z = w.take<float>(B * 16);
@@ -290,84 +254,44 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   return (w.off + 255) & ~(size_t)255;
 }
 
-template <int NT>
-int launch_gemm_nt(ada_ctx *x, int epi, GemmArgs &a, dim3 grid, size_t smem) {
-  switch (epi) {
-    case EPI_STORE: LAUNCH(x, (k_gemm<NT, EPI_STORE>), grid, 128, smem, a); break;
-    case EPI_RESID: LAUNCH(x, (k_gemm<NT, EPI_RESID>), grid, 128, smem, a); break;
-    case EPI_SWIGLU: LAUNCH(x, (k_gemm<NT, EPI_SWIGLU>), grid, 128, smem, a); break;
-    default: LAUNCH(x, (k_gemm<NT, EPI_ARGMAX>), grid, 128, smem, a); break;
+// Y = X W^T with one of the epilogues.  W0..W2: row segments (STORE) or gate/up (SWIGLU).  False (with the context's
+// error text set) if an operand has no tensor map; every operand of the path is registered at initialisation.
+bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, int nseg, int Nseg, int K,
+          const bf16 *Xhi, const bf16 *Xlo, float *Y, int ldy, bf16 *Ohi, bf16 *Olo, int ldo, float *logits,
+          int use_lm_rows) {
+  GemmTcArgs t;
+  memset(&t, 0, sizeof(t));
+  const bf16 *Ws[3] = {W0, W1, W2};
+  auto map_of = [&](const void *base) -> const TensorMap128 * {
+    auto it = x->tcmap_of.find(base);
+    return it == x->tcmap_of.end() ? nullptr : x->d_tcmaps + it->second;
+  };
+  for (int i = 0; i < 3; ++i)
+    if (Ws[i]) t.wmap[i] = map_of(Ws[i]);
+  t.xhi_map = map_of(Xhi);
+  t.xlo_map = map_of(Xlo);
+  if (!t.wmap[0] || (W1 && !t.wmap[1]) || (W2 && !t.wmap[2]) || !t.xhi_map || !t.xlo_map) {
+    x->err = "gemm: operand without a tensor map";
+    x->enqueue_failed = 1;
+    return false;
   }
-  return 0;
-}
-
-template <int NT>
-cudaError_t gemm_attr_nt(int bytes) {
-  cudaError_t e;
-  e = cudaFuncSetAttribute(k_gemm<NT, EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_gemm<NT, EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_gemm<NT, EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_gemm<NT, EPI_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-}
-
-// Y = X W^T with one of the epilogues.  W0..W2: row segments (STORE) or gate/up (SWIGLU).
-void gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, int nseg, int Nseg, int K,
-          const bf16 *Xhi, const bf16 *Xlo, int ldx, float *Y, int ldy, bf16 *Ohi, bf16 *Olo, int ldo,
-          float *logits, int use_lm_rows) {
-  if (x->NT != 2) {
-    GemmTcArgs t;
-    memset(&t, 0, sizeof(t));
-    const bf16 *Ws[3] = {W0, W1, W2};
-    auto map_of = [&](const void *base) -> const TensorMap128 * {
-      auto it = x->tcmap_of.find(base);
-      return it == x->tcmap_of.end() ? nullptr : x->d_tcmaps + it->second;
-    };
-    for (int i = 0; i < 3; ++i)
-      if (Ws[i]) t.wmap[i] = map_of(Ws[i]);
-    t.xhi_map = map_of(Xhi);
-    t.xlo_map = map_of(Xlo);
-    if (!t.wmap[0] || (W1 && !t.wmap[1]) || (W2 && !t.wmap[2]) || !t.xhi_map || !t.xlo_map) {
-      x->err = "gemm: operand without a tensor map";   // (every operand of the path is registered at initialisation)
-      return;
+  t.epi = epi; t.nseg = nseg; t.Nseg = Nseg; t.K = K;
+  const int tiles = tc_tiles(epi, nseg, Nseg);
+  t.S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tiles, K);
+  t.Y = Y; t.ldy = ldy; t.Ohi = Ohi; t.Olo = Olo; t.ldo = ldo;
+  t.part = x->gemm_part;
+  t.logits = logits; t.ldl = x->c.vocab; t.amax = x->amax;
+  t.pass = x->pass; t.use_lm_rows = use_lm_rows; t.cnts = x->cnt;
+  const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
+  timed(x, 0, wb, [&] {
+    LAUNCH(x, k_gemm_tc, dim3(tiles, t.S), kTcThreads, kTcSmemBytes, t);
+    if (t.S > 1) {   // the splits' partial sums, added in split order, then the epilogue
+      const int ncol = epi == EPI_SWIGLU ? Nseg : nseg * Nseg;
+      const int blocks = (kTcRows * (ncol / 4) + 255) / 256;
+      LAUNCH(x, k_tc_reduce, blocks < 1184 ? blocks : 1184, 256, 0, t);
     }
-    t.epi = epi; t.nseg = nseg; t.Nseg = Nseg; t.K = K;
-    const int tiles = tc_tiles(epi, nseg, Nseg);
-    t.S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tiles, K);
-    t.Y = Y; t.ldy = ldy; t.Ohi = Ohi; t.Olo = Olo; t.ldo = ldo;
-    t.part = x->gemm_part;
-    t.logits = logits; t.ldl = x->c.vocab; t.amax = x->amax;
-    t.pass = x->pass; t.use_lm_rows = use_lm_rows; t.cnts = x->cnt;
-    const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
-    timed(x, 0, wb, [&] {
-      LAUNCH(x, k_gemm_tc, dim3(tiles, t.S), kTcThreads, kTcSmemBytes, t);
-      if (t.S > 1) {   // the splits' partial sums, added in split order, then the epilogue
-        const int ncol = epi == EPI_SWIGLU ? Nseg : nseg * Nseg;
-        const int blocks = (kTcRows * (ncol / 4) + 255) / 256;
-        LAUNCH(x, k_tc_reduce, blocks < 1184 ? blocks : 1184, 256, 0, t);
-      }
-    });
-    return;
-  }
-  GemmArgs a;
-  memset(&a, 0, sizeof(a));
-  a.W[0] = W0; a.W[1] = W1; a.W[2] = W2;
-  a.nseg = nseg; a.Nseg = Nseg; a.K = K;
-  const int tiles_per_seg = (Nseg + 63) / 64;
-  const int tiles = epi == EPI_SWIGLU ? tiles_per_seg : tiles_per_seg * nseg;
-  GemmPlan p = plan_gemm(x->NT, K, tiles);
-  a.KC = p.KC; a.KS = p.KS; a.S = p.S;
-  a.Xhi = Xhi; a.Xlo = Xlo; a.ldx = ldx;
-  a.Y = Y; a.ldy = ldy; a.Ohi = Ohi; a.Olo = Olo; a.ldo = ldo;
-  a.part = x->gemm_part; a.cnt = x->gemm_cnt;
-  a.logits = logits; a.ldl = x->c.vocab; a.amax = x->amax;
-  a.pass = x->pass; a.use_lm_rows = use_lm_rows;
-  const size_t smem = (size_t)2 * x->NT * 8 * (p.KC * 2 + 64);
-  dim3 grid(tiles, p.S);
-  const double wbytes = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
-  timed(x, 0, wbytes, [&] { launch_gemm_nt<2>(x, epi, a, grid, smem); });   // (16-row passes without the persistent kernel)
+  });
+  return true;
 }
 
 void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
@@ -394,15 +318,14 @@ void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L,
   const ada_config &c = x->c;
   const int d = c.d_model, F = c.d_ffn;
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.na, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
-  gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->ldx, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
+  gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rope_kv, x->TM, 256, 0, x->pass, x->qkv, x->rope, x->qrot, kpool, vpool, x->page_table,
          x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim), x->use_pass);
   attention(x, kpool, vpool, L, layer);
-  gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->ldx, x->h, d, nullptr, nullptr, 0, nullptr, 0);
+  gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.nm, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
-  gemm(x, EPI_SWIGLU, w.wg, w.wu, nullptr, 1, F, d, x->xhi, x->xlo, x->ldx, nullptr, 0, x->x2hi, x->x2lo, x->ldx2,
-       nullptr, 0);
-  gemm(x, EPI_RESID, w.wd, nullptr, nullptr, 1, d, F, x->x2hi, x->x2lo, x->ldx2, x->h, d, nullptr, nullptr, 0, nullptr, 0);
+  gemm(x, EPI_SWIGLU, w.wg, w.wu, nullptr, 1, F, d, x->xhi, x->xlo, nullptr, 0, x->x2hi, x->x2lo, x->ldx2, nullptr, 0);
+  gemm(x, EPI_RESID, w.wd, nullptr, nullptr, 1, d, F, x->x2hi, x->x2lo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
 }
 
 // Target over the rows of x->pass: embedding, all layers, final norm (features kept per position).
@@ -415,13 +338,13 @@ void target_rows(ada_ctx *x) {
 }
 
 // Shared LM head + greedy choice over the rows staged in (xhi, xlo).
-void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int ldx, int use_lm_rows, int *tok_out, float2 *top_out,
+void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int use_lm_rows, int *tok_out, float2 *top_out,
              const int *forced, float *logits) {
   const ada_config &c = x->c;
-  gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, ldx, nullptr, 0, nullptr, nullptr,
-       0, logits, use_lm_rows);
-  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, x->NT != 2 ? (c.vocab + 255) / 256 : (c.vocab + 63) / 64, x->NT * 8,
-         x->pass, use_lm_rows, tok_out, top_out, forced);
+  gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, nullptr, 0, nullptr, nullptr, 0,
+       logits, use_lm_rows);
+  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 255) / 256, kTcRows, x->pass, use_lm_rows, tok_out, top_out,
+         forced);
 }
 
 // Draft head over the rows of x->pass (already built for `step`).
@@ -430,12 +353,11 @@ void draft_rows(ada_ctx *x, int step, bool with_lm) {
   const int d = c.d_model;
   LAUNCH(x, k_eagle_input, x->TM, 256, 0, x->pass, x->embed, x->feat, c.kv_capacity, x->dfeat, c.n_max, step, d, x->xhi,
          x->xlo, x->ldx);
-  gemm(x, EPI_STORE, x->eagle_fc, nullptr, nullptr, 1, d, 2 * d, x->xhi, x->xlo, x->ldx, x->h, d, nullptr, nullptr, 0,
-       nullptr, 0);
+  gemm(x, EPI_STORE, x->eagle_fc, nullptr, nullptr, 1, d, 2 * d, x->xhi, x->xlo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
   decoder_block(x, x->eagle, x->dk, x->dv, 1, 0);
   if (with_lm) {
     LAUNCH(x, k_split_lm_rows, x->B, 256, 0, x->pass, x->h, d, x->x2hi, x->x2lo, x->ldx2, x->dfeat, c.n_max, step);
-    lm_head(x, x->x2hi, x->x2lo, x->ldx2, 1, x->draft, x->dtop, x->force_draft, nullptr);
+    lm_head(x, x->x2hi, x->x2lo, 1, x->draft, x->dtop, x->force_draft, nullptr);
   }
 }
 
@@ -615,17 +537,24 @@ void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
     run_pass(x, 0, 0, 1, d_logits, x->target, x->vtop, nullptr);
   } else {
     target_rows(x);
-    lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->target, x->vtop, nullptr, d_logits);
+    lm_head(x, x->xhi, x->xlo, 0, x->target, x->vtop, nullptr, d_logits);
   }
 }
 
-bool cuda_ok(ada_ctx *x, const char *what) {
+// Status of an API call after its launches: ADA_ERR_STATE if a helper refused to enqueue part of it, ADA_ERR_CUDA if
+// a launch failed, else ADA_OK.
+int finish(ada_ctx *x, const char *what) {
+  if (x->enqueue_failed) {
+    x->enqueue_failed = 0;
+    cudaGetLastError();
+    return ADA_ERR_STATE;
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     x->err = std::string(what) + ": " + cudaGetErrorString(e);
-    return false;
+    return ADA_ERR_CUDA;
   }
-  return true;
+  return ADA_OK;
 }
 
 }  // namespace
@@ -679,7 +608,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   x->force_draft = nullptr; x->has_force_n = 0; x->launches = 0; x->graph = nullptr; x->graph_launches = 0;
   x->graph_key = -1;
   x->capture_stream = nullptr;
-  x->prof = 0; x->ev_used = 0;
+  x->prof = 0; x->ev_used = 0; x->enqueue_failed = 0;
 
   // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as (cos, sin) floats
   const int half = cfg->head_dim / 2, cap = cfg->kv_capacity;
@@ -701,7 +630,6 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess) e = cudaMemsetAsync(x->st, 0, sizeof(SeqState) * x->B, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->cnt, 0, sizeof(Counters), x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->pass, 0, sizeof(Pass), x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->gemm_cnt, 0, sizeof(int) * 4096, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->tok, 0, sizeof(int) * (size_t)x->B * cap, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->draft, 0, sizeof(int) * x->B * cfg->n_max, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->target, 0, sizeof(int) * x->B * (cfg->n_max + 1), x->stream);
@@ -712,9 +640,9 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);  // host vectors go out of scope
-  // persistent pass kernel: used when a pass never has more than 16 rows (batch 1)
+  // persistent pass kernel: one sequence, at most 16 rows per pass (its attention phase reads one sequence's cache)
   x->use_pass = 0;
-  if (e == cudaSuccess && x->NT == 2) {
+  if (e == cudaSuccess && cfg->max_batch == 1 && x->TM <= 16) {
     int dev = 0, sms = 0, per_sm = 0;
     e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -763,19 +691,13 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
       if (e == cudaSuccess) e = cudaMemset(x->gbar, 0, 64 * sizeof(unsigned));
     }
   }
-  // passes of more than 16 rows: the tensor-core GEMM
-  x->use_tc = 0;
-  const bool tc_fits = cfg->d_model >= 128 && cfg->d_ffn >= 128 && cfg->vocab >= 128;   // boxes are 128 rows high
-  if (e == cudaSuccess && !tc_fits && x->NT != 2) e = cudaErrorInvalidValue;
-  if (e == cudaSuccess && tc_fits) {
+  // the multi-row path (prompts of every engine, decode passes of batches): tensor maps of its GEMM operands
+  if (e == cudaSuccess) {
     e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
     std::vector<TensorMap128> maps;
     if (e == cudaSuccess && !build_tc_maps(x, maps)) e = cudaErrorUnknown;
     if (e == cudaSuccess) e = cudaMemcpy(x->d_tcmaps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) x->use_tc = 1;
   }
-  const int gemm_smem = 2 * x->NT * 8 * ((x->NT == 2 ? 1024 : 256) * 2 + 64);
-  if (e == cudaSuccess && x->NT == 2) e = gemm_attr_nt<2>(gemm_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_attn_rows<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<128>());
   if (e == cudaSuccess)
@@ -800,52 +722,48 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
   LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
   int last_rows = 0;
-  // A prompt is a many-row pass: an engine whose decode passes have 16 rows takes it through the multi-row kernels
-  // (tensor-core GEMM, 88 rows per chunk: a sixth of the weight passes) when their tensor maps exist.
-  const bool wide = x->NT == 2 && x->use_tc;
-  const bool by_pass = x->use_pass && !wide;
-  const int TM0 = x->TM, NT0 = x->NT;
-  if (wide) { x->TM = kTcRows; x->NT = kTcRows / 8; }
+  // A prompt is a many-row pass: every engine takes it through the multi-row kernels, 88 rows per chunk.
+  const int TM0 = x->TM;
+  x->TM = kTcRows;
   for (int p0 = 0; p0 < m; p0 += x->TM) {
     const int R = (m - p0 < x->TM) ? m - p0 : x->TM;
     LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
-    if (by_pass) {  // the LM phase also writes the features; its choices matter only in the last chunk
-      run_pass(x, 0, 0, 1, nullptr, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr);
-      if (p0 + R == m) last_rows = R;
-    } else {
-      target_rows(x);
-      if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
-        lm_head(x, x->xhi, x->xlo, x->ldx, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
-        last_rows = R;
-      }
+    target_rows(x);
+    if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
+      lm_head(x, x->xhi, x->xlo, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
+      last_rows = R;
     }
     // draft head on positions p0 .. min(p0+R, m-1)-1 (needs the token after each position)
     const int Rd = (p0 + R <= m - 1) ? R : (m - 1 - p0);
     if (Rd > 0) {
       LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
-      if (by_pass) run_pass(x, 1, 0, 0, nullptr, nullptr, nullptr, nullptr);
-      else draft_rows(x, 0, false);
+      draft_rows(x, 0, false);
     }
   }
-  x->TM = TM0; x->NT = NT0;
+  x->TM = TM0;
   LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),
          d_first_token);
-  return cuda_ok(x, "ada_prefill") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_prefill");
 }
 
 extern "C" int ada_ldlp_predict(ada_ctx *x, int32_t *d_n) {
   if (!x || !d_n) return ADA_ERR_NULL;
   enqueue_ldlp(x, d_n);
-  return cuda_ok(x, "ada_ldlp_predict") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_ldlp_predict");
 }
 
 extern "C" int ada_draft(ada_ctx *x, const int32_t *d_n, int32_t *d_draft) {
   if (!x || !d_n || !d_draft) return ADA_ERR_NULL;
   const ada_config &c = x->c;
+  if (x->has_force_n) {   // forced plain autoregressive decoding: the draft head is not kept up to date
+    bool all_ar = true;
+    for (int b = 0; b < x->B; ++b) all_ar = all_ar && x->host_force_n[b] == 0;
+    if (all_ar) return fail(x, ADA_ERR_STATE, "ada_draft: draft lengths are forced to 0 (ada_force_n)");
+  }
   LAUNCH(x, k_set_n, 1, 32, 0, x->st, d_n, x->B, c.n_max, c.kv_capacity, x->cnt);
   enqueue_draft(x);
   LAUNCH(x, k_copy_i32, 1, 128, 0, d_draft, x->draft, x->B * c.n_max);
-  return cuda_ok(x, "ada_draft") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_draft");
 }
 
 extern "C" int ada_label(ada_ctx *x, int32_t *d_k) {
@@ -855,13 +773,13 @@ extern "C" int ada_label(ada_ctx *x, int32_t *d_k) {
   enqueue_draft(x);
   enqueue_verify(x, -1, nullptr);
   LAUNCH(x, k_label, 1, 32, 0, x->st, x->draft, x->target, c.n_max, x->B, d_k);
-  return cuda_ok(x, "ada_label") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_label");
 }
 
 extern "C" int ada_draft_lengths(ada_ctx *x, int32_t *d_n) {
   if (!x || !d_n) return ADA_ERR_NULL;
   LAUNCH(x, k_gather_n, 1, 32, 0, x->st, d_n, x->B);
-  return cuda_ok(x, "ada_draft_lengths") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_draft_lengths");
 }
 
 extern "C" int ada_verify(ada_ctx *x, const int32_t *d_draft, const int32_t *d_n, int32_t *d_target_tok,
@@ -872,7 +790,7 @@ extern "C" int ada_verify(ada_ctx *x, const int32_t *d_draft, const int32_t *d_n
   if (d_draft && d_draft != x->draft) LAUNCH(x, k_copy_i32, 1, 128, 0, x->draft, d_draft, x->B * c.n_max);
   enqueue_verify(x, -1, d_logits);
   LAUNCH(x, k_copy_i32, 1, 128, 0, d_target_tok, x->target, x->B * (c.n_max + 1));
-  return cuda_ok(x, "ada_verify") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_verify");
 }
 
 extern "C" int ada_accept(ada_ctx *x, int32_t *d_accept_len, int32_t *d_emitted, int32_t *d_n_emitted) {
@@ -880,7 +798,7 @@ extern "C" int ada_accept(ada_ctx *x, int32_t *d_accept_len, int32_t *d_emitted,
   const ada_config &c = x->c;
   LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, -1,
          (const int *)nullptr, 0, d_accept_len, d_emitted, d_n_emitted, (int *)nullptr);
-  return cuda_ok(x, "ada_accept") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_accept");
 }
 
 extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, int32_t *d_n_used,
@@ -933,7 +851,7 @@ extern "C" int ada_step(ada_ctx *x, int32_t *d_emitted, int32_t *d_n_emitted, in
   if (d_n_emitted) LAUNCH(x, k_copy_i32, 1, 32, 0, d_n_emitted, x->out_nemit, x->B);
   if (d_n_used) LAUNCH(x, k_copy_i32, 1, 32, 0, d_n_used, x->out_nused, x->B);
   if (d_accept_len) LAUNCH(x, k_copy_i32, 1, 32, 0, d_accept_len, x->out_acc, x->B);
-  return cuda_ok(x, "ada_step") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_step");
 }
 
 extern "C" int ada_force_n(ada_ctx *x, const int32_t *n) {
@@ -971,7 +889,7 @@ extern "C" int ada_force_commit(ada_ctx *x, int seq, const int32_t *d_tokens, in
   enqueue_verify(x, seq, nullptr);
   LAUNCH(x, k_accept, 1, 32, 0, x->st, x->tok, c.kv_capacity, x->draft, x->target, c.n_max, x->B, x->cnt, seq, d_tokens,
          count, (int *)nullptr, (int *)nullptr, (int *)nullptr, (int *)nullptr);
-  return cuda_ok(x, "ada_force_commit") ? ADA_OK : ADA_ERR_CUDA;
+  return finish(x, "ada_force_commit");
 }
 
 extern "C" int ada_get_counters(ada_ctx *x, int64_t out[8]) {
@@ -983,6 +901,24 @@ extern "C" int ada_get_counters(ada_ctx *x, int64_t out[8]) {
   out[0] = (int64_t)h.n_target; out[1] = (int64_t)h.n_draft; out[2] = (int64_t)h.n_waste; out[3] = (int64_t)h.n_tokens;
   out[4] = h.status; out[5] = x->launches; out[6] = 0; out[7] = 0;
   return ADA_OK;
+}
+
+extern "C" int ada_reset_status(ada_ctx *x) {
+  if (!x) return ADA_ERR_NULL;
+  if (cudaMemsetAsync(&x->cnt->status, 0, sizeof(int), x->stream) != cudaSuccess)
+    return fail(x, ADA_ERR_CUDA, "ada_reset_status: memset failed");
+  return ADA_OK;
+}
+
+extern "C" int ada_selftest_bounded_wait(ada_ctx *x, int32_t mode, uint32_t spin_limit, int32_t *d_result) {
+  if (!x || !d_result) return ADA_ERR_NULL;
+  if (mode < 0 || mode > 1 || spin_limit < 1 || spin_limit > (1u << 22))
+    return fail(x, ADA_ERR_RANGE, "ada_selftest_bounded_wait: mode 0..1, 1 <= spin_limit <= 2^22");
+  // a counter word of its own (not the pass kernel's), zero before the launch
+  unsigned *word = x->gbar + 32;
+  cudaMemsetAsync(word, 0, sizeof(unsigned), x->stream);
+  LAUNCH(x, k_wait_selftest, 1, kPassThreads, 0, word, x->cnt, spin_limit, mode, d_result);
+  return finish(x, "ada_selftest_bounded_wait");
 }
 
 extern "C" int ada_debug_buffer(ada_ctx *x, int which, void **d_ptr, size_t *bytes) {

@@ -120,265 +120,8 @@ __device__ __forceinline__ Top2 top2_shfl_xor(Top2 a, int m) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Skinny GEMM  Y[t][n] = sum_k X[t][k] * W[n][k],  t < T <= 8*NT rows, W bf16 [N][K] streamed once.
-// The weight tile is the 16-row operand of mma.sync m16n8k16 (swap-AB) and is loaded straight from
-// global memory with 128-bit loads: lane (g, q) reads 8 consecutive k of rows g and g+8, and the
-// same k permutation is applied to the activation operand, so no shared-memory staging of W is
-// needed.  Activations (hi and lo halves) sit in shared memory for the CTA's K chunk.
-// A CTA = 4 warps = 64 weight rows; grid.y splits K; partial sums go to a scratch buffer and the
-// CTA that arrives last adds them in split order and runs the epilogue (deterministic).
+// Epilogues of the multi-row GEMM (ada_gemm_tc.cuh).
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_ARGMAX = 3 };
-
-struct GemmArgs {
-  const __nv_bfloat16 *W[3];  // STORE: up to 3 row segments; SWIGLU: W[0] = gate, W[1] = up
-  int nseg, Nseg, K;
-  int KS;                     // k range of one split (multiple of KC)
-  int KC;                     // k chunk held in shared memory (multiple of 64)
-  int S;                      // splits
-  const __nv_bfloat16 *Xhi, *Xlo;
-  int ldx;
-  float *Y;                   // STORE / RESID target
-  int ldy;
-  __nv_bfloat16 *Ohi, *Olo;   // SWIGLU target
-  int ldo;
-  float *part;                // [S][8*NT][Ntot] partial sums
-  int *cnt;                   // [tiles] arrival counters (zero between launches)
-  float *logits;              // ARGMAX: optional logits [slot][ldl]
-  int ldl;
-  float4 *amax;               // ARGMAX: [tiles][8*NT] (v1, i1, v2)
-  const Pass *pass;
-  int use_lm_rows;            // ARGMAX in the draft: T = pass->lmT, slots = pass->lm_out
-};
-
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-      "{%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint4 ldg_stream(const void *p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-
-template <int NT, int EPI>
-__global__ void __launch_bounds__(128) k_gemm(const GemmArgs a) {
-  constexpr int NA = (EPI == EPI_SWIGLU) ? 2 : 1;  // weight matrices per warp
-  constexpr int U = (NT > 2) ? 2 : 4;              // 32-k blocks in flight per thread
-  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
-  if (T <= 0) return;
-  const int nt_act = (T + 7) >> 3;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q = lane & 3;
-
-  extern __shared__ __align__(16) unsigned char smem[];
-  const int xstride = a.KC * 2 + 64;  // bytes per activation row in shared memory
-  unsigned char *xs_hi = smem;
-  unsigned char *xs_lo = smem + (size_t)NT * 8 * xstride;
-  __shared__ int s_last;
-  __shared__ Top2 s_top[4][NT * 8];
-
-  const int tiles_per_seg = (a.Nseg + 63) >> 6;
-  const int seg = (EPI == EPI_SWIGLU) ? 0 : blockIdx.x / tiles_per_seg;
-  const int tile = (EPI == EPI_SWIGLU) ? blockIdx.x : blockIdx.x % tiles_per_seg;
-  const int n0 = tile * 64 + warp * 16;
-  const int ra = n0 + g, rb = n0 + g + 8;
-  const bool va = ra < a.Nseg, vb = rb < a.Nseg;
-
-  const int kbeg = blockIdx.y * a.KS;
-  const int kend = min(a.K, kbeg + a.KS);
-
-  float acc[NA][NT][4];
-#pragma unroll
-  for (int m = 0; m < NA; ++m)
-#pragma unroll
-    for (int i = 0; i < NT; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[m][i][j] = 0.f;
-
-  const __nv_bfloat16 *wa[NA], *wb[NA];
-#pragma unroll
-  for (int m = 0; m < NA; ++m) {
-    const __nv_bfloat16 *base = (EPI == EPI_SWIGLU) ? a.W[m] : a.W[seg];
-    wa[m] = base + (size_t)(va ? ra : 0) * a.K + 8 * q;
-    wb[m] = base + (size_t)(vb ? rb : 0) * a.K + 8 * q;
-  }
-
-  for (int kc = kbeg; kc < kend; kc += a.KC) {
-    const int kc_end = min(kend, kc + a.KC);
-    __syncthreads();
-    {  // stage activations [nt_act*8][KC] (hi, lo); 16-byte granules, zero beyond K
-      const int gran = a.KC >> 3;
-      const int total = nt_act * 8 * gran * 2;
-      for (int i = tid; i < total; i += 128) {
-        const int which = i / (nt_act * 8 * gran);
-        const int rem = i - which * (nt_act * 8 * gran);
-        const int row = rem / gran, gk = rem - row * gran;
-        const int k = kc + gk * 8;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (k < kc_end) v = *reinterpret_cast<const uint4 *>((which ? a.Xlo : a.Xhi) + (size_t)row * a.ldx + k);
-        *reinterpret_cast<uint4 *>((which ? xs_lo : xs_hi) + (size_t)row * xstride + gk * 16) = v;
-      }
-    }
-    __syncthreads();
-
-    const int nblk = (kc_end - kc + 31) >> 5;
-    uint4 A0[NA][U], A1[NA][U];
-    auto load_blocks = [&](uint4 (&P0)[NA][U], uint4 (&P1)[NA][U], int blk0) {
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int k = kc + (blk0 + u) * 32 + 8 * q;
-        const bool ok = (blk0 + u) < nblk && k < kc_end;
-#pragma unroll
-        for (int m = 0; m < NA; ++m) {
-          P0[m][u] = (ok && va) ? ldg_stream(wa[m] + kc + (blk0 + u) * 32) : make_uint4(0, 0, 0, 0);
-          P1[m][u] = (ok && vb) ? ldg_stream(wb[m] + kc + (blk0 + u) * 32) : make_uint4(0, 0, 0, 0);
-        }
-      }
-    };
-    load_blocks(A0, A1, 0);
-    for (int blk = 0; blk < nblk; blk += U) {
-      uint4 N0[NA][U], N1[NA][U];
-      load_blocks(N0, N1, blk + U);
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        if (blk + u < nblk) {
-          const int koff = ((blk + u) * 32 + 8 * q) * 2;
-#pragma unroll
-          for (int i = 0; i < NT; ++i) {
-            if (i < nt_act) {
-              const uint4 bh = *reinterpret_cast<const uint4 *>(xs_hi + (size_t)(i * 8 + g) * xstride + koff);
-              const uint4 bl = *reinterpret_cast<const uint4 *>(xs_lo + (size_t)(i * 8 + g) * xstride + koff);
-#pragma unroll
-              for (int m = 0; m < NA; ++m) {
-                mma_bf16(acc[m][i], A0[m][u].x, A1[m][u].x, A0[m][u].y, A1[m][u].y, bh.x, bh.y);
-                mma_bf16(acc[m][i], A0[m][u].z, A1[m][u].z, A0[m][u].w, A1[m][u].w, bh.z, bh.w);
-                mma_bf16(acc[m][i], A0[m][u].x, A1[m][u].x, A0[m][u].y, A1[m][u].y, bl.x, bl.y);
-                mma_bf16(acc[m][i], A0[m][u].z, A1[m][u].z, A0[m][u].w, A1[m][u].w, bl.z, bl.w);
-              }
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < U; ++u)
-#pragma unroll
-        for (int m = 0; m < NA; ++m) {
-          A0[m][u] = N0[m][u];
-          A1[m][u] = N1[m][u];
-        }
-    }
-  }
-
-  // element (m, i, j) of acc: weight row n = n0 + g + 8*(j>>1), pass row t = 8*i + 2*q + (j&1)
-  const int Ntot = (EPI == EPI_SWIGLU) ? 2 * a.Nseg : a.nseg * a.Nseg;
-  if (a.S > 1) {
-    const int TP = NT * 8;
-#pragma unroll
-    for (int m = 0; m < NA; ++m)
-#pragma unroll
-      for (int i = 0; i < NT; ++i)
-        if (i < nt_act)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
-            if (n < a.Nseg) {
-              const int col = ((EPI == EPI_SWIGLU) ? m : seg) * a.Nseg + n;
-              __stcg(a.part + ((size_t)blockIdx.y * TP + t) * Ntot + col, acc[m][i][j]);
-            }
-          }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(a.cnt + blockIdx.x, 1) == a.S - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-#pragma unroll
-    for (int m = 0; m < NA; ++m)
-#pragma unroll
-      for (int i = 0; i < NT; ++i)
-        if (i < nt_act)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
-            float s = 0.f;
-            if (n < a.Nseg) {
-              const int col = ((EPI == EPI_SWIGLU) ? m : seg) * a.Nseg + n;
-              for (int sp = 0; sp < a.S; ++sp) s += __ldcg(a.part + ((size_t)sp * TP + t) * Ntot + col);
-            }
-            acc[m][i][j] = s;
-          }
-    if (tid == 0) a.cnt[blockIdx.x] = 0;
-  }
-
-  if (EPI == EPI_STORE || EPI == EPI_RESID) {
-#pragma unroll
-    for (int i = 0; i < NT; ++i)
-      if (i < nt_act)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
-          if (n < a.Nseg && t < T) {
-            float *p = a.Y + (size_t)t * a.ldy + seg * a.Nseg + n;
-            if (EPI == EPI_RESID) *p += acc[0][i][j]; else *p = acc[0][i][j];
-          }
-        }
-  } else if (EPI == EPI_SWIGLU) {
-#pragma unroll
-    for (int i = 0; i < NT; ++i)
-      if (i < nt_act)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int n = n0 + g + 8 * (j >> 1), t = 8 * i + 2 * q + (j & 1);
-          if (n < a.Nseg && t < T) {
-            const float gt = acc[0][i][j], up = acc[NA - 1][i][j];
-            const float o = (gt / (1.f + __expf(-gt))) * up;
-            __nv_bfloat16 hi, lo;
-            split_bf16(o, hi, lo);
-            a.Ohi[(size_t)t * a.ldo + n] = hi;
-            a.Olo[(size_t)t * a.ldo + n] = lo;
-          }
-        }
-  } else {  // EPI_ARGMAX
-#pragma unroll
-    for (int i = 0; i < NT; ++i) {
-      if (i < nt_act) {
-#pragma unroll
-        for (int jj = 0; jj < 2; ++jj) {
-          const int t = 8 * i + 2 * q + jj;
-          const int slot = (t < T) ? (a.use_lm_rows ? a.pass->lm_out[t] : a.pass->row_out[t]) : 0;
-          Top2 best;
-          best.v1 = -INFINITY; best.i1 = 0x7fffffff; best.v2 = -INFINITY;
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int n = n0 + g + 8 * h;
-            if (n < a.Nseg) {
-              const float v = acc[0][i][jj + 2 * h];
-              if (a.logits && t < T) a.logits[(size_t)slot * a.ldl + n] = v;
-              Top2 c; c.v1 = v; c.i1 = n; c.v2 = -INFINITY;
-              best = top2_merge(best, c);
-            }
-          }
-          best = top2_shfl_xor(best, 4);
-          best = top2_shfl_xor(best, 8);
-          best = top2_shfl_xor(best, 16);
-          if (g == 0) s_top[warp][t] = best;
-        }
-      }
-    }
-    __syncthreads();
-    if (tid < nt_act * 8) {
-      Top2 b = s_top[0][tid];
-      for (int w = 1; w < 4; ++w) b = top2_merge(b, s_top[w][tid]);
-      a.amax[(size_t)blockIdx.x * (NT * 8) + tid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
-    }
-  }
-}
 
 // Final greedy choice per row: merge the per-tile candidates in tile order.
 // tok_out[slot] = argmax; top_out[slot] = (top1, top2).  forced (optional) overrides the token.

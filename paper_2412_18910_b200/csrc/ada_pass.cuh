@@ -164,8 +164,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, unsigned parity) {
 }
 // (the spin is kept out of line: the kernel's phases together exceed the instruction cache, so every
 // copy of cold code that is not inlined into them makes the hot part smaller)
-__device__ __noinline__ void mbar_spin(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
-  for (unsigned i = 0; i < kSpinLimit; ++i) {
+__device__ __noinline__ void mbar_spin(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag,
+                                       unsigned limit = kSpinLimit) {
+  for (unsigned i = 0; i < limit; ++i) {
     if (mbar_try(bar, parity)) return;
     if (*abort_flag) return;
     if (i > 64) __nanosleep(40);
@@ -173,9 +174,10 @@ __device__ __noinline__ void mbar_spin(uint64_t *bar, unsigned parity, Counters 
   *abort_flag = 1;
   atomicOr(&cnt->status, kStatTimeout);
 }
-__device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag) {
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, unsigned parity, Counters *cnt, volatile int *abort_flag,
+                                          unsigned limit = kSpinLimit) {
   if (mbar_test(bar, parity)) return;
-  mbar_spin(bar, parity, cnt, abort_flag);
+  mbar_spin(bar, parity, cnt, abort_flag, limit);
 }
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -475,7 +477,7 @@ __device__ __forceinline__ void tile_source(const GemmDesc &g, const Slab &s, in
 
 // Warp 1 and the eight worker warps (288 threads) take part; the producers' and the issuer's warps do not.
 __device__ __noinline__ void grid_barrier_body(unsigned *gbar, Counters *cnt, unsigned long long *phase_ns, unsigned epoch, int tid,
-                                              volatile int *abort_flag) {
+                                              volatile int *abort_flag, unsigned limit = kSpinLimit) {
   named_bar(2, (kNumXWarps + kNumCWarps) * 32);
   if (tid == 32) {
     // arrive with release semantics (the named barrier above ordered the other threads' writes before this
@@ -483,7 +485,7 @@ __device__ __noinline__ void grid_barrier_body(unsigned *gbar, Counters *cnt, un
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(gbar) : "memory");
     const unsigned target = epoch * gridDim.x;
     bool ok = false;
-    for (unsigned i = 0; i < kSpinLimit && !*abort_flag; ++i) {
+    for (unsigned i = 0; i < limit && !*abort_flag; ++i) {
       if (ld_acquire(gbar) >= target) { ok = true; break; }
       if ((i & 63) == 63 && (ld_acquire(reinterpret_cast<const unsigned *>(&cnt->status)) & kStatTimeout)) break;
       if (i > 4096) __nanosleep(64);   // a barrier normally completes within a few polls
@@ -1322,6 +1324,31 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
   if (!is_xprod) {
     tc_fence_before();
     named_bar(5, 32 + kNumCWarps * 32);
+  }
+}
+
+// Self-test of the bounded waits: the same wait routines as the pass kernel, on a barrier nobody arrives at (mode 0:
+// an mbarrier phase that never completes; mode 1: a grid-barrier count that is never reached), with a small limit.
+// Both give up, set the time-out bit of the status word and return; result[mode] receives 1 when the wait returned.
+__global__ void __launch_bounds__(kPassThreads, 1) k_wait_selftest(unsigned *gbar, Counters *cnt, unsigned limit, int mode,
+                                                                   int *result) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (mode == 0) {
+    if (tid == 0) {
+      mbar_wait(&bar, 0u, cnt, &abort_flag, limit);
+      result[0] = 1;
+    }
+  } else if (warp == 1 || warp >= kFirstWorker) {   // the threads that take part in the pass kernel's grid barrier
+    grid_barrier_body(gbar, cnt, nullptr, 2u, tid, &abort_flag, limit);   // one CTA arrives, two are awaited
+    if (tid == 32) result[1] = 1;
   }
 }
 

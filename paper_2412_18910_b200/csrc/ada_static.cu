@@ -15,6 +15,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "ada.h"
 
 namespace {
@@ -23,7 +25,7 @@ static __device__ __align__(256) float g_ldlp_hidden[ADA_STATIC_MAX_HIDDEN];
 
 // In host code the name above is only a handle; the device address is looked up once per device.
 constexpr int kMaxDevices = 64;
-float *g_scratch_addr[kMaxDevices] = {nullptr};
+std::atomic<float *> g_scratch_addr[kMaxDevices];   // (zero-initialised; threads racing on the first call store the same address)
 
 __device__ __forceinline__ float warp_total(float v) {
 #pragma unroll
@@ -71,12 +73,11 @@ extern "C" int ada_ldlp_eval_static(const void *d_w1, const void *d_b1, const vo
   if (d_model < 1 || hidden < 1 || n_max < 1 || n_max > ADA_MAX_NMAX) return ADA_ERR_RANGE;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ADA_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {  // first call on this device (it is the current one): look the array up
-    float *p = nullptr;
-    if (cudaGetSymbolAddress((void **)&p, g_ldlp_hidden) != cudaSuccess || !p) return ADA_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+  float *scratch = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {  // first call on this device (it is the current one): look the array up
+    if (cudaGetSymbolAddress((void **)&scratch, g_ldlp_hidden) != cudaSuccess || !scratch) return ADA_ERR_CUDA;
+    g_scratch_addr[dev].store(scratch, std::memory_order_release);
   }
-  float *scratch = g_scratch_addr[dev];
   cudaStream_t st = (cudaStream_t)cuda_stream;
   k_static_hidden<<<(hidden + 7) / 8, 256, 0, st>>>((const __nv_bfloat16 *)d_w1, (const __nv_bfloat16 *)d_b1,
                                                     (const __nv_bfloat16 *)d_embed_row, d_feature, d_model, hidden,

@@ -4,8 +4,8 @@
 
 For each configuration the oracle prefills the seeded prompt(s) and runs lock-step iterations; per iteration
 the file keeps the draft length, the drafts, the target's choices, the accepted length, the emitted tokens,
-the top-1/top-2 logits of every draft step and verify row (the margins decide which positions are exempt) and
-the predictor's outputs.  Lengths:
+the top-1/top-2 logits of every draft step and verify row (the margins decide which positions are exempt), the
+root mean square of the draft head's feature at every step, and the predictor's outputs.  Lengths:
 
     7b      the configuration's 256 new tokens
     13b     64 iterations
@@ -37,8 +37,14 @@ LOGIT_ROWS = {"7b": [(0, 2, -1), (0, 200, 0)], "13b": [(0, 1, -1), (0, 60, 0)],
 TF_LOGIT_ROWS = [(10, 0, -1), (5, 7, 0)]   # (forced length, iteration of that sweep, row)
 
 
-def it_json(it):
-    return dict(j=int(it["j"]), n=int(it["n"]), k=int(it["k"]), emitted=[int(t) for t in it["emitted"]],
+def it_json(it, seq=None):
+    extra = {}
+    if seq is not None and it["n"] > 0:
+        # root mean square of the draft head's output at every step: the head feeds on its own unnormalised output,
+        # so the scale of its features, and with it of the draft logits, grows along the chain
+        f = seq.draft_features(int(it["n"])).astype(np.float64)
+        extra["d_rms"] = [float(x) for x in np.sqrt((f * f).mean(axis=1))]
+    return dict(extra, j=int(it["j"]), n=int(it["n"]), k=int(it["k"]), emitted=[int(t) for t in it["emitted"]],
                 draft=[int(t) for t in it["draft"]], target=[int(t) for t in it["target"]],
                 v_top1=[float(x) for x in it["v_top1"]], v_top2=[float(x) for x in it["v_top2"]],
                 d_top1=[float(x) for x in it["d_top1"]], d_top2=[float(x) for x in it["d_top2"]],
@@ -108,7 +114,7 @@ def main(names):
                         else:
                             it = seq.step(n, forced)
                         assert it["k"] == n
-                        sweep["iters"].append(it_json(it))
+                        sweep["iters"].append(it_json(it, seq))
                     rec["sweeps"].append(sweep)
                     dlen = len(prompt) - 1   # the draft head's prompt rows stay valid for the later sweeps
                     print(name, "n", n, "done at %.0f s" % (time.time() - t0), flush=True)
@@ -126,7 +132,7 @@ def main(names):
                         keep("seq%d_it%d" % (b, r), it, lg, want[0][2])
                     else:
                         it = seq.step(-1)
-                    rec["iters"].append(it_json(it))
+                    rec["iters"].append(it_json(it, seq))
                     emitted += len(it["emitted"])
                     r += 1
                     if r % 16 == 0:

@@ -17,10 +17,11 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
 def _golden(name):
-    path = os.path.join(GOLDEN, name + ".json")
-    if not os.path.exists(path):
-        pytest.skip("golden %s.json not generated yet" % name)
-    return json.load(open(path))
+    path, npz = os.path.join(GOLDEN, name + ".json"), os.path.join(GOLDEN, name + "_logits.npz")
+    if not os.path.exists(path) or not os.path.exists(npz):
+        pytest.skip("golden %s.json / %s_logits.npz not generated yet" % (name, name))
+    rows = np.load(npz)
+    return json.load(open(path)), rows
 
 
 @pytest.fixture(scope="module")
@@ -28,49 +29,61 @@ def w7b():
     return si.make_weights(si.SHAPES["7b"])
 
 
-def _run(sh, weights, golden, batch, **kw):
+def _run(sh, weights, golden, rows, batch):
+    """Replays a stored oracle trajectory through the C ABI in the engine configuration bench.py times; prints how many
+    positions were compared and how many of them were exempt (inside the oracle's own margin)."""
     from paper_2412_18910_b200 import Engine
     prompts = si.make_prompts(sh)
     assert [len(p) for p in prompts] == golden["prompt_lens"]
     e = Engine(sh, weights, max_batch=batch, kv_capacity=sh.kv_capacity)
     try:
-        for b, p in enumerate(prompts):
-            first = e.prefill(b, p)
-            assert first == golden["seqs"][b]["first"], "first token of sequence %d differs from the oracle's" % b
-        streams = [s.get("greedy") for s in golden["seqs"]] if kw.pop("teacher", False) else None
-        res = lockstep.run_golden(e, golden, prompts, greedy_streams=streams, **kw)
+        if "sweeps" not in golden["seqs"][0]:
+            for b, p in enumerate(prompts):
+                first = e.prefill(b, p)
+                assert first == golden["seqs"][b]["first"], "first token of sequence %d differs from the oracle's" % b
+        res = lockstep.run_golden(e, golden, prompts, logit_rows=rows)
         c = e.ada_get_counters()
     finally:
         e.close()
+    print("%s: iterations %d exempt %d; %s" % (golden["config"], res["iterations"], res["exempt"],
+                                              lockstep.format_stats(res["stats"])))
     assert c["status"] == 0
     assert not res["failures"], res["failures"]
+    assert res["stats"]["logit_rows"] == len(golden["logit_rows"]) == 2
     assert res["exempt"] <= max(1, res["iterations"] // 3)
-    print("iterations %d exempt %d max top-1 logit diff %.4f" % (res["iterations"], res["exempt"], res["max_top1_diff"]))
     return res
 
 
-def test_7b_predictor_lengths(w7b):
-    _run(si.SHAPES["7b"], w7b, _golden("7b"), 1)
+def test_7b_predictor_lengths_full_256_tokens(w7b):
+    g, rows = _golden("7b")
+    res = _run(si.SHAPES["7b"], w7b, g, rows, 1)
+    assert 1 + sum(len(it["emitted"]) for it in g["seqs"][0]["iters"]) >= si.SHAPES["7b"].max_new
+    assert res["iterations"] == len(g["seqs"][0]["iters"]) >= 200
 
 
 def test_7b_teacher_forced_every_length(w7b):
-    g = _golden("7b_tf")
+    """Drafts forced to the oracle's greedy continuation, length forced to each of 1..n_max, 8 iterations per length,
+    every sweep from the same prefilled 1024-token prompt: every draft is accepted, tau = n + 1."""
+    g, rows = _golden("7b_tf")
     sh = si.SHAPES["7b_tf"]
-    sched = [n for n in range(1, sh.n_max + 1) for _ in range(2)]
-    res = _run(sh, w7b, g, 1, forced_n_schedule=sched, teacher=True)
-    assert all(it["k"] == it["n"] for it in g["seqs"][0]["iters"])   # the oracle accepted every forced draft
-    assert res["exempt"] <= 2
+    res = _run(sh, w7b, g, rows, 1)
+    sweeps = g["seqs"][0]["sweeps"]
+    assert [sw["n"] for sw in sweeps] == list(range(1, sh.n_max + 1)) and all(len(sw["iters"]) >= 8 for sw in sweeps)
+    assert all(it["k"] == it["n"] for sw in sweeps for it in sw["iters"])   # the oracle accepted every forced draft
+    assert res["exempt"] <= 4
 
 
 def test_13b_predictor_lengths():
-    g = _golden("13b")
+    g, rows = _golden("13b")
     sh = si.SHAPES["13b"]
-    _run(sh, si.make_weights(sh), g, 1)
+    res = _run(sh, si.make_weights(sh), g, rows, 1)
+    assert res["iterations"] >= 64
 
 
 def test_7b_batch8_ragged(w7b):
-    g = _golden("7b_b8")
-    _run(si.SHAPES["7b_b8"], w7b, g, 8)
+    g, rows = _golden("7b_b8")
+    res = _run(si.SHAPES["7b_b8"], w7b, g, rows, 8)
+    assert res["iterations"] >= 8 * 16
 
 
 @pytest.mark.parametrize("name", ["7b", "13b"])
@@ -96,12 +109,58 @@ def test_full_width_two_layers_against_the_live_oracle(name):
             assert t_o == t_g
             feats.append(f)
             res = lockstep.run_lockstep(e, [seq], 8)
+            rel = _draft_chain_deviation(e, seq, sh)
             assert e.ada_get_counters()["status"] == 0
         finally:
             e.close()
         assert not res["failures"], res["failures"]
         assert res["exempt"] <= 2
+        # draft-head features of every step of a full-length chain, relative to the scale of the oracle's feature
+        assert max(rel) < 2e-2, rel
     assert np.array_equal(feats[0], feats[1])
+
+
+def _draft_chain_deviation(e, seq, sh):
+    """A full-length draft chain on both sides, fed the same tokens (the oracle's): per step the largest deviation of
+    the library's draft-head feature from the oracle's, divided by max(1, root mean square of the oracle's feature)."""
+    n = sh.n_max
+    d_o, _, _ = seq.draft(n)
+    ft = torch.zeros(1, n, dtype=torch.int32)
+    ft[0] = torch.from_numpy(d_o)
+    e.ada_force_draft(ft.to(e.dev))
+    e.d_n.fill_(n)
+    e.ada_draft(e.d_n, e.d_draft)
+    e.ada_force_draft(None)
+    fo = seq.draft_features(n).astype(np.float64)
+    fg = e.ada_debug_buffer(4, torch.float32, (1, n, sh.d_model))[0].cpu().numpy().astype(np.float64)
+    rms = np.sqrt((fo * fo).mean(axis=1))
+    rel = (np.abs(fo - fg).max(axis=1) / np.maximum(1.0, rms)).tolist()
+    print("draft chain: feature rms %s, max deviation / rms %s" % (np.round(rms, 2).tolist(), np.round(rel, 4).tolist()))
+    return rel
+
+
+def test_draft_chain_deviation_at_full_depth_7b():
+    """All 32 layers of the 7B shape against the live oracle on a short prompt.  The draft head feeds on its own
+    output, which no norm rescales: the oracle's feature grows about x1.33 per step (root mean square 2.6 at step 1, 35
+    at step 10), and the deviation the library inherits from its 16-bit target cache (target features within 2e-2 of
+    the oracle's, root mean square error about 2e-3) grows with it.  Relative to that scale it stays below 4e-2."""
+    import oracle
+    from paper_2412_18910_b200 import Engine
+    sh = si.SHAPES["7b"]
+    w = si.make_weights(sh)
+    prompt = si.make_prompts(sh)[0][:48]
+    m = oracle.Model(sh, w)
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
+    try:
+        seq = m.new_seq(128)
+        assert seq.prefill(prompt) == e.prefill(0, prompt)
+        f = e.ada_debug_buffer(0, torch.float32, (1, sh.kv_capacity, sh.d_model))[0, :len(prompt)].cpu().numpy()
+        assert np.abs(f - seq.features(0, len(prompt))).max() < 2e-2
+        rel = _draft_chain_deviation(e, seq, sh)
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
+    assert max(rel) < 4e-2, rel
 
 
 def test_full_width_ddd_stopping_rule_against_the_live_oracle():

@@ -83,6 +83,7 @@ def test_step_lockstep(tiny, eng, n_forced):
     eng.ada_force_n(None if n_forced < 0 else [n_forced])
     res = lockstep.run_lockstep(eng, [seq], 24, n_forced=n_forced)
     eng.ada_force_n(None)
+    print(lockstep.format_stats(res["stats"]))
     assert not res["failures"], res["failures"]
     assert res["exempt"] <= res["iterations"] // 2
 
@@ -109,7 +110,7 @@ def test_scalar_form_predictor_lockstep(tiny):
             assert t_o == t_g
             zbuf = e.ada_debug_buffer(1, torch.float32, (1, 16))
             for it in range(10):   # the scalar itself, before any decision
-                o = seq.step()
+                o = lockstep.with_draft_scale(seq.step(), seq)
                 g = e.step()
                 assert abs(float(zbuf[0, 0]) - float(o["ldlp_z"][0])) < 2e-2
                 ok, ex, resync, msg = lockstep.compare_iteration(o, g["n"][0], *_bufs(e), g["k"][0], g["emitted"][0],
@@ -193,12 +194,52 @@ def test_ragged_batch_matches_per_sequence_oracle(tiny):
             seqs.append(s)
         res = lockstep.run_lockstep(e, seqs, 10)
         assert not res["failures"], res["failures"]
+        # per-sequence forced lengths: the verify block is ragged (2, 6 and 9 rows); every sequence's drafts, target
+        # choices, accepted length and emitted tokens against its own batch-1 oracle run
         e.ada_force_n([1, 5, 8])
-        for b in range(B):       # per-sequence lengths: the verify block is ragged
-            pass
-        olist = [s.step(n) for s, n in zip(seqs, (1, 5, 8))]
-        g = e.step()
-        assert g["n"] == [1, 5, 8]
+        draft_buf = e.ada_debug_buffer(7, torch.int32, (B, sh.n_max))
+        target_buf = e.ada_debug_buffer(8, torch.int32, (B, sh.n_max + 1))
+        stats = lockstep.new_stats(sh.n_max)
+        for it in range(3):
+            olist = [lockstep.with_draft_scale(s.step(n), s) for s, n in zip(seqs, (1, 5, 8))]
+            g = e.step()
+            assert g["n"] == [1, 5, 8]
+            gd, gt = draft_buf.cpu().numpy(), target_buf.cpu().numpy()
+            for b, o in enumerate(olist):
+                ok, ex, resync, msg = lockstep.compare_iteration(o, g["n"][b], gd[b], gt[b], g["k"][b], g["emitted"][b],
+                                                                 sh.n_max, forced_n=True, stats=stats)
+                assert ok, (it, b, msg)
+                if resync:
+                    em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(e.dev)
+                    e.ada_force_commit(b, em, len(o["emitted"]))
+        print(lockstep.format_stats(stats))
+        assert sum(stats["draft_compared"]) >= 3 * 10 and stats["target_compared"] >= 9
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
+
+
+def test_batch_of_two_with_sixteen_rows_matches_per_sequence_oracle():
+    """max_batch = 2 with n_max = 7: a decode pass has at most 16 rows, as at batch 1, but two sequences: it must take
+    the multi-kernel path (the persistent pass kernel's attention reads one sequence's cache)."""
+    from paper_2412_18910_b200 import Engine
+    sh = si.scaled(si.SHAPES["tiny"], n_max=7)
+    w = si.make_weights(sh)
+    m = oracle.Model(sh, w)
+    prompts = [si.uniform_ids(13, "two%d" % b, L, sh.vocab) for b, L in enumerate((23, 70))]
+    e = Engine(sh, w, max_batch=2, kv_capacity=256)
+    try:
+        seqs = []
+        for b in range(2):
+            s = m.new_seq(256)
+            assert s.prefill(prompts[b]) == e.prefill(b, prompts[b])
+            seqs.append(s)
+        res = lockstep.run_lockstep(e, seqs, 6)
+        assert not res["failures"], res["failures"]
+        e.ada_force_n([7, 7])             # both sequences at full length: 16 rows
+        res = lockstep.run_lockstep(e, seqs, 4, n_forced=7)
+        assert not res["failures"], res["failures"]
+        assert res["stats"]["draft_compared"][6] > 0
         assert e.ada_get_counters()["status"] == 0
     finally:
         e.close()
@@ -298,7 +339,7 @@ def test_ddd_stopping_rule_lockstep(tiny, thr, n_forced):
         lens = set()
         lpbuf = e.ada_debug_buffer(10, torch.float32, (1, sh.n_max))
         for it in range(10):
-            o = seq.step(n_forced=n_forced)
+            o = lockstep.with_draft_scale(seq.step(n_forced=n_forced), seq)
             g = e.step()
             ok, ex, resync, msg = lockstep.compare_iteration(o, g["n"][0], *_bufs(e), g["k"][0], g["emitted"][0],
                                                              sh.n_max, ddd=thr)
@@ -369,3 +410,29 @@ def test_label_pass_matches_the_oracle_label_on_own_drafts(tiny, eng):
         assert int(d_k.cpu()[0]) == seq.label()
         res = lockstep.run_lockstep(eng, [seq], 1)
         assert not res["failures"], res["failures"]
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_bounded_waits_give_up_and_the_context_stays_usable(tiny, eng, mode):
+    """Failure detection: the pass kernel's wait routines (mode 0: mbarrier wait, mode 1: grid barrier) on a barrier
+    that nothing completes, with a limit of 1000 polls.  The wait returns, the status word gets the time-out bit, and
+    after ada_reset_status the same context decodes in lock step with the oracle again."""
+    sh, w, prompt, m = tiny
+    with pytest.raises(Exception):
+        eng.ada_selftest_bounded_wait(2, 1000, torch.zeros(2, dtype=torch.int32, device=eng.dev))   # no such mode
+    res = torch.zeros(2, dtype=torch.int32, device=eng.dev)
+    eng.ada_reset_status()
+    assert eng.ada_get_counters()["status"] == 0
+    eng.ada_selftest_bounded_wait(mode, 1000, res)
+    c = eng.ada_get_counters()
+    assert c["status"] & 4, c
+    assert int(res.cpu()[mode]) == 1
+    eng.ada_reset_status()
+    assert eng.ada_get_counters()["status"] == 0
+    seq, t_o, t_g = _prefill_both(eng, m, prompt)
+    assert t_o == t_g
+    eng.ada_force_n(None)
+    eng.ada_force_draft(None)
+    out = lockstep.run_lockstep(eng, [seq], 4)
+    assert not out["failures"], out["failures"]
+    assert eng.ada_get_counters()["status"] == 0

@@ -39,15 +39,15 @@ def test_scalar_predictor_configuration_is_validated():
     assert L.ada_workspace_bytes(C.byref(pkg.Config(*base, 2, 1, 4096, 64, 2, 1))) == 0     # unknown mode
 
 
-def test_batch_configurations_need_matrices_of_at_least_one_weight_box():
-    """Passes of more than 16 rows go through the tensor-core GEMM, whose weight boxes are 128 rows high: a batch
-    configuration of a narrower model is refused; the same model at batch 1 (16-row passes) is accepted, and the
-    workspace of a batch-1 engine holds the 88-row scratch of its prompt pass."""
+def test_configurations_need_matrices_of_at_least_one_weight_box():
+    """Prompts (every engine) and batches go through the multi-row tensor-core GEMM, whose weight boxes are 128 rows
+    high: a model with a narrower matrix is refused at any batch size; the workspace of a batch-1 engine holds the
+    88-row scratch of its prompt pass."""
     import ctypes as C
     import paper_2412_18910_b200 as pkg
     L = pkg.lib()
     narrow = (2, 64, 1, 64, 176, 4096, 1e4, 1e-6, 128, 8, 0)
-    assert L.ada_workspace_bytes(C.byref(pkg.Config(*narrow, 1, 256, 64))) > 0
+    assert L.ada_workspace_bytes(C.byref(pkg.Config(*narrow, 1, 256, 64))) == 0
     assert L.ada_workspace_bytes(C.byref(pkg.Config(*narrow, 3, 256, 64))) == 0
     tiny = (2, 256, 4, 64, 688, 4096, 1e4, 1e-6, 128, 8, 0)
     one = L.ada_workspace_bytes(C.byref(pkg.Config(*tiny, 1, 256, 64)))

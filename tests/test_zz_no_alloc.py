@@ -4,7 +4,8 @@ Such callers (a plugin inside an application that owns all device memory, code r
 another allocator holds the GPU) cannot give the library a workspace, so this entry point keeps
 its scratch in a fixed array inside the library.  The test calls it through the C ABI twice in a
 row, on different inputs, and checks each result against ada_ldlp_predict of a context fed the same
-inputs.  This file sorts last so that a run stopping at the first failure has run everything else.
+inputs and against the CPU oracle's predictor on the same decoding state.  This file sorts last so that
+a run stopping at the first failure has run everything else.
 """
 import numpy as np
 import pytest
@@ -20,7 +21,8 @@ def test_static_predictor_matches_the_context_predictor_twice(tiny):
     sh, w, prompt, m = tiny
     e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
     try:
-        e.prefill(0, prompt)
+        seq = m.new_seq(sh.kv_capacity)
+        assert seq.prefill(prompt) == e.prefill(0, prompt)
         feat = e.ada_debug_buffer(0, torch.float32, (1, sh.kv_capacity, sh.d_model))
         toks = e.ada_debug_buffer(2, torch.int32, (1, sh.kv_capacity))
         lens = e.ada_debug_buffer(3, torch.int32, (1, 8))
@@ -39,8 +41,15 @@ def test_static_predictor_matches_the_context_predictor_twice(tiny):
             torch.cuda.synchronize()
             assert int(n_out.cpu()[0]) == int(e.d_n.cpu()[0])
             assert np.abs(z_out.cpu().numpy() - zbuf[0, : sh.n_max].cpu().numpy()).max() <= Z_TOL
+            n_o, z_o = seq.ldlp()                               # the oracle's predictor on the same state
+            assert int(n_out.cpu()[0]) == n_o
+            assert np.abs(z_out.cpu().numpy() - z_o[: sh.n_max]).max() <= Z_TOL
             seen.append(z_out.cpu().numpy().copy())
-            e.step()                                            # move on: the second call sees other inputs
+            o = seq.step()                                      # move on: the second call sees other inputs
+            g = e.step()
+            if list(g["emitted"][0]) != [int(t) for t in o["emitted"]]:   # a flip inside the oracle's margin: follow the oracle
+                em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(e.dev)
+                e.ada_force_commit(0, em, len(o["emitted"]))
         assert not np.array_equal(seen[0], seen[1])
     finally:
         e.close()
