@@ -158,32 +158,35 @@ def batch8_sample(weights, dev, peak, iters: int = 30):
     for _ in range(5):
         eng.ada_step()
     c0 = eng.ada_get_counters()
-    lens = eng.ada_debug_buffer(3, torch.int32, (sh8.batch, 8))
-    # per iteration, on the device and in stream order: cached positions read by the verify pass (len - 1 per sequence)
-    # and the number of draft steps that ran (the longest draft length of the iteration)
-    ctx_acc = torch.zeros(1, dtype=torch.int64, device=dev)
-    steps_acc = torch.zeros(1, dtype=torch.int64, device=dev)
+    lens0 = eng.ada_debug_buffer(3, torch.int32, (sh8.batch, 8))[:, 0].cpu().to(torch.int64)   # committed tokens per sequence
+    # per iteration the library itself writes the draft lengths used and the tokens emitted into rows of these arrays
+    nused = torch.zeros(iters, sh8.batch, dtype=torch.int32, device=dev)
+    nemit = torch.zeros(iters, sh8.batch, dtype=torch.int32, device=dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(dev)
     e0.record(eng.stream)
-    for _ in range(iters):
-        ctx_acc += (lens[:, 0].to(torch.int64) - 1).sum()
-        eng.ada_step(None, None, eng.d_nused, None)
-        steps_acc += eng.d_nused.max().to(torch.int64)
+    for i in range(iters):
+        eng.ada_step(None, nemit[i], nused[i], None)
     e1.record(eng.stream)
     torch.cuda.synchronize(dev)
     c1 = eng.ada_get_counters()
     ms = e0.elapsed_time(e1)
-    kv = int(ctx_acc.item()) * kv_bytes_per_token(sh8)
-    dkv = int(ctx_acc.item()) * 2 * 2 * sh8.d_model          # the draft head's one-layer cache, read by its first step
-    bytes_total = iters * verify_weight_bytes(sh8) + kv + int(steps_acc.item()) * draft_step_bytes(sh8) + dkv
+    # cached positions read by the verify pass of iteration t: len - 1 per sequence, len growing by the tokens emitted;
+    # draft steps that ran in it: the longest draft length of the iteration
+    ne = nemit.cpu().to(torch.int64)
+    before = torch.cumsum(ne, dim=0) - ne
+    ctx_total = int(((lens0 - 1).unsqueeze(0) + before).sum())
+    steps_total = int(nused.cpu().max(dim=1).values.sum())
+    kv = ctx_total * kv_bytes_per_token(sh8)
+    dkv = ctx_total * 2 * 2 * sh8.d_model          # the draft head's one-layer cache, read by its first step
+    bytes_total = iters * verify_weight_bytes(sh8) + kv + steps_total * draft_step_bytes(sh8) + dkv
     gbs = bytes_total / (ms * 1e-3) / 1e9
     out = {"workload": "7b shape, 8 sequences, prompts %s, predictor-chosen draft lengths" % [len(p) for p in prompts],
            "iterations": iters, "ms_per_iteration": ms / iters,
            "tokens_per_s": (c1["n_tokens"] - c0["n_tokens"]) / (ms * 1e-3),
            "mean_draft_len": (c1["n_draft"] - c0["n_draft"]) / max(1, c1["n_target"] - c0["n_target"]),
            "bytes_per_iteration": bytes_total / iters, "kv_bytes_per_iteration": kv / iters,
-           "draft_steps_per_iteration": int(steps_acc.item()) / iters, "gbs": gbs, "frac_of_measured": gbs / peak,
+           "draft_steps_per_iteration": steps_total / iters, "gbs": gbs, "frac_of_measured": gbs / peak,
            "status": c1["status"]}
     eng.close()
     return out

@@ -120,6 +120,21 @@ int ada_draft(ada_ctx *ctx, const int32_t *d_n, int32_t *d_draft);
  * draft head recomputes the row of the last verified position).  d_k: [max_batch]. */
 int ada_label(ada_ctx *ctx, int32_t *d_k);
 
+/* Labels for a range of start positions of an already decoded sequence (Section 3.3, data collection: for every
+ * position j of a target output, k^j = the length of the longest common prefix of a k_max-token draft started at j and
+ * the target's own continuation).  For j = j0 .. j0 + count - 1, with token j of sequence `seq` taken as the pending
+ * token and tokens 0..j as the committed prefix, the draft head drafts n_max tokens (fewer at the end of the cache), the
+ * target verifies them, and d_k[j - j0] receives the accepted length; d_drafts [count][n_max] and d_targets
+ * [count][n_max+1] (optional) receive the drafts and the target's choices, -1 past the draft length.  The positions
+ * run one after another, last first, each through the draft and verify kernels of the decode iteration; afterwards
+ * the cache rows and features from j0 on are recomputed from the committed tokens (multi-row chunks), so the sequence
+ * continues exactly as if the call had not been made.  1 <= j0, j0 + count - 1 <= index of the pending token; the
+ * draft head must be up to date (the sequence was decoded with drafts): ADA_ERR_STATE otherwise.  Teacher forcing
+ * (ada_force_draft) applies as in ada_label.  This call reads the sequence's length from the device: it synchronises
+ * the stream once before it enqueues. */
+int ada_label_positions(ada_ctx *ctx, int seq, int32_t j0, int32_t count, int32_t *d_k, int32_t *d_drafts,
+                        int32_t *d_targets);
+
 /* The draft lengths in force after ada_draft: d_n itself, or, with ddd_threshold < 0 (Section 4), the lengths
  * the stopping rule settled on; these are the lengths to hand to ada_verify.  d_n: [max_batch]. */
 int ada_draft_lengths(ada_ctx *ctx, int32_t *d_n);

@@ -72,7 +72,7 @@ def _load():
     L.orc_accept.argtypes = [vp, vp, i32p, i32p, C.c_int, i32p, i32p]
     L.orc_step.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, f32p, f32p, f32p]
     L.orc_draft_dyn.argtypes = [vp, vp, C.c_int, i32p, i32p, f32p, f32p, f32p, i32p]
-    L.orc_label.argtypes = [vp, vp]
+    L.orc_label.argtypes = [vp, vp, i32p, i32p, i32p]
     L.orc_rewind.argtypes = [vp, C.c_int, C.c_int]
     L.orc_forward_nocache.argtypes = [vp, i32p, C.c_int, f32p, f32p]
     L.orc_draft_rows.argtypes = [vp, i32p, f32p, C.c_int, C.c_int, f32p, f32p, f32p]
@@ -286,9 +286,30 @@ class Seq:
     def label(self) -> int:
         """The optimal draft length for the current state (longest confirmed prefix of a full-length draft);
         the sequence is left unchanged."""
-        k = self.lib.orc_label(self.m.h, self.h)
+        k = self.lib.orc_label(self.m.h, self.h, None, None, None)
         assert k >= 0, "label failed rc=%d" % k
         return k
+
+    def label_tokens(self):
+        """As label(), also returning what it was decided on: (k, drafted tokens [n], target choices [n + 1])."""
+        nm = max(self.m.shape.n_max, 1)
+        dr, tg = np.zeros(nm, dtype=np.int32), np.zeros(nm + 1, dtype=np.int32)
+        n = C.c_int32(0)
+        k = self.lib.orc_label(self.m.h, self.h, dr.ctypes.data, tg.ctypes.data, C.addressof(n))
+        assert k >= 0, "label failed rc=%d" % k
+        return k, dr[: n.value].copy(), tg[: n.value + 1].copy()
+
+    def label_positions(self, j0: int, count: int) -> dict:
+        """Labels of Section 3.3 for start positions j0 .. j0 + count - 1 of this sequence's committed tokens: for each
+        j the sequence is rolled back to the state in which token j was pending and labelled (Seq.label_tokens: the
+        label, the drafts, the target's choices).  Positions
+        run from the last to the first, so that a label never reads a cache row a later position's passes wrote.
+        The sequence is left rolled back to j0: use a sequence kept for this purpose."""
+        out = {}
+        for j in range(j0 + count - 1, j0 - 1, -1):
+            self.rewind(j + 1, min(self.dlen, j - 1))
+            out[j] = self.label_tokens()
+        return out
 
     def rewind(self, length: int, dlen: int) -> None:
         """Back to an earlier state of this sequence: `length` committed tokens (the last one pending), `dlen`

@@ -555,8 +555,9 @@ int orc_step(const orc_model *m, orc_seq *s, int n_forced, const int32_t *forced
  * allowed (n_max, or what the cache still holds), verify them, and return the length of the longest prefix of the
  * draft that the target confirms -- the optimal draft length for this iteration.  Nothing is committed: the
  * sequence is left as it was (the draft head's rows of true features are recomputed identically by the next
- * draft, the target's rows are overwritten by the next verify). */
-int orc_label(const orc_model *m, orc_seq *s) {
+ * draft, the target's rows are overwritten by the next verify).  draft_out / target_out / n_out (optional) receive
+ * the drafted tokens, the target's choices after each row, and the draft length. */
+int orc_label(const orc_model *m, orc_seq *s, int32_t *draft_out, int32_t *target_out, int32_t *n_out) {
   int32_t draft[64], target[65];
   const int j = s->len - 1;
   int n = m->c.n_max;
@@ -566,6 +567,9 @@ int orc_label(const orc_model *m, orc_seq *s) {
   if (draft_impl(m, s, n, 0, NULL, draft, NULL, NULL, NULL, NULL)) return -1;
   if (orc_verify(m, s, draft, n, target, NULL, NULL, NULL)) return -2;
   s->dlen = dlen0;
+  if (draft_out) memcpy(draft_out, draft, sizeof(int32_t) * (size_t)n);
+  if (target_out) memcpy(target_out, target, sizeof(int32_t) * (size_t)(n + 1));
+  if (n_out) *n_out = n;
   int k = 0;
   while (k < n && draft[k] == target[k]) ++k;
   return k;

@@ -15,7 +15,7 @@ ADA_ERRORS = {0: "ADA_OK", -1: "ADA_ERR_BAD_CONFIG", -2: "ADA_ERR_NULL", -3: "AD
               -5: "ADA_ERR_CUDA", -6: "ADA_ERR_WORKSPACE", -7: "ADA_ERR_STATE",
               -8: "ADA_ERR_TOO_LARGE (a size exceeds a fixed maximum of the library)"}
 
-exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_draft_lengths", "ada_label",
+exported_symbols = ("ada_workspace_bytes", "ada_init", "ada_prefill", "ada_ldlp_predict", "ada_draft", "ada_draft_lengths", "ada_label", "ada_label_positions",
                     "ada_verify",
                     "ada_accept", "ada_step", "ada_force_n", "ada_force_draft", "ada_force_commit",
                     "ada_get_counters", "ada_debug_buffer", "ada_profile", "ada_get_profile", "ada_last_error",
@@ -65,6 +65,7 @@ def lib():
     L.ada_draft.argtypes = [vp, vp, vp]
     L.ada_draft_lengths.argtypes = [vp, vp]
     L.ada_label.argtypes = [vp, vp]
+    L.ada_label_positions.argtypes = [vp, C.c_int, i32, i32, vp, vp, vp]
     L.ada_verify.argtypes = [vp, vp, vp, vp, vp]
     L.ada_accept.argtypes = [vp, vp, vp, vp]
     L.ada_step.argtypes = [vp, vp, vp, vp, vp]
@@ -200,6 +201,10 @@ class Engine:
 
     def ada_label(self, d_k):
         self._check(self.L.ada_label(self.h, _dp(d_k)), "ada_label")
+
+    def ada_label_positions(self, seq: int, j0: int, count: int, d_k, d_drafts=None, d_targets=None):
+        self._check(self.L.ada_label_positions(self.h, seq, j0, count, _dp(d_k), _dp(d_drafts), _dp(d_targets)),
+                    "ada_label_positions")
 
     def ada_draft_lengths(self, d_n):
         self._check(self.L.ada_draft_lengths(self.h, _dp(d_n)), "ada_draft_lengths")

@@ -541,6 +541,33 @@ void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
   }
 }
 
+// Multi-row passes over committed positions of one sequence, 88 rows per chunk: the target over positions
+// [p_begin, p_end) (cache rows and features), the draft head over those of them below d_end (each needs the token after
+// its position).  with_choice: the greedy choice after position p_end - 1 goes to chunk_tok.  Returns the rows of the
+// last chunk.
+int enqueue_chunks(ada_ctx *x, int seq, int p_begin, int p_end, int d_end, bool with_choice) {
+  const ada_config &c = x->c;
+  int last_rows = 0;
+  const int TM0 = x->TM;
+  x->TM = kTcRows;
+  for (int p0 = p_begin; p0 < p_end; p0 += x->TM) {
+    const int R = (p_end - p0 < x->TM) ? p_end - p0 : x->TM;
+    LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
+    target_rows(x);
+    if (p0 + R == p_end) {  // the chunk that holds the last position: greedy choice after it
+      if (with_choice) lm_head(x, x->xhi, x->xlo, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
+      last_rows = R;
+    }
+    const int Rd = (p0 + R <= d_end) ? R : (d_end - p0);
+    if (Rd > 0) {
+      LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
+      draft_rows(x, 0, false);
+    }
+  }
+  x->TM = TM0;
+  return last_rows;
+}
+
 // Status of an API call after its launches: ADA_ERR_STATE if a helper refused to enqueue part of it, ADA_ERR_CUDA if
 // a launch failed, else ADA_OK.
 int finish(ada_ctx *x, const char *what) {
@@ -721,26 +748,7 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   if (m < 1) return fail(x, ADA_ERR_RANGE, "ada_prefill: empty prompt");
   if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
   LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
-  int last_rows = 0;
-  // A prompt is a many-row pass: every engine takes it through the multi-row kernels, 88 rows per chunk.
-  const int TM0 = x->TM;
-  x->TM = kTcRows;
-  for (int p0 = 0; p0 < m; p0 += x->TM) {
-    const int R = (m - p0 < x->TM) ? m - p0 : x->TM;
-    LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
-    target_rows(x);
-    if (p0 + R == m) {  // the chunk that holds the last prompt token: greedy choice after it
-      lm_head(x, x->xhi, x->xlo, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
-      last_rows = R;
-    }
-    // draft head on positions p0 .. min(p0+R, m-1)-1 (needs the token after each position)
-    const int Rd = (p0 + R <= m - 1) ? R : (m - 1 - p0);
-    if (Rd > 0) {
-      LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
-      draft_rows(x, 0, false);
-    }
-  }
-  x->TM = TM0;
+  const int last_rows = enqueue_chunks(x, seq, 0, m, m - 1, true);
   LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),
          d_first_token);
   return finish(x, "ada_prefill");
@@ -774,6 +782,39 @@ extern "C" int ada_label(ada_ctx *x, int32_t *d_k) {
   enqueue_verify(x, -1, nullptr);
   LAUNCH(x, k_label, 1, 32, 0, x->st, x->draft, x->target, c.n_max, x->B, d_k);
   return finish(x, "ada_label");
+}
+
+extern "C" int ada_label_positions(ada_ctx *x, int seq, int32_t j0, int32_t count, int32_t *d_k, int32_t *d_drafts,
+                                   int32_t *d_targets) {
+  if (!x || !d_k) return ADA_ERR_NULL;
+  const ada_config &c = x->c;
+  if (seq < 0 || seq >= x->B) return fail(x, ADA_ERR_RANGE, "ada_label_positions: seq out of range");
+  if (j0 < 1 || count < 1) return fail(x, ADA_ERR_RANGE, "ada_label_positions: j0 >= 1 and count >= 1");
+  // the sequence's lengths live on the device: this call reads them back (it synchronises the stream)
+  SeqState s0;
+  if (cudaMemcpyAsync(&s0, x->st + seq, sizeof(SeqState), cudaMemcpyDeviceToHost, x->stream) != cudaSuccess ||
+      cudaStreamSynchronize(x->stream) != cudaSuccess)
+    return fail(x, ADA_ERR_CUDA, "ada_label_positions: cannot read the sequence state");
+  if (s0.len < 2) return fail(x, ADA_ERR_STATE, "ada_label_positions: the sequence has no committed tokens");
+  if (j0 + count - 1 > s0.len - 1) return fail(x, ADA_ERR_RANGE, "ada_label_positions: start positions past the pending token");
+  if (s0.stale || s0.len - 1 - s0.dlen > c.n_max + 1)
+    return fail(x, ADA_ERR_STATE, "ada_label_positions: the draft head is behind the sequence (it was decoded without drafts)");
+  // Start positions from the last to the first: the passes of position j write cache rows and features at positions
+  // >= j only (draft head: >= j - 1, that row from true inputs), which no earlier start position reads.
+  for (int j = j0 + count - 1; j >= j0; --j) {
+    const int dl = s0.dlen < j - 1 ? s0.dlen : j - 1;
+    LAUNCH(x, k_label_begin, 1, 32, 0, x->st, seq, x->B, j + 1, dl, c.n_max, c.kv_capacity);
+    enqueue_draft(x);
+    enqueue_verify(x, seq, nullptr);
+    const int i = j - j0;
+    LAUNCH(x, k_label_one, 1, 32, 0, x->st, x->draft, x->target, c.n_max, seq, d_k + i,
+           d_drafts ? d_drafts + (size_t)i * c.n_max : (int *)nullptr,
+           d_targets ? d_targets + (size_t)i * (c.n_max + 1) : (int *)nullptr);
+  }
+  // the sequence's own state again: cache rows and features from the first start position on, from the committed tokens
+  LAUNCH(x, k_label_end, 1, 32, 0, x->st, seq, s0.len, s0.dlen, s0.n, s0.j_prev);
+  enqueue_chunks(x, seq, j0, s0.len - 1, s0.dlen, false);
+  return finish(x, "ada_label_positions");
 }
 
 extern "C" int ada_draft_lengths(ada_ctx *x, int32_t *d_n) {

@@ -608,6 +608,43 @@ __global__ void k_label(const SeqState *st, const int *draft, const int *target,
   k_out[b] = k;
 }
 
+// Label collection over start positions (Section 3.3): sequence `seq` is put into the state it had when token j was
+// pending (len = j + 1; the draft head's rows of true features up to dlen), with a full-length draft ahead; every
+// other sequence of the batch sits the pass out.
+__global__ void k_label_begin(SeqState *st, int seq, int B, int len_j, int dlen_j, int nmax, int cap) {
+  const int b = threadIdx.x;
+  if (b >= B) return;
+  if (b != seq) { st[b].n = 0; return; }
+  st[b].len = len_j;
+  st[b].dlen = dlen_j;
+  st[b].j_prev = -1;
+  st[b].n = max(0, min(nmax, cap - len_j - 1));
+}
+// ... the label of that start position (and, optionally, the drafts and the target's choices it came from) ...
+__global__ void k_label_one(const SeqState *st, const int *draft, const int *target, int nmax, int seq, int *k_out,
+                            int *draft_out, int *target_out) {
+  if (threadIdx.x != 0) return;
+  const int n = st[seq].n;
+  int k = 0;
+  while (k < n && draft[seq * nmax + k] == target[seq * (nmax + 1) + k]) ++k;
+  *k_out = k;
+  for (int i = 0; i < nmax; ++i) {
+    if (draft_out) draft_out[i] = i < n ? draft[seq * nmax + i] : -1;
+  }
+  for (int i = 0; i <= nmax; ++i) {
+    if (target_out) target_out[i] = i <= n ? target[seq * (nmax + 1) + i] : -1;
+  }
+}
+// ... and the sequence's own state back (the cache rows and features past the first start position are recomputed
+// by the caller's chunk passes).
+__global__ void k_label_end(SeqState *st, int seq, int len0, int dlen0, int n0, int j_prev0) {
+  if (threadIdx.x != 0) return;
+  st[seq].len = len0;
+  st[seq].dlen = dlen0;
+  st[seq].n = n0;
+  st[seq].j_prev = j_prev0;
+}
+
 __global__ void k_gather_n(const SeqState *st, int *out, int B) {
   if (threadIdx.x < B) out[threadIdx.x] = st[threadIdx.x].n;
 }

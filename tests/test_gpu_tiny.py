@@ -436,3 +436,56 @@ def test_bounded_waits_give_up_and_the_context_stays_usable(tiny, eng, mode):
     out = lockstep.run_lockstep(eng, [seq], 4)
     assert not out["failures"], out["failures"]
     assert eng.ada_get_counters()["status"] == 0
+
+
+def test_labels_over_start_positions_match_the_oracle_and_leave_the_state_alone(tiny):
+    """Section 3.3, data collection: ada_label_positions over the generated part of a decoded sequence against the
+    oracle's Seq.label_positions (label, drafts and target choices of every start position), then the sequence goes on
+    decoding in lock step as if nothing had happened."""
+    from paper_2412_18910_b200 import Engine
+    sh, w, prompt, m = tiny
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
+    try:
+        seq, t_o, t_g = _prefill_both(e, m, prompt)
+        assert t_o == t_g
+        res = lockstep.run_lockstep(e, [seq], 12)          # a decoded sequence, the two sides on the same tokens
+        assert not res["failures"], res["failures"]
+        toks = seq.tokens()
+        j0, count = len(prompt) + 1, len(toks) - 1 - len(prompt)     # up to and including the pending token
+        shadow = m.new_seq(512)                                        # the oracle's copy for the roll-backs
+        shadow.prefill(prompt)
+        while shadow.len < seq.len:
+            shadow.step(-1)
+        assert np.array_equal(shadow.tokens(), toks)
+        want = shadow.label_positions(j0, count)
+        d_k = torch.full((count,), -9, dtype=torch.int32, device=e.dev)
+        d_dr = torch.zeros(count, sh.n_max, dtype=torch.int32, device=e.dev)
+        d_tg = torch.zeros(count, sh.n_max + 1, dtype=torch.int32, device=e.dev)
+        e.ada_label_positions(0, j0, count, d_k, d_dr, d_tg)
+        k_g, dr_g, tg_g = d_k.cpu().numpy(), d_dr.cpu().numpy(), d_tg.cpu().numpy()
+        same = 0
+        for i in range(count):
+            k_o, dr_o, tg_o = want[j0 + i]
+            n = len(dr_o)
+            # drafts may flip only inside the oracle's margins, which this call does not return: count the positions
+            # that agree token for token and demand that nearly all do; where the drafts agree, so must the rest
+            if np.array_equal(dr_g[i, :n], dr_o):
+                same += 1
+                assert k_g[i] == k_o
+                assert tg_g[i, 0] == tg_o[0]
+                if j0 + i + 1 < len(toks):
+                    assert tg_o[0] == toks[j0 + i + 1]       # row 0 is committed token j: the target repeats its choice
+            assert np.all(dr_g[i, n:] == -1) and np.all(tg_g[i, n + 1:] == -1)
+        assert same >= count - 3, (same, count)
+        # out-of-range requests are refused on the host
+        from paper_2412_18910_b200 import AdaError
+        with pytest.raises(AdaError):
+            e.ada_label_positions(0, 0, 1, d_k)
+        with pytest.raises(AdaError):
+            e.ada_label_positions(0, len(toks) - 1, 2, d_k)
+        # the state is as before: the next iterations match the oracle's
+        res = lockstep.run_lockstep(e, [seq], 6)
+        assert not res["failures"], res["failures"]
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()

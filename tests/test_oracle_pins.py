@@ -493,3 +493,22 @@ def test_told_the_label_no_draft_is_wasted(tiny):
     assert run["counters"]["n_waste"] == 0
     for n in (1, 4, sh.n_max):
         assert run["counters"]["n_target"] <= oracle.decode(m, prompt, 32, n_policy=n)["counters"]["n_target"]
+
+
+def test_labels_over_start_positions_equal_labels_after_fresh_prefills(tiny):
+    """Section 3.3, data collection: Seq.label_positions (roll back to each start position, last first) gives, for
+    every position of a generated sequence, the label, drafts and target choices that a sequence freshly prefilled up
+    to that position gives."""
+    sh, w, prompt, m = tiny
+    dec = oracle.decode(m, prompt, 14, n_policy=-1)
+    seq = dec["seq"]
+    toks = seq.tokens()
+    j0, count = len(prompt) + 1, len(toks) - 1 - len(prompt) - 1
+    assert count >= 8
+    got = seq.label_positions(j0, count)
+    for j in range(j0, j0 + count):
+        fresh = m.new_seq(256)
+        assert fresh.prefill(toks[:j]) == toks[j]          # the sequence is the model's own greedy output
+        k, dr, tg = fresh.label_tokens()
+        assert got[j][0] == k and np.array_equal(got[j][1], dr) and np.array_equal(got[j][2], tg), j
+        assert len(dr) == sh.n_max and tg[0] == toks[j + 1]   # row 0 is the committed token j: the target repeats its choice
