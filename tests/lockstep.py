@@ -166,13 +166,14 @@ def _np_iter(o):
                 v_top1=np.asarray(o["v_top1"]), v_top2=np.asarray(o["v_top2"]), d_rms=np.asarray(o.get("d_rms", [])))
 
 
-def run_golden(engine, golden, prompts, logit_rows=None):
+def run_golden(engine, golden, prompts, logit_rows=None, row_tol=LOGIT_TOL):
     """Replays stored oracle iterations (tests/golden/*.json, written by make_goldens.py) in lock step.
 
     golden: the parsed file; prompts: the same seeded prompts (already prefilled into the engine unless the file holds
     teacher-forced sweeps, each of which starts from a fresh prefill made here).  logit_rows: the opened
     <config>_logits.npz; at the iterations it names the library runs the four separate calls, with the oracle's drafts
-    forced so that every row sees the same inputs, and the complete logit row must agree within LOGIT_TOL.
+    forced so that every row sees the same inputs, and the complete logit row must agree within row_tol (LOGIT_TOL
+    unless the caller states a measured deviation); the top-1 logit of every comparable row within LOGIT_TOL.
     Returns dict(iterations, exempt, failures, stats).
     """
     B, nmax, V = engine.B, engine.nmax, engine.shape.vocab
@@ -248,7 +249,7 @@ def run_golden(engine, golden, prompts, logit_rows=None):
                     diff = float(np.abs(d_logits[b, row].cpu().numpy() - logit_rows[key]).max())
                     stats["logit_rows"] += 1
                     stats["max_logit_diff"] = max(stats["max_logit_diff"], diff)
-                    if diff > LOGIT_TOL:
+                    if diff > row_tol:
                         failures.append("%s: complete logit row differs by %.4f" % (key, diff))
                 if resync:
                     em = torch.as_tensor(np.asarray(o["emitted"], dtype=np.int32)).to(dev)
