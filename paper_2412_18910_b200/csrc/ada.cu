@@ -303,11 +303,11 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
     LAUNCH(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, x->cnt);
     LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   } else {
     LAUNCH(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, x->use_pass, nrg);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, x->cnt);
     LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
   }
   });
@@ -320,7 +320,7 @@ void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L,
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.na, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
   gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rope_kv, x->TM, 256, 0, x->pass, x->qkv, x->rope, x->qrot, kpool, vpool, x->page_table,
-         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim), x->use_pass);
+         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim));
   attention(x, kpool, vpool, L, layer);
   gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.nm, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
@@ -655,6 +655,14 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(x->page_table, pt.data(), pt.size() * sizeof(int), cudaMemcpyHostToDevice, x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->st, 0, sizeof(SeqState) * x->B, x->stream);
+  // cache rows start finite (zero): the attention kernels copy whole blocks, and a masked key still multiplies its value row by 0
+  {
+    const size_t pool = (size_t)x->n_pages * cfg->n_heads * cfg->page_size * cfg->head_dim * sizeof(bf16);
+    if (e == cudaSuccess) e = cudaMemsetAsync(x->tk, 0, pool * cfg->n_layers, x->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(x->tv, 0, pool * cfg->n_layers, x->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(x->dk, 0, pool, x->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(x->dv, 0, pool, x->stream);
+  }
   if (e == cudaSuccess) e = cudaMemsetAsync(x->cnt, 0, sizeof(Counters), x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->pass, 0, sizeof(Pass), x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->tok, 0, sizeof(int) * (size_t)x->B * cap, x->stream);

@@ -2,30 +2,36 @@
 // head over one split of the cache, 16 query rows per CTA (row groups of a long pass across grid.z).
 //
 // Row r (absolute position pos0 + r) sees cache positions 0 .. pos0 + r: the whole history and the earlier rows
-// of its own block (every row's key and value are in the cache before this kernel runs).  A warp takes 32-key
-// blocks of the split: it copies the block's key and value rows to its own shared-memory area with 16-byte loads
-// (a block lies in one cache page), then walks it 8 keys at a time -- scores = q k^T as m16n8k16 products per 16
-// channels, online softmax on the accumulator fragments, weighted values as m16n8k8 products per 8 channels.
-// Cache elements are 16-bit halves and enter the products as they are; q and the softmax weights are fp32 and
-// enter as a (hi, lo) pair of halves, so each product is issued twice and the sums are fp32 (error 2^-22
-// relative).  Key rows sit in shared memory with their 16-byte chunks XORed by (row & 7), which makes ldmatrix
-// of 8 consecutive keys conflict-free (caches kept in that layout are copied as they are).
+// of its own block (every row's key and value are in the cache before this kernel runs).  The cache splits of a
+// sequence follow from its length alone (about 256 keys each, at most 8), so a short context is not cut into
+// slivers that cost more to set up and merge than to compute.  A warp takes 32-key blocks of the split, in halves
+// of 16 keys: one bulk copy brings a half's key rows and one its value rows (they are contiguous in the cache page)
+// into one of the warp's two buffers, so the next half is in flight while this one is computed -- scores = q k^T
+// as m16n8k16 products per 16 channels, online softmax on the accumulator fragments, weighted values as m16n8k8
+// products per 8 channels, 8 keys at a time.  Cache elements are 16-bit halves and enter the products as they are;
+// q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, so each product is issued twice and
+// the sums are fp32 (error 2^-22 relative).  Key rows are kept in the cache with their 16-byte chunks XORed by
+// (slot & 7), which makes ldmatrix of 8 consecutive keys conflict-free and lets the copy be verbatim.  A copy always
+// takes 16 whole rows: rows past the sequence are masked out of the softmax, and every cache row is finite (the
+// pools are cleared at initialisation), so they add exact zeros.
 // Partial (m, l, o[hd]) per (head, split, row) goes to `part`; k_attn_combine merges the splits in split order.
 #pragma once
 #include "ada_pass.cuh"
 
 namespace ada {
 
+constexpr int kAttnHalf = 16;   // keys per copy
+
 template <int HD>
 constexpr int attn_rows_smem_bytes() {
-  return 2 * kRowGroup * HD * 2 + 4 * 2 * 32 * HD * 2 + 2 * 4 * kRowGroup * 4;
+  return 2 * kRowGroup * HD * 2 + 4 * 2 * 2 * kAttnHalf * HD * 2 + 2 * 4 * kRowGroup * 4 + 4 * 2 * 8;
 }
 
 template <int HD>
 __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
                                                    const __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
-                                                   int page_size, int L, int layer, int H, float *part, int kswz,
-                                                   int nrg) {
+                                                   int page_size, int L, int layer, int H, float *part, int nrg,
+                                                   Counters *cnt) {
   static_assert(HD == 64 || HD == 128, "head width");
   constexpr int CH = HD / 8;   // 16-byte chunks per row
   // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
@@ -35,26 +41,53 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
   const int row0 = pass->seq_row0[b];
   const int pos0 = pass->row_pos[row0];
   const int nkeys = pos0 + R;
-  int chunk = (nkeys + kAttnSplits - 1) / kAttnSplits;
-  chunk = ((chunk + 31) / 32) * 32;
+  const int chunk = attn_split_keys(nkeys);
   const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
+  if (kbeg >= nkeys) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int d = H * HD;
 
   extern __shared__ __align__(128) unsigned char attn_rows_smem[];
   __half *qh_s = reinterpret_cast<__half *>(attn_rows_smem);          // q hi [16][HD], chunks XORed with row & 7
   __half *ql_s = qh_s + kRowGroup * HD;                               // q lo, same layout
-  __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(ql_s + kRowGroup * HD);   // [4 warps][K, V][32 keys][HD]
-  __nv_bfloat16 *kst = stg + (size_t)warp * 2 * 32 * HD, *vst = kst + 32 * HD;
+  __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(ql_s + kRowGroup * HD);   // [4 warps][2 buffers][K, V][16 keys][HD]
+  __nv_bfloat16 *wst = stg + (size_t)warp * 2 * 2 * kAttnHalf * HD;
   float (*o_s)[kRowGroup][HD] = reinterpret_cast<float (*)[kRowGroup][HD]>(stg);    // merge area, over the staging areas
-  float (*m_s)[kRowGroup] = reinterpret_cast<float (*)[kRowGroup]>(attn_rows_smem + 2 * kRowGroup * HD * 2 + 4 * 2 * 32 * HD * 2);
+  unsigned char *tail = attn_rows_smem + 2 * kRowGroup * HD * 2 + 4 * 2 * 2 * kAttnHalf * HD * 2;
+  float (*m_s)[kRowGroup] = reinterpret_cast<float (*)[kRowGroup]>(tail);
   float (*l_s)[kRowGroup] = m_s + 4;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(tail + 2 * 4 * kRowGroup * 4) + warp * 2;   // this warp's two buffers
+  __shared__ int abort_s;
   const int g8r = lane >> 2, t4 = lane & 3;
   const uint32_t qh_u = smem_u32(qh_s), ql_u = smem_u32(ql_s);
+  if (threadIdx.x == 0) abort_s = 0;
+  if (lane == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  unsigned uses[2] = {0, 0};   // completed phases of the two buffers' barriers
+  const size_t head_off = ((size_t)layer * H + hh) * page_size * HD;   // inside a page: [layer][head][slot][HD]
+  const size_t page_stride = (size_t)L * H * page_size * HD;
 
   for (int rg = rgi * kRowGroup; rg < R; rg += nrg * kRowGroup) {
     const int nr = min(kRowGroup, R - rg);
-    __syncthreads();   // the previous group's merge has read the shared areas
+    __syncthreads();   // the previous group's merge has read the shared areas; the barriers are initialised
+    const int last_pos = pos0 + rg + nr - 1;   // the last position any row of the group sees
+    // half h of this warp: keys key0(h) .. key0(h) + 15
+    auto key0_of = [&](int h) { return kbeg + 32 * (warp + 4 * (h >> 1)) + kAttnHalf * (h & 1); };
+    auto valid = [&](int h) { const int k0 = key0_of(h); return k0 < kend && k0 <= last_pos; };
+    auto issue = [&](int h) {   // one lane: the half's key rows and value rows into buffer h & 1
+      const int k0 = key0_of(h);
+      const int page = page_table[b * pages_per_seq + k0 / page_size];
+      const size_t off = (size_t)page * page_stride + head_off + (size_t)(k0 % page_size) * HD;
+      __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
+      mbar_expect_tx(&bars[h & 1], (unsigned)(2 * kAttnHalf * HD * 2));
+      bulk_g2s(kst, kpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
+      bulk_g2s(kst + kAttnHalf * HD, vpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
+    };
+    if (lane == 0 && valid(0)) issue(0);   // flies under the staging of q
     {   // the group's query rows as (hi, lo) halves; rows past nr are zero
       constexpr int PER = kRowGroup * HD / 4 / 128;
       float4 qv[PER];
@@ -91,39 +124,21 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
     float o[CH][4];
 #pragma unroll
     for (int nt = 0; nt < CH; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-    const int last_pos = pos0 + rg + nr - 1;   // the last position any row of the group sees
     const int qp0 = pos0 + rg + g8r, qp1 = qp0 + 8;
 
-    for (int kb = kbeg + warp * 32; kb < kend; kb += 128) {
-      if (kb > last_pos) break;
-      // a block of 32 keys starts at a multiple of 32 and lies in one cache page
-      const int blk_page = page_table[b * pages_per_seq + kb / page_size];
-      const size_t blk_off = (((size_t)blk_page * L + layer) * H + hh) * page_size * HD + (size_t)(kb % page_size) * HD;
-      const int nk = min(32, kend - kb);
-      __syncwarp();   // the previous block has been read
-#pragma unroll 4
-      for (int idx = lane; idx < 32 * CH; idx += 32) {   // rows past the split are zero (they may never have been written)
-        const int r = idx / CH, pc = idx - r * CH;
-        uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
-        if (r < nk) {
-          kk = *reinterpret_cast<const uint4 *>(kpool + blk_off + (size_t)r * HD + pc * 8);
-          vv = *reinterpret_cast<const uint4 *>(vpool + blk_off + (size_t)r * HD + pc * 8);
-        }
-        // piece pc of a cache key row is channel chunk pc ^ (slot & 7) in the swizzled cache layout (slot & 7 = r & 7:
-        // blocks start at multiples of 32), chunk pc otherwise; in shared memory chunk c sits at c ^ (r & 7)
-        const int c = kswz ? (pc ^ (r & 7)) : pc;
-        *reinterpret_cast<uint4 *>(kst + r * HD + ((c ^ (r & 7)) << 3)) = kk;
-        *reinterpret_cast<uint4 *>(vst + r * HD + pc * 8) = vv;
-      }
-      __syncwarp();
-
-      for (int sub = 0; sub < 4; ++sub) {
+    for (int h = 0; valid(h); ++h) {
+      if (lane == 0 && valid(h + 1)) issue(h + 1);   // the other buffer: every lane left it at the end of the last turn
+      const __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD, *vst = kst + kAttnHalf * HD;
+      mbar_wait(&bars[h & 1], (uses[h & 1]++) & 1u, cnt, &abort_s);
+      const int kb = key0_of(h);
+#pragma unroll
+      for (int sub = 0; sub < 2; ++sub) {
         const int key0 = kb + 8 * sub;          // first of these 8 keys
         if (key0 >= kend || key0 > last_pos) break;
         // ---- scores: 16 rows x 8 keys
         float sc[4] = {0.f, 0.f, 0.f, 0.f};
         const uint32_t krow = smem_u32(kst + (size_t)(8 * sub + (lane & 7)) * HD);
-        const int ksw = lane & 7;
+        const int ksw = lane & 7;               // = slot & 7: halves start at multiples of 16
         const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
         for (int kp = 0; kp < HD / 32; ++kp) {    // pairs of 16-channel steps
@@ -179,6 +194,7 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
           }
         }
       }
+      __syncwarp();   // every lane is done with this buffer
     }
 
     // per-warp partials -> shared (over the staging areas, once every warp has left them), merged in warp order

@@ -226,11 +226,11 @@ __global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bf
 // Rotary embedding (rotate-half pairing) of q and k, scaling of q by 1/sqrt(hd), and the write of
 // k, v (bf16) into the paged cache.  qkv: [T][3d] fp32.  rope: [cap][hd/2] (cos, sin).
 // Cache element (page, layer, head, slot, i): ((page*L + layer)*H + head)*page_size*hd + slot*hd + i.
-// kswz: key rows are stored with their 16-byte chunks XORed by (slot & 7), the layout the persistent pass kernel
-// keeps its caches in (an engine that decodes with that kernel and takes prompts through this one).
+// Key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared memory, eight
+// consecutive keys then sit in eight different bank groups (the layout both attention kernels read).
 __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope, float *qout,
                           __nv_bfloat16 *kpool, __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
-                          int page_size, int L, int layer, int H, int hd, float qscale, int kswz) {
+                          int page_size, int L, int layer, int H, int hd, float qscale) {
   const int t = blockIdx.x;
   if (t >= pass->T) return;
   const int d = H * hd, half = hd >> 1;
@@ -238,7 +238,7 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
   const int page = page_table[b * pages_per_seq + pos / page_size], slot = pos % page_size;
   const float *__restrict__ q = qkv + (size_t)t * 3 * d;
   const float *__restrict__ k = q + d, *__restrict__ v = k + d;
-  const int sw = kswz ? (slot & 7) : 0;
+  const int sw = slot & 7;
   for (int idx0 = threadIdx.x; idx0 < H * half; idx0 += 4 * blockDim.x) {
     // the loads of four steps first, so that they are in flight together
     float qa[4], qb[4], ka[4], kb[4], va[4], vb[4];
@@ -272,6 +272,14 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
   }
 }
 
+// Keys per cache split of a sequence that holds nkeys keys (the result is a multiple of 32), and with it the number of splits.
+__host__ __device__ __forceinline__ int attn_split_keys(int nkeys) {
+  int nsp = (nkeys + 255) / 256;
+  nsp = nsp < 1 ? 1 : (nsp > kAttnSplits ? kAttnSplits : nsp);
+  const int chunk = (nkeys + nsp - 1) / nsp;
+  return ((chunk + 31) / 32) * 32;
+}
+
 // Merge the cache splits in split order and emit the attention output row as hi/lo halves.
 template <int HD>
 __global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat16 *xhi, __nv_bfloat16 *xlo,
@@ -283,8 +291,7 @@ __global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat1
   const size_t sstride = (size_t)kMaxRows * (HD + 2);
   const int b = pass->row_seq[t];
   const int nkeys = pass->row_pos[pass->seq_row0[b]] + pass->seq_rows[b];
-  int chunk = (nkeys + kAttnSplits - 1) / kAttnSplits;
-  chunk = ((chunk + 31) / 32) * 32;
+  const int chunk = attn_split_keys(nkeys);
   const int nsp = (nkeys + chunk - 1) / chunk;  // splits that held keys
   float M = -INFINITY;
   for (int s = 0; s < nsp; ++s) M = fmaxf(M, base[s * sstride + HD]);
