@@ -89,7 +89,7 @@ size_t ada_workspace_bytes(const ada_config *cfg);
  * With max_batch = 1 every decode pass (draft step, verify) is one persistent kernel launched
  * cooperatively in thread-block clusters of two, one CTA per SM; ada_init checks that the whole grid
  * can be resident and uses the multi-kernel path otherwise.  Batches (max_batch > 1: that kernel's
- * attention reads one sequence's cache) and the prompt of every engine, 88 rows at a time, run the
+ * attention reads one sequence's cache) and the prompt of every engine, 128 rows at a time, run the
  * multi-kernel path with its tensor-core GEMM, whose weight boxes are 128 rows high: d_model, d_ffn and
  * vocab must be at least 128 (ADA_ERR_BAD_CONFIG otherwise).  The environment variable ADA_PASS_NONCOOP
  * (any value) drops the cooperative launch attribute, for profilers that refuse it together with
@@ -98,7 +98,7 @@ int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights *w, void *d
              size_t workspace_bytes, void *cuda_stream);
 
 /* Algorithm 1, first pass (draft length 0): the target reads the m prompt tokens of sequence
- * `seq` (in chunks of up to 88 positions), fills its cache and emits the first new token, which
+ * `seq` (in chunks of up to 128 positions), fills its cache and emits the first new token, which
  * becomes the pending token; the draft head is brought up to date on prompt positions 0..m-2.  d_first_token (optional)
  * receives that token.  1 <= m, m + n_max + 2 <= kv_capacity. */
 int ada_prefill(ada_ctx *ctx, int seq, const int32_t *d_prompt, int32_t m, int32_t *d_first_token);

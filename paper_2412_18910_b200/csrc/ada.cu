@@ -65,7 +65,7 @@ struct ada_ctx {
   // the activation planes, found by base pointer
   TensorMap128 *d_tcmaps;
   int n_tcmaps;
-  std::unordered_map<const void *, int> tcmap_of;
+  std::unordered_map<const void *, int> tcmap_of, tcmap_wide_of;   // (wide: the planes in boxes of 128 rows)
   LayerPtrs *d_layers, *d_eagle;
   TensorMap128 *d_maps;
   int n_maps;
@@ -171,7 +171,7 @@ int tc_tiles(int epi, int nseg, int Nseg) { return epi == EPI_SWIGLU ? (Nseg + 1
 size_t part_need_tc(int epi, int nseg, int Nseg, int K) {
   const int S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tc_tiles(epi, nseg, Nseg), K);
   const size_t Ntot = epi == EPI_SWIGLU ? 2 * (size_t)Nseg : (size_t)nseg * Nseg;
-  return S > 1 ? (size_t)S * kTcRows * Ntot : 0;
+  return S > 1 ? (size_t)S * kTcRowsMax * Ntot : 0;
 }
 
 // Lays the workspace out; with base == nullptr only measures it.
@@ -180,7 +180,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   const size_t d = c->d_model, F = c->d_ffn, V = c->vocab, L = c->n_layers, H = c->n_heads, hd = c->head_dim;
   const size_t B = c->max_batch, cap = c->kv_capacity, ps = c->page_size;
   const int TM = rows_per_pass(c);
-  const size_t TP = kTcRows;   // row scratch holds the largest pass of any engine: prompts go through 88-row chunks
+  const size_t TP = kTcRowsMax;   // row scratch holds the largest pass of any engine: prompts go through 128-row chunks
   const size_t pps = cap / ps, pages = pps * B;
   x->B = (int)B; x->TM = TM; x->pages_per_seq = (int)pps; x->n_pages = (int)pages;
   x->tk = w.take<bf16>(pages * L * H * ps * hd);
@@ -239,7 +239,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->d_eagle = w.take<LayerPtrs>(1);
   x->n_maps = (int)(7 * (L + 1) + 2 + 8);
   x->d_maps = w.take<TensorMap128>(x->n_maps);
-  x->n_tcmaps = (int)(7 * (L + 1) + 2 + 4);
+  x->n_tcmaps = (int)(7 * (L + 1) + 2 + 8);
   x->d_tcmaps = w.take<TensorMap128>(x->n_tcmaps);
   x->xa = w.take<bf16>(((d + 63) / 64) * 2048);
   x->at = w.take<bf16>(((d + 63) / 64) * 2048);
@@ -262,14 +262,20 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   GemmTcArgs t;
   memset(&t, 0, sizeof(t));
   const bf16 *Ws[3] = {W0, W1, W2};
+  const bool wide = x->TM > kTcRows;   // a prompt chunk: planes in boxes of 128 rows
   auto map_of = [&](const void *base) -> const TensorMap128 * {
     auto it = x->tcmap_of.find(base);
     return it == x->tcmap_of.end() ? nullptr : x->d_tcmaps + it->second;
   };
+  auto plane_of = [&](const void *base) -> const TensorMap128 * {
+    if (!wide) return map_of(base);
+    auto it = x->tcmap_wide_of.find(base);
+    return it == x->tcmap_wide_of.end() ? nullptr : x->d_tcmaps + it->second;
+  };
   for (int i = 0; i < 3; ++i)
     if (Ws[i]) t.wmap[i] = map_of(Ws[i]);
-  t.xhi_map = map_of(Xhi);
-  t.xlo_map = map_of(Xlo);
+  t.xhi_map = plane_of(Xhi);
+  t.xlo_map = plane_of(Xlo);
   if (!t.wmap[0] || (W1 && !t.wmap[1]) || (W2 && !t.wmap[2]) || !t.xhi_map || !t.xlo_map) {
     x->err = "gemm: operand without a tensor map";
     x->enqueue_failed = 1;
@@ -284,10 +290,11 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   t.pass = x->pass; t.use_lm_rows = use_lm_rows; t.cnts = x->cnt;
   const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
   timed(x, 0, wb, [&] {
-    LAUNCH(x, k_gemm_tc, dim3(tiles, t.S), kTcThreads, kTcSmemBytes, t);
+    if (wide) LAUNCH(x, k_gemm_tc<kTcRowsMax>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRowsMax>::kSmemBytes, t);
+    else LAUNCH(x, k_gemm_tc<kTcRows>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRows>::kSmemBytes, t);
     if (t.S > 1) {   // the splits' partial sums, added in split order, then the epilogue
       const int ncol = epi == EPI_SWIGLU ? Nseg : nseg * Nseg;
-      const int blocks = (kTcRows * (ncol / 4) + 255) / 256;
+      const int blocks = ((wide ? kTcRowsMax : kTcRows) * (ncol / 4) + 255) / 256;
       LAUNCH(x, k_tc_reduce, blocks < 1184 ? blocks : 1184, 256, 0, t);
     }
   });
@@ -297,7 +304,8 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
 void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   const ada_config &c = x->c;
   // query rows of a sequence in groups of 16 across grid.z (a prompt chunk is one sequence with up to 88 rows)
-  const int nrg = (x->TM / x->B + kRowGroup - 1) / kRowGroup;
+  // (a prompt chunk is one sequence with up to 128 rows, whatever the batch size of the engine)
+  const int nrg = x->TM > kTcRows ? (x->TM + kRowGroup - 1) / kRowGroup : (x->TM / x->B + kRowGroup - 1) / kRowGroup;
   dim3 g1(c.n_heads, kAttnSplits, x->B * nrg);
   dim3 g2(c.n_heads, x->TM);
   timed(x, 1, 0.0, [&] {
@@ -343,7 +351,7 @@ void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int use_lm_rows, int 
   const ada_config &c = x->c;
   gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, nullptr, 0, nullptr, nullptr, 0,
        logits, use_lm_rows);
-  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 255) / 256, kTcRows, x->pass, use_lm_rows, tok_out, top_out,
+  LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 255) / 256, kTcRowsMax, x->pass, use_lm_rows, tok_out, top_out,
          forced);
 }
 
@@ -438,8 +446,14 @@ bool build_tc_maps(ada_ctx *x, std::vector<TensorMap128> &maps) {
   layer(x->eagle);
   add(x->eagle_fc, d, 2 * d, 128);
   add(x->lm_head, V, d, 128);
-  add(x->xhi, kTcRows, x->ldx, kTcRows); add(x->xlo, kTcRows, x->ldx, kTcRows);
-  add(x->x2hi, kTcRows, x->ldx2, kTcRows); add(x->x2lo, kTcRows, x->ldx2, kTcRows);
+  add(x->xhi, kTcRowsMax, x->ldx, kTcRows); add(x->xlo, kTcRowsMax, x->ldx, kTcRows);
+  add(x->x2hi, kTcRowsMax, x->ldx2, kTcRows); add(x->x2lo, kTcRowsMax, x->ldx2, kTcRows);
+  x->tcmap_wide_of.clear();
+  auto add_wide = [&](const void *base, size_t cols) {
+    ok = ok && next < x->n_tcmaps && encode_map(fn, &maps[next], base, kTcRowsMax, cols, kTcRowsMax);
+    x->tcmap_wide_of[base] = next++;
+  };
+  add_wide(x->xhi, x->ldx); add_wide(x->xlo, x->ldx); add_wide(x->x2hi, x->ldx2); add_wide(x->x2lo, x->ldx2);
   return ok;
 }
 
@@ -541,7 +555,7 @@ void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
   }
 }
 
-// Multi-row passes over committed positions of one sequence, 88 rows per chunk: the target over positions
+// Multi-row passes over committed positions of one sequence, 128 rows per chunk: the target over positions
 // [p_begin, p_end) (cache rows and features), the draft head over those of them below d_end (each needs the token after
 // its position).  with_choice: the greedy choice after position p_end - 1 goes to chunk_tok.  Returns the rows of the
 // last chunk.
@@ -549,7 +563,7 @@ int enqueue_chunks(ada_ctx *x, int seq, int p_begin, int p_end, int d_end, bool 
   const ada_config &c = x->c;
   int last_rows = 0;
   const int TM0 = x->TM;
-  x->TM = kTcRows;
+  x->TM = kTcRowsMax;
   for (int p0 = p_begin; p0 < p_end; p0 += x->TM) {
     const int R = (p_end - p0 < x->TM) ? p_end - p0 : x->TM;
     LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
@@ -670,10 +684,10 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   if (e == cudaSuccess) e = cudaMemsetAsync(x->target, 0, sizeof(int) * x->B * (cfg->n_max + 1), x->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->force_n_dev, 0, sizeof(int) * x->B, x->stream);
   // activation staging rows beyond the live ones are read by the tensor-core tiles: keep them finite
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->xhi, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->xlo, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)kTcRows * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xhi, 0, sizeof(bf16) * (size_t)kTcRowsMax * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->xlo, 0, sizeof(bf16) * (size_t)kTcRowsMax * x->ldx, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2hi, 0, sizeof(bf16) * (size_t)kTcRowsMax * x->ldx2, x->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(x->x2lo, 0, sizeof(bf16) * (size_t)kTcRowsMax * x->ldx2, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);  // host vectors go out of scope
   // persistent pass kernel: one sequence, at most 16 rows per pass (its attention phase reads one sequence's cache)
   x->use_pass = 0;
@@ -728,7 +742,9 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   }
   // the multi-row path (prompts of every engine, decode passes of batches): tensor maps of its GEMM operands
   if (e == cudaSuccess) {
-    e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    e = cudaFuncSetAttribute(k_gemm_tc<kTcRows>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcShape<kTcRows>::kSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_gemm_tc<kTcRowsMax>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcShape<kTcRowsMax>::kSmemBytes);
     std::vector<TensorMap128> maps;
     if (e == cudaSuccess && !build_tc_maps(x, maps)) e = cudaErrorUnknown;
     if (e == cudaSuccess) e = cudaMemcpy(x->d_tcmaps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);

@@ -1,5 +1,6 @@
-// Multi-row GEMM on the 5th-generation tensor cores for passes of up to 88 rows (ragged batches, prompt chunks):
-//   Y[t][n] = sum_k X[t][k] * W[n][k],  t < T <= 88,  W bf16 [N][K] streamed once from HBM.
+// Multi-row GEMM on the 5th-generation tensor cores for passes of up to ROWS rows (ROWS = 88: decode passes of a
+// ragged batch; ROWS = 128: prompt chunks):
+//   Y[t][n] = sum_k X[t][k] * W[n][k],  t < T <= ROWS,  W bf16 [N][K] streamed once from HBM.
 //
 // With this many rows the activation operand is no longer small next to the weights (88 rows x {hi, lo} = 22 KB per
 // 64 k against 16 KB for 128 weight rows), so a CTA takes a tall tile -- two m tiles of 128 weight rows that share
@@ -7,14 +8,15 @@
 // (grid.y splits); level-2 to shared-memory traffic then stays below 1.7 times the weight bytes.
 //
 //   warp 0   producer, one thread: per 64 k one stage = weight boxes (TMA tiled loads, 128-byte swizzle, box 64 k x 128
-//            rows) + the hi plane box and the lo plane box of the activations (64 k x 88 rows each, stacked so that they
-//            form one K-major operand of 176 rows); 4 stages of 54 KB, mbarrier transaction counts
-//   warp 1   one elected thread issues tcgen05.mma (M = 128, N = 176, K = 16) per m tile and 16 k straight from the
-//            TMA-written tiles; accumulators in tensor memory (m tile i in columns [256 i, 256 i + 176));
+//            rows) + the hi plane box and the lo plane box of the activations (64 k x ROWS rows each, stacked so that
+//            they form one K-major operand of 2 ROWS rows); 4 stages of 54 KB (ROWS = 88) or 3 of 64 KB (ROWS = 128),
+//            mbarrier transaction counts
+//   warp 1   one elected thread issues tcgen05.mma (M = 128, N = 2 ROWS, K = 16) per m tile and 16 k straight from the
+//            TMA-written tiles; accumulators in tensor memory (m tile i in columns [256 i, 256 i + 2 ROWS));
 //            tcgen05.commit frees the stage and, at the end, signals the accumulators
 //   warp 2   owns the tensor-memory allocation (512 columns)
 //   warps 4..11  epilogue: thread = one weight row (tensor-memory lane), tcgen05.ld eight pass rows at a time,
-//            column t (hi) + column 88 + t (lo)
+//            column t (hi) + column ROWS + t (lo)
 //
 // K splits leave their partial sums in a scratch buffer and k_tc_reduce, launched next, adds them in split order
 // and runs the epilogue over the whole grid (a last-arriving CTA per tile doing this alone was measured to take
@@ -25,35 +27,42 @@
 
 namespace ada {
 
-constexpr int kTcRows = 88;                          // rows of a pass at most = box height of the plane maps
-constexpr int kTcN = 2 * kTcRows;                    // MMA N: hi rows then lo rows
+constexpr int kTcRows = 88;                          // rows of a decode pass of a batch at most (8 sequences x 11 rows)
+constexpr int kTcRowsMax = 128;                      // rows of a prompt chunk; row scratch, partial sums and candidates are strided by it
 constexpr int kTcABytes = 128 * 128;                 // one weight box: 128 rows x 64 k bf16
-constexpr int kTcBBytes = kTcRows * 128;             // one plane box
-constexpr int kTcStageBytes = 2 * kTcABytes + 2 * kTcBBytes;   // 55296
-constexpr int kTcStages = 4;
 constexpr int kTcThreads = 12 * 32;
-constexpr int kTcSmemBytes = 1024 + kTcStages * kTcStageBytes + 256;
 constexpr int kTcTmemCols = 512;
-static_assert(kTcBBytes % 1024 == 0, "the lo plane must start on a swizzle-atom boundary");
-static_assert(kTcSmemBytes <= 227 * 1024, "shared memory budget");
+// Shapes of the two instantiations: ROWS = 88 (N = 176, four 54 KB stages) and ROWS = 128 (N = 256, the largest N of one
+// product and exactly the 2 x 256 accumulator columns; three 64 KB stages).
+template <int ROWS>
+struct TcShape {
+  static constexpr int kN = 2 * ROWS;                          // MMA N: hi rows then lo rows
+  static constexpr int kBBytes = ROWS * 128;                   // one plane box
+  static constexpr int kStageBytes = 2 * kTcABytes + 2 * kBBytes;
+  static constexpr int kStages = ROWS <= 88 ? 4 : 3;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
+  static_assert(kBBytes % 1024 == 0, "the lo plane must start on a swizzle-atom boundary");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+  static_assert(kN <= 256 && kN % 16 == 0, "N of one product");
+};
 
 struct GemmTcArgs {
   const TensorMap128 *wmap[3];   // box {64 k, 128 rows}; STORE: up to 3 row segments; SWIGLU: gate, up
-  const TensorMap128 *xhi_map, *xlo_map;   // planes [88][ld]: box {64 k, 88 rows}
+  const TensorMap128 *xhi_map, *xlo_map;   // planes [128][ld]: box {64 k, ROWS rows}
   int epi;                    // EPI_STORE / EPI_RESID / EPI_SWIGLU / EPI_ARGMAX
   int nseg, Nseg, K;
   int S;                      // K splits (grid.y)
   float *Y; int ldy;          // STORE / RESID target
   __nv_bfloat16 *Ohi, *Olo; int ldo;   // SWIGLU target planes
-  float *part;                // [S][88][Ntot] partial sums (S > 1; ARGMAX is never split)
+  float *part;                // [S][128][Ntot] partial sums (S > 1; ARGMAX is never split)
   float *logits; int ldl;     // ARGMAX: optional logits [slot][ldl]
-  float4 *amax;               // ARGMAX: [tiles][88] (v1, i1, v2)
+  float4 *amax;               // ARGMAX: [tiles][128] (v1, i1, v2)
   const Pass *pass;
   int use_lm_rows;            // ARGMAX in the draft: T = pass->lmT, slots = pass->lm_out
   Counters *cnts;             // status word for waits that gave up
 };
 
-// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = 128, N = 176, K = 16
+// D(f32, tensor memory) (+)= A(bf16, smem) * B(bf16, smem)^T, M = m, N = n, K = 16
 __host__ __device__ constexpr uint32_t umma_idesc_mn(uint32_t m, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
@@ -69,7 +78,10 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+template <int ROWS>
 __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
+  using Sh = TcShape<ROWS>;
+  constexpr int kTcStages = Sh::kStages, kTcStageBytes = Sh::kStageBytes, kTcBBytes = Sh::kBBytes, kTcN = Sh::kN;
   const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
   if (T <= 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -176,12 +188,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
       for (int i = 0; i < 8; ++i) { y[i] = 0.f; u[i] = 0.f; }
       if (!active_warp || kb1 <= kb0) return;     // (warp-uniform)
       tmem_ld8(taddr + (uint32_t)(8 * j), hi);
-      tmem_ld8(taddr + (uint32_t)(kTcRows + 8 * j), lo);
+      tmem_ld8(taddr + (uint32_t)(ROWS + 8 * j), lo);
 #pragma unroll
       for (int i = 0; i < 8; ++i) y[i] = hi[i] + lo[i];
       if (sw) {
         tmem_ld8(taddr + 256u + (uint32_t)(8 * j), hi);
-        tmem_ld8(taddr + 256u + (uint32_t)(kTcRows + 8 * j), lo);
+        tmem_ld8(taddr + 256u + (uint32_t)(ROWS + 8 * j), lo);
 #pragma unroll
         for (int i = 0; i < 8; ++i) u[i] = hi[i] + lo[i];
       }
@@ -196,7 +208,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
           for (int i = 0; i < 8; ++i) {
             const int t = 8 * j + i;
             if (t < T) {
-              float *pp = a.part + ((size_t)blockIdx.y * kTcRows + t) * Ntot;
+              float *pp = a.part + ((size_t)blockIdx.y * kTcRowsMax + t) * Ntot;
               __stcg(pp + col, y[i]);
               if (sw) __stcg(pp + a.Nseg + n, u[i]);
             }
@@ -204,7 +216,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
         }
       }
     } else {
-      Top2 *s_top = reinterpret_cast<Top2 *>(smem);   // [8 warps][88]: the stages are idle by now
+      Top2 *s_top = reinterpret_cast<Top2 *>(smem);   // [8 warps][128]: the stages are idle by now
       if (a.epi == EPI_ARGMAX) named_bar(3, 256);
       for (int j = 0; j < nblk; ++j) {
         float y[8], u[8];
@@ -237,7 +249,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
-            if (lane == 0) s_top[cw * kTcRows + t] = b;
+            if (lane == 0) s_top[cw * kTcRowsMax + t] = b;
           }
         }
       }
@@ -245,8 +257,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
         named_bar(3, 256);
         if (ctid < T) {
           Top2 b = s_top[ctid];
-          for (int w = 1; w < 8; ++w) b = top2_merge(b, s_top[w * kTcRows + ctid]);
-          a.amax[(size_t)blockIdx.x * kTcRows + ctid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+          for (int w = 1; w < 8; ++w) b = top2_merge(b, s_top[w * kTcRowsMax + ctid]);
+          a.amax[(size_t)blockIdx.x * kTcRowsMax + ctid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
         }
       }
     }
@@ -270,7 +282,7 @@ __global__ void __launch_bounds__(256) k_tc_reduce(const GemmTcArgs a) {
     const int t = idx / c4, col = (idx - t * c4) << 2;
     float4 y = make_float4(0.f, 0.f, 0.f, 0.f), u = y;
     for (int sp = 0; sp < a.S; ++sp) {
-      const float *pp = a.part + ((size_t)sp * kTcRows + t) * Ntot + col;
+      const float *pp = a.part + ((size_t)sp * kTcRowsMax + t) * Ntot + col;
       const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp));
       y.x += v.x; y.y += v.y; y.z += v.z; y.w += v.w;
       if (sw) {

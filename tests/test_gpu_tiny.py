@@ -279,11 +279,11 @@ def test_cache_full_clips_the_draft_length(tiny):
         e.close()
 
 
-@pytest.mark.parametrize("plen", [88, 89, 200, 333, 420, 451, 1500])
+@pytest.mark.parametrize("plen", [88, 128, 129, 200, 333, 420, 451, 1500])
 def test_long_context_attention_spans_blocks_and_rounds(tiny, plen):
     """Contexts of several hundred positions: every KV split holds more than one 32-key block.  The prompt pass
-    takes 88 rows at a time through the multi-row tensor-core GEMM (88: one full chunk; 89: a one-row tail; the
-    others: several chunks and a ragged tail) and writes the caches that the 16-row decode passes then read."""
+    takes 128 rows at a time through the multi-row tensor-core GEMM (88: a partial chunk; 128: one full chunk; 129: a
+    one-row tail; the others: several chunks and a ragged tail) and writes the caches that the 16-row decode passes then read."""
     from paper_2412_18910_b200 import Engine
     sh, w, prompt, m = tiny
     long_prompt = si.uniform_ids(5, "long%d" % plen, plen, sh.vocab)

@@ -42,7 +42,7 @@ def test_scalar_predictor_configuration_is_validated():
 def test_configurations_need_matrices_of_at_least_one_weight_box():
     """Prompts (every engine) and batches go through the multi-row tensor-core GEMM, whose weight boxes are 128 rows
     high: a model with a narrower matrix is refused at any batch size; the workspace of a batch-1 engine holds the
-    88-row scratch of its prompt pass."""
+    128-row scratch of its prompt pass."""
     import ctypes as C
     import paper_2412_18910_b200 as pkg
     L = pkg.lib()
@@ -52,4 +52,4 @@ def test_configurations_need_matrices_of_at_least_one_weight_box():
     tiny = (2, 256, 4, 64, 688, 4096, 1e4, 1e-6, 128, 8, 0)
     one = L.ada_workspace_bytes(C.byref(pkg.Config(*tiny, 1, 256, 64)))
     three = L.ada_workspace_bytes(C.byref(pkg.Config(*tiny, 3, 256, 64)))
-    assert one > 88 * (3 * 256) * 4 and three > one
+    assert one > 128 * (3 * 256) * 4 and three > one
