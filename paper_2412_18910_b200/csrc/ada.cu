@@ -518,8 +518,8 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
 
 void enqueue_ldlp(ada_ctx *x, int *d_n) {
   const ada_config &c = x->c;
-  dim3 g((c.ldlp_hidden + 7) / 8, x->B);
-  LAUNCH(x, k_ldlp_hidden, g, 256, 0, x->st, x->tok, x->feat, c.kv_capacity, x->embed, x->ldlp_w1, x->ldlp_b1,
+  dim3 g((c.ldlp_hidden + 7) / 8, x->B), g4((c.ldlp_hidden + 3) / 4, x->B);
+  LAUNCH(x, k_ldlp_hidden, g4, 128, 0, x->st, x->tok, x->feat, c.kv_capacity, x->embed, x->ldlp_w1, x->ldlp_b1,
          c.d_model, c.ldlp_hidden, x->ldlp_h);
   float *hin = x->ldlp_h, *hout = x->ldlp_h2;
   if (c.ldlp_mode == 1)
@@ -528,7 +528,7 @@ void enqueue_ldlp(ada_ctx *x, int *d_n) {
              x->ldlp_br + (size_t)blk * c.ldlp_hidden, c.ldlp_hidden);
       float *t = hin; hin = hout; hout = t;
     }
-  LAUNCH(x, k_ldlp_out, x->B, 32, 0, x->st, hin, x->ldlp_w2, x->ldlp_b2, c.ldlp_hidden, c.n_max, c.ldlp_mode, c.k_min,
+  LAUNCH(x, k_ldlp_out, x->B, 512, 0, x->st, hin, x->ldlp_w2, x->ldlp_b2, c.ldlp_hidden, c.n_max, c.ldlp_mode, c.k_min,
          c.kv_capacity, x->force_n_dev, x->has_force_n, x->ldlp_z, d_n, x->cnt);
 }
 

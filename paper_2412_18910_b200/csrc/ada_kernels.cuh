@@ -94,6 +94,15 @@ __device__ __forceinline__ float block_sum(float v, float *sh) {
   return t;
 }
 
+// 128-bit streaming load (read once: no level-1 allocation)
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
 // ---------------------------------------------------------------------------------------------
 // top-2 bookkeeping for the greedy choice: (v1, i1) best value / lowest index among equals, v2 second
 struct Top2 {
@@ -339,21 +348,43 @@ __global__ void k_eagle_input(const Pass *pass, const __nv_bfloat16 *embed, cons
 
 // ---------------------------------------------------------------------------------------------
 // Length predictor (Eq. 3), class-logit form.  Stage 1: hidden unit per warp:
-// h[b][u] = ReLU(W1[u] . [e(tok[len-2]) ; f[len-2]] + b1[u]).
-__global__ void k_ldlp_hidden(const SeqState *st, const int *tok, const float *feat, int cap,
-                              const __nv_bfloat16 *embed, const __nv_bfloat16 *w1, const __nv_bfloat16 *b1, int d,
-                              int hid, float *hbuf) {
+// h[b][u] = ReLU(W1[u] . [e(tok[len-2]) ; f[len-2]] + b1[u]).  The 2d weights of a unit are streamed with 128-bit
+// loads (8 bf16 per lane and step; d is a multiple of 64), all of a lane's loads of a step in flight together.
+__device__ __forceinline__ float dot8_bf16(uint4 w, uint4 x) {
+  const __nv_bfloat162 *wp = reinterpret_cast<const __nv_bfloat162 *>(&w), *xp = reinterpret_cast<const __nv_bfloat162 *>(&x);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 a = __bfloat1622float2(wp[i]), c = __bfloat1622float2(xp[i]);
+    s += a.x * c.x + a.y * c.y;
+  }
+  return s;
+}
+__device__ __forceinline__ float dot8_bf16_f32(uint4 w, float4 x0, float4 x1) {
+  const __nv_bfloat162 *wp = reinterpret_cast<const __nv_bfloat162 *>(&w);
+  const float2 a = __bfloat1622float2(wp[0]), b = __bfloat1622float2(wp[1]), c = __bfloat1622float2(wp[2]), e = __bfloat1622float2(wp[3]);
+  return (a.x * x0.x + a.y * x0.y) + (b.x * x0.z + b.y * x0.w) + (c.x * x1.x + c.y * x1.y) + (e.x * x1.z + e.y * x1.w);
+}
+__global__ void __launch_bounds__(128) k_ldlp_hidden(const SeqState *st, const int *tok, const float *feat, int cap,
+                                                     const __nv_bfloat16 *embed, const __nv_bfloat16 *w1, const __nv_bfloat16 *b1,
+                                                     int d, int hid, float *hbuf) {
   const int b = blockIdx.y;
   const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int p = st[b].len - 2;
   if (u >= hid || p < 0) return;
-  const __nv_bfloat16 *e = embed + (size_t)tok[(size_t)b * cap + p] * d;
-  const float *f = feat + ((size_t)b * cap + p) * d;
-  const __nv_bfloat16 *w = w1 + (size_t)u * 2 * d;
+  const uint4 *e8 = reinterpret_cast<const uint4 *>(embed + (size_t)tok[(size_t)b * cap + p] * d);
+  const float4 *f4 = reinterpret_cast<const float4 *>(feat + ((size_t)b * cap + p) * d);
+  const uint4 *we = reinterpret_cast<const uint4 *>(w1 + (size_t)u * 2 * d), *wf = we + (d >> 3);
   float s = 0.f;
-  for (int i = lane; i < d; i += 32) s += __bfloat162float(w[i]) * __bfloat162float(e[i]);
-  for (int i = lane; i < d; i += 32) s += __bfloat162float(w[d + i]) * f[i];
+  const int n8 = d >> 3;   // groups of 8 elements per half of the input
+#pragma unroll 8
+  for (int i = lane; i < n8; i += 32) {
+    const uint4 w_e = ldg_stream(we + i), w_f = ldg_stream(wf + i);
+    const uint4 xe = e8[i];
+    const float4 x0 = f4[2 * i], x1 = f4[2 * i + 1];
+    s += dot8_bf16(w_e, xe) + dot8_bf16_f32(w_f, x0, x1);
+  }
   s = warp_sum(s);
   if (lane == 0) hbuf[(size_t)b * hid + u] = fmaxf(s + __bfloat162float(b1[u]), 0.f);
 }
@@ -375,24 +406,27 @@ __global__ void k_ldlp_block(const SeqState *st, const float *hin, float *hout, 
 
 // Stage 2: z = W2 h + b2, then n = argmax + 1 (class form, lowest index among equals) or
 // n = clip(round-half-even(z_0), k_min, n_max) (scalar form, Eq. 3), then the override and the clip to the
-// cache capacity.  One warp per sequence.
-__global__ void k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 *w2, const __nv_bfloat16 *b2,
-                           int hid, int nmax, int mode, int kmin, int cap, const int *force_n, int has_force, float *zbuf,
-                           int *n_out, Counters *cnt) {
-  const int b = blockIdx.x, lane = threadIdx.x;
+// cache capacity.  One CTA per sequence, one warp per output (16 warps: n_max <= 15).
+__global__ void __launch_bounds__(512) k_ldlp_out(SeqState *st, const float *hbuf, const __nv_bfloat16 *w2, const __nv_bfloat16 *b2,
+                                                  int hid, int nmax, int mode, int kmin, int cap, const int *force_n, int has_force,
+                                                  float *zbuf, int *n_out, Counters *cnt) {
+  __shared__ float zs[16];
+  const int b = blockIdx.x, lane = threadIdx.x & 31, c = threadIdx.x >> 5;
   const int len = st[b].len;
-  if (len < 2) { if (lane == 0) { st[b].n = 0; if (n_out) n_out[b] = 0; } return; }
-  float best = -INFINITY;
-  int bi = 0;
+  if (len < 2) { if (threadIdx.x == 0) { st[b].n = 0; if (n_out) n_out[b] = 0; } return; }
   const int nz = mode == 0 ? nmax : 1;
-  for (int c = 0; c < nz; ++c) {
+  if (c < nz) {
     float s = 0.f;
     for (int i = lane; i < hid; i += 32) s += __bfloat162float(w2[(size_t)c * hid + i]) * hbuf[(size_t)b * hid + i];
     s = warp_sum(s) + __bfloat162float(b2[c]);
-    if (lane == 0) zbuf[b * 16 + c] = s;
-    if (s > best) { best = s; bi = c; }
+    if (lane == 0) { zs[c] = s; zbuf[b * 16 + c] = s; }
   }
-  if (lane == 0) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float best = -INFINITY;
+    int bi = 0;
+    for (int i = 0; i < nz; ++i)
+      if (zs[i] > best) { best = zs[i]; bi = i; }
     int n = bi + 1;
     if (mode != 0) n = (int)fminf(fmaxf(rintf(best), (float)kmin), (float)nmax);   // best = z_0
     if (has_force) n = force_n[b];
