@@ -60,7 +60,7 @@ struct ada_ctx {
   int host_force_n[ADA_MAX_BATCH];
   size_t part_floats;
   // persistent pass kernel (batch 1): device copies of the layer pointer tables and its scratch
-  int use_pass, n_sm, attn_splits;
+  int use_pass, n_sm;
   // tensor-core GEMM of the multi-row path (passes of up to 88 rows): tensor maps of every weight matrix and of
   // the activation planes, found by base pointer
   TensorMap128 *d_tcmaps;
@@ -246,7 +246,7 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->ac = w.take<bf16>(((F + 63) / 64) * 2048);
   x->fc = w.take<bf16>(((2 * d + 63) / 64) * 2048);
   x->ss_part = w.take<float>(256 * 16);
-  x->attn_part2 = w.take<float>(H * 8 * 16 * (hd + 2));
+  x->attn_part2 = w.take<float>(H * kPassMaxSplits * 16 * (hd + 2));
   x->attn_cnt = w.take<int>(H);
   x->amax2 = w.take<float4>(256 * 16);
   x->gbar = w.take<unsigned>(64);
@@ -311,12 +311,12 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
     LAUNCH(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, x->cnt);
-    LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
+    LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
   } else {
     LAUNCH(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, x->cnt);
-    LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx);
+           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
+    LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
   }
   });
 }
@@ -491,7 +491,7 @@ void run_pass(ada_ctx *x, int mode, int step, int with_lm, float *logits, int *t
   p.rope = x->rope;
   p.kpool = mode == 0 ? x->tk : x->dk; p.vpool = mode == 0 ? x->tv : x->dv;
   p.page_table = x->page_table; p.pages_per_seq = x->pages_per_seq; p.page_size = c.page_size;
-  p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt; p.attn_splits = x->attn_splits;
+  p.attn_part = x->attn_part2; p.attn_cnt = x->attn_cnt;
   p.amax = x->amax2; p.logits = logits; p.tok_out = tok_out; p.top_out = top_out; p.forced = forced;
   p.gbar = x->gbar; p.cnt = x->cnt;
   p.lp_out = (mode == 1 && with_lm && x->c.ddd_threshold < 0.f) ? x->dlp : nullptr; p.tok_logit = x->dfl;
@@ -557,16 +557,16 @@ void enqueue_verify(ada_ctx *x, int only_seq, float *d_logits) {
 
 // Multi-row passes over committed positions of one sequence, 128 rows per chunk: the target over positions
 // [p_begin, p_end) (cache rows and features), the draft head over those of them below d_end (each needs the token after
-// its position).  with_choice: the greedy choice after position p_end - 1 goes to chunk_tok.  Returns the rows of the
-// last chunk.
-int enqueue_chunks(ada_ctx *x, int seq, int p_begin, int p_end, int d_end, bool with_choice) {
+// its position).  with_choice: the greedy choice after position p_end - 1 goes to chunk_tok.  chunk: the sequence's
+// attention split size.  Returns the rows of the last chunk.
+int enqueue_chunks(ada_ctx *x, int seq, int p_begin, int p_end, int d_end, bool with_choice, int chunk) {
   const ada_config &c = x->c;
   int last_rows = 0;
   const int TM0 = x->TM;
   x->TM = kTcRowsMax;
   for (int p0 = p_begin; p0 < p_end; p0 += x->TM) {
     const int R = (p_end - p0 < x->TM) ? p_end - p0 : x->TM;
-    LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B);
+    LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, R, 0, x->B, chunk);
     target_rows(x);
     if (p0 + R == p_end) {  // the chunk that holds the last position: greedy choice after it
       if (with_choice) lm_head(x, x->xhi, x->xlo, 0, x->chunk_tok, x->vtop + x->B * (c.n_max + 1), nullptr, nullptr);
@@ -574,7 +574,7 @@ int enqueue_chunks(ada_ctx *x, int seq, int p_begin, int p_end, int d_end, bool 
     }
     const int Rd = (p0 + R <= d_end) ? R : (d_end - p0);
     if (Rd > 0) {
-      LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B);
+      LAUNCH(x, k_rows_chunk, 1, 32, 0, x->pass, x->tok, c.kv_capacity, seq, p0, Rd, 1, x->B, chunk);
       draft_rows(x, 0, false);
     }
   }
@@ -716,8 +716,6 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
     if (e == cudaSuccess && per_sm >= 1 && sms <= 256 && fits && max_clusters >= grid / 2) {
       x->use_pass = 1;
       x->n_sm = grid;
-      int sp = sms / cfg->n_heads;
-      x->attn_splits = sp < 1 ? 1 : (sp > 8 ? 8 : sp);
       std::vector<LayerPtrs> lp(cfg->n_layers);
       for (int l = 0; l < cfg->n_layers; ++l) {
         const LayerW &a = x->layers[l];
@@ -772,8 +770,9 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   if (m < 1) return fail(x, ADA_ERR_RANGE, "ada_prefill: empty prompt");
   if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
   LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
-  const int last_rows = enqueue_chunks(x, seq, 0, m, m - 1, true);
-  LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, x->chunk_tok + (last_rows - 1),
+  const int chunk = attn_chunk_for_prompt(m, c.kv_capacity);   // attention split size of this sequence from now on
+  const int last_rows = enqueue_chunks(x, seq, 0, m, m - 1, true, chunk);
+  LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, chunk, x->chunk_tok + (last_rows - 1),
          d_first_token);
   return finish(x, "ada_prefill");
 }
@@ -837,7 +836,7 @@ extern "C" int ada_label_positions(ada_ctx *x, int seq, int32_t j0, int32_t coun
   }
   // the sequence's own state again: cache rows and features from the first start position on, from the committed tokens
   LAUNCH(x, k_label_end, 1, 32, 0, x->st, seq, s0.len, s0.dlen, s0.n, s0.j_prev);
-  enqueue_chunks(x, seq, j0, s0.len - 1, s0.dlen, false);
+  enqueue_chunks(x, seq, j0, s0.len - 1, s0.dlen, false, s0.chunk);
   return finish(x, "ada_label_positions");
 }
 

@@ -2,9 +2,10 @@
 // head over one split of the cache, 16 query rows per CTA (row groups of a long pass across grid.z).
 //
 // Row r (absolute position pos0 + r) sees cache positions 0 .. pos0 + r: the whole history and the earlier rows
-// of its own block (every row's key and value are in the cache before this kernel runs).  The cache splits of a
-// sequence follow from its length alone (about 256 keys each, at most 8), so a short context is not cut into
-// slivers that cost more to set up and merge than to compute.  A warp takes 32-key blocks of the split, in halves
+// of its own block (every row's key and value are in the cache before this kernel runs).  The size of a sequence's
+// cache splits is fixed when its prompt is read (a quarter of the prompt and its expected continuation, at least an
+// eighth of the capacity), so the split a key falls in does not depend on the pass, and a short context is not cut
+// into slivers that cost more to set up and merge than to compute.  A warp takes 32-key blocks of the split, in halves
 // of 16 keys: one bulk copy brings a half's key rows and one its value rows (they are contiguous in the cache page)
 // into one of the warp's two buffers, so the next half is in flight while this one is computed -- scores = q k^T
 // as m16n8k16 products per 16 channels, online softmax on the accumulator fragments, weighted values as m16n8k8
@@ -31,7 +32,7 @@ template <int HD>
 __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
                                                    const __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
                                                    int page_size, int L, int layer, int H, float *part, int nrg,
-                                                   Counters *cnt) {
+                                                   int cap, Counters *cnt) {
   static_assert(HD == 64 || HD == 128, "head width");
   constexpr int CH = HD / 8;   // 16-byte chunks per row
   // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
@@ -41,7 +42,7 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
   const int row0 = pass->seq_row0[b];
   const int pos0 = pass->row_pos[row0];
   const int nkeys = pos0 + R;
-  const int chunk = attn_split_keys(nkeys);
+  const int chunk = attn_rows_chunk(pass->seq_chunk[b], cap);
   const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
   if (kbeg >= nkeys) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -33,7 +33,7 @@ struct SeqState {
   int j_prev;  // index of the pending token when the last verify started
   int n_emit;  // tokens emitted by the last accept
   int stale;   // draft head is behind by more rows than one pass holds
-  int pad;
+  int chunk;   // keys per attention split of this sequence's caches, fixed when its prompt was read (multiple of 32)
 };
 
 struct Counters {
@@ -54,6 +54,7 @@ struct Pass {
   int lm_out[kMaxRows];    // draft: output slot of LM row i
   int seq_row0[kMaxBatch];
   int seq_rows[kMaxBatch];
+  int seq_chunk[kMaxBatch];   // keys per attention split of the sequence (SeqState::chunk)
 };
 
 // KV-cache element: 16 bits per value like the weights, but IEEE half (11-bit significand) rather than bf16
@@ -281,18 +282,30 @@ __global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope
   }
 }
 
-// Keys per cache split of a sequence that holds nkeys keys (the result is a multiple of 32), and with it the number of splits.
-__host__ __device__ __forceinline__ int attn_split_keys(int nkeys) {
-  int nsp = (nkeys + 255) / 256;
-  nsp = nsp < 1 ? 1 : (nsp > kAttnSplits ? kAttnSplits : nsp);
-  const int chunk = (nkeys + nsp - 1) / nsp;
-  return ((chunk + 31) / 32) * 32;
+// Keys per attention split of a sequence whose prompt has m tokens, in a cache of `cap` positions: four splits cover
+// the prompt and the tokens expected after it (a quarter as many again, at least 256, within the capacity); at least
+// cap / 32 so that no sequence has more than 32 splits.  Chosen once per sequence, from its prompt alone: the split a
+// key falls in must not depend on the shape of the pass that reads it (a one-row step and a block of drafts then sum in
+// the same order).
+__host__ __device__ __forceinline__ int attn_chunk_for_prompt(int m, int cap) {
+  const int grow = m / 4 > 256 ? m / 4 : 256;
+  const int total = m + grow < cap ? m + grow : cap;
+  int chunk = ((total + 3) / 4 + 31) / 32 * 32;
+  const int least = ((cap + 31) / 32 + 31) / 32 * 32;
+  return chunk < least ? least : chunk;
+}
+// The multi-row attention kernel takes at most kAttnSplits splits per sequence: its split size is the sequence's, or
+// cap / kAttnSplits if that is larger (again independent of the pass).
+__host__ __device__ __forceinline__ int attn_rows_chunk(int seq_chunk, int cap) {
+  const int least = ((cap + kAttnSplits - 1) / kAttnSplits + 31) / 32 * 32;
+  const int c = seq_chunk < 32 ? 32 : seq_chunk;
+  return c < least ? least : c;
 }
 
 // Merge the cache splits in split order and emit the attention output row as hi/lo halves.
 template <int HD>
 __global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat16 *xhi, __nv_bfloat16 *xlo,
-                               int ldx) {
+                               int ldx, int cap) {
   const int hh = blockIdx.x, t = blockIdx.y;
   if (t >= pass->T) return;
   const int c = threadIdx.x;
@@ -300,7 +313,7 @@ __global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat1
   const size_t sstride = (size_t)kMaxRows * (HD + 2);
   const int b = pass->row_seq[t];
   const int nkeys = pass->row_pos[pass->seq_row0[b]] + pass->seq_rows[b];
-  const int chunk = attn_split_keys(nkeys);
+  const int chunk = attn_rows_chunk(pass->seq_chunk[b], cap);
   const int nsp = (nkeys + chunk - 1) / chunk;  // splits that held keys
   float M = -INFINITY;
   for (int s = 0; s < nsp; ++s) M = fmaxf(M, base[s * sstride + HD]);
@@ -459,6 +472,7 @@ __global__ void k_rows_verify(Pass *pass, SeqState *st, const int *tok, int cap,
   for (int b = 0; b < B; ++b) {
     pass->seq_row0[b] = T;
     pass->seq_rows[b] = 0;
+    pass->seq_chunk[b] = st[b].chunk;
     if (only_seq >= 0 && b != only_seq) continue;
     const int len = st[b].len;
     if (len < 1) continue;
@@ -479,9 +493,9 @@ __global__ void k_rows_verify(Pass *pass, SeqState *st, const int *tok, int cap,
 }
 
 // Prefill chunk: rows pos0..pos0+R-1 of sequence b, tokens from the committed-token array.
-__global__ void k_rows_chunk(Pass *pass, const int *tok, int cap, int b, int pos0, int R, int tok_shift, int B) {
+__global__ void k_rows_chunk(Pass *pass, const int *tok, int cap, int b, int pos0, int R, int tok_shift, int B, int chunk) {
   if (threadIdx.x != 0) return;
-  for (int i = 0; i < B; ++i) { pass->seq_row0[i] = 0; pass->seq_rows[i] = 0; }
+  for (int i = 0; i < B; ++i) { pass->seq_row0[i] = 0; pass->seq_rows[i] = 0; pass->seq_chunk[i] = chunk; }
   for (int i = 0; i < R; ++i) {
     pass->row_seq[i] = b;
     pass->row_pos[i] = pos0 + i;
@@ -505,6 +519,7 @@ __global__ void k_rows_draft(Pass *pass, SeqState *st, const int *tok, int cap, 
   for (int b = 0; b < B; ++b) {
     pass->seq_row0[b] = T;
     pass->seq_rows[b] = 0;
+    pass->seq_chunk[b] = st[b].chunk;
     const int n = st[b].n, j = st[b].len - 1;
     if (n <= step || j < 1) continue;
     if (step == 0) {
@@ -593,7 +608,7 @@ __global__ void k_copy_prompt(int *tok, int cap, int b, const int *prompt, int m
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < m; i += gridDim.x * blockDim.x)
     tok[(size_t)b * cap + i] = prompt[i];
 }
-__global__ void k_finish_prefill(SeqState *st, int *tok, int cap, int b, int m, const int *first_tok_slot,
+__global__ void k_finish_prefill(SeqState *st, int *tok, int cap, int b, int m, int chunk, const int *first_tok_slot,
                                  int *user_out) {
   if (threadIdx.x != 0) return;
   const int t = first_tok_slot[0];
@@ -601,6 +616,7 @@ __global__ void k_finish_prefill(SeqState *st, int *tok, int cap, int b, int m, 
   st[b].len = m + 1;
   st[b].dlen = m - 1;
   st[b].n = 0; st[b].k_acc = 0; st[b].j_prev = -1; st[b].n_emit = 0; st[b].stale = 0;
+  st[b].chunk = chunk;
   if (user_out) *user_out = t;
 }
 __global__ void k_rewind(SeqState *st, int b, int count, const int *forced_tok, int *draft, int nmax,

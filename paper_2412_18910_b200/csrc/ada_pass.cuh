@@ -59,7 +59,8 @@ constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA 
 // attention scratch lives where the activation buffers and the reduction buffer are (both idle
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
 constexpr int kAttnLoopBytes = 4 * 16 * 128 * 2 + 2 * 2 * 2 * 32 * 128 * 2;   // q hi, q lo, new k, v rows; two buffers of staged keys and values
-constexpr int kAttnPartBytes = 8 * 16 * 130 * 4 + 2 * 8 * 16 * 4;   // per-warp partial results, merge weights
+constexpr int kPassMaxSplits = 32;                // cache splits of a sequence at most (its split size is at least capacity / 32)
+constexpr int kAttnPartBytes = 8 * 16 * 130 * 4 + 8 * 16 * 4 + kPassMaxSplits * 16 * 4;   // per-warp partial results, merge weights
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
@@ -113,7 +114,6 @@ struct PassParams {
   const int *page_table; int pages_per_seq, page_size;
   float *attn_part;            // [H][splits][16][hd+2]
   int *attn_cnt;               // [H] arrival counters (zero between passes)
-  int attn_splits;
   // LM head
   float4 *amax;                // [grid][16]
   float *logits;               // optional [slot][V]
@@ -775,10 +775,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         // each (a block is contiguous in its cache page) into one of two buffers, so the copies of the next
         // round fly while this one is computed.
         const int R = T, pos0 = p.pass->row_pos[0], HD = p.hd, d = p.d, half = HD >> 1;
-        const int nkeys = pos0 + R, nsp = p.attn_splits;
-        int chunk = (nkeys + nsp - 1) / nsp;
-        chunk = ((chunk + 31) / 32) * 32;
+        // The cache is cut into splits of a size fixed per sequence when its prompt was read (a multiple of 32 keys), so
+        // the split a key falls in, and with it every sum of this phase, does not depend on how many rows a pass holds:
+        // a row's result is the same bit for bit in a one-row pass and in a block of drafts.
         const int b = p.pass->row_seq[0];
+        const int nkeys = pos0 + R, chunk = max(32, p.pass->seq_chunk[b]);
+        const int nsp = min(kPassMaxSplits, (nkeys + chunk - 1) / chunk);
         __half *qh_s = reinterpret_cast<__half *>(xbuf);                              // q hi [16][128], 16-byte chunks XORed with row & 7
         __half *ql_s = qh_s + 16 * 128;                                              // q lo, same layout
         __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(ql_s + 16 * 128);    // new rows, rotated [16][128]
@@ -786,7 +788,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         __nv_bfloat16 *stg = v_s + 16 * 128;                                         // [2 buffers][K, V][2 blocks][32 keys][128]
         float *part_s = reinterpret_cast<float *>(xbuf);                              // [8 warps][16 rows][130], reuses the above
         float *lw_s = part_s + 8 * 16 * 130;                                          // [8 warps][16 rows] merge weights
-        float *wgt = lw_s + 8 * 16;                                                   // [8 splits][16 rows] (cross-CTA merge)
+        float *wgt = lw_s + 8 * 16;                                                   // [splits][16 rows] (cross-CTA merge)
         const int g8r = lane >> 2, t4 = lane & 3;
         const int bw = cw >> 2, kq = cw & 3;
         const size_t head_stride = (size_t)p.page_size * HD;
@@ -998,35 +1000,62 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const int r = ctid;
               const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2);
               const size_t sst = (size_t)16 * (HD + 2);
-              float ms[8], ls[8];
+              // (eight splits at a time, their loads in flight together; more than eight splits only in long contexts)
+              float M = -INFINITY, lo = 0.f;
+              if (nsp <= 8) {   // one batch of loads serves both passes
+                float ms[8], ls[8];
 #pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) {
-                ms[s2] = s2 < nsp ? __ldcg(gp + s2 * sst + HD) : -INFINITY;
-                ls[s2] = s2 < nsp ? __ldcg(gp + s2 * sst + HD + 1) : 0.f;
+                for (int u = 0; u < 8; ++u) {
+                  ms[u] = u < nsp ? __ldcg(gp + u * sst + HD) : -INFINITY;
+                  ls[u] = u < nsp ? __ldcg(gp + u * sst + HD + 1) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) M = fmaxf(M, ms[u]);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const float e = ms[u] > -INFINITY ? __expf(ms[u] - M) : 0.f;
+                  if (u < nsp) wgt[u * 16 + r] = e;
+                  lo += ls[u] * e;
+                }
+              } else {
+                for (int s0 = 0; s0 < nsp; s0 += 8) {
+                  float ms[8];
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) ms[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst + HD) : -INFINITY;
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) M = fmaxf(M, ms[u]);
+                }
+                for (int s0 = 0; s0 < nsp; s0 += 8) {
+                  float ms[8], ls[8];
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) {
+                    ms[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst + HD) : -INFINITY;
+                    ls[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst + HD + 1) : 0.f;
+                  }
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) {
+                    const float e = ms[u] > -INFINITY ? __expf(ms[u] - M) : 0.f;
+                    if (s0 + u < nsp) wgt[(s0 + u) * 16 + r] = e;
+                    lo += ls[u] * e;
+                  }
+                }
               }
-              float M = -INFINITY;
-#pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) M = fmaxf(M, ms[s2]);
-              float lo = 0.f;
-#pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) {
-                ms[s2] = ms[s2] > -INFINITY ? __expf(ms[s2] - M) : 0.f;
-                lo += ls[s2] * ms[s2];
-              }
-#pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) wgt[s2 * 16 + r] = ms[s2] / lo;
+              const float inv = 1.f / lo;
+              for (int s2 = 0; s2 < nsp; ++s2) wgt[s2 * 16 + r] *= inv;
             }
             named_bar(3, kNumCWarps * 32);
             for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
               const int r = i / HD, c = i - r * HD;
               const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2) + c;
               const size_t sst = (size_t)16 * (HD + 2);
-              float ov[8];
-#pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) ov[s2] = s2 < nsp ? __ldcg(gp + s2 * sst) : 0.f;
               float oo = 0.f;
+              for (int s0 = 0; s0 < nsp; s0 += 8) {
+                float ov[8];
 #pragma unroll
-              for (int s2 = 0; s2 < 8; ++s2) oo += ov[s2] * wgt[s2 * 16 + r];
+                for (int u = 0; u < 8; ++u) ov[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst) : 0.f;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) oo += s0 + u < nsp ? ov[u] * wgt[(s0 + u) * 16 + r] : 0.f;
+              }
               xstore(p.at, r, hh * HD + c, oo);
             }
             if (ctid == 0) p.attn_cnt[hh] = 0;

@@ -191,3 +191,42 @@ def test_full_width_ddd_stopping_rule_against_the_live_oracle():
     assert not res["failures"], res["failures"]
     assert res["exempt"] <= 2
     assert c["n_draft"] > c["n_target"]          # drafts did grow past n = 1
+
+
+def test_block_verify_equals_one_row_steps_bit_for_bit():
+    """Lossless on the GPU itself, at the 7B widths (two layers): the greedy stream of plain one-row steps, then
+    teacher-forced blocks of n + 1 rows over the same positions.  Every draft must be accepted and the features of every
+    position must be the same bit for bit: no sum in the pass depends on how many rows share it (the attention splits
+    of a sequence are fixed when its prompt is read).  The run crosses several split and page boundaries."""
+    from paper_2412_18910_b200 import Engine
+    sh = si.scaled(si.SHAPES["7b"], n_layers=2)
+    w = si.make_weights(sh)
+    prompt = si.make_prompts(sh)[0][:300]
+    e = Engine(sh, w, max_batch=1, kv_capacity=sh.kv_capacity)
+    try:
+        feat = e.ada_debug_buffer(0, torch.float32, (1, sh.kv_capacity, sh.d_model))
+        new = 264
+        first = e.prefill(0, prompt)
+        e.ada_force_n([0])
+        stream = [first]
+        while len(stream) < new + sh.n_max + 2:
+            stream.extend(e.step()["emitted"][0])
+        f_ar = feat[0, : len(prompt) + new].clone()
+        st = torch.tensor(stream + [0] * sh.n_max, dtype=torch.int32, device=e.dev)
+        for n in (3, sh.n_max):
+            assert e.prefill(0, prompt) == first
+            e.ada_force_n([n])
+            off, iters = 1, 0
+            while off + n + 1 <= new:
+                e.ada_force_draft(st[off: off + sh.n_max].view(1, sh.n_max))
+                g = e.step()
+                assert g["k"][0] == n and g["emitted"][0] == stream[off: off + n + 1], (n, iters, off)
+                off += n + 1
+                iters += 1
+            assert iters >= 20
+            assert torch.equal(feat[0, : len(prompt) + off - 1], f_ar[: len(prompt) + off - 1])
+        e.ada_force_n(None)
+        e.ada_force_draft(None)
+        assert e.ada_get_counters()["status"] == 0
+    finally:
+        e.close()
