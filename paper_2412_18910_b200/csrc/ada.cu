@@ -49,7 +49,7 @@ struct ada_ctx {
   SeqState *st;                     // [B]
   Counters *cnt;
   Pass *pass;
-  float *h, *qkv, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z, *dlp, *dfl, *dcum;
+  float *h, *qkv, *ss_rows, *qrot, *attn_part, *gemm_part, *ldlp_h, *ldlp_h2, *ldlp_z, *dlp, *dfl, *dcum;
   bf16 *xhi, *xlo, *x2hi, *x2lo;    // [TP][ldx], [TP][ldx2]
   int ldx, ldx2;
   float4 *amax;
@@ -133,6 +133,7 @@ bool config_ok(const ada_config *c) {
   if (c->n_layers < 1 || c->n_layers > ADA_MAX_LAYERS) return false;
   if (c->head_dim != 64 && c->head_dim != 128) return false;
   if (c->n_heads < 1 || c->d_model != c->n_heads * c->head_dim) return false;
+  if (c->d_model > 1024 * kSsSegs) return false;   // the rows' sums of squares are kept per 1024-column segment
   if (c->d_model % 64 || c->d_ffn % 16 || c->d_ffn < 16 || c->vocab % 16 || c->vocab < 16) return false;
   if (c->ldlp_hidden < 1 || c->n_max < 1 || c->n_max > ADA_MAX_NMAX) return false;
   if (c->ldlp_mode != 0 && c->ldlp_mode != 1) return false;
@@ -171,7 +172,7 @@ int tc_tiles(int epi, int nseg, int Nseg) { return epi == EPI_SWIGLU ? (Nseg + 1
 size_t part_need_tc(int epi, int nseg, int Nseg, int K) {
   const int S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tc_tiles(epi, nseg, Nseg), K);
   const size_t Ntot = epi == EPI_SWIGLU ? 2 * (size_t)Nseg : (size_t)nseg * Nseg;
-  return S > 1 ? (size_t)S * kTcRowsMax * Ntot : 0;
+  return epi == EPI_ARGMAX ? 0 : (size_t)S * kTcRowsMax * Ntot;   // (every GEMM but the LM head leaves its sums here)
 }
 
 // Lays the workspace out; with base == nullptr only measures it.
@@ -196,7 +197,8 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   x->cnt = w.take<Counters>(1);
   x->pass = w.take<Pass>(1);
   x->h = w.take<float>(TP * d);
-  x->qkv = w.take<float>(TP * 3 * d);
+  x->qkv = w.take<float>(16 * 3 * d);   // the persistent pass kernel's q, k, v rows
+  x->ss_rows = w.take<float>(TP * kSsSegs);
   x->qrot = w.take<float>(TP * d);
   x->attn_part = w.take<float>(H * kAttnSplits * (size_t)kMaxRows * (hd + 2));
   const size_t ldx = 2 * d, ldx2 = ((F + 63) / 64) * 64 > d ? ((F + 63) / 64) * 64 : d;
@@ -254,11 +256,22 @@ size_t carve(ada_ctx *x, const ada_config *c, char *base) {
   return (w.off + 255) & ~(size_t)255;
 }
 
-// Y = X W^T with one of the epilogues.  W0..W2: row segments (STORE) or gate/up (SWIGLU).  False (with the context's
-// error text set) if an operand has no tensor map; every operand of the path is registered at initialisation.
+// What follows a GEMM's sums (the reduction kernel launched after it).
+struct Reduce {
+  enum Kind { QKV_ROPE, H, SWIGLU, NONE } kind;
+  // H: residual add or plain store, and the norm whose input planes are written (null: none)
+  int resid; const bf16 *gain;
+  // QKV_ROPE: the cache the rows go to
+  bf16 *kpool, *vpool; int L, layer;
+};
+
+// Sums of X W^T into the scratch buffer (tensor-core GEMM, K splits), then the reduction kernel `r`; the LM head
+// (EPI_ARGMAX, r.kind NONE) reduces the greedy choice itself.  W0..W2: row segments (STORE) or gate/up (SWIGLU).
+// False (with the context's error text set) if an operand has no tensor map; every operand of the path is registered
+// at initialisation.
 bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, int nseg, int Nseg, int K,
-          const bf16 *Xhi, const bf16 *Xlo, float *Y, int ldy, bf16 *Ohi, bf16 *Olo, int ldo, float *logits,
-          int use_lm_rows) {
+          const bf16 *Xhi, const bf16 *Xlo, const Reduce &r, float *logits, int use_lm_rows) {
+  const ada_config &c = x->c;
   GemmTcArgs t;
   memset(&t, 0, sizeof(t));
   const bf16 *Ws[3] = {W0, W1, W2};
@@ -284,18 +297,34 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   t.epi = epi; t.nseg = nseg; t.Nseg = Nseg; t.K = K;
   const int tiles = tc_tiles(epi, nseg, Nseg);
   t.S = epi == EPI_ARGMAX ? 1 : plan_tc_splits(tiles, K);
-  t.Y = Y; t.ldy = ldy; t.Ohi = Ohi; t.Olo = Olo; t.ldo = ldo;
+  t.to_part = epi != EPI_ARGMAX;
   t.part = x->gemm_part;
-  t.logits = logits; t.ldl = x->c.vocab; t.amax = x->amax;
+  t.logits = logits; t.ldl = c.vocab; t.amax = x->amax;
   t.pass = x->pass; t.use_lm_rows = use_lm_rows; t.cnts = x->cnt;
+  const int rows = wide ? kTcRowsMax : kTcRows;
+  const int d = c.d_model;
   const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
   timed(x, 0, wb, [&] {
     if (wide) LAUNCH(x, k_gemm_tc<kTcRowsMax>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRowsMax>::kSmemBytes, t);
     else LAUNCH(x, k_gemm_tc<kTcRows>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRows>::kSmemBytes, t);
-    if (t.S > 1) {   // the splits' partial sums, added in split order, then the epilogue
-      const int ncol = epi == EPI_SWIGLU ? Nseg : nseg * Nseg;
-      const int blocks = ((wide ? kTcRowsMax : kTcRows) * (ncol / 4) + 255) / 256;
-      LAUNCH(x, k_tc_reduce, blocks < 1184 ? blocks : 1184, 256, 0, t);
+    if (r.kind == Reduce::H) {
+      ReduceHArgs a;
+      a.part = x->gemm_part; a.S = t.S; a.Ntot = Nseg; a.h = x->h; a.d = d; a.resid = r.resid; a.gain = r.gain;
+      a.xhi = x->xhi; a.xlo = x->xlo; a.ldx = x->ldx; a.ss_part = x->ss_rows; a.pass = x->pass;
+      LAUNCH(x, k_reduce_h, dim3((d + 1023) / 1024, rows), 256, 0, a);
+    } else if (r.kind == Reduce::QKV_ROPE) {
+      ReduceQkvArgs a;
+      a.part = x->gemm_part; a.S = t.S; a.ss_part = x->ss_rows; a.eps = c.rms_eps; a.rope = x->rope; a.qout = x->qrot;
+      a.kpool = r.kpool; a.vpool = r.vpool; a.page_table = x->page_table; a.pages_per_seq = x->pages_per_seq;
+      a.page_size = c.page_size; a.L = r.L; a.layer = r.layer; a.H = c.n_heads; a.hd = c.head_dim;
+      a.qscale = 1.0f / sqrtf((float)c.head_dim); a.pass = x->pass;
+      LAUNCH(x, k_reduce_qkv, dim3((c.n_heads * (c.head_dim / 2) + 255) / 256, rows), 256, 0, a);
+    } else if (r.kind == Reduce::SWIGLU) {
+      ReduceSwigluArgs a;
+      a.part = x->gemm_part; a.S = t.S; a.F = Nseg; a.ss_part = x->ss_rows; a.eps = c.rms_eps; a.d = d;
+      a.ohi = x->x2hi; a.olo = x->x2lo; a.ldo = x->ldx2; a.pass = x->pass;
+      const int blocks = (rows * (Nseg / 4) + 255) / 256;
+      LAUNCH(x, k_reduce_swiglu, blocks < 1184 ? blocks : 1184, 256, 0, a);
     }
   });
   return true;
@@ -321,26 +350,30 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   });
 }
 
-// One pre-norm decoder block over the rows of x->pass; residual stream in x->h.
-void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L, int layer) {
+// One pre-norm decoder block over the rows of x->pass.  On entry the residual stream is in x->h, the planes hold
+// split(h * norm_attn gain) and the rows' sums of squares are in x->ss_rows (written by whatever produced h); on exit
+// the same holds for `next_gain`, the norm that follows the block (null: none, planes are left alone).
+void decoder_block(ada_ctx *x, const LayerW &w, bf16 *kpool, bf16 *vpool, int L, int layer, const bf16 *next_gain) {
   const ada_config &c = x->c;
   const int d = c.d_model, F = c.d_ffn;
-  LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.na, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
-  gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, x->qkv, 3 * d, nullptr, nullptr, 0, nullptr, 0);
-  LAUNCH(x, k_rope_kv, x->TM, 256, 0, x->pass, x->qkv, x->rope, x->qrot, kpool, vpool, x->page_table,
-         x->pages_per_seq, c.page_size, L, layer, c.n_heads, c.head_dim, 1.0f / sqrtf((float)c.head_dim));
+  Reduce qkv{Reduce::QKV_ROPE, 0, nullptr, kpool, vpool, L, layer};
+  gemm(x, EPI_STORE, w.wq, w.wk, w.wv, 3, d, d, x->xhi, x->xlo, qkv, nullptr, 0);
   attention(x, kpool, vpool, L, layer);
-  gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
-  LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, w.nm, c.rms_eps, d, x->xhi, x->xlo, x->ldx, (float *)nullptr, 0);
-  gemm(x, EPI_SWIGLU, w.wg, w.wu, nullptr, 1, F, d, x->xhi, x->xlo, nullptr, 0, x->x2hi, x->x2lo, x->ldx2, nullptr, 0);
-  gemm(x, EPI_RESID, w.wd, nullptr, nullptr, 1, d, F, x->x2hi, x->x2lo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
+  Reduce o{Reduce::H, 1, w.nm, nullptr, nullptr, 0, 0};
+  gemm(x, EPI_RESID, w.wo, nullptr, nullptr, 1, d, d, x->xhi, x->xlo, o, nullptr, 0);
+  Reduce sw{Reduce::SWIGLU, 0, nullptr, nullptr, nullptr, 0, 0};
+  gemm(x, EPI_SWIGLU, w.wg, w.wu, nullptr, 1, F, d, x->xhi, x->xlo, sw, nullptr, 0);
+  Reduce down{Reduce::H, 1, next_gain, nullptr, nullptr, 0, 0};
+  gemm(x, EPI_RESID, w.wd, nullptr, nullptr, 1, d, F, x->x2hi, x->x2lo, down, nullptr, 0);
 }
 
 // Target over the rows of x->pass: embedding, all layers, final norm (features kept per position).
 void target_rows(ada_ctx *x) {
   const ada_config &c = x->c;
-  LAUNCH(x, k_embed, x->TM, 256, 0, x->pass, x->embed, x->h, c.d_model);
-  for (int l = 0; l < c.n_layers; ++l) decoder_block(x, x->layers[l], x->tk, x->tv, c.n_layers, l);
+  LAUNCH(x, k_embed, x->TM, 256, 0, x->pass, x->embed, x->h, c.d_model, x->layers[0].na, x->xhi, x->xlo, x->ldx, x->ss_rows,
+         kSsSegs);
+  for (int l = 0; l < c.n_layers; ++l)
+    decoder_block(x, x->layers[l], x->tk, x->tv, c.n_layers, l, l + 1 < c.n_layers ? x->layers[l + 1].na : nullptr);
   LAUNCH(x, k_rmsnorm, x->TM, 256, 0, x->pass, x->h, x->final_norm, c.rms_eps, c.d_model, x->xhi, x->xlo, x->ldx,
          x->feat, c.kv_capacity);
 }
@@ -349,8 +382,8 @@ void target_rows(ada_ctx *x) {
 void lm_head(ada_ctx *x, const bf16 *Xhi, const bf16 *Xlo, int use_lm_rows, int *tok_out, float2 *top_out,
              const int *forced, float *logits) {
   const ada_config &c = x->c;
-  gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, nullptr, 0, nullptr, nullptr, 0,
-       logits, use_lm_rows);
+  Reduce none{Reduce::NONE, 0, nullptr, nullptr, nullptr, 0, 0};
+  gemm(x, EPI_ARGMAX, x->lm_head, nullptr, nullptr, 1, c.vocab, c.d_model, Xhi, Xlo, none, logits, use_lm_rows);
   LAUNCH(x, k_argmax_final, x->TM, 32, 0, x->amax, (c.vocab + 255) / 256, kTcRowsMax, x->pass, use_lm_rows, tok_out, top_out,
          forced);
 }
@@ -361,8 +394,9 @@ void draft_rows(ada_ctx *x, int step, bool with_lm) {
   const int d = c.d_model;
   LAUNCH(x, k_eagle_input, x->TM, 256, 0, x->pass, x->embed, x->feat, c.kv_capacity, x->dfeat, c.n_max, step, d, x->xhi,
          x->xlo, x->ldx);
-  gemm(x, EPI_STORE, x->eagle_fc, nullptr, nullptr, 1, d, 2 * d, x->xhi, x->xlo, x->h, d, nullptr, nullptr, 0, nullptr, 0);
-  decoder_block(x, x->eagle, x->dk, x->dv, 1, 0);
+  Reduce fc{Reduce::H, 0, x->eagle.na, nullptr, nullptr, 0, 0};   // h = fc([e ; f]), planes for the head's layer
+  gemm(x, EPI_STORE, x->eagle_fc, nullptr, nullptr, 1, d, 2 * d, x->xhi, x->xlo, fc, nullptr, 0);
+  decoder_block(x, x->eagle, x->dk, x->dv, 1, 0, nullptr);
   if (with_lm) {
     LAUNCH(x, k_split_lm_rows, x->B, 256, 0, x->pass, x->h, d, x->x2hi, x->x2lo, x->ldx2, x->dfeat, c.n_max, step);
     lm_head(x, x->x2hi, x->x2lo, 1, x->draft, x->dtop, x->force_draft, nullptr);

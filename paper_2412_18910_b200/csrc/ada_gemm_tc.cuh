@@ -18,9 +18,10 @@
 //   warps 4..11  epilogue: thread = one weight row (tensor-memory lane), tcgen05.ld eight pass rows at a time,
 //            column t (hi) + column ROWS + t (lo)
 //
-// K splits leave their partial sums in a scratch buffer and k_tc_reduce, launched next, adds them in split order
-// and runs the epilogue over the whole grid (a last-arriving CTA per tile doing this alone was measured to take
-// longer than the products: 16 CTAs walking 9 x 88 x 256 values each).  Every output element depends only on its
+// Every CTA leaves its sums in a scratch buffer and a reduction kernel, launched next, adds the K splits in split
+// order and runs everything up to the next GEMM's input over the whole grid (k_reduce_h, k_reduce_qkv,
+// k_reduce_swiglu; a last-arriving CTA per tile doing the sum alone was measured to take longer than the products:
+// 16 CTAs walking 9 x 88 x 256 values each).  Only the LM head is never split: its CTAs reduce the greedy choice.  Every output element depends only on its
 // own input row and on the fixed split of K.  Every wait is bounded.
 #pragma once
 #include "ada_pass.cuh"
@@ -49,11 +50,10 @@ struct TcShape {
 struct GemmTcArgs {
   const TensorMap128 *wmap[3];   // box {64 k, 128 rows}; STORE: up to 3 row segments; SWIGLU: gate, up
   const TensorMap128 *xhi_map, *xlo_map;   // planes [128][ld]: box {64 k, ROWS rows}
-  int epi;                    // EPI_STORE / EPI_RESID / EPI_SWIGLU / EPI_ARGMAX
+  int epi;                    // EPI_STORE / EPI_RESID / EPI_SWIGLU (sums go to `part`) / EPI_ARGMAX
   int nseg, Nseg, K;
   int S;                      // K splits (grid.y)
-  float *Y; int ldy;          // STORE / RESID target
-  __nv_bfloat16 *Ohi, *Olo; int ldo;   // SWIGLU target planes
+  int to_part;                // the CTA leaves its sums in `part` for a reduction kernel (always, except ARGMAX)
   float *part;                // [S][128][Ntot] partial sums (S > 1; ARGMAX is never split)
   float *logits; int ldl;     // ARGMAX: optional logits [slot][ldl]
   float4 *amax;               // ARGMAX: [tiles][128] (v1, i1, v2)
@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
       }
     };
 
-    if (a.S > 1) {
+    if (a.to_part) {
       for (int j = 0; j < nblk; ++j) {
         float y[8], u[8];
         from_tmem(j, y, u);
@@ -215,9 +215,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
           }
         }
       }
-    } else {
+    } else {   // LM head (never split): the warp's two largest logits of every pass row, merged per CTA
       Top2 *s_top = reinterpret_cast<Top2 *>(smem);   // [8 warps][128]: the stages are idle by now
-      if (a.epi == EPI_ARGMAX) named_bar(3, 256);
+      named_bar(3, 256);
       for (int j = 0; j < nblk; ++j) {
         float y[8], u[8];
         from_tmem(j, y, u);
@@ -225,41 +225,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
         for (int i = 0; i < 8; ++i) {
           const int t = 8 * j + i;
           if (t >= T) continue;     // (uniform over the CTA)
-          if (a.epi == EPI_STORE) {
-            if (valid) a.Y[(size_t)t * a.ldy + col] = y[i];
-          } else if (a.epi == EPI_RESID) {
-            if (valid) a.Y[(size_t)t * a.ldy + col] += y[i];
-          } else if (sw) {
-            if (valid) {
-              const float o = (y[i] / (1.f + __expf(-y[i]))) * u[i];
-              __nv_bfloat16 hi, lo;
-              split_bf16(o, hi, lo);
-              a.Ohi[(size_t)t * a.ldo + n] = hi;
-              a.Olo[(size_t)t * a.ldo + n] = lo;
+          Top2 b;
+          b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
+          if (valid) {
+            if (a.logits) {
+              const int slot = a.use_lm_rows ? a.pass->lm_out[t] : a.pass->row_out[t];
+              a.logits[(size_t)slot * a.ldl + n] = y[i];
             }
-          } else {   // EPI_ARGMAX: the warp's two largest logits of this pass row
-            Top2 b;
-            b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
-            if (valid) {
-              if (a.logits) {
-                const int slot = a.use_lm_rows ? a.pass->lm_out[t] : a.pass->row_out[t];
-                a.logits[(size_t)slot * a.ldl + n] = y[i];
-              }
-              b.v1 = y[i]; b.i1 = n;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
-            if (lane == 0) s_top[cw * kTcRowsMax + t] = b;
+            b.v1 = y[i]; b.i1 = n;
           }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
+          if (lane == 0) s_top[cw * kTcRowsMax + t] = b;
         }
       }
-      if (a.epi == EPI_ARGMAX) {
-        named_bar(3, 256);
-        if (ctid < T) {
-          Top2 b = s_top[ctid];
-          for (int w = 1; w < 8; ++w) b = top2_merge(b, s_top[w * kTcRowsMax + ctid]);
-          a.amax[(size_t)blockIdx.x * kTcRowsMax + ctid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
-        }
+      named_bar(3, 256);
+      if (ctid < T) {
+        Top2 b = s_top[ctid];
+        for (int w = 1; w < 8; ++w) b = top2_merge(b, s_top[w * kTcRowsMax + ctid]);
+        a.amax[(size_t)blockIdx.x * kTcRowsMax + ctid] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
       }
     }
   }
@@ -271,43 +255,151 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   if (warp == 2) tmem_dealloc(tmem_base, kTcTmemCols);
 }
 
-// Sum of the K splits' partial sums in split order, then the epilogue; one thread per (pass row, 4 output columns).
-__global__ void __launch_bounds__(256) k_tc_reduce(const GemmTcArgs a) {
-  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
-  const bool sw = a.epi == EPI_SWIGLU;
-  const int Ntot = sw ? 2 * a.Nseg : a.nseg * a.Nseg;
-  const int ncol = sw ? a.Nseg : Ntot;           // output columns
-  const int c4 = ncol >> 2;                       // (column counts are multiples of 16)
+// ---------------------------------------------------------------------------------------------
+// Reduction kernels: the K splits' partial sums added in split order, then everything that follows the GEMM up to
+// the next GEMM's input, so that no row-wise kernel runs between two GEMMs of a layer.
+//
+// RMSNorm is folded around the GEMMs: the kernel that produces the residual stream h also stores the next GEMM's input
+// planes split(h * gain) and, per row, partial sums of squares of h (one per 1024-column segment, kSsSegs slots per
+// row); the kernel that consumes the next GEMM's sums multiplies them by 1 / rms(row).
+constexpr int kSsSegs = 8;   // segments of 1024 columns per row (d <= 8192)
+
+__device__ __forceinline__ float inv_rms_of(const float *ss_part, int t, int d, float eps) {
+  const int nseg = (d + 1023) >> 10;
+  float s = 0.f;
+  for (int i = 0; i < nseg; ++i) s += __ldcg(ss_part + (size_t)t * kSsSegs + i);   // fixed order
+  return rsqrtf(s / (float)d + eps);
+}
+
+// h = (resid ? h : 0) + sum of the splits; planes = split(h * gain) (if gain); partial sums of squares.
+// Block (segment of 1024 columns, pass row); thread = 4 columns.
+struct ReduceHArgs {
+  const float *part; int S, Ntot;      // [S][128][Ntot]
+  float *h; int d;                      // residual stream [rows][d]
+  int resid;
+  const __nv_bfloat16 *gain;            // norm that follows (null: none)
+  __nv_bfloat16 *xhi, *xlo; int ldx;   // planes of the next GEMM's input
+  float *ss_part;                       // [rows][kSsSegs]
+  const Pass *pass;
+};
+__global__ void __launch_bounds__(256) k_reduce_h(const ReduceHArgs a) {
+  __shared__ float sh[32];
+  const int t = blockIdx.y, seg = blockIdx.x;
+  if (t >= a.pass->T) return;
+  const int col = seg * 1024 + threadIdx.x * 4;
+  float ss = 0.f;
+  if (col < a.d) {
+    float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp = 0; sp < a.S; ++sp) {
+      const float4 v = __ldcg(reinterpret_cast<const float4 *>(a.part + ((size_t)sp * kTcRowsMax + t) * a.Ntot + col));
+      y.x += v.x; y.y += v.y; y.z += v.z; y.w += v.w;
+    }
+    float4 *hp = reinterpret_cast<float4 *>(a.h + (size_t)t * a.d + col);
+    float4 hv = y;
+    if (a.resid) {
+      const float4 o = *hp;
+      hv.x = o.x + y.x; hv.y = o.y + y.y; hv.z = o.z + y.z; hv.w = o.w + y.w;
+    }
+    *hp = hv;
+    ss = (hv.x * hv.x + hv.y * hv.y) + (hv.z * hv.z + hv.w * hv.w);
+    if (a.gain) {
+      const uint2 gg = *reinterpret_cast<const uint2 *>(a.gain + col);
+      const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x), g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
+      const float x[4] = {hv.x * __bfloat162float(g01.x), hv.y * __bfloat162float(g01.y), hv.z * __bfloat162float(g23.x),
+                          hv.w * __bfloat162float(g23.y)};
+      __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) split_bf16(x[i], hi[i], lo[i]);
+      uint2 ph, pl;
+      ph.x = (uint32_t)__bfloat16_as_ushort(hi[0]) | ((uint32_t)__bfloat16_as_ushort(hi[1]) << 16);
+      ph.y = (uint32_t)__bfloat16_as_ushort(hi[2]) | ((uint32_t)__bfloat16_as_ushort(hi[3]) << 16);
+      pl.x = (uint32_t)__bfloat16_as_ushort(lo[0]) | ((uint32_t)__bfloat16_as_ushort(lo[1]) << 16);
+      pl.y = (uint32_t)__bfloat16_as_ushort(lo[2]) | ((uint32_t)__bfloat16_as_ushort(lo[3]) << 16);
+      *reinterpret_cast<uint2 *>(a.xhi + (size_t)t * a.ldx + col) = ph;
+      *reinterpret_cast<uint2 *>(a.xlo + (size_t)t * a.ldx + col) = pl;
+    }
+  }
+  if (a.gain) {
+    ss = block_sum(ss, sh);
+    if (threadIdx.x == 0) a.ss_part[(size_t)t * kSsSegs + seg] = ss;
+  }
+}
+
+// QKV: sums of the splits times 1 / rms(row), then rotary embedding of q and k (rotate-half pairing), q scaled by
+// 1 / sqrt(hd) to qout, k and v as 16-bit cache elements into the paged pools (key rows with their 16-byte chunks XORed
+// by slot & 7).  Block (group of 256 (head, i) pairs, pass row); thread = one pair (i, i + hd / 2) of one head.
+struct ReduceQkvArgs {
+  const float *part; int S;            // [S][128][3 d]
+  const float *ss_part; float eps;
+  const float2 *rope; float *qout;
+  __nv_bfloat16 *kpool, *vpool;
+  const int *page_table; int pages_per_seq, page_size, L, layer, H, hd;
+  float qscale;
+  const Pass *pass;
+};
+__global__ void __launch_bounds__(256) k_reduce_qkv(const ReduceQkvArgs a) {
+  const int t = blockIdx.y;
+  if (t >= a.pass->T) return;
+  const int d = a.H * a.hd, half = a.hd >> 1;
+  const int idx = blockIdx.x * 256 + threadIdx.x;
+  if (idx >= a.H * half) return;
+  const int hh = idx / half, i = idx - hh * half, o = hh * a.hd + i;
+  float v[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // q_i, q_i+half, k_i, k_i+half, v_i, v_i+half
+  for (int sp = 0; sp < a.S; ++sp) {
+    const float *pp = a.part + ((size_t)sp * kTcRowsMax + t) * (3 * d);
+    v[0] += __ldcg(pp + o); v[1] += __ldcg(pp + o + half);
+    v[2] += __ldcg(pp + d + o); v[3] += __ldcg(pp + d + o + half);
+    v[4] += __ldcg(pp + 2 * d + o); v[5] += __ldcg(pp + 2 * d + o + half);
+  }
+  const float inv = inv_rms_of(a.ss_part, t, d, a.eps);
+#pragma unroll
+  for (int j = 0; j < 6; ++j) v[j] *= inv;
+  const int pos = a.pass->row_pos[t], b = a.pass->row_seq[t];
+  const float2 cs = a.rope[(size_t)pos * half + i];
+  a.qout[(size_t)t * d + o] = (v[0] * cs.x - v[1] * cs.y) * a.qscale;
+  a.qout[(size_t)t * d + o + half] = (v[1] * cs.x + v[0] * cs.y) * a.qscale;
+  const int page = a.page_table[b * a.pages_per_seq + pos / a.page_size], slot = pos % a.page_size;
+  const size_t base = (((size_t)page * a.L + a.layer) * a.H + hh) * a.page_size * a.hd + (size_t)slot * a.hd;
+  const int sw = slot & 7;
+  a.kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[2] * cs.x - v[3] * cs.y);
+  a.kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[3] * cs.x + v[2] * cs.y);
+  a.vpool[base + i] = kv_store(v[4]);
+  a.vpool[base + i + half] = kv_store(v[5]);
+}
+
+// SwiGLU: gate and up sums of the splits times 1 / rms(row), silu(gate) * up as hi / lo planes.
+// One thread per (pass row, 4 columns), grid-stride.
+struct ReduceSwigluArgs {
+  const float *part; int S, F;         // [S][128][2 F]: gate columns then up columns
+  const float *ss_part; float eps; int d;
+  __nv_bfloat16 *ohi, *olo; int ldo;
+  const Pass *pass;
+};
+__global__ void __launch_bounds__(256) k_reduce_swiglu(const ReduceSwigluArgs a) {
+  const int T = a.pass->T;
+  const int c4 = a.F >> 2;
   for (int idx = blockIdx.x * 256 + threadIdx.x; idx < T * c4; idx += gridDim.x * 256) {
     const int t = idx / c4, col = (idx - t * c4) << 2;
     float4 y = make_float4(0.f, 0.f, 0.f, 0.f), u = y;
     for (int sp = 0; sp < a.S; ++sp) {
-      const float *pp = a.part + ((size_t)sp * kTcRowsMax + t) * Ntot + col;
+      const float *pp = a.part + ((size_t)sp * kTcRowsMax + t) * (2 * (size_t)a.F) + col;
       const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp));
+      const float4 w = __ldcg(reinterpret_cast<const float4 *>(pp + a.F));
       y.x += v.x; y.y += v.y; y.z += v.z; y.w += v.w;
-      if (sw) {
-        const float4 w = __ldcg(reinterpret_cast<const float4 *>(pp + a.Nseg));
-        u.x += w.x; u.y += w.y; u.z += w.z; u.w += w.w;
-      }
+      u.x += w.x; u.y += w.y; u.z += w.z; u.w += w.w;
     }
-    if (a.epi == EPI_STORE) {
-      *reinterpret_cast<float4 *>(a.Y + (size_t)t * a.ldy + col) = y;
-    } else if (a.epi == EPI_RESID) {
-      float4 *yp = reinterpret_cast<float4 *>(a.Y + (size_t)t * a.ldy + col);
-      float4 h = *yp;
-      h.x += y.x; h.y += y.y; h.z += y.z; h.w += y.w;
-      *yp = h;
-    } else if (sw) {
-      const float yy[4] = {y.x, y.y, y.z, y.w}, uu[4] = {u.x, u.y, u.z, u.w};
+    const float inv = inv_rms_of(a.ss_part, t, a.d, a.eps);
+    const float yy[4] = {y.x * inv, y.y * inv, y.z * inv, y.w * inv}, uu[4] = {u.x * inv, u.y * inv, u.z * inv, u.w * inv};
+    __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float o = (yy[i] / (1.f + __expf(-yy[i]))) * uu[i];
-        __nv_bfloat16 hi, lo;
-        split_bf16(o, hi, lo);
-        a.Ohi[(size_t)t * a.ldo + col + i] = hi;
-        a.Olo[(size_t)t * a.ldo + col + i] = lo;
-      }
-    }
+    for (int i = 0; i < 4; ++i) split_bf16((yy[i] / (1.f + __expf(-yy[i]))) * uu[i], hi[i], lo[i]);
+    uint2 ph, pl;
+    ph.x = (uint32_t)__bfloat16_as_ushort(hi[0]) | ((uint32_t)__bfloat16_as_ushort(hi[1]) << 16);
+    ph.y = (uint32_t)__bfloat16_as_ushort(hi[2]) | ((uint32_t)__bfloat16_as_ushort(hi[3]) << 16);
+    pl.x = (uint32_t)__bfloat16_as_ushort(lo[0]) | ((uint32_t)__bfloat16_as_ushort(lo[1]) << 16);
+    pl.y = (uint32_t)__bfloat16_as_ushort(lo[2]) | ((uint32_t)__bfloat16_as_ushort(lo[3]) << 16);
+    *reinterpret_cast<uint2 *>(a.ohi + (size_t)t * a.ldo + col) = ph;
+    *reinterpret_cast<uint2 *>(a.olo + (size_t)t * a.ldo + col) = pl;
   }
 }
 

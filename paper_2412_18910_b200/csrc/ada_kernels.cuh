@@ -157,14 +157,28 @@ __global__ void k_argmax_final(const float4 *amax, int tiles, int TP, const Pass
 }
 
 // ---------------------------------------------------------------------------------------------
-// h[t][:] = embedding of row_tok[t]
-__global__ void k_embed(const Pass *pass, const __nv_bfloat16 *embed, float *h, int d) {
+// h[t][:] = embedding of row_tok[t]; planes = split(h * gain) of the first layer's norm; the row's sum of squares
+// (slot 0 of the row's segments, the others zero: see the reduction kernels of the multi-row GEMM).
+__global__ void k_embed(const Pass *pass, const __nv_bfloat16 *embed, float *h, int d, const __nv_bfloat16 *gain,
+                        __nv_bfloat16 *xhi, __nv_bfloat16 *xlo, int ldx, float *ss_part, int ss_segs) {
+  __shared__ float sh[32];
   const int t = blockIdx.x;
   if (t >= pass->T) return;
   const __nv_bfloat16 *__restrict__ e = embed + (size_t)pass->row_tok[t] * d;
   float *__restrict__ hr = h + (size_t)t * d;
+  float ss = 0.f;
 #pragma unroll 8
-  for (int i = threadIdx.x; i < d; i += blockDim.x) hr[i] = __bfloat162float(e[i]);   // (loads of a row in flight together)
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {   // (loads of a row in flight together)
+    const float v = __bfloat162float(e[i]);
+    hr[i] = v;
+    ss += v * v;
+    __nv_bfloat16 hi, lo;
+    split_bf16(v * __bfloat162float(gain[i]), hi, lo);
+    xhi[(size_t)t * ldx + i] = hi;
+    xlo[(size_t)t * ldx + i] = lo;
+  }
+  ss = block_sum(ss, sh);
+  if (threadIdx.x < ss_segs) ss_part[(size_t)t * ss_segs + threadIdx.x] = threadIdx.x == 0 ? ss : 0.f;
 }
 
 // x = h / sqrt(mean(h^2) + eps) * gain  ->  hi/lo halves; optionally also fp32 rows to
@@ -230,55 +244,6 @@ __global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bf
     xhi[(size_t)i * ldx + c] = hi;
     xlo[(size_t)i * ldx + c] = lo;
     fo[c] = x;
-  }
-}
-
-// Rotary embedding (rotate-half pairing) of q and k, scaling of q by 1/sqrt(hd), and the write of
-// k, v (bf16) into the paged cache.  qkv: [T][3d] fp32.  rope: [cap][hd/2] (cos, sin).
-// Cache element (page, layer, head, slot, i): ((page*L + layer)*H + head)*page_size*hd + slot*hd + i.
-// Key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared memory, eight
-// consecutive keys then sit in eight different bank groups (the layout both attention kernels read).
-__global__ void k_rope_kv(const Pass *pass, const float *qkv, const float2 *rope, float *qout,
-                          __nv_bfloat16 *kpool, __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
-                          int page_size, int L, int layer, int H, int hd, float qscale) {
-  const int t = blockIdx.x;
-  if (t >= pass->T) return;
-  const int d = H * hd, half = hd >> 1;
-  const int pos = pass->row_pos[t], b = pass->row_seq[t];
-  const int page = page_table[b * pages_per_seq + pos / page_size], slot = pos % page_size;
-  const float *__restrict__ q = qkv + (size_t)t * 3 * d;
-  const float *__restrict__ k = q + d, *__restrict__ v = k + d;
-  const int sw = slot & 7;
-  for (int idx0 = threadIdx.x; idx0 < H * half; idx0 += 4 * blockDim.x) {
-    // the loads of four steps first, so that they are in flight together
-    float qa[4], qb[4], ka[4], kb[4], va[4], vb[4];
-    float2 cs[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int idx = idx0 + u * blockDim.x;
-      qa[u] = qb[u] = ka[u] = kb[u] = va[u] = vb[u] = 0.f;
-      cs[u] = make_float2(1.f, 0.f);
-      if (idx < H * half) {
-        const int hh = idx / half, i = idx - hh * half;
-        const int o = hh * hd + i;
-        cs[u] = rope[(size_t)pos * half + i];
-        qa[u] = q[o]; qb[u] = q[o + half]; ka[u] = k[o]; kb[u] = k[o + half]; va[u] = v[o]; vb[u] = v[o + half];
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int idx = idx0 + u * blockDim.x;
-      if (idx >= H * half) continue;
-      const int hh = idx / half, i = idx - hh * half;
-      const int o = hh * hd + i;
-      qout[(size_t)t * d + o] = (qa[u] * cs[u].x - qb[u] * cs[u].y) * qscale;
-      qout[(size_t)t * d + o + half] = (qb[u] * cs[u].x + qa[u] * cs[u].y) * qscale;
-      const size_t base = (((size_t)page * L + layer) * H + hh) * page_size * hd + (size_t)slot * hd;
-      kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(ka[u] * cs[u].x - kb[u] * cs[u].y);
-      kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(kb[u] * cs[u].x + ka[u] * cs[u].y);
-      vpool[base + i] = kv_store(va[u]);
-      vpool[base + i + half] = kv_store(vb[u]);
-    }
   }
 }
 
