@@ -8,8 +8,8 @@
 // into slivers that cost more to set up and merge than to compute.  A warp takes 32-key blocks of the split, in halves
 // of 16 keys: one bulk copy brings a half's key rows and one its value rows (they are contiguous in the cache page)
 // into one of the warp's two buffers, so the next half is in flight while this one is computed -- scores = q k^T
-// as m16n8k16 products per 16 channels, online softmax on the accumulator fragments, weighted values as m16n8k8
-// products per 8 channels, 8 keys at a time.  Cache elements are 16-bit halves and enter the products as they are;
+// as m16n8k16 products per 16 channels (two tiles of 8 keys), online softmax on the accumulator fragments, weighted
+// values as m16n8k16 products over the 16 keys per 8 channels, 16 keys at a time.  Cache elements are 16-bit halves and enter the products as they are;
 // q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, so each product is issued twice and
 // the sums are fp32 (error 2^-22 relative).  Key rows are kept in the cache with their 16-byte chunks XORed by
 // (slot & 7), which makes ldmatrix of 8 consecutive keys conflict-free and lets the copy be verbatim.  A copy always
@@ -131,68 +131,92 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
       if (lane == 0 && valid(h + 1)) issue(h + 1);   // the other buffer: every lane left it at the end of the last turn
       const __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD, *vst = kst + kAttnHalf * HD;
       mbar_wait(&bars[h & 1], (uses[h & 1]++) & 1u, cnt, &abort_s);
-      const int kb = key0_of(h);
-#pragma unroll
-      for (int sub = 0; sub < 2; ++sub) {
-        const int key0 = kb + 8 * sub;          // first of these 8 keys
-        if (key0 >= kend || key0 > last_pos) break;
-        // ---- scores: 16 rows x 8 keys
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t krow = smem_u32(kst + (size_t)(8 * sub + (lane & 7)) * HD);
+      const int key0 = key0_of(h);            // first of these 16 keys
+      {
+        // ---- scores: 16 rows x 16 keys as two tiles of 8 keys (sa: keys 0..7, sb: keys 8..15)
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t krow = smem_u32(kst + (size_t)(lane & 7) * HD);
         const int ksw = lane & 7;               // = slot & 7: halves start at multiples of 16
         const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
         for (int kp = 0; kp < HD / 32; ++kp) {    // pairs of 16-channel steps
-          uint32_t kb0, kb1, kb2, kb3;
-          ldmatrix_x4(krow + (((kp * 4 + (lane >> 3)) ^ ksw) << 4), kb0, kb1, kb2, kb3);
+          uint32_t ka0, ka1, ka2, ka3, kb0, kb1, kb2, kb3;
+          const uint32_t koff = (uint32_t)(((kp * 4 + (lane >> 3)) ^ ksw) << 4);
+          ldmatrix_x4(krow + koff, ka0, ka1, ka2, ka3);
+          ldmatrix_x4(krow + 8 * HD * 2 + koff, kb0, kb1, kb2, kb3);
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
             const int ks = kp * 2 + h2;
             const uint32_t aoff = (uint32_t)(arow * (HD * 2) + (((ks * 2 + (lane >> 4)) ^ (arow & 7)) << 4));
             uint32_t a0, a1, a2, a3;
             ldmatrix_x4(qh_u + aoff, a0, a1, a2, a3);
-            mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+            mma_f16_k16(sa, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
+            mma_f16_k16(sb, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
             ldmatrix_x4(ql_u + aoff, a0, a1, a2, a3);
-            mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+            mma_f16_k16(sa, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
+            mma_f16_k16(sb, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
           }
         }
-        // ---- online softmax: this thread holds keys kc, kc + 1 of rows g8r and g8r + 8
+        // ---- online softmax: this thread holds keys kc, kc + 1, kc + 8, kc + 9 of rows g8r and g8r + 8
         const int kc = key0 + 2 * t4;
-        const bool s00 = kc < kend && kc <= qp0, s01 = kc + 1 < kend && kc + 1 <= qp0;
-        const bool s10 = kc < kend && kc <= qp1, s11 = kc + 1 < kend && kc + 1 <= qp1;
-        float mx0 = fmaxf(s00 ? sc[0] : -INFINITY, s01 ? sc[1] : -INFINITY);
-        float mx1 = fmaxf(s10 ? sc[2] : -INFINITY, s11 ? sc[3] : -INFINITY);
+        bool ok0[4], ok1[4];    // [key slot] for row g8r / g8r + 8
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int k = kc + (j & 1) + 8 * (j >> 1);
+          ok0[j] = k < kend && k <= qp0;
+          ok1[j] = k < kend && k <= qp1;
+        }
+        const float s0[4] = {sa[0], sa[1], sb[0], sb[1]}, s1[4] = {sa[2], sa[3], sb[2], sb[3]};
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          mx0 = fmaxf(mx0, ok0[j] ? s0[j] : -INFINITY);
+          mx1 = fmaxf(mx1, ok1[j] ? s1[j] : -INFINITY);
+        }
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
         const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-        float p00 = 0.f, p01 = 0.f, p10 = 0.f, p11 = 0.f, c0 = 1.f, c1 = 1.f;
-        if (mn0 > -INFINITY) { p00 = s00 ? __expf(sc[0] - mn0) : 0.f; p01 = s01 ? __expf(sc[1] - mn0) : 0.f; c0 = __expf(m0 - mn0); }
-        if (mn1 > -INFINITY) { p10 = s10 ? __expf(sc[2] - mn1) : 0.f; p11 = s11 ? __expf(sc[3] - mn1) : 0.f; c1 = __expf(m1 - mn1); }
-        float ps0 = p00 + p01, ps1 = p10 + p11;
+        float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f}, c0 = 1.f, c1 = 1.f;
+        if (mn0 > -INFINITY) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) p0[j] = ok0[j] ? __expf(s0[j] - mn0) : 0.f;
+          c0 = __expf(m0 - mn0);
+        }
+        if (mn1 > -INFINITY) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) p1[j] = ok1[j] ? __expf(s1[j] - mn1) : 0.f;
+          c1 = __expf(m1 - mn1);
+        }
+        float ps0 = (p0[0] + p0[1]) + (p0[2] + p0[3]), ps1 = (p1[0] + p1[1]) + (p1[2] + p1[3]);
         ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1); ps1 += __shfl_xor_sync(0xffffffffu, ps1, 1);
         ps0 += __shfl_xor_sync(0xffffffffu, ps0, 2); ps1 += __shfl_xor_sync(0xffffffffu, ps1, 2);
         l0 = l0 * c0 + ps0; l1 = l1 * c1 + ps1;
         m0 = mn0; m1 = mn1;
-        // weights as (hi, lo) halves: A operand rows g8r, g8r + 8, k = keys 2 t4, 2 t4 + 1
-        const __half2 ph0 = __floats2half2_rn(p00, p01), ph1 = __floats2half2_rn(p10, p11);
-        const float2 pf0 = __half22float2(ph0), pf1 = __half22float2(ph1);
-        const __half2 pl0 = __floats2half2_rn(p00 - pf0.x, p01 - pf0.y), pl1 = __floats2half2_rn(p10 - pf1.x, p11 - pf1.y);
-        const uint32_t ah0 = *reinterpret_cast<const uint32_t *>(&ph0), ah1 = *reinterpret_cast<const uint32_t *>(&ph1);
-        const uint32_t al0 = *reinterpret_cast<const uint32_t *>(&pl0), al1 = *reinterpret_cast<const uint32_t *>(&pl1);
-        // ---- values: out[16 rows][HD] += w[16 x 8 keys] v[8 keys x HD]
-        const uint32_t vrow = smem_u32(vst + (size_t)(8 * sub + (lane & 7)) * HD);
+        // weights as (hi, lo) halves: A operand of a k = 16 product: a0 = row g8r keys 0..7, a1 = row g8r + 8 keys 0..7,
+        // a2 = row g8r keys 8..15, a3 = row g8r + 8 keys 8..15 (this thread's pair of each)
+        uint32_t ah[4], al[4];
 #pragma unroll
-        for (int nq = 0; nq < HD / 32; ++nq) {      // four 8-channel tiles per load
-          uint32_t v0, v1, v2, v3;
-          ldmatrix_x4_trans(vrow + ((nq * 4 + (lane >> 3)) << 4), v0, v1, v2, v3);
+        for (int j = 0; j < 4; ++j) {
+          const float x = (j & 1) ? p1[2 * (j >> 1)] : p0[2 * (j >> 1)], y = (j & 1) ? p1[2 * (j >> 1) + 1] : p0[2 * (j >> 1) + 1];
+          const __half2 ph = __floats2half2_rn(x, y);
+          const float2 pf = __half22float2(ph);
+          const __half2 pl = __floats2half2_rn(x - pf.x, y - pf.y);
+          ah[j] = *reinterpret_cast<const uint32_t *>(&ph);
+          al[j] = *reinterpret_cast<const uint32_t *>(&pl);
+        }
+        // ---- values: out[16 rows][HD] += w[16 x 16 keys] v[16 keys x HD], two 8-channel tiles per load
+        const uint32_t vrow = smem_u32(vst + (size_t)((lane & 7) + 8 * ((lane >> 3) & 1)) * HD);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float *oo = o[nq * 4 + j];
-            oo[0] *= c0; oo[1] *= c0; oo[2] *= c1; oo[3] *= c1;
-            const uint32_t vb = j == 0 ? v0 : j == 1 ? v1 : j == 2 ? v2 : v3;
-            mma_f16_k8(oo, ah0, ah1, vb);
-            mma_f16_k8(oo, al0, al1, vb);
-          }
+        for (int c2 = 0; c2 < HD / 16; ++c2) {
+          uint32_t v0, v1, v2, v3;   // (keys 0..7, keys 8..15) of channel tile 2 c2, then of tile 2 c2 + 1
+          ldmatrix_x4_trans(vrow + ((2 * c2 + (lane >> 4)) << 4), v0, v1, v2, v3);
+          float *oa = o[2 * c2], *ob = o[2 * c2 + 1];
+          oa[0] *= c0; oa[1] *= c0; oa[2] *= c1; oa[3] *= c1;
+          ob[0] *= c0; ob[1] *= c0; ob[2] *= c1; ob[3] *= c1;
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), ah[0], ah[1], ah[2], ah[3], v0, v1);
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), al[0], al[1], al[2], al[3], v0, v1);
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(ob), ah[0], ah[1], ah[2], ah[3], v2, v3);
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(ob), al[0], al[1], al[2], al[3], v2, v3);
         }
       }
       __syncwarp();   // every lane is done with this buffer
