@@ -18,6 +18,7 @@
 #include "ada_attn_rows.cuh"
 
 #include <unordered_map>
+#include <utility>
 
 using namespace ada;
 typedef __nv_bfloat16 bf16;
@@ -83,6 +84,7 @@ struct ada_ctx {
   int *out_acc, *out_emit, *out_nemit, *out_nused;   // internal outputs of ada_step
   // per-kernel timing for roofline reports (off by default): event pairs around GEMM / attention launches
   int prof;
+  int pdl;                      // 1: the multi-row chain is launched with programmatic serialization (ADA_NO_PDL unset)
   std::vector<cudaEvent_t> ev_pool;
   struct ProfRec { int cls; int ev; double bytes; };
   std::vector<ProfRec> prof_recs;
@@ -103,6 +105,22 @@ int fail(ada_ctx *ctx, int code, const char *msg) {
     kernel<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);              \
     (ctx)->launches++;                                                      \
   } while (0)
+
+// Launch with the programmatic-serialization attribute: the kernel may begin while the kernel before it in the stream
+// still runs and waits inside (pdl_wait) before it touches anything that kernel writes.  Only for kernels that wait in
+// every thread before their first dependent access and before returning.
+template <typename... KArgs, typename... Args>
+void launch_pdl(ada_ctx *x, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args &&...args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = x->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = x->pdl;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+  x->launches++;
+}
 
 // Event pair around the launches made by `body` when profiling is on.
 template <typename F>
@@ -305,26 +323,26 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
   const int d = c.d_model;
   const double wb = 2.0 * (double)Nseg * (double)K * (epi == EPI_SWIGLU ? 2 : nseg);
   timed(x, 0, wb, [&] {
-    if (wide) LAUNCH(x, k_gemm_tc<kTcRowsMax>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRowsMax>::kSmemBytes, t);
-    else LAUNCH(x, k_gemm_tc<kTcRows>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRows>::kSmemBytes, t);
+    if (wide) launch_pdl(x, k_gemm_tc<kTcRowsMax>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRowsMax>::kSmemBytes, t);
+    else launch_pdl(x, k_gemm_tc<kTcRows>, dim3(tiles, t.S), kTcThreads, TcShape<kTcRows>::kSmemBytes, t);
     if (r.kind == Reduce::H) {
       ReduceHArgs a;
       a.part = x->gemm_part; a.S = t.S; a.Ntot = Nseg; a.h = x->h; a.d = d; a.resid = r.resid; a.gain = r.gain;
       a.xhi = x->xhi; a.xlo = x->xlo; a.ldx = x->ldx; a.ss_part = x->ss_rows; a.pass = x->pass;
-      LAUNCH(x, k_reduce_h, dim3((d + 1023) / 1024, rows), 256, 0, a);
+      launch_pdl(x, k_reduce_h, dim3((d + 1023) / 1024, rows), 256, 0, a);
     } else if (r.kind == Reduce::QKV_ROPE) {
       ReduceQkvArgs a;
       a.part = x->gemm_part; a.S = t.S; a.ss_part = x->ss_rows; a.eps = c.rms_eps; a.rope = x->rope; a.qout = x->qrot;
       a.kpool = r.kpool; a.vpool = r.vpool; a.page_table = x->page_table; a.pages_per_seq = x->pages_per_seq;
       a.page_size = c.page_size; a.L = r.L; a.layer = r.layer; a.H = c.n_heads; a.hd = c.head_dim;
       a.qscale = 1.0f / sqrtf((float)c.head_dim); a.pass = x->pass;
-      LAUNCH(x, k_reduce_qkv, dim3((c.n_heads * (c.head_dim / 2) + 255) / 256, rows), 256, 0, a);
+      launch_pdl(x, k_reduce_qkv, dim3((c.n_heads * (c.head_dim / 2) + 255) / 256, rows), 256, 0, a);
     } else if (r.kind == Reduce::SWIGLU) {
       ReduceSwigluArgs a;
       a.part = x->gemm_part; a.S = t.S; a.F = Nseg; a.ss_part = x->ss_rows; a.eps = c.rms_eps; a.d = d;
       a.ohi = x->x2hi; a.olo = x->x2lo; a.ldo = x->ldx2; a.pass = x->pass;
       const int blocks = (rows * (Nseg / 4) + 255) / 256;
-      LAUNCH(x, k_reduce_swiglu, blocks < 1184 ? blocks : 1184, 256, 0, a);
+      launch_pdl(x, k_reduce_swiglu, dim3(blocks < 1184 ? blocks : 1184), 256, 0, a);
     }
   });
   return true;
@@ -339,13 +357,13 @@ void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   dim3 g2(c.n_heads, x->TM);
   timed(x, 1, 0.0, [&] {
   if (c.head_dim == 128) {
-    LAUNCH(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+    launch_pdl(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
-    LAUNCH(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
+    launch_pdl(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
   } else {
-    LAUNCH(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
+    launch_pdl(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
            x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
-    LAUNCH(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
+    launch_pdl(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
   }
   });
 }
@@ -684,6 +702,7 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
   x->graph_key = -1;
   x->capture_stream = nullptr;
   x->prof = 0; x->ev_used = 0; x->enqueue_failed = 0;
+  x->pdl = getenv("ADA_NO_PDL") ? 0 : 1;
 
   // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as (cos, sin) floats
   const int half = cfg->head_dim / 2, cap = cfg->kv_capacity;

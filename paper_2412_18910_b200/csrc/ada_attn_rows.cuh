@@ -34,15 +34,16 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
                                                    int page_size, int L, int layer, int H, float *part, int nrg,
                                                    int cap, Counters *cnt) {
   static_assert(HD == 64 || HD == 128, "head width");
+  pdl_launch_dependents();
+  pdl_wait();                  // queries and the new cache rows come from the kernel before this one
   constexpr int CH = HD / 8;   // 16-byte chunks per row
   // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
   const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / nrg, rgi = blockIdx.z - b * nrg;
-  const int R = pass->seq_rows[b];
-  if (pass->T <= 0 || R <= 0) return;
-  const int row0 = pass->seq_row0[b];
-  const int pos0 = pass->row_pos[row0];
+  const int4 si = pass->seq_info[b];   // (first row, rows, split size, first position) in one load
+  const int row0 = si.x, R = si.y, pos0 = si.w;
+  if (R <= 0) return;
   const int nkeys = pos0 + R;
-  const int chunk = attn_rows_chunk(pass->seq_chunk[b], cap);
+  const int chunk = attn_rows_chunk(si.z, cap);
   const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
   if (kbeg >= nkeys) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -75,12 +76,13 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
     const int nr = min(kRowGroup, R - rg);
     __syncthreads();   // the previous group's merge has read the shared areas; the barriers are initialised
     const int last_pos = pos0 + rg + nr - 1;   // the last position any row of the group sees
-    // half h of this warp: keys key0(h) .. key0(h) + 15
-    auto key0_of = [&](int h) { return kbeg + 32 * (warp + 4 * (h >> 1)) + kAttnHalf * (h & 1); };
+    // half h of this warp: keys key0(h) .. key0(h) + 15 (the split's halves are dealt to the four warps in turn)
+    auto key0_of = [&](int h) { return kbeg + kAttnHalf * (warp + 4 * h); };
     auto valid = [&](int h) { const int k0 = key0_of(h); return k0 < kend && k0 <= last_pos; };
-    auto issue = [&](int h) {   // one lane: the half's key rows and value rows into buffer h & 1
+    // cache pages of the warp's halves 32 i + lane, fetched 32 at a time so that no copy waits for a table lookup
+    int pages = valid(lane) ? page_table[b * pages_per_seq + key0_of(lane) / page_size] : 0;
+    auto issue = [&](int h, int page) {   // one lane: the half's key rows and value rows into buffer h & 1
       const int k0 = key0_of(h);
-      const int page = page_table[b * pages_per_seq + k0 / page_size];
       const size_t off = (size_t)page * page_stride + head_off + (size_t)(k0 % page_size) * HD;
       __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
@@ -88,7 +90,11 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
       bulk_g2s(kst, kpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
       bulk_g2s(kst + kAttnHalf * HD, vpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
     };
-    if (lane == 0 && valid(0)) issue(0);   // flies under the staging of q
+    {   // both buffers are free: the first two halves fly under the staging of q
+      const int p0 = __shfl_sync(0xffffffffu, pages, 0), p1 = __shfl_sync(0xffffffffu, pages, 1);
+      if (lane == 0 && valid(0)) issue(0, p0);
+      if (lane == 0 && valid(1)) issue(1, p1);
+    }
     {   // the group's query rows as (hi, lo) halves; rows past nr are zero
       constexpr int PER = kRowGroup * HD / 4 / 128;
       float4 qv[PER];
@@ -128,7 +134,6 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
     const int qp0 = pos0 + rg + g8r, qp1 = qp0 + 8;
 
     for (int h = 0; valid(h); ++h) {
-      if (lane == 0 && valid(h + 1)) issue(h + 1);   // the other buffer: every lane left it at the end of the last turn
       const __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD, *vst = kst + kAttnHalf * HD;
       mbar_wait(&bars[h & 1], (uses[h & 1]++) & 1u, cnt, &abort_s);
       const int key0 = key0_of(h);            // first of these 16 keys
@@ -219,7 +224,10 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(ob), al[0], al[1], al[2], al[3], v2, v3);
         }
       }
-      __syncwarp();   // every lane is done with this buffer
+      __syncwarp();   // every lane is done with this buffer: the half after the next one goes into it
+      if (((h + 2) & 31) == 0) pages = valid(h + 2 + lane) ? page_table[b * pages_per_seq + key0_of(h + 2 + lane) / page_size] : 0;
+      const int pnext = __shfl_sync(0xffffffffu, pages, (h + 2) & 31);
+      if (lane == 0 && valid(h + 2)) issue(h + 2, pnext);
     }
 
     // per-warp partials -> shared (over the staging areas, once every warp has left them), merged in warp order

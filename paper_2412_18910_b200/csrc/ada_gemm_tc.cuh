@@ -78,12 +78,25 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 32 consecutive accumulator columns of this thread's tensor-memory lane: requested here, valid after tmem_ld_wait
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+      "%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 template <int ROWS>
 __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   using Sh = TcShape<ROWS>;
   constexpr int kTcStages = Sh::kStages, kTcStageBytes = Sh::kStageBytes, kTcBBytes = Sh::kBBytes, kTcN = Sh::kN;
-  const int T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
-  if (T <= 0) return;
+  pdl_launch_dependents();   // the next kernel may start its prologue; it waits for this grid to complete before it reads
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool sw = a.epi == EPI_SWIGLU;
 
@@ -110,23 +123,49 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   const TensorMap128 *m0 = sw ? a.wmap[0] : a.wmap[seg];
   const TensorMap128 *m1 = sw ? a.wmap[1] : a.wmap[seg];
   const unsigned tx = (unsigned)(mtiles * kTcABytes + 2 * kTcBBytes);
-  auto load_stage = [&](int kb, int s) {
+  auto load_weights = [&](int kb, int s) {   // arms the stage's barrier for the whole stage
     unsigned char *st = smem + (size_t)s * kTcStageBytes;
     mbar_expect_tx(&full[s], tx);
     tma_load_2d(st, m0, kb * 64, row0, &full[s]);                 // rows past the matrix and k past K read as zero
     if (mtiles > 1) tma_load_2d(st + kTcABytes, m1, kb * 64, row1, &full[s]);
+  };
+  auto load_planes = [&](int kb, int s) {
+    unsigned char *st = smem + (size_t)s * kTcStageBytes;
     tma_load_2d(st + 2 * kTcABytes, a.xhi_map, kb * 64, 0, &full[s]);
     tma_load_2d(st + 2 * kTcABytes + kTcBBytes, a.xlo_map, kb * 64, 0, &full[s]);
   };
+  // Weights depend on no earlier kernel: the first stages' weight boxes are requested before this grid waits for
+  // the grid before it (programmatic dependent launch), the activation boxes after; the tensor memory is allocated
+  // meanwhile.  The row count read before the wait is only a hint (it may be stale): it decides whether to run ahead,
+  // so that a pass without rows costs next to nothing; the count read after the wait decides what is computed.
+  // Nothing else of this kernel reads or writes global memory before the wait.
   const int nfirst = min(kTcStages, kb1 - kb0);
+  __shared__ int ahead_s;      // one read for the whole CTA: every thread takes the same branch
+  if (tid == 0) ahead_s = (a.use_lm_rows ? a.pass->lmT : a.pass->T) > 0;
+  __syncthreads();
+  const bool ahead = ahead_s != 0;
+  int T;
   if (tid == 0) {
     *abort_s = 0;
     for (int i = 0; i < kTcStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(accfull, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int i = 0; i < nfirst; ++i) load_stage(kb0 + i, i);
+    if (ahead)
+      for (int i = 0; i < nfirst; ++i) load_weights(kb0 + i, i);
+    pdl_wait();
+    T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
+    for (int i = 0; i < nfirst && (ahead || T > 0); ++i) {
+      if (!ahead) load_weights(kb0 + i, i);
+      load_planes(kb0 + i, i);     // (also for a pass that turned out empty: the armed barrier must complete)
+    }
+  } else {
+    if (warp == 2 && ahead) tmem_alloc(tmem_slot, kTcTmemCols);
+    pdl_wait();
+    T = a.use_lm_rows ? a.pass->lmT : a.pass->T;
+    if (warp == 2 && !ahead && T > 0) tmem_alloc(tmem_slot, kTcTmemCols);
   }
-  if (warp == 2) tmem_alloc(tmem_slot, kTcTmemCols);
+  const bool idle = T <= 0;   // a pass without rows: requested stages are awaited, nothing is computed or stored
+  if (idle && !ahead) return; // (uniform over the grid) nothing was requested or allocated
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -135,16 +174,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
   if (warp == 0) {
     // ------------------------------------------------------------- producer
     if (lane == 0) {
-      for (int kb = kb0 + nfirst, i = nfirst; kb < kb1; ++kb, ++i) {
+      for (int kb = kb0 + nfirst, i = nfirst; kb < kb1 && !idle; ++kb, ++i) {
         const int s = i % kTcStages;
         mbar_wait(&empty[s], ((unsigned)(i / kTcStages) & 1u) ^ 1u, a.cnts, abort_s);
-        load_stage(kb, s);
+        load_weights(kb, s);
+        load_planes(kb, s);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------- tensor-core issuer
     const uint32_t idesc = umma_idesc_mn(128u, (uint32_t)kTcN);
-    for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
+    if (idle)
+      for (int i = 0; i < nfirst; ++i) mbar_wait(&full[i], 0u, a.cnts, abort_s);   // no copy may outlive the CTA
+    for (int kb = kb0, i = 0; kb < kb1 && !idle; ++kb, ++i) {
       const int s = i % kTcStages;
       mbar_wait(&full[s], (unsigned)(i / kTcStages) & 1u, a.cnts, abort_s);
       tc_fence_after();
@@ -161,11 +203,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
       }
       __syncwarp();
     }
-    if (elect_one()) umma_commit(accfull);
+    if (!idle && elect_one()) umma_commit(accfull);
     __syncwarp();
   }
 
-  if (warp >= 4) {
+  if (warp >= 4 && !idle) {
     // ------------------------------------------------------------- epilogue
     const int cw = warp - 4, quarter = warp & 3;
     const int ctid = tid - 128;
@@ -174,53 +216,56 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const GemmTcArgs a) {
     const int n = (mi ? row1 : row0) + quarter * 32 + lane;         // weight row inside the segment
     const bool valid = active_warp && n < a.Nseg;
     const int Ntot = sw ? 2 * a.Nseg : a.nseg * a.Nseg;
-    const int col = seg * a.Nseg + n;                                  // output column (SWIGLU: gate column)
     const int nblk = (T + 7) >> 3;
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * 256);
 
     if (kb1 > kb0) mbar_wait(accfull, 0u, a.cnts, abort_s);
     tc_fence_after();
 
-    // pass rows 8 j .. 8 j + 7 of this thread's weight row: y (and u, the up projection, for SWIGLU)
-    auto from_tmem = [&](int j, float (&y)[8], float (&u)[8]) {
+    // pass rows 8 j .. 8 j + 7 of this thread's weight row (LM head)
+    auto from_tmem = [&](int j, float (&y)[8]) {
       float hi[8], lo[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { y[i] = 0.f; u[i] = 0.f; }
+      for (int i = 0; i < 8; ++i) y[i] = 0.f;
       if (!active_warp || kb1 <= kb0) return;     // (warp-uniform)
       tmem_ld8(taddr + (uint32_t)(8 * j), hi);
       tmem_ld8(taddr + (uint32_t)(ROWS + 8 * j), lo);
 #pragma unroll
       for (int i = 0; i < 8; ++i) y[i] = hi[i] + lo[i];
-      if (sw) {
-        tmem_ld8(taddr + 256u + (uint32_t)(8 * j), hi);
-        tmem_ld8(taddr + 256u + (uint32_t)(ROWS + 8 * j), lo);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) u[i] = hi[i] + lo[i];
-      }
     };
 
     if (a.to_part) {
-      for (int j = 0; j < nblk; ++j) {
-        float y[8], u[8];
-        from_tmem(j, y, u);
-        if (valid) {
+      // 32 pass rows per round: both planes' columns are requested before the one wait, then a warp stores 128
+      // contiguous bytes (32 weight rows) per pass row.  SWIGLU: warps 4..7 take the gate tile, 8..11 the up tile.
+      const int pmi = cw >> 2;
+      const int pn = (sw || !pmi ? row0 : row1) + quarter * 32 + lane;
+      const bool pvalid = (sw || pmi < mtiles) && pn < a.Nseg;
+      const int pcol = sw ? pmi * a.Nseg + pn : seg * a.Nseg + pn;
+      const uint32_t paddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(pmi * 256);
+      const bool have = (sw || pmi < mtiles) && kb1 > kb0;     // (warp-uniform)
+      float *pp = a.part + (size_t)blockIdx.y * kTcRowsMax * Ntot + pcol;
+      for (int c0 = 0; c0 < T; c0 += 32) {
+        uint32_t hi[32], lo[32];
+        if (have) {
+          tmem_ld32_issue(paddr + (uint32_t)c0, hi);
+          tmem_ld32_issue(paddr + (uint32_t)(ROWS + c0), lo);
+          tmem_ld_wait();
+        } else {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int t = 8 * j + i;
-            if (t < T) {
-              float *pp = a.part + ((size_t)blockIdx.y * kTcRowsMax + t) * Ntot;
-              __stcg(pp + col, y[i]);
-              if (sw) __stcg(pp + a.Nseg + n, u[i]);
-            }
-          }
+          for (int i = 0; i < 32; ++i) hi[i] = lo[i] = 0u;
+        }
+        if (pvalid) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i < T) __stcg(pp + (size_t)(c0 + i) * Ntot, __uint_as_float(hi[i]) + __uint_as_float(lo[i]));
         }
       }
     } else {   // LM head (never split): the warp's two largest logits of every pass row, merged per CTA
       Top2 *s_top = reinterpret_cast<Top2 *>(smem);   // [8 warps][128]: the stages are idle by now
       named_bar(3, 256);
       for (int j = 0; j < nblk; ++j) {
-        float y[8], u[8];
-        from_tmem(j, y, u);
+        float y[8];
+        from_tmem(j, y);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int t = 8 * j + i;
@@ -284,6 +329,8 @@ struct ReduceHArgs {
 };
 __global__ void __launch_bounds__(256) k_reduce_h(const ReduceHArgs a) {
   __shared__ float sh[32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.y, seg = blockIdx.x;
   if (t >= a.pass->T) return;
   const int col = seg * 1024 + threadIdx.x * 4;
@@ -338,6 +385,8 @@ struct ReduceQkvArgs {
   const Pass *pass;
 };
 __global__ void __launch_bounds__(256) k_reduce_qkv(const ReduceQkvArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.y;
   if (t >= a.pass->T) return;
   const int d = a.H * a.hd, half = a.hd >> 1;
@@ -376,6 +425,8 @@ struct ReduceSwigluArgs {
   const Pass *pass;
 };
 __global__ void __launch_bounds__(256) k_reduce_swiglu(const ReduceSwigluArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int T = a.pass->T;
   const int c4 = a.F >> 2;
   for (int idx = blockIdx.x * 256 + threadIdx.x; idx < T * c4; idx += gridDim.x * 256) {

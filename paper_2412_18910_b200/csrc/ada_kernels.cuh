@@ -55,7 +55,16 @@ struct Pass {
   int seq_row0[kMaxBatch];
   int seq_rows[kMaxBatch];
   int seq_chunk[kMaxBatch];   // keys per attention split of the sequence (SeqState::chunk)
+  int4 seq_info[kMaxBatch];   // (seq_row0, seq_rows, seq_chunk, position of the first row): one load for the attention kernels
 };
+
+// Last step of every kernel that fills a row list.
+__device__ __forceinline__ void pass_seal(Pass *pass, int B) {
+  for (int b = 0; b < B; ++b) {
+    const int r0 = pass->seq_row0[b], n = pass->seq_rows[b];
+    pass->seq_info[b] = make_int4(r0, n, pass->seq_chunk[b], n > 0 ? pass->row_pos[r0] : 0);
+  }
+}
 
 // KV-cache element: 16 bits per value like the weights, but IEEE half (11-bit significand) rather than bf16
 // (8-bit): with bf16 keys and values the logits of a 32-layer stack were measured 0.03-0.05 away from the
@@ -66,6 +75,14 @@ __device__ __forceinline__ __nv_bfloat16 kv_store(float x) {
 }
 __device__ __forceinline__ float kv_lo(uint32_t pair) { return __half2float(__ushort_as_half((unsigned short)(pair & 0xffffu))); }
 __device__ __forceinline__ float kv_hi(uint32_t pair) { return __half2float(__ushort_as_half((unsigned short)(pair >> 16))); }
+
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may start while the
+// kernel before it in the stream still runs; pdl_wait returns once that kernel has completed and its writes are
+// visible (at once if there is no such dependency).  Every thread of such a kernel waits before it touches memory
+// another kernel writes and before it returns, so completion of a kernel implies completion of all before it.
+// pdl_launch_dependents lets the kernel after this one begin its own prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
   hi = __float2bfloat16_rn(x);
@@ -271,23 +288,34 @@ __host__ __device__ __forceinline__ int attn_rows_chunk(int seq_chunk, int cap) 
 template <int HD>
 __global__ void k_attn_combine(const Pass *pass, const float *part, __nv_bfloat16 *xhi, __nv_bfloat16 *xlo,
                                int ldx, int cap) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int hh = blockIdx.x, t = blockIdx.y;
   if (t >= pass->T) return;
   const int c = threadIdx.x;
   const float *base = part + (((size_t)hh * kAttnSplits) * kMaxRows + t) * (HD + 2);
   const size_t sstride = (size_t)kMaxRows * (HD + 2);
-  const int b = pass->row_seq[t];
-  const int nkeys = pass->row_pos[pass->seq_row0[b]] + pass->seq_rows[b];
-  const int chunk = attn_rows_chunk(pass->seq_chunk[b], cap);
-  const int nsp = (nkeys + chunk - 1) / chunk;  // splits that held keys
-  float M = -INFINITY;
-  for (int s = 0; s < nsp; ++s) M = fmaxf(M, base[s * sstride + HD]);
-  float l = 0.f, o = 0.f;
-  for (int s = 0; s < nsp; ++s) {
-    const float e = __expf(base[s * sstride + HD] - M);
-    l += base[s * sstride + HD + 1] * e;
-    o += base[s * sstride + c] * e;
+  const int4 si = pass->seq_info[pass->row_seq[t]];
+  const int nkeys = si.w + si.y;
+  const int chunk = attn_rows_chunk(si.z, cap);
+  const int nsp = (nkeys + chunk - 1) / chunk;  // splits that held keys (at most kAttnSplits)
+  float ms[kAttnSplits], ls[kAttnSplits], os[kAttnSplits];
+#pragma unroll
+  for (int s = 0; s < kAttnSplits; ++s) {       // all loads first: one round trip
+    ms[s] = -INFINITY; ls[s] = 0.f; os[s] = 0.f;
+    if (s < nsp) { ms[s] = base[s * sstride + HD]; ls[s] = base[s * sstride + HD + 1]; os[s] = base[s * sstride + c]; }
   }
+  float M = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < kAttnSplits; ++s) M = fmaxf(M, ms[s]);
+  float l = 0.f, o = 0.f;
+#pragma unroll
+  for (int s = 0; s < kAttnSplits; ++s)
+    if (s < nsp) {
+      const float e = __expf(ms[s] - M);
+      l += ls[s] * e;
+      o += os[s] * e;
+    }
   const float x = o / l;
   __nv_bfloat16 hi, lo;
   split_bf16(x, hi, lo);
@@ -455,6 +483,7 @@ __global__ void k_rows_verify(Pass *pass, SeqState *st, const int *tok, int cap,
   }
   pass->T = T;
   pass->lmT = T;
+  pass_seal(pass, B);
 }
 
 // Prefill chunk: rows pos0..pos0+R-1 of sequence b, tokens from the committed-token array.
@@ -472,6 +501,7 @@ __global__ void k_rows_chunk(Pass *pass, const int *tok, int cap, int b, int pos
   pass->seq_rows[b] = R;
   pass->T = R;
   pass->lmT = R;
+  pass_seal(pass, B);
 }
 
 // Draft (Eq. 2).  step 0: catch-up rows p = dlen..j-1 of every sequence with n >= 1; row p pairs the
@@ -517,6 +547,7 @@ __global__ void k_rows_draft(Pass *pass, SeqState *st, const int *tok, int cap, 
   }
   pass->T = T;
   pass->lmT = lmT;
+  pass_seal(pass, B);
 }
 
 // ---------------------------------------------------------------------------------------------

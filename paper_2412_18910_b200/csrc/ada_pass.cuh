@@ -798,8 +798,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           const int kbeg = split * chunk, kend = min(nkeys, kbeg + chunk);
           const int nround = kend > kbeg ? (kend - kbeg + 63) >> 6 : 0;
           named_bar(3, kNumCWarps * 32);
-          // round rd -> buffer rd & 1: keys then values, two blocks each
-          auto issue_round = [&](int rd) {
+          // cache pages of the item's 32-key blocks 32 i + lane, fetched 32 at a time by the first worker warp, so that
+          // no copy waits for a chain of table lookups
+          int pages = 0;
+          if (cw == 0 && kbeg + 32 * lane < kend) pages = p.page_table[b * p.pages_per_seq + (kbeg + 32 * lane) / p.page_size];
+          // round rd -> buffer rd & 1: keys then values, two blocks each (pg0, pg1: the blocks' pages)
+          auto issue_round = [&](int rd, int pg0, int pg1) {
             const int r0 = kbeg + 64 * rd;
             const int nblk = min(2, (kend - r0 + 31) >> 5);
             uint64_t *bar = attn_bar + (rd & 1);
@@ -808,15 +812,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             mbar_expect_tx(bar, (unsigned)(2 * nblk * 32 * HD * 2));
             for (int bb = 0; bb < nblk; ++bb) {
               const int key0 = r0 + 32 * bb;
-              const int page = p.page_table[b * p.pages_per_seq + key0 / p.page_size], slot = key0 % p.page_size;
+              const int page = bb ? pg1 : pg0, slot = key0 % p.page_size;
               const size_t off = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
               bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), bar);
               bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), bar);
             }
           };
-          if (ctid == 0) {   // the first two rounds fly under the staging below
-            if (nround > 0) issue_round(0);
-            if (nround > 1) issue_round(1);
+          if (cw == 0) {   // the first two rounds fly under the staging below
+            const int q0 = __shfl_sync(0xffffffffu, pages, 0), q1 = __shfl_sync(0xffffffffu, pages, 1);
+            const int q2 = __shfl_sync(0xffffffffu, pages, 2), q3 = __shfl_sync(0xffffffffu, pages, 3);
+            if (lane == 0) {
+              if (nround > 0) issue_round(0, q0, q1);
+              if (nround > 1) issue_round(1, q2, q3);
+            }
           }
           // q (scaled), k, v of the block rows with rotary embedding; rows past R are zero
           const float qscale = rsqrtf((float)HD);
@@ -948,7 +956,15 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               }
             }
             named_bar(3, kNumCWarps * 32);   // every warp is done with this buffer
-            if (ctid == 0 && rd + 2 < nround) issue_round(rd + 2);
+            if (cw == 0) {
+              const int nb = 2 * (rd + 2);   // first block of the round that goes into the freed buffer
+              if ((nb & 31) == 0) {
+                const int k0 = kbeg + 32 * (nb + lane);
+                pages = k0 < kend ? p.page_table[b * p.pages_per_seq + k0 / p.page_size] : 0;
+              }
+              const int pa = __shfl_sync(0xffffffffu, pages, nb & 31), pb = __shfl_sync(0xffffffffu, pages, (nb + 1) & 31);
+              if (lane == 0 && rd + 2 < nround) issue_round(rd + 2, pa, pb);
+            }
           }
           // per-warp partials -> shared (over the staging areas, which every warp has left), merged over
           // the eight warps in warp order, stored per (head, split)
