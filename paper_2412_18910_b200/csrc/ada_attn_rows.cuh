@@ -139,7 +139,9 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
       const int key0 = key0_of(h);            // first of these 16 keys
       {
         // ---- scores: 16 rows x 16 keys as two tiles of 8 keys (sa: keys 0..7, sb: keys 8..15)
+        // (the hi and the lo products have accumulators of their own, added at the end: four chains of 8 products)
         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        float sal[4] = {0.f, 0.f, 0.f, 0.f}, sbl[4] = {0.f, 0.f, 0.f, 0.f};
         const uint32_t krow = smem_u32(kst + (size_t)(lane & 7) * HD);
         const int ksw = lane & 7;               // = slot & 7: halves start at multiples of 16
         const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -158,39 +160,53 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
             mma_f16_k16(sa, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
             mma_f16_k16(sb, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
             ldmatrix_x4(ql_u + aoff, a0, a1, a2, a3);
-            mma_f16_k16(sa, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
-            mma_f16_k16(sb, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+            mma_f16_k16(sal, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
+            mma_f16_k16(sbl, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
           }
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { sa[j] += sal[j]; sb[j] += sbl[j]; }
         // ---- online softmax: this thread holds keys kc, kc + 1, kc + 8, kc + 9 of rows g8r and g8r + 8
         const int kc = key0 + 2 * t4;
-        bool ok0[4], ok1[4];    // [key slot] for row g8r / g8r + 8
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int k = kc + (j & 1) + 8 * (j >> 1);
-          ok0[j] = k < kend && k <= qp0;
-          ok1[j] = k < kend && k <= qp1;
-        }
         const float s0[4] = {sa[0], sa[1], sb[0], sb[1]}, s1[4] = {sa[2], sa[3], sb[2], sb[3]};
-        float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          mx0 = fmaxf(mx0, ok0[j] ? s0[j] : -INFINITY);
-          mx1 = fmaxf(mx1, ok1[j] ? s1[j] : -INFINITY);
-        }
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
         float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f}, c0 = 1.f, c1 = 1.f;
-        if (mn0 > -INFINITY) {
+        float mn0, mn1;
+        if (key0 + kAttnHalf <= kend && key0 + kAttnHalf - 1 <= pos0 + rg) {
+          // every row of the group sees all 16 keys (warp-uniform): no masks
+          float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s0[2], s0[3])), mx1 = fmaxf(fmaxf(s1[0], s1[1]), fmaxf(s1[2], s1[3]));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+          mn0 = fmaxf(m0, mx0); mn1 = fmaxf(m1, mx1);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) p0[j] = ok0[j] ? __expf(s0[j] - mn0) : 0.f;
-          c0 = __expf(m0 - mn0);
-        }
-        if (mn1 > -INFINITY) {
+          for (int j = 0; j < 4; ++j) { p0[j] = __expf(s0[j] - mn0); p1[j] = __expf(s1[j] - mn1); }
+          c0 = __expf(m0 - mn0); c1 = __expf(m1 - mn1);
+        } else {
+          bool ok0[4], ok1[4];    // [key slot] for row g8r / g8r + 8
 #pragma unroll
-          for (int j = 0; j < 4; ++j) p1[j] = ok1[j] ? __expf(s1[j] - mn1) : 0.f;
-          c1 = __expf(m1 - mn1);
+          for (int j = 0; j < 4; ++j) {
+            const int k = kc + (j & 1) + 8 * (j >> 1);
+            ok0[j] = k < kend && k <= qp0;
+            ok1[j] = k < kend && k <= qp1;
+          }
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            mx0 = fmaxf(mx0, ok0[j] ? s0[j] : -INFINITY);
+            mx1 = fmaxf(mx1, ok1[j] ? s1[j] : -INFINITY);
+          }
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+          mn0 = fmaxf(m0, mx0); mn1 = fmaxf(m1, mx1);
+          if (mn0 > -INFINITY) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) p0[j] = ok0[j] ? __expf(s0[j] - mn0) : 0.f;
+            c0 = __expf(m0 - mn0);
+          }
+          if (mn1 > -INFINITY) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) p1[j] = ok1[j] ? __expf(s1[j] - mn1) : 0.f;
+            c1 = __expf(m1 - mn1);
+          }
         }
         float ps0 = (p0[0] + p0[1]) + (p0[2] + p0[3]), ps1 = (p1[0] + p1[1]) + (p1[2] + p1[3]);
         ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1); ps1 += __shfl_xor_sync(0xffffffffu, ps1, 1);
@@ -211,13 +227,15 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
         }
         // ---- values: out[16 rows][HD] += w[16 x 16 keys] v[16 keys x HD], two 8-channel tiles per load
         const uint32_t vrow = smem_u32(vst + (size_t)((lane & 7) + 8 * ((lane >> 3) & 1)) * HD);
+        if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {   // some running maximum moved: rescale the sums so far
+#pragma unroll
+          for (int nt = 0; nt < CH; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c1; o[nt][3] *= c1; }
+        }
 #pragma unroll
         for (int c2 = 0; c2 < HD / 16; ++c2) {
           uint32_t v0, v1, v2, v3;   // (keys 0..7, keys 8..15) of channel tile 2 c2, then of tile 2 c2 + 1
           ldmatrix_x4_trans(vrow + ((2 * c2 + (lane >> 4)) << 4), v0, v1, v2, v3);
           float *oa = o[2 * c2], *ob = o[2 * c2 + 1];
-          oa[0] *= c0; oa[1] *= c0; oa[2] *= c1; oa[3] *= c1;
-          ob[0] *= c0; ob[1] *= c0; ob[2] *= c1; ob[3] *= c1;
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), ah[0], ah[1], ah[2], ah[3], v0, v1);
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), al[0], al[1], al[2], al[3], v0, v1);
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(ob), ah[0], ah[1], ah[2], ah[3], v2, v3);
