@@ -350,21 +350,28 @@ bool gemm(ada_ctx *x, int epi, const bf16 *W0, const bf16 *W1, const bf16 *W2, i
 
 void attention(ada_ctx *x, bf16 *kpool, bf16 *vpool, int L, int layer) {
   const ada_config &c = x->c;
-  // query rows of a sequence in groups of 16 across grid.z (a prompt chunk is one sequence with up to 88 rows)
-  // (a prompt chunk is one sequence with up to 128 rows, whatever the batch size of the engine)
-  const int nrg = x->TM > kTcRows ? (x->TM + kRowGroup - 1) / kRowGroup : (x->TM / x->B + kRowGroup - 1) / kRowGroup;
+  // Query rows of a sequence in groups across grid.z.  A prompt chunk is one sequence with up to 128 rows (whatever the
+  // batch size of the engine): groups of 16 rows.  Decode passes have at most n_max + 1 rows per sequence: groups of 8
+  // rows whose hi and lo halves share one 16-row tile (half the products per key); every decode row of a sequence goes
+  // through this form, whatever the shape of its pass.
+  const bool wide = x->TM > kTcRows;
+  const int nrg = wide ? (x->TM + kRowGroup - 1) / kRowGroup : (x->TM / x->B + 7) / 8;
   dim3 g1(c.n_heads, kAttnSplits, x->B * nrg);
   dim3 g2(c.n_heads, x->TM);
+  auto rows_kernel = [&](auto kernel, int smem) {
+    launch_pdl(x, kernel, g1, dim3(128), (size_t)smem, x->pass, x->qrot, kpool, vpool, x->page_table, x->pages_per_seq,
+               c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
+  };
   timed(x, 1, 0.0, [&] {
-  if (c.head_dim == 128) {
-    launch_pdl(x, k_attn_rows<128>, g1, 128, attn_rows_smem_bytes<128>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
-    launch_pdl(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
-  } else {
-    launch_pdl(x, k_attn_rows<64>, g1, 128, attn_rows_smem_bytes<64>(), x->pass, x->qrot, kpool, vpool, x->page_table,
-           x->pages_per_seq, c.page_size, L, layer, c.n_heads, x->attn_part, nrg, c.kv_capacity, x->cnt);
-    launch_pdl(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
-  }
+    if (c.head_dim == 128) {
+      if (wide) rows_kernel(k_attn_rows<128, false>, attn_rows_smem_bytes<128>());
+      else rows_kernel(k_attn_rows<128, true>, attn_rows_smem_bytes<128>());
+      launch_pdl(x, k_attn_combine<128>, g2, 128, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
+    } else {
+      if (wide) rows_kernel(k_attn_rows<64, false>, attn_rows_smem_bytes<64>());
+      else rows_kernel(k_attn_rows<64, true>, attn_rows_smem_bytes<64>());
+      launch_pdl(x, k_attn_combine<64>, g2, 64, 0, x->pass, x->attn_part, x->xhi, x->xlo, x->ldx, c.kv_capacity);
+    }
   });
 }
 
@@ -801,9 +808,13 @@ extern "C" int ada_init(ada_ctx **out, const ada_config *cfg, const ada_weights 
     if (e == cudaSuccess) e = cudaMemcpy(x->d_tcmaps, maps.data(), sizeof(TensorMap128) * maps.size(), cudaMemcpyHostToDevice);
   }
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_attn_rows<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<128>());
+    e = cudaFuncSetAttribute(k_attn_rows<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<128>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_attn_rows<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<64>());
+    e = cudaFuncSetAttribute(k_attn_rows<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<128>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_attn_rows<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<64>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_attn_rows<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_rows_smem_bytes<64>());
   if (e != cudaSuccess) {
     delete x;
     return ADA_ERR_CUDA;

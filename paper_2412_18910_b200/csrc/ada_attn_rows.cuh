@@ -11,8 +11,8 @@
 // as m16n8k16 products per 16 channels (two tiles of 8 keys), online softmax on the accumulator fragments, weighted
 // values as m16n8k16 products over the 16 keys per 8 channels, 16 keys at a time.  Cache elements are 16-bit halves and enter the products as they are;
 // q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, so each product is issued twice and
-// the sums are fp32 (error 2^-22 relative).  Key rows are kept in the cache with their 16-byte chunks XORed by
-// (slot & 7), which makes ldmatrix of 8 consecutive keys conflict-free and lets the copy be verbatim.  A copy always
+// the sums are fp32 (error 2^-22 relative).  Key and value rows are kept in the cache with their 16-byte chunks XORed by
+// (slot & 7), which makes ldmatrix of 8 consecutive keys (plain or transposed) conflict-free and lets the copy be verbatim.  A copy always
 // takes 16 whole rows: rows past the sequence are masked out of the softmax, and every cache row is finite (the
 // pools are cleared at initialisation), so they add exact zeros.
 // Partial (m, l, o[hd]) per (head, split, row) goes to `part`; k_attn_combine merges the splits in split order.
@@ -28,7 +28,7 @@ constexpr int attn_rows_smem_bytes() {
   return 2 * kRowGroup * HD * 2 + 4 * 2 * 2 * kAttnHalf * HD * 2 + 2 * 4 * kRowGroup * 4 + 4 * 2 * 8;
 }
 
-template <int HD>
+template <int HD, bool PACK>
 __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
                                                    const __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
                                                    int page_size, int L, int layer, int H, float *part, int nrg,
@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
   pdl_launch_dependents();
   pdl_wait();                  // queries and the new cache rows come from the kernel before this one
   constexpr int CH = HD / 8;   // 16-byte chunks per row
+  constexpr int RG = PACK ? 8 : kRowGroup;   // query rows per group
   // grid.z = sequences x nrg: CTA (b, rgi) takes the row groups rgi, rgi + nrg, ... of sequence b
   const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / nrg, rgi = blockIdx.z - b * nrg;
   const int4 si = pass->seq_info[b];   // (first row, rows, split size, first position) in one load
@@ -72,8 +73,8 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
   const size_t head_off = ((size_t)layer * H + hh) * page_size * HD;   // inside a page: [layer][head][slot][HD]
   const size_t page_stride = (size_t)L * H * page_size * HD;
 
-  for (int rg = rgi * kRowGroup; rg < R; rg += nrg * kRowGroup) {
-    const int nr = min(kRowGroup, R - rg);
+  for (int rg = rgi * RG; rg < R; rg += nrg * RG) {
+    const int nr = min(RG, R - rg);
     __syncthreads();   // the previous group's merge has read the shared areas; the barriers are initialised
     const int last_pos = pos0 + rg + nr - 1;   // the last position any row of the group sees
     // half h of this warp: keys key0(h) .. key0(h) + 15 (the split's halves are dealt to the four warps in turn)
@@ -95,8 +96,8 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
       if (lane == 0 && valid(0)) issue(0, p0);
       if (lane == 0 && valid(1)) issue(1, p1);
     }
-    {   // the group's query rows as (hi, lo) halves; rows past nr are zero
-      constexpr int PER = kRowGroup * HD / 4 / 128;
+    {   // the group's query rows as (hi, lo) halves; rows past nr are zero.  PACK: hi of row r in tile row r, lo in row r + 8
+      constexpr int PER = RG * HD / 4 / 128;
       float4 qv[PER];
 #pragma unroll
       for (int u = 0; u < PER; ++u) {
@@ -121,23 +122,106 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
         pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
         pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
         *reinterpret_cast<uint2 *>(qh_s + o) = ph;
-        *reinterpret_cast<uint2 *>(ql_s + o) = pl;
+        *reinterpret_cast<uint2 *>((PACK ? qh_s + 8 * HD : ql_s) + o) = pl;
       }
     }
     __syncthreads();
 
     // running maxima, sums and outputs of rows g8r and g8r + 8 over this warp's keys
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float m0 = -INFINITY, l0 = 0.f;
+    [[maybe_unused]] float m1 = -INFINITY, l1 = 0.f;
     float o[CH][4];
 #pragma unroll
     for (int nt = 0; nt < CH; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-    const int qp0 = pos0 + rg + g8r, qp1 = qp0 + 8;
+    const int qp0 = pos0 + rg + g8r;
+    [[maybe_unused]] const int qp1 = qp0 + 8;
 
     for (int h = 0; valid(h); ++h) {
       const __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD, *vst = kst + kAttnHalf * HD;
       mbar_wait(&bars[h & 1], (uses[h & 1]++) & 1u, cnt, &abort_s);
       const int key0 = key0_of(h);            // first of these 16 keys
-      {
+      if constexpr (PACK) {
+        // ---- 8 query rows: tile row r holds the hi half of row r, tile row r + 8 its lo half, so one product gives
+        // both parts; this thread's row is g8r, its hi sums are accumulator elements 0, 1 and its lo sums 2, 3
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t krow = smem_u32(kst + (size_t)(lane & 7) * HD);
+        const int ksw = lane & 7;
+        const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int kp = 0; kp < HD / 32; ++kp) {
+          uint32_t ka0, ka1, ka2, ka3, kb0, kb1, kb2, kb3;
+          const uint32_t koff = (uint32_t)(((kp * 4 + (lane >> 3)) ^ ksw) << 4);
+          ldmatrix_x4(krow + koff, ka0, ka1, ka2, ka3);
+          ldmatrix_x4(krow + 8 * HD * 2 + koff, kb0, kb1, kb2, kb3);
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int ks = kp * 2 + h2;
+            const uint32_t aoff = (uint32_t)(arow * (HD * 2) + (((ks * 2 + (lane >> 4)) ^ (arow & 7)) << 4));
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(qh_u + aoff, a0, a1, a2, a3);
+            mma_f16_k16(sa, a0, a1, a2, a3, h2 ? ka2 : ka0, h2 ? ka3 : ka1);
+            mma_f16_k16(sb, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+          }
+        }
+        // ---- online softmax of row g8r: keys kc, kc + 1, kc + 8, kc + 9
+        const int kc = key0 + 2 * t4;
+        const float s0[4] = {sa[0] + sa[2], sa[1] + sa[3], sb[0] + sb[2], sb[1] + sb[3]};
+        float p0[4] = {0.f, 0.f, 0.f, 0.f}, c0 = 1.f, mn0;
+        if (key0 + kAttnHalf <= kend && key0 + kAttnHalf - 1 <= pos0 + rg) {   // every row sees all 16 keys (warp-uniform)
+          float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s0[2], s0[3]));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+          mn0 = fmaxf(m0, mx0);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) p0[j] = __expf(s0[j] - mn0);
+          c0 = __expf(m0 - mn0);
+        } else {
+          bool ok0[4];
+          float mx0 = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int k = kc + (j & 1) + 8 * (j >> 1);
+            ok0[j] = k < kend && k <= qp0;
+            mx0 = fmaxf(mx0, ok0[j] ? s0[j] : -INFINITY);
+          }
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+          mn0 = fmaxf(m0, mx0);
+          if (mn0 > -INFINITY) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) p0[j] = ok0[j] ? __expf(s0[j] - mn0) : 0.f;
+            c0 = __expf(m0 - mn0);
+          }
+        }
+        float ps0 = (p0[0] + p0[1]) + (p0[2] + p0[3]);
+        ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1);
+        ps0 += __shfl_xor_sync(0xffffffffu, ps0, 2);
+        l0 = l0 * c0 + ps0;
+        m0 = mn0;
+        // weights: A operand rows g8r (hi halves) and g8r + 8 (lo halves); a0, a1: keys 0..7, a2, a3: keys 8..15
+        uint32_t aw[4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const __half2 ph = __floats2half2_rn(p0[2 * j], p0[2 * j + 1]);
+          const float2 pf = __half22float2(ph);
+          const __half2 pl = __floats2half2_rn(p0[2 * j] - pf.x, p0[2 * j + 1] - pf.y);
+          aw[2 * j] = *reinterpret_cast<const uint32_t *>(&ph);
+          aw[2 * j + 1] = *reinterpret_cast<const uint32_t *>(&pl);
+        }
+        // ---- values: elements 0, 1 of a tile collect the hi weights' sums of row g8r, elements 2, 3 the lo weights' sums
+        const uint32_t vrow = smem_u32(vst + (size_t)((lane & 7) + 8 * ((lane >> 3) & 1)) * HD);
+        if (__any_sync(0xffffffffu, c0 != 1.f)) {
+#pragma unroll
+          for (int nt = 0; nt < CH; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c0; o[nt][3] *= c0; }
+        }
+#pragma unroll
+        for (int c2 = 0; c2 < HD / 16; ++c2) {
+          uint32_t v0, v1, v2, v3;
+          ldmatrix_x4_trans(vrow + (((2 * c2 + (lane >> 4)) ^ (lane & 7)) << 4), v0, v1, v2, v3);
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(o[2 * c2]), aw[0], aw[1], aw[2], aw[3], v0, v1);
+          mma_f16_k16(*reinterpret_cast<float (*)[4]>(o[2 * c2 + 1]), aw[0], aw[1], aw[2], aw[3], v2, v3);
+        }
+      } else {
         // ---- scores: 16 rows x 16 keys as two tiles of 8 keys (sa: keys 0..7, sb: keys 8..15)
         // (the hi and the lo products have accumulators of their own, added at the end: four chains of 8 products)
         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
@@ -234,7 +318,7 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
 #pragma unroll
         for (int c2 = 0; c2 < HD / 16; ++c2) {
           uint32_t v0, v1, v2, v3;   // (keys 0..7, keys 8..15) of channel tile 2 c2, then of tile 2 c2 + 1
-          ldmatrix_x4_trans(vrow + ((2 * c2 + (lane >> 4)) << 4), v0, v1, v2, v3);
+          ldmatrix_x4_trans(vrow + (((2 * c2 + (lane >> 4)) ^ (lane & 7)) << 4), v0, v1, v2, v3);
           float *oa = o[2 * c2], *ob = o[2 * c2 + 1];
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), ah[0], ah[1], ah[2], ah[3], v0, v1);
           mma_f16_k16(*reinterpret_cast<float (*)[4]>(oa), al[0], al[1], al[2], al[3], v0, v1);
@@ -252,12 +336,16 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
     __syncthreads();
 #pragma unroll
     for (int nt = 0; nt < CH; ++nt) {
-      *reinterpret_cast<float2 *>(&o_s[warp][g8r][nt * 8 + 2 * t4]) = make_float2(o[nt][0], o[nt][1]);
-      *reinterpret_cast<float2 *>(&o_s[warp][g8r + 8][nt * 8 + 2 * t4]) = make_float2(o[nt][2], o[nt][3]);
+      if constexpr (PACK) {   // hi and lo sums of the row
+        *reinterpret_cast<float2 *>(&o_s[warp][g8r][nt * 8 + 2 * t4]) = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
+      } else {
+        *reinterpret_cast<float2 *>(&o_s[warp][g8r][nt * 8 + 2 * t4]) = make_float2(o[nt][0], o[nt][1]);
+        *reinterpret_cast<float2 *>(&o_s[warp][g8r + 8][nt * 8 + 2 * t4]) = make_float2(o[nt][2], o[nt][3]);
+      }
     }
     if (t4 == 0) {
       m_s[warp][g8r] = m0; l_s[warp][g8r] = l0;
-      m_s[warp][g8r + 8] = m1; l_s[warp][g8r + 8] = l1;
+      if constexpr (!PACK) { m_s[warp][g8r + 8] = m1; l_s[warp][g8r + 8] = l1; }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < nr * HD; i += 128) {

@@ -373,7 +373,7 @@ __global__ void __launch_bounds__(256) k_reduce_h(const ReduceHArgs a) {
 }
 
 // QKV: sums of the splits times 1 / rms(row), then rotary embedding of q and k (rotate-half pairing), q scaled by
-// 1 / sqrt(hd) to qout, k and v as 16-bit cache elements into the paged pools (key rows with their 16-byte chunks XORed
+// 1 / sqrt(hd) to qout, k and v as 16-bit cache elements into the paged pools (rows with their 16-byte chunks XORed
 // by slot & 7).  Block (group of 256 (head, i) pairs, pass row); thread = one pair (i, i + hd / 2) of one head.
 struct ReduceQkvArgs {
   const float *part; int S;            // [S][128][3 d]
@@ -412,8 +412,8 @@ __global__ void __launch_bounds__(256) k_reduce_qkv(const ReduceQkvArgs a) {
   const int sw = slot & 7;
   a.kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[2] * cs.x - v[3] * cs.y);
   a.kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[3] * cs.x + v[2] * cs.y);
-  a.vpool[base + i] = kv_store(v[4]);
-  a.vpool[base + i + half] = kv_store(v[5]);
+  a.vpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[4]);          // value rows: the same chunk order as key rows
+  a.vpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[5]);
 }
 
 // SwiGLU: gate and up sums of the splits times 1 / rms(row), silu(gate) * up as hi / lo planes.

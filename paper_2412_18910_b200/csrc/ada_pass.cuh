@@ -865,12 +865,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                 const int pos = pos0 + r;
                 const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
                 const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
-                // key rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to shared
-                // memory, eight consecutive keys then sit in eight different bank groups
+                // key and value rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to
+                // shared memory, eight consecutive rows then sit in eight different bank groups (ldmatrix of 8 keys'
+                // chunk, plain for the scores and transposed for the weighted values, is conflict-free)
                 const int sw = slot & 7;
                 p.kpool[base + ((((c >> 3) ^ sw) << 3) | (c & 7))] = k0;
                 p.kpool[base + (((((c + half) >> 3) ^ sw) << 3) | (c & 7))] = k1;
-                p.vpool[base + c] = v0; p.vpool[base + c + half] = v1;
+                p.vpool[base + ((((c >> 3) ^ sw) << 3) | (c & 7))] = v0;
+                p.vpool[base + (((((c + half) >> 3) ^ sw) << 3) | (c & 7))] = v1;
               }
             }
           }
@@ -943,7 +945,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               for (int nq = 0; nq < 4; ++nq) {            // four 8-channel tiles per load
                 if (nq * 32 < HD) {
                   uint32_t v0, v1, v2, v3;
-                  ldmatrix_x4_trans(vrow + ((nq * 4 + (lane >> 3)) << 4), v0, v1, v2, v3);
+                  ldmatrix_x4_trans(vrow + (((nq * 4 + (lane >> 3)) ^ ksw) << 4), v0, v1, v2, v3);
 #pragma unroll
                   for (int j = 0; j < 4; ++j) {
                     float *oo = o[nq * 4 + j];
