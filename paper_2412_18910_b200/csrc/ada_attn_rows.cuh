@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
   __half *ql_s = qh_s + kRowGroup * HD;                               // q lo, same layout
   __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(ql_s + kRowGroup * HD);   // [4 warps][2 buffers][K, V][16 keys][HD]
   __nv_bfloat16 *wst = stg + (size_t)warp * 2 * 2 * kAttnHalf * HD;
-  float (*o_s)[kRowGroup][HD] = reinterpret_cast<float (*)[kRowGroup][HD]>(stg);    // merge area, over the staging areas
+  float (*o_s)[kRowGroup][HD + 8] = reinterpret_cast<float (*)[kRowGroup][HD + 8]>(stg);   // merge area, over the staging areas (rows padded: the fragment stores of 8 rows fall into different banks)
   unsigned char *tail = attn_rows_smem + 2 * kRowGroup * HD * 2 + 4 * 2 * 2 * kAttnHalf * HD * 2;
   float (*m_s)[kRowGroup] = reinterpret_cast<float (*)[kRowGroup]>(tail);
   float (*l_s)[kRowGroup] = m_s + 4;

@@ -60,7 +60,8 @@ constexpr int kMiscBytes = 3072;                 // mbarriers and small per-CTA 
 // during the attention phase); the ring is NOT reused: the producer keeps filling it meanwhile
 constexpr int kAttnLoopBytes = 4 * 16 * 128 * 2 + 2 * 2 * 2 * 32 * 128 * 2;   // q hi, q lo, new k, v rows; two buffers of staged keys and values
 constexpr int kPassMaxSplits = 32;                // cache splits of a sequence at most (its split size is at least capacity / 32)
-constexpr int kAttnPartBytes = 8 * 16 * 130 * 4 + 8 * 16 * 4 + kPassMaxSplits * 16 * 4;   // per-warp partial results, merge weights
+constexpr int kPartRow = 136;   // floats per row of a warp's partial result: 128 sums, m, l, padded so that a half-warp's fragment stores (4 rows x 4 column pairs) fall into 32 different banks
+constexpr int kAttnPartBytes = 8 * 16 * kPartRow * 4 + 8 * 16 * 4 + kPassMaxSplits * 16 * 4;   // per-warp partial results, merge weights
 constexpr int kAttnBytes = kAttnPartBytes > kAttnLoopBytes ? kAttnPartBytes : kAttnLoopBytes;
 // (a tensor-core read of 128 tile rows may run a few KB past the last ring stage: the areas below follow the ring)
 constexpr int kScratchBytes = (kXBufs * kXBufBytes + kRedBytes) > kAttnBytes ? (kXBufs * kXBufBytes + kRedBytes) : kAttnBytes;
@@ -786,8 +787,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         __nv_bfloat16 *k_s = reinterpret_cast<__nv_bfloat16 *>(ql_s + 16 * 128);    // new rows, rotated [16][128]
         __nv_bfloat16 *v_s = k_s + 16 * 128;
         __nv_bfloat16 *stg = v_s + 16 * 128;                                         // [2 buffers][K, V][2 blocks][32 keys][128]
-        float *part_s = reinterpret_cast<float *>(xbuf);                              // [8 warps][16 rows][130], reuses the above
-        float *lw_s = part_s + 8 * 16 * 130;                                          // [8 warps][16 rows] merge weights
+        float *part_s = reinterpret_cast<float *>(xbuf);                              // [8 warps][16 rows][kPartRow], reuses the above
+        float *lw_s = part_s + 8 * 16 * kPartRow;                                          // [8 warps][16 rows] merge weights
         float *wgt = lw_s + 8 * 16;                                                   // [splits][16 rows] (cross-CTA merge)
         const int g8r = lane >> 2, t4 = lane & 3;
         const int bw = cw >> 2, kq = cw & 3;
@@ -859,8 +860,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const __nv_bfloat16 k0 = kv_store(ka[u] * cs[u].x - kb[u] * cs[u].y);   // 16-bit cache elements (see kv_store)
               const __nv_bfloat16 k1 = kv_store(kb[u] * cs[u].x + ka[u] * cs[u].y);
               const __nv_bfloat16 v0 = kv_store(va[u]), v1 = kv_store(vb[u]);
-              k_s[r * 128 + c] = k0; k_s[r * 128 + c + half] = k1;
-              v_s[r * 128 + c] = v0; v_s[r * 128 + c + half] = v1;
+              k_s[o0] = k0; k_s[o1] = k1;      // (the staged rows have their chunks XORed by row & 7, like q)
+              v_s[o0] = v0; v_s[o1] = v1;
               if (split == 0 && r < R) {  // one item per head stores the new rows in the cache
                 const int pos = pos0 + r;
                 const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
@@ -893,10 +894,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               // ---- scores: 16 rows x 8 keys
               float sc[4] = {0.f, 0.f, 0.f, 0.f};
               const int myk = key0 + (lane & 7);          // key whose row address this lane supplies
-              const bool fresh = myk >= pos0;             // a row of this pass: from the staged new rows, natural layout
+              const bool fresh = myk >= pos0;             // a row of this pass: from the staged new rows
               const uint32_t krow = fresh ? smem_u32(k_s + (size_t)min(myk - pos0, 15) * 128)
                                           : smem_u32(kst + (size_t)(bw * 32 + 8 * kq + (lane & 7)) * HD);
-              const int ksw = fresh ? 0 : (lane & 7);     // = slot & 7: blocks start at multiples of 32
+              const int ksw = fresh ? ((myk - pos0) & 7) : (lane & 7);     // cache rows: slot & 7 (blocks start at multiples of 32); staged rows: row & 7
               const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
               for (int kp = 0; kp < 4; ++kp) {            // pairs of 16-channel steps
@@ -973,24 +974,24 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
 #pragma unroll
           for (int nt = 0; nt < 16; ++nt)
             if (nt * 8 < HD) {
-              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r) * 130 + nt * 8 + 2 * t4) = make_float2(o[nt][0], o[nt][1]);
-              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r + 8) * 130 + nt * 8 + 2 * t4) = make_float2(o[nt][2], o[nt][3]);
+              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r) * kPartRow + nt * 8 + 2 * t4) = make_float2(o[nt][0], o[nt][1]);
+              *reinterpret_cast<float2 *>(part_s + (cw * 16 + g8r + 8) * kPartRow + nt * 8 + 2 * t4) = make_float2(o[nt][2], o[nt][3]);
             }
           if (t4 == 0) {
-            part_s[(cw * 16 + g8r) * 130 + 128] = m0; part_s[(cw * 16 + g8r) * 130 + 129] = l0;
-            part_s[(cw * 16 + g8r + 8) * 130 + 128] = m1; part_s[(cw * 16 + g8r + 8) * 130 + 129] = l1;
+            part_s[(cw * 16 + g8r) * kPartRow + 128] = m0; part_s[(cw * 16 + g8r) * kPartRow + 129] = l0;
+            part_s[(cw * 16 + g8r + 8) * kPartRow + 128] = m1; part_s[(cw * 16 + g8r + 8) * kPartRow + 129] = l1;
           }
           named_bar(3, kNumCWarps * 32);
           if (ctid < 16) {   // per row: maximum over the warps, each warp's weight, the merged sum
             const int r = ctid;
             float M = -INFINITY;
-            for (int w8 = 0; w8 < kNumCWarps; ++w8) M = fmaxf(M, part_s[(w8 * 16 + r) * 130 + 128]);
+            for (int w8 = 0; w8 < kNumCWarps; ++w8) M = fmaxf(M, part_s[(w8 * 16 + r) * kPartRow + 128]);
             float lo = 0.f;
             for (int w8 = 0; w8 < kNumCWarps; ++w8) {
-              const float mw = part_s[(w8 * 16 + r) * 130 + 128];
+              const float mw = part_s[(w8 * 16 + r) * kPartRow + 128];
               const float e = mw > -INFINITY ? __expf(mw - M) : 0.f;
               lw_s[w8 * 16 + r] = e;
-              lo += part_s[(w8 * 16 + r) * 130 + 129] * e;
+              lo += part_s[(w8 * 16 + r) * kPartRow + 129] * e;
             }
             if (r < R) {
               float *gp = p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2);
@@ -1002,7 +1003,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const int r = i / HD, c = i - r * HD;
             float oo = 0.f;
 #pragma unroll
-            for (int w8 = 0; w8 < kNumCWarps; ++w8) oo += part_s[(w8 * 16 + r) * 130 + c] * lw_s[w8 * 16 + r];
+            for (int w8 = 0; w8 < kNumCWarps; ++w8) oo += part_s[(w8 * 16 + r) * kPartRow + c] * lw_s[w8 * 16 + r];
             __stcg(p.attn_part + (((size_t)hh * nsp + split) * 16 + r) * (HD + 2) + c, oo);
           }
           // the item that arrives last for this head merges the splits in split order
