@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "decode tokens/sec at batch 1 (device-timed)"
 UNIT = "tokens/s"
 # measured dram__bytes_read+write over algorithmic bytes of k_pass (None once the kernel changed since the capture)
-TRAFFIC_PER_ALGORITHMIC_BYTE = 1.012
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.011
 
 
 def load_peaks():
@@ -309,6 +309,9 @@ def main():
     ap.add_argument("--no-teacher-forced", action="store_true", help="skip the teacher-forced sweep n = 1..n_max (7b workload only)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (a reduced case for profiler captures)")
     ap.add_argument("--profile-only", action="store_true", help="prefill, a few verify passes, exit (for ncu)")
+    ap.add_argument("--profile-batch8", action="store_true",
+                    help="with --profile-only: the ragged batch of 8 (multi-row path) instead of batch 1: the 8 prompts, then "
+                         "--steps iterations through the separate calls")
     args = ap.parse_args()
 
     import numpy as np
@@ -352,6 +355,20 @@ def main():
     dev = torch.device("cuda:%d" % local)
     torch.cuda.set_device(dev)
     weights = si.make_weights(sh)
+    if args.profile_only and args.profile_batch8:
+        sh8 = si.scaled(si.SHAPES["7b_b8"], n_layers=sh.n_layers, name="7b_b8-%dlayers" % sh.n_layers)
+        eng = Engine(sh8, weights, max_batch=sh8.batch, kv_capacity=sh8.kv_capacity, device=str(dev))
+        for b, pr in enumerate(si.make_prompts(sh8)):
+            eng.ada_prefill(b, torch.from_numpy(pr).to(dev), None)
+        for _ in range(max(1, K)):
+            eng.ada_ldlp_predict(eng.d_n)
+            eng.ada_draft(eng.d_n, eng.d_draft)
+            eng.ada_verify(eng.d_draft, eng.d_n, eng.d_target)
+            eng.ada_accept()
+        torch.cuda.synchronize(dev)
+        print(json.dumps({"profile_only": True, "batch": sh8.batch, "status": eng.ada_get_counters()["status"]}))
+        eng.close()
+        return 0
     prompt = si.uniform_ids(si.DEFAULT_SEED + rank, "prompt0", sh.prompt_len, sh.vocab)
     eng = Engine(sh, weights, max_batch=1, kv_capacity=sh.kv_capacity, device=str(dev))
     per_episode = max(1, (sh.kv_capacity - sh.prompt_len - sh.n_max - 4) // (sh.n_max + 1))
