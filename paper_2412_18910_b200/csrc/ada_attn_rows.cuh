@@ -31,9 +31,10 @@ constexpr int attn_rows_smem_bytes() {
 template <int HD, bool PACK>
 __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float *q, const __nv_bfloat16 *kpool,
                                                    const __nv_bfloat16 *vpool, const int *page_table, int pages_per_seq,
-                                                   int page_size, int L, int layer, int H, float *part, int nrg,
+                                                   int /*page_size = kPageSize*/, int L, int layer, int H, float *part, int nrg,
                                                    int cap, Counters *cnt) {
   static_assert(HD == 64 || HD == 128, "head width");
+  constexpr int page_size = kPageSize;
   pdl_launch_dependents();
   pdl_wait();                  // queries and the new cache rows come from the kernel before this one
   constexpr int CH = HD / 8;   // 16-byte chunks per row

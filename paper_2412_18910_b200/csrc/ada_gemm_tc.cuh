@@ -407,8 +407,8 @@ __global__ void __launch_bounds__(256) k_reduce_qkv(const ReduceQkvArgs a) {
   const float2 cs = a.rope[(size_t)pos * half + i];
   a.qout[(size_t)t * d + o] = (v[0] * cs.x - v[1] * cs.y) * a.qscale;
   a.qout[(size_t)t * d + o + half] = (v[1] * cs.x + v[0] * cs.y) * a.qscale;
-  const int page = a.page_table[b * a.pages_per_seq + pos / a.page_size], slot = pos % a.page_size;
-  const size_t base = (((size_t)page * a.L + a.layer) * a.H + hh) * a.page_size * a.hd + (size_t)slot * a.hd;
+  const int page = a.page_table[b * a.pages_per_seq + pos / kPageSize], slot = pos % kPageSize;
+  const size_t base = (((size_t)page * a.L + a.layer) * a.H + hh) * kPageSize * a.hd + (size_t)slot * a.hd;
   const int sw = slot & 7;
   a.kpool[base + ((((i >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[2] * cs.x - v[3] * cs.y);
   a.kpool[base + (((((i + half) >> 3) ^ sw) << 3) | (i & 7))] = kv_store(v[3] * cs.x + v[2] * cs.y);

@@ -17,6 +17,7 @@
 namespace ada {
 
 constexpr int kMaxBatch = 8;
+constexpr int kPageSize = 64;   // positions per cache page (the configuration accepts no other): divisions by it are shifts
 constexpr int kMaxRows = 128;   // rows of one pass (all sequences together)
 constexpr int kAttnSplits = 8;  // KV splits per (sequence, head)
 constexpr int kRowGroup = 16;   // query rows of one attention CTA (one m16 tile)

@@ -792,7 +792,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
         float *wgt = lw_s + 8 * 16;                                                   // [splits][16 rows] (cross-CTA merge)
         const int g8r = lane >> 2, t4 = lane & 3;
         const int bw = cw >> 2, kq = cw & 3;
-        const size_t head_stride = (size_t)p.page_size * HD;
+        const size_t head_stride = (size_t)kPageSize * HD;
         const uint32_t qh_u = smem_u32(qh_s), ql_u = smem_u32(ql_s);
         for (int item = cta; item < p.H * nsp; item += ncta) {
           const int hh = item / nsp, split = item - hh * nsp;
@@ -802,7 +802,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           // cache pages of the item's 32-key blocks 32 i + lane, fetched 32 at a time by the first worker warp, so that
           // no copy waits for a chain of table lookups
           int pages = 0;
-          if (cw == 0 && kbeg + 32 * lane < kend) pages = p.page_table[b * p.pages_per_seq + (kbeg + 32 * lane) / p.page_size];
+          if (cw == 0 && kbeg + 32 * lane < kend) pages = p.page_table[b * p.pages_per_seq + (kbeg + 32 * lane) / kPageSize];
           // round rd -> buffer rd & 1: keys then values, two blocks each (pg0, pg1: the blocks' pages)
           auto issue_round = [&](int rd, int pg0, int pg1) {
             const int r0 = kbeg + 64 * rd;
@@ -813,7 +813,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             mbar_expect_tx(bar, (unsigned)(2 * nblk * 32 * HD * 2));
             for (int bb = 0; bb < nblk; ++bb) {
               const int key0 = r0 + 32 * bb;
-              const int page = bb ? pg1 : pg0, slot = key0 % p.page_size;
+              const int page = bb ? pg1 : pg0, slot = key0 % kPageSize;
               const size_t off = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
               bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), bar);
               bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), bar);
@@ -864,7 +864,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               v_s[o0] = v0; v_s[o1] = v1;
               if (split == 0 && r < R) {  // one item per head stores the new rows in the cache
                 const int pos = pos0 + r;
-                const int page = p.page_table[b * p.pages_per_seq + pos / p.page_size], slot = pos % p.page_size;
+                const int page = p.page_table[b * p.pages_per_seq + pos / kPageSize], slot = pos % kPageSize;
                 const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
                 // key and value rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to
                 // shared memory, eight consecutive rows then sit in eight different bank groups (ldmatrix of 8 keys'
@@ -963,7 +963,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const int nb = 2 * (rd + 2);   // first block of the round that goes into the freed buffer
               if ((nb & 31) == 0) {
                 const int k0 = kbeg + 32 * (nb + lane);
-                pages = k0 < kend ? p.page_table[b * p.pages_per_seq + k0 / p.page_size] : 0;
+                pages = k0 < kend ? p.page_table[b * p.pages_per_seq + k0 / kPageSize] : 0;
               }
               const int pa = __shfl_sync(0xffffffffu, pages, nb & 31), pb = __shfl_sync(0xffffffffu, pages, (nb + 1) & 31);
               if (lane == 0 && rd + 2 < nround) issue_round(rd + 2, pa, pb);
