@@ -829,11 +829,18 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           }
           // q (scaled), k, v of the block rows with rotary embedding; rows past R are zero
           const float qscale = rsqrtf((float)HD);
-          for (int i0 = 0; i0 < 16 * half; i0 += 2 * kNumCWarps * 32) {
-            float qa[2], qb[2], ka[2], kb[2], va[2], vb[2];
-            float2 cs[2];
+          // (all loads of a thread's four elements, and the pages its cache rows go to, in one round trip)
+          const int pos_last = pos0 + R - 1;
+          int page_first = 0, page_last = 0;
+          if (split == 0) {
+            page_first = p.page_table[b * p.pages_per_seq + pos0 / kPageSize];
+            page_last = p.page_table[b * p.pages_per_seq + pos_last / kPageSize];
+          }
+          for (int i0 = 0; i0 < 16 * half; i0 += 4 * kNumCWarps * 32) {
+            float qa[4], qb[4], ka[4], kb[4], va[4], vb[4];
+            float2 cs[4];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {   // all loads of two elements first
+            for (int u = 0; u < 4; ++u) {
               const int i = i0 + u * kNumCWarps * 32 + ctid;
               const int r = i / half, c = i - r * half;
               qa[u] = qb[u] = ka[u] = kb[u] = va[u] = vb[u] = 0.f;
@@ -847,7 +854,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               }
             }
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < 4; ++u) {
               const int i = i0 + u * kNumCWarps * 32 + ctid;
               if (i >= 16 * half) continue;
               const int r = i / half, c = i - r * half;
@@ -864,7 +871,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               v_s[o0] = v0; v_s[o1] = v1;
               if (split == 0 && r < R) {  // one item per head stores the new rows in the cache
                 const int pos = pos0 + r;
-                const int page = p.page_table[b * p.pages_per_seq + pos / kPageSize], slot = pos % kPageSize;
+                // (at most 16 rows: they lie in the page of the first row or in the page of the last)
+                const int page = pos / kPageSize == pos0 / kPageSize ? page_first : page_last, slot = pos % kPageSize;
                 const size_t base = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
                 // key and value rows are stored with their 16-byte chunks XORed by (slot & 7): copied verbatim to
                 // shared memory, eight consecutive rows then sit in eight different bank groups (ldmatrix of 8 keys'
@@ -892,7 +900,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const int key0 = r0 + 32 * bw + 8 * kq;     // first of this warp's 8 keys
             if (bw < nblk && key0 < kend) {
               // ---- scores: 16 rows x 8 keys
-              float sc[4] = {0.f, 0.f, 0.f, 0.f};
+              float sc[4] = {0.f, 0.f, 0.f, 0.f}, scl[4] = {0.f, 0.f, 0.f, 0.f};   // hi and lo products apart: two chains of 8
               const int myk = key0 + (lane & 7);          // key whose row address this lane supplies
               const bool fresh = myk >= pos0;             // a row of this pass: from the staged new rows
               const uint32_t krow = fresh ? smem_u32(k_s + (size_t)min(myk - pos0, 15) * 128)
@@ -912,10 +920,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
                     ldmatrix_x4(qh_u + aoff, a0, a1, a2, a3);
                     mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
                     ldmatrix_x4(ql_u + aoff, a0, a1, a2, a3);
-                    mma_f16_k16(sc, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
+                    mma_f16_k16(scl, a0, a1, a2, a3, h2 ? kb2 : kb0, h2 ? kb3 : kb1);
                   }
                 }
               }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) sc[j] += scl[j];
               // ---- online softmax: this thread holds keys kc, kc + 1 of rows g8r and g8r + 8
               const int kc = key0 + 2 * t4;
               const bool s00 = kc < kend && kc <= pos0 + g8r, s01 = kc + 1 < kend && kc + 1 <= pos0 + g8r;
@@ -1063,19 +1073,44 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               for (int s2 = 0; s2 < nsp; ++s2) wgt[s2 * 16 + r] *= inv;
             }
             named_bar(3, kNumCWarps * 32);
-            for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
-              const int r = i / HD, c = i - r * HD;
-              const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2) + c;
-              const size_t sst = (size_t)16 * (HD + 2);
-              float oo = 0.f;
-              for (int s0 = 0; s0 < nsp; s0 += 8) {
-                float ov[8];
+            const size_t sst = (size_t)16 * (HD + 2);
+            if (nsp <= 8) {
+              // four output elements per thread and batch: all their splits' loads are in flight together
+              for (int k0 = 0; k0 < R * HD; k0 += 4 * kNumCWarps * 32) {
+                float ov[4][8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) ov[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst) : 0.f;
+                for (int k = 0; k < 4; ++k) {
+                  const int i = k0 + k * kNumCWarps * 32 + ctid;
+                  const int r = i / HD, c = i - r * HD;
+                  const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2) + c;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) oo += s0 + u < nsp ? ov[u] * wgt[(s0 + u) * 16 + r] : 0.f;
+                  for (int u = 0; u < 8; ++u) ov[k][u] = (i < R * HD && u < nsp) ? __ldcg(gp + u * sst) : 0.f;
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int i = k0 + k * kNumCWarps * 32 + ctid;
+                  if (i >= R * HD) continue;
+                  const int r = i / HD, c = i - r * HD;
+                  float oo = 0.f;
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) oo += u < nsp ? ov[k][u] * wgt[u * 16 + r] : 0.f;
+                  xstore(p.at, r, hh * HD + c, oo);
+                }
               }
-              xstore(p.at, r, hh * HD + c, oo);
+            } else {
+              for (int i = ctid; i < R * HD; i += kNumCWarps * 32) {
+                const int r = i / HD, c = i - r * HD;
+                const float *gp = p.attn_part + (((size_t)hh * nsp) * 16 + r) * (HD + 2) + c;
+                float oo = 0.f;
+                for (int s0 = 0; s0 < nsp; s0 += 8) {
+                  float ov[8];
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) ov[u] = s0 + u < nsp ? __ldcg(gp + (s0 + u) * sst) : 0.f;
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) oo += s0 + u < nsp ? ov[u] * wgt[(s0 + u) * 16 + r] : 0.f;
+                }
+                xstore(p.at, r, hh * HD + c, oo);
+              }
             }
             if (ctid == 0) p.attn_cnt[hh] = 0;
           }
