@@ -245,6 +245,54 @@ def test_batch_of_two_with_sixteen_rows_matches_per_sequence_oracle():
         e.close()
 
 
+def test_launch_chain_equals_plain_stream_order_bit_for_bit(monkeypatch):
+    """The multi-kernel path launches a layer's kernels with programmatic dependent launch (each may start while the
+    one before it runs and waits inside before it touches that kernel's data).  With ADA_NO_PDL set at ada_init the
+    same kernels run in plain stream order: prompt features, draft features, tokens and all verify logits of a ragged
+    batch must be the same bits, through the separate calls and through the step graph."""
+    from paper_2412_18910_b200 import Engine
+    sh = si.SHAPES["tiny"]
+    w = si.make_weights(sh)
+    prompts = [si.uniform_ids(17, "pdl%d" % b, L, sh.vocab) for b, L in enumerate((150, 33, 64))]
+    runs = []
+    for no_pdl in (False, True):
+        if no_pdl:
+            monkeypatch.setenv("ADA_NO_PDL", "1")
+        else:
+            monkeypatch.delenv("ADA_NO_PDL", raising=False)
+        e = Engine(sh, w, max_batch=3, kv_capacity=256)
+        try:
+            rec = []
+            for b in range(3):
+                rec.append(e.prefill(b, prompts[b]))
+            feat = e.ada_debug_buffer(0, torch.float32, (3, 256, sh.d_model))
+            rec.append(feat[0, :150].cpu().numpy().copy())
+            e.ada_force_n([3, 8, 5])
+            logits = torch.zeros(3 * (sh.n_max + 1), sh.vocab, dtype=torch.float32, device=e.dev)
+            for it in range(3):                     # separate calls, with the logits of every verify row
+                e.ada_ldlp_predict(e.d_n)
+                e.ada_draft(e.d_n, e.d_draft)
+                e.ada_verify(e.d_draft, e.d_n, e.d_target, logits)
+                e.ada_accept()
+                torch.cuda.synchronize()
+                rec.append(e.d_draft.cpu().numpy().copy())
+                rec.append(e.d_target.cpu().numpy().copy())
+                rec.append(logits.cpu().numpy().copy())
+            dfeat = e.ada_debug_buffer(4, torch.float32, (3, sh.n_max, sh.d_model))
+            for b, n in enumerate((3, 8, 5)):       # (rows past a sequence's draft length are never written)
+                rec.append(dfeat[b, :n].cpu().numpy().copy())
+            for it in range(4):                     # the step graph
+                g = e.step()
+                rec.append(np.asarray(g["k"])); rec.append(np.asarray([t for em in g["emitted"] for t in em]))
+            assert e.ada_get_counters()["status"] == 0
+            runs.append(rec)
+        finally:
+            e.close()
+    assert len(runs[0]) == len(runs[1])
+    for i, (a, b) in enumerate(zip(runs[0], runs[1])):
+        assert np.array_equal(np.asarray(a), np.asarray(b)), "record %d differs between launch modes" % i
+
+
 def test_argument_errors_are_reported_not_launched(tiny, eng):
     import ctypes as C
     from paper_2412_18910_b200 import AdaError, Config, lib
