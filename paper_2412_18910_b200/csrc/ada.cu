@@ -176,11 +176,16 @@ int rows_per_pass(const ada_config *c) {
 int plan_tc_splits(int tiles, int K) {
   const int sms = 148;   // B200; the split is part of the arithmetic (summation order), so it follows the shape alone
   const int kboxes = (K + 63) / 64;
+  // Cost of a launch relative to its weight bytes at full rate: how full the waves of one CTA per SM are, plus what
+  // every further split adds in partial sums written and read back (128 rows x 4 bytes per output column against
+  // 2 K bytes of weights, at about a third of the streaming rate).  Measured on the 7B shapes: gate-up (86 tiles,
+  // K = 4096) is 8 % faster with 3 splits (1.7 waves) than with 5 (2.9 waves); O / down (16 tiles) are best at 8-9.
+  const double per_split = 384.0 / (double)K;
   int best = 1;
   double best_cost = 1e30;
   for (int S = 1; S <= 16 && S * 4 <= (kboxes > 4 ? kboxes : 4); ++S) {
     const int ctas = tiles * S, waves = (ctas + sms - 1) / sms;
-    const double cost = (double)waves * sms / ctas + 0.03 * (S - 1);
+    const double cost = (double)waves * sms / ctas + per_split * (S - 1);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = S; }
   }
   return best;
