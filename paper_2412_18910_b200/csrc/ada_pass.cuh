@@ -193,6 +193,25 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const TensorMap128 *map, 
       "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+// The same load with a level-2 eviction policy.  Weights are read once per pass: with evict-first they do not push the
+// data that is read again (activation planes, partial sums, the cache) out of level 2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const TensorMap128 *map, int x, int y, uint64_t *bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
@@ -576,6 +595,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
     uint32_t *st_off = st_rec + pidx * 2 * kFlight, *st_end = st_off + kFlight;   // this producer's own record of the stages
     RingRetire rr;   // both producers place and retire every stage of the schedule (see ada_ring.h)
     rr.init();
+    const uint64_t pol_w = l2_policy_evict_first();   // weights are read once per pass
     for (int ph = 0; ph < nphase; ++ph) {
       int layer;
       const int kind = phase_kind(p, ph, layer);
@@ -609,11 +629,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const uint32_t dst = smem_u32(ring) + off, bar = smem_u32(&full[slot]);
             const unsigned long long mp = mi ? m1 : m0;
             const int y = mi ? row1 : row0;
-            for (int b = 0; b < nb; ++b)   // rows past the matrix and k past K read as zero
+            for (int b = 0; b < nb; ++b)   // rows past the matrix and k past K read as zero; evict-first in level 2
               asm volatile(
-                  "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                  "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(
                       dst + (uint32_t)(b * region)),
-                  "l"(mp), "r"(c * kKc + (b0 + b) * kBoxK), "r"(y), "r"(bar)
+                  "l"(mp), "r"(c * kKc + (b0 + b) * kBoxK), "r"(y), "r"(bar), "l"(pol_w)
                   : "memory");
           }
         }
