@@ -89,8 +89,13 @@ __global__ void __launch_bounds__(128) k_attn_rows(const Pass *pass, const float
       __nv_bfloat16 *kst = wst + (size_t)(h & 1) * 2 * kAttnHalf * HD;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the buffer come first
       mbar_expect_tx(&bars[h & 1], (unsigned)(2 * kAttnHalf * HD * 2));
-      bulk_g2s(kst, kpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
-      bulk_g2s(kst + kAttnHalf * HD, vpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
+      if constexpr (PACK) {   // a decode pass reads a sequence's cache rows once: evict-first in level 2
+        bulk_g2s_hint(kst, kpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1], l2_policy_evict_first());
+        bulk_g2s_hint(kst + kAttnHalf * HD, vpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1], l2_policy_evict_first());
+      } else {                // a prompt chunk's row groups read the same rows again
+        bulk_g2s(kst, kpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
+        bulk_g2s(kst + kAttnHalf * HD, vpool + off, (unsigned)(kAttnHalf * HD * 2), &bars[h & 1]);
+      }
     };
     {   // both buffers are free: the first two halves fly under the staging of q
       const int p0 = __shfl_sync(0xffffffffu, pages, 0), p1 = __shfl_sync(0xffffffffu, pages, 1);

@@ -186,6 +186,12 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+__device__ __forceinline__ void bulk_g2s_hint(void *dst, const void *src, unsigned bytes, uint64_t *bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
+               : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(void *dst, const TensorMap128 *map, int x, int y, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
@@ -835,8 +841,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
               const int key0 = r0 + 32 * bb;
               const int page = bb ? pg1 : pg0, slot = key0 % kPageSize;
               const size_t off = (((size_t)page * p.cache_layers + layer) * p.H + hh) * head_stride + (size_t)slot * HD;
-              bulk_g2s(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), bar);
-              bulk_g2s(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), bar);
+              // (a layer's cache rows are read once per pass: evict-first, like the weights)
+              bulk_g2s_hint(kst + (size_t)bb * 32 * HD, p.kpool + off, (unsigned)(32 * HD * 2), bar, l2_policy_evict_first());
+              bulk_g2s_hint(vst + (size_t)bb * 32 * HD, p.vpool + off, (unsigned)(32 * HD * 2), bar, l2_policy_evict_first());
             }
           };
           if (cw == 0) {   // the first two rounds fly under the staging below
@@ -1157,8 +1164,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
             const int nbox = (min(kKc, g.K - c * kKc) + kBoxK - 1) / kBoxK;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffer doubles as attention scratch
             mbar_expect_tx(&xfull[buf], (unsigned)(nbox * kXBoxBytes));
-            bulk_g2s(xbuf + (size_t)buf * kXBufBytes, g.xt + (size_t)c * (kKc / kBoxK) * (kXBoxBytes / 2),
-                     (unsigned)(nbox * kXBoxBytes), &xfull[buf]);
+            // (every CTA reads the same input tiles: evict-last)
+            bulk_g2s_hint(xbuf + (size_t)buf * kXBufBytes, g.xt + (size_t)c * (kKc / kBoxK) * (kXBoxBytes / 2),
+                          (unsigned)(nbox * kXBoxBytes), &xfull[buf], l2_policy_evict_last());
           }
           __syncwarp();
         }
