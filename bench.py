@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "decode tokens/sec at batch 1 (device-timed)"
 UNIT = "tokens/s"
 # measured dram__bytes_read+write over algorithmic bytes of k_pass (None once the kernel changed since the capture)
-TRAFFIC_PER_ALGORITHMIC_BYTE = 1.011
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.006
 
 
 def load_peaks():

@@ -839,7 +839,7 @@ extern "C" int ada_prefill(ada_ctx *x, int seq, const int32_t *d_prompt, int32_t
   if (m < 1) return fail(x, ADA_ERR_RANGE, "ada_prefill: empty prompt");
   if (m + c.n_max + 2 > c.kv_capacity) return fail(x, ADA_ERR_KV_FULL, "ada_prefill: prompt does not fit the cache");
   LAUNCH(x, k_copy_prompt, 8, 256, 0, x->tok, c.kv_capacity, seq, d_prompt, m);
-  const int chunk = attn_chunk_for_prompt(m, c.kv_capacity);   // attention split size of this sequence from now on
+  const int chunk = attn_chunk_for_prompt(m, c.kv_capacity, c.n_heads);   // attention split size of this sequence from now on
   const int last_rows = enqueue_chunks(x, seq, 0, m, m - 1, true, chunk);
   LAUNCH(x, k_finish_prefill, 1, 32, 0, x->st, x->tok, c.kv_capacity, seq, m, chunk, x->chunk_tok + (last_rows - 1),
          d_first_token);

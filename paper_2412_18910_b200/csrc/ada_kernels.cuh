@@ -265,15 +265,18 @@ __global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bf
   }
 }
 
-// Keys per attention split of a sequence whose prompt has m tokens, in a cache of `cap` positions: four splits cover
-// the prompt and the tokens expected after it (a quarter as many again, at least 256, within the capacity); at least
-// cap / 32 so that no sequence has more than 32 splits.  Chosen once per sequence, from its prompt alone: the split a
-// key falls in must not depend on the shape of the pass that reads it (a one-row step and a block of drafts then sum in
-// the same order).
-__host__ __device__ __forceinline__ int attn_chunk_for_prompt(int m, int cap) {
+// Keys per attention split of a sequence whose prompt has m tokens, in a cache of `cap` positions, for a model of H
+// heads: as many splits as keep heads x splits within the persistent kernel's 148 CTAs (four at most: 32 heads -> 4,
+// 40 heads -> 3) cover the prompt and the tokens expected after it (a quarter as many again, at least 256, within the
+// capacity); at least cap / 32 so that no sequence has more than 32 splits.  Chosen once per sequence, from its prompt
+// alone: the split a key falls in must not depend on the shape of the pass that reads it (a one-row step and a block of
+// drafts then sum in the same order).
+__host__ __device__ __forceinline__ int attn_chunk_for_prompt(int m, int cap, int H) {
   const int grow = m / 4 > 256 ? m / 4 : 256;
   const int total = m + grow < cap ? m + grow : cap;
-  int chunk = ((total + 3) / 4 + 31) / 32 * 32;
+  int nsplit = H > 0 ? 148 / H : 4;
+  nsplit = nsplit < 1 ? 1 : (nsplit > 4 ? 4 : nsplit);
+  int chunk = ((total + nsplit - 1) / nsplit + 31) / 32 * 32;
   const int least = ((cap + 31) / 32 + 31) / 32 * 32;
   return chunk < least ? least : chunk;
 }
