@@ -160,10 +160,16 @@ __global__ void k_argmax_final(const float4 *amax, int tiles, int TP, const Pass
   if (t >= T) return;
   Top2 b;
   b.v1 = -INFINITY; b.i1 = 0x7fffffff; b.v2 = -INFINITY;
-  for (int i = threadIdx.x; i < tiles; i += 32) {
-    const float4 c = amax[(size_t)i * TP + t];
-    Top2 x; x.v1 = c.x; x.i1 = __float_as_int(c.y); x.v2 = c.z;
-    b = top2_merge(b, x);
+  for (int i0 = threadIdx.x; i0 < tiles; i0 += 4 * 32) {   // a lane's four candidates of a round in flight together
+    float4 c[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      c[u] = i0 + 32 * u < tiles ? amax[(size_t)(i0 + 32 * u) * TP + t] : make_float4(-INFINITY, __int_as_float(0x7fffffff), -INFINITY, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      Top2 x; x.v1 = c[u].x; x.i1 = __float_as_int(c[u].y); x.v2 = c[u].z;
+      b = top2_merge(b, x);
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) b = top2_shfl_xor(b, o);
@@ -253,14 +259,16 @@ __global__ void k_split_lm_rows(const Pass *pass, const float *h, int d, __nv_bf
   if (i >= pass->lmT) return;
   const int t = pass->lm_row[i];
   const int b = pass->row_seq[t];
-  const float *hr = h + (size_t)t * d;
-  float *fo = dfeat + ((size_t)b * nmax + step) * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+  const float *__restrict__ hr = h + (size_t)t * d;
+  float *__restrict__ fo = dfeat + ((size_t)b * nmax + step) * d;
+  __nv_bfloat16 *__restrict__ oh = xhi + (size_t)i * ldx, *__restrict__ ol = xlo + (size_t)i * ldx;
+#pragma unroll 8
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {   // (loads of eight steps in flight together)
     const float x = hr[c];
     __nv_bfloat16 hi, lo;
     split_bf16(x, hi, lo);
-    xhi[(size_t)i * ldx + c] = hi;
-    xlo[(size_t)i * ldx + c] = lo;
+    oh[c] = hi;
+    ol[c] = lo;
     fo[c] = x;
   }
 }
