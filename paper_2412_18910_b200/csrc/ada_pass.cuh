@@ -1322,9 +1322,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
           p.h[(size_t)t * p.d + vrow] = hn;
           xstore(p.xa, t, vrow, hn * gn);
         }
-        // sum of squares per pass row: over the warp's 32 weight rows, then over the warps in order (below)
-        const float r = warp_sum(hn * hn);
-        if (lane == 0) ssw[cw * 16 + t] = r;
+        // squares parked in the thread's column of the (now read) old-residual area; summed per pass row below
+        hs[t * 256] = hn * hn;
       } else if (sw) {
         if (act) {
           const float up = us[t * 256] * sc;
@@ -1356,12 +1355,20 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const PassParams p) {
       }
     }
     if (has_ss) {
-      if (lane >= Tg && lane < 16) ssw[cw * 16 + lane] = 0.f;
+      // sum of squares per pass row over the CTA's 256 weight-row slots: warp w takes rows 2 w and 2 w + 1, a lane eight
+      // slots of each (fixed order), one warp reduction per row instead of one per row and warp inside the loop above
       named_bar(3, kNumCWarps * 32);
-      if (cw == 0 && lane < 16) {
+      const float *sq = reinterpret_cast<const float *>(xbuf) + 2 * 16 * 256;
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int t = 2 * cw + k;
         float r = 0.f;
-        for (int w = 0; w < kNumCWarps; ++w) r += ssw[w * 16 + lane];
-        p.ss_part[(size_t)cta * 16 + lane] = r;
+        if (t < Tg) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) r += sq[t * 256 + j * 32 + lane];
+        }
+        r = warp_sum(r);
+        if (lane == 0) p.ss_part[(size_t)cta * 16 + t] = r;
       }
     } else if (epi == EPI_ARGMAX_LM) {
       if (lane >= Tg && lane < 16) {
