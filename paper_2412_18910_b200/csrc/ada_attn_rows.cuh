@@ -1,20 +1,27 @@
-// Attention of the multi-row path (ragged batches, prompt chunks) on mma.sync: the rows of one sequence for one
-// head over one split of the cache, 16 query rows per CTA (row groups of a long pass across grid.z).
+// Attention of the multi-row path (ragged batches, prompt chunks) on mma.sync: a group of query rows of one sequence
+// for one head over one split of the cache per CTA (the row groups of a pass across grid.z).
 //
 // Row r (absolute position pos0 + r) sees cache positions 0 .. pos0 + r: the whole history and the earlier rows
 // of its own block (every row's key and value are in the cache before this kernel runs).  The size of a sequence's
-// cache splits is fixed when its prompt is read (a quarter of the prompt and its expected continuation, at least an
-// eighth of the capacity), so the split a key falls in does not depend on the pass, and a short context is not cut
-// into slivers that cost more to set up and merge than to compute.  A warp takes 32-key blocks of the split, in halves
-// of 16 keys: one bulk copy brings a half's key rows and one its value rows (they are contiguous in the cache page)
-// into one of the warp's two buffers, so the next half is in flight while this one is computed -- scores = q k^T
-// as m16n8k16 products per 16 channels (two tiles of 8 keys), online softmax on the accumulator fragments, weighted
-// values as m16n8k16 products over the 16 keys per 8 channels, 16 keys at a time.  Cache elements are 16-bit halves and enter the products as they are;
-// q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, so each product is issued twice and
-// the sums are fp32 (error 2^-22 relative).  Key and value rows are kept in the cache with their 16-byte chunks XORed by
-// (slot & 7), which makes ldmatrix of 8 consecutive keys (plain or transposed) conflict-free and lets the copy be verbatim.  A copy always
-// takes 16 whole rows: rows past the sequence are masked out of the softmax, and every cache row is finite (the
-// pools are cleared at initialisation), so they add exact zeros.
+// cache splits is fixed when its prompt is read (the prompt and its expected continuation cut into at most four, at
+// least an eighth of the capacity), so the split a key falls in does not depend on the pass, and a short context is not
+// cut into slivers that cost more to set up and merge than to compute.  The split's 16-key halves are dealt to the four
+// warps in turn: one bulk copy brings a half's key rows and one its value rows (they are contiguous in the cache page)
+// into one of the warp's two buffers, so the next half is in flight while this one is computed -- scores = q k^T as
+// m16n8k16 products per 16 channels (two tiles of 8 keys), online softmax on the accumulator fragments, weighted values
+// as m16n8k16 products over the 16 keys per 8 channels.  Cache elements are 16-bit halves and enter the products as
+// they are; q and the softmax weights are fp32 and enter as a (hi, lo) pair of halves, the sums are fp32 (error 2^-22
+// relative).  Two forms (template parameter PACK):
+//   PACK = false  16 query rows per group; every product is issued twice, for the hi and for the lo halves (prompt
+//                 chunks)
+//   PACK = true   8 query rows per group: tile rows 0..7 hold their hi halves, rows 8..15 their lo halves, so one
+//                 product yields both parts and half as many products and q loads are issued per key (decode passes of
+//                 a batch, at most n_max + 1 rows per sequence; every decode row goes through this form whatever the
+//                 shape of its pass, so a row's sums do not depend on the pass)
+// Key and value rows are kept in the cache with their 16-byte chunks XORed by (slot & 7), which makes ldmatrix of 8
+// consecutive keys (plain or transposed) conflict-free and lets the copy be verbatim.  A copy always takes 16 whole
+// rows: rows past the sequence are masked out of the softmax, and every cache row is finite (the pools are cleared at
+// initialisation), so they add exact zeros.
 // Partial (m, l, o[hd]) per (head, split, row) goes to `part`; k_attn_combine merges the splits in split order.
 #pragma once
 #include "ada_pass.cuh"
